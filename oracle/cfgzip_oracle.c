@@ -1,0 +1,192 @@
+/*
+ * CPU oracle for the CFGzip per-decode-step wrapper path.
+ *
+ * TEST INFRASTRUCTURE ONLY. This file is the slow, element-by-element
+ * statement of what the path computes, written from the paper's Section 3.1
+ * ("Pre-Computation" and "Inference" paragraphs) and Section 2.2. It shares
+ * no code, header, table or helper with the CUDA library and is never called
+ * from the product path. Floating-point reductions are carried in double.
+ *
+ * Conventions (where the paper is silent, the reading taken is stated):
+ *   - c[i]  : class id of token i, 0 <= c[i] < K      (Section 3.1, vector c)
+ *   - r[k]  : token id representing class k            (Section 3.1, vector r)
+ *   - masks are packed 32-bit words, bit j of word w <-> index 32*w + j,
+ *     1 = allowed. Class-mask bits >= K are ignored; vocab-mask bits >= V
+ *     inside the last word are written 0.
+ *   - the paper's "z_i <- z_i * m_{c_i}" with m in {-inf, 1} is read as a
+ *     select: a disallowed logit becomes -inf (Section 2.2 says exactly
+ *     that), an allowed logit keeps its bits.
+ *   - the token choice is greedy: largest allowed value, ties to the lowest
+ *     token id, comparison on values (so -0.0 == +0.0).
+ *   - a row with nothing allowed yields argmax = rep = -1 and -inf log
+ *     quantities; a row whose allowed logits are all -inf yields the lowest
+ *     allowed token id and -inf log quantities.
+ *
+ * Parity pins: every function here is pinned by tests/test_oracle_pins.py
+ * (closed forms, invariants, a library log-softmax, brute force); nothing in
+ * this file is "parity unpinned".
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+enum { ORACLE_F32 = 0, ORACLE_BF16 = 1 };
+
+/* bfloat16 -> float is exact: the 16 bits are the top half of the float. */
+static float bf16_to_float(uint16_t h) {
+    uint32_t u = (uint32_t)h << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return f;
+}
+
+static float load_logit(const void* z, int dtype, int64_t idx) {
+    if (dtype == ORACLE_BF16) return bf16_to_float(((const uint16_t*)z)[idx]);
+    return ((const float*)z)[idx];
+}
+
+static void store_neg_inf(void* z, int dtype, int64_t idx) {
+    if (dtype == ORACLE_BF16) {
+        ((uint16_t*)z)[idx] = 0xFF80u;
+    } else {
+        uint32_t u = 0xFF800000u;
+        memcpy((float*)z + idx, &u, sizeof u);
+    }
+}
+
+static int get_bit(const uint32_t* words, int64_t i) { return (int)((words[i >> 5] >> (i & 31)) & 1u); }
+
+/*
+ * Gather-expansion of the class mask into a token mask (Section 3.1,
+ * "Inference": the mask entry used for token i is m_{c_i}).
+ * vocab_mask row b receives ceil(V/32) words.
+ */
+void oracle_expand_mask(const int32_t* c, int32_t V, int32_t K, const uint32_t* class_mask,
+                        int64_t class_stride_words, uint32_t* vocab_mask, int64_t vocab_stride_words,
+                        int32_t B) {
+    (void)K;
+    int32_t VW = (V + 31) / 32;
+    for (int32_t b = 0; b < B; ++b) {
+        const uint32_t* m = class_mask + (int64_t)b * class_stride_words;
+        uint32_t* v = vocab_mask + (int64_t)b * vocab_stride_words;
+        for (int32_t w = 0; w < VW; ++w) v[w] = 0u;
+        for (int32_t i = 0; i < V; ++i) {
+            int allowed = get_bit(m, c[i]);
+            v[i >> 5] |= (uint32_t)allowed << (i & 31);
+        }
+    }
+}
+
+/*
+ * Inverse of c: for class k, tok[off[k] .. off[k+1]) lists its tokens in
+ * ascending token id. Follows from the definition of c (Section 3.1).
+ */
+void oracle_build_csr(const int32_t* c, int32_t V, int32_t K, int32_t* off, int32_t* tok) {
+    for (int32_t k = 0; k <= K; ++k) off[k] = 0;
+    for (int32_t i = 0; i < V; ++i) off[c[i] + 1] += 1;
+    for (int32_t k = 0; k < K; ++k) off[k + 1] += off[k];
+    /* visiting tokens in ascending id keeps every class list ascending */
+    int32_t* next = (int32_t*)malloc((size_t)K * sizeof(int32_t));
+    for (int32_t k = 0; k < K; ++k) next[k] = off[k];
+    for (int32_t i = 0; i < V; ++i) tok[next[c[i]]++] = i;
+    free(next);
+}
+
+/*
+ * The same token mask reached from the class side: clear the row, then for
+ * every allowed class set the bit of each of its members.
+ */
+void oracle_expand_mask_csr(const int32_t* off, const int32_t* tok, int32_t V, int32_t K,
+                            const uint32_t* class_mask, int64_t class_stride_words, uint32_t* vocab_mask,
+                            int64_t vocab_stride_words, int32_t B) {
+    int32_t VW = (V + 31) / 32;
+    for (int32_t b = 0; b < B; ++b) {
+        const uint32_t* m = class_mask + (int64_t)b * class_stride_words;
+        uint32_t* v = vocab_mask + (int64_t)b * vocab_stride_words;
+        for (int32_t w = 0; w < VW; ++w) v[w] = 0u;
+        for (int32_t k = 0; k < K; ++k) {
+            if (!get_bit(m, k)) continue;
+            for (int32_t j = off[k]; j < off[k + 1]; ++j) v[tok[j] >> 5] |= 1u << (tok[j] & 31);
+        }
+    }
+}
+
+/*
+ * Logit masking (Section 2.2: the logit of a disallowed token is set to
+ * -inf; Section 3.1 applies it through the token mask). In place; elements
+ * at index >= V of a row are not touched.
+ */
+void oracle_mask_logits(void* logits, int dtype, int64_t row_stride_elems, int32_t B, int32_t V,
+                        const uint32_t* vocab_mask, int64_t vocab_stride_words) {
+    for (int32_t b = 0; b < B; ++b) {
+        const uint32_t* v = vocab_mask + (int64_t)b * vocab_stride_words;
+        for (int32_t i = 0; i < V; ++i)
+            if (!get_bit(v, i)) store_neg_inf(logits, dtype, (int64_t)b * row_stride_elems + i);
+    }
+}
+
+/*
+ * Greedy choice and log-softmax renormalised over the allowed set, from
+ * logits that are already masked. lse = log sum_{allowed} exp(z_i);
+ * logp_i = z_i - lse; logp_argmax = z_best - lse = -log sum exp(z_i - z_best).
+ * logp_full (nullable) is [B, V] doubles with row stride V.
+ */
+void oracle_logsoftmax_argmax(const void* logits, int dtype, int64_t row_stride_elems, int32_t B, int32_t V,
+                              const uint32_t* vocab_mask, int64_t vocab_stride_words, int32_t* argmax,
+                              double* lse, double* logp_argmax, double* logp_full) {
+    for (int32_t b = 0; b < B; ++b) {
+        const uint32_t* v = vocab_mask + (int64_t)b * vocab_stride_words;
+        int64_t base = (int64_t)b * row_stride_elems;
+        int32_t best = -1;
+        for (int32_t i = 0; i < V; ++i) {
+            if (!get_bit(v, i)) continue;
+            if (best < 0 || load_logit(logits, dtype, base + i) > load_logit(logits, dtype, base + best)) best = i;
+        }
+        argmax[b] = best;
+        double M = best < 0 ? -INFINITY : (double)load_logit(logits, dtype, base + best);
+        double S = 0.0;
+        if (best >= 0 && M > -INFINITY)
+            for (int32_t i = 0; i < V; ++i)
+                if (get_bit(v, i)) S += exp((double)load_logit(logits, dtype, base + i) - M);
+        int finite = best >= 0 && M > -INFINITY;
+        lse[b] = finite ? M + log(S) : -INFINITY;
+        logp_argmax[b] = finite ? -log(S) : -INFINITY;
+        if (logp_full) {
+            for (int32_t i = 0; i < V; ++i) {
+                double lp = -INFINITY;
+                if (finite && get_bit(v, i)) lp = (double)load_logit(logits, dtype, base + i) - lse[b];
+                logp_full[(int64_t)b * V + i] = lp;
+            }
+        }
+    }
+}
+
+/*
+ * Token -> representative of its class, r_{c_t} (Section 3.1, "Inference";
+ * Figure 1a). A token id outside [0, V) maps to -1.
+ */
+void oracle_map_tokens(const int32_t* c, const int32_t* r, int32_t V, int32_t K, const int32_t* tokens,
+                       int32_t* reps, int32_t B) {
+    (void)K;
+    for (int32_t b = 0; b < B; ++b) {
+        int32_t t = tokens[b];
+        reps[b] = (t >= 0 && t < V) ? r[c[t]] : -1;
+    }
+}
+
+/*
+ * One whole decode step for rows that share one partition: the four steps
+ * above in the order the paper gives them (expand, mask, choose/normalise,
+ * map to representative). vocab_mask must hold B rows of ceil(V/32) words.
+ */
+void oracle_decode_step(const int32_t* c, const int32_t* r, int32_t V, int32_t K, const uint32_t* class_mask,
+                        int64_t class_stride_words, void* logits, int dtype, int64_t row_stride_elems,
+                        int32_t B, uint32_t* vocab_mask, int64_t vocab_stride_words, int32_t* argmax,
+                        int32_t* rep, double* lse, double* logp_argmax, double* logp_full) {
+    oracle_expand_mask(c, V, K, class_mask, class_stride_words, vocab_mask, vocab_stride_words, B);
+    oracle_mask_logits(logits, dtype, row_stride_elems, B, V, vocab_mask, vocab_stride_words);
+    oracle_logsoftmax_argmax(logits, dtype, row_stride_elems, B, V, vocab_mask, vocab_stride_words, argmax, lse,
+                             logp_argmax, logp_full);
+    oracle_map_tokens(c, r, V, K, argmax, rep, B);
+}

@@ -1,0 +1,342 @@
+"""Pins for the CPU oracle: it is checked against things other than itself.
+
+Closed forms, algebraic invariants, the corollary of the paper's Theorem 1 (a token and
+the representative of its class always share a mask bit), a library log-softmax in
+float64 on the case where the path reduces to a textbook one, a hand-worked example and
+per-bit brute force on tiny shapes whose V and K are not multiples of 32.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth
+from synth import rng
+
+NEG_INF_F32 = np.uint32(0xFF800000)
+NEG_INF_BF16 = np.uint16(0xFF80)
+
+
+def _popcount_rows(words):
+    return np.unpackbits(np.ascontiguousarray(words).view(np.uint8), axis=-1).sum(axis=-1)
+
+
+def _rand_mask(K, B, p, *ids):
+    return synth.class_mask_bernoulli(K, B, p, rng.stream_key(991, *ids))
+
+
+SHAPES = [(1, 1), (31, 2), (32, 31), (33, 32), (63, 33), (64, 5), (65, 64), (1000, 37), (4099, 130)]
+
+
+# ---------------------------------------------------------------- expand
+
+def test_hand_worked_example():
+    # six tokens, three classes; classes 0 and 2 allowed
+    c = np.array([0, 1, 0, 2, 1, 2], dtype=np.int32)
+    r = np.array([0, 1, 3], dtype=np.int32)
+    cm = np.array([[0b101]], dtype=np.uint32)
+    vm = oracle.expand_mask(c, 3, cm)
+    assert vm.tolist() == [[0b101101]]  # tokens 0, 2, 3, 5
+    z = np.array([[1.0, 5.0, 2.0, 0.0, 9.0, 2.0]], dtype=np.float32)
+    oracle.mask_logits(z, 6, vm)
+    assert z[0, [0, 2, 3, 5]].tolist() == [1.0, 2.0, 0.0, 2.0]
+    assert np.all(np.isneginf(z[0, [1, 4]]))
+    am, lse, lpa, full = oracle.logsoftmax_argmax(z, 6, vm, want_full=True)
+    assert am.tolist() == [2]  # 2.0 appears at tokens 2 and 5: the lower id wins
+    want_lse = math.log(math.e + 2 * math.e ** 2 + 1.0)
+    assert abs(lse[0] - want_lse) < 1e-12
+    assert abs(lpa[0] - (2.0 - want_lse)) < 1e-12
+    assert abs(full[0, 3] - (0.0 - want_lse)) < 1e-12 and np.isneginf(full[0, 1])
+    assert oracle.map_tokens(c, r, am).tolist() == [0]
+
+
+@pytest.mark.parametrize("V,K", SHAPES)
+def test_expand_brute_force_per_bit(V, K):
+    K = min(K, V)
+    part = synth.zipf_partition(V, K, 1.1, seed=V + K)
+    cm = _rand_mask(K, 3, 0.4, V, K)
+    vm = oracle.expand_mask(part.c, K, cm)
+    assert vm.shape == (3, (V + 31) // 32)
+    for b in range(3):
+        for i in range(V):
+            k = int(part.c[i])
+            want = (int(cm[b, k // 32]) >> (k % 32)) & 1
+            got = (int(vm[b, i // 32]) >> (i % 32)) & 1
+            assert got == want, (b, i)
+        for i in range(V, 32 * vm.shape[1]):  # tail bits of the last word are zero
+            assert (int(vm[b, i // 32]) >> (i % 32)) & 1 == 0
+
+
+@pytest.mark.parametrize("V,K", [(1000, 37), (32000, 256), (128256, 2048)])
+def test_expand_popcount_equals_allowed_class_sizes(V, K):
+    part = synth.zipf_partition(V, K, 1.1, seed=3)
+    sizes = np.bincount(part.c, minlength=K)
+    cm = _rand_mask(K, 4, 0.3, V)
+    vm = oracle.expand_mask(part.c, K, cm)
+    allowed = synth.unpack_bits(cm, K)
+    assert _popcount_rows(vm).tolist() == (allowed * sizes[None, :]).sum(axis=1).tolist()
+
+
+@pytest.mark.parametrize("V,K", SHAPES)
+def test_expand_all_ones_all_zeros_and_ignored_tail_bits(V, K):
+    K = min(K, V)
+    part = synth.zipf_partition(V, K, 1.1, seed=1)
+    KW = (K + 31) // 32
+    ones = np.full((1, KW), 0xFFFFFFFF, dtype=np.uint32)  # includes garbage bits >= K
+    vm = oracle.expand_mask(part.c, K, ones)
+    assert synth.unpack_bits(vm, 32 * vm.shape[1])[0].tolist() == [i < V for i in range(32 * vm.shape[1])]
+    assert not oracle.expand_mask(part.c, K, np.zeros((1, KW), dtype=np.uint32)).any()
+    cm = _rand_mask(K, 2, 0.5, V, K, 7)
+    dirty = cm.copy()
+    if K % 32:
+        dirty[:, -1] |= np.uint32((0xFFFFFFFF << (K % 32)) & 0xFFFFFFFF)
+    assert np.array_equal(oracle.expand_mask(part.c, K, cm), oracle.expand_mask(part.c, K, dirty))
+
+
+@pytest.mark.parametrize("V", [1, 31, 32, 33, 100, 1024])
+def test_expand_identity_partition_copies_the_class_mask(V):
+    part = synth.identity_partition(V)
+    cm = _rand_mask(V, 3, 0.5, V)
+    assert np.array_equal(oracle.expand_mask(part.c, V, cm), cm)
+
+
+def test_expand_single_class_is_all_or_nothing():
+    c = np.zeros(77, dtype=np.int32)
+    on = oracle.expand_mask(c, 1, np.array([[1]], dtype=np.uint32))
+    off = oracle.expand_mask(c, 1, np.array([[0]], dtype=np.uint32))
+    assert _popcount_rows(on).tolist() == [77] and _popcount_rows(off).tolist() == [0]
+
+
+def test_expand_is_a_boolean_homomorphism():
+    V, K = 5003, 211
+    part = synth.zipf_partition(V, K, 1.1, seed=5)
+    a, b = _rand_mask(K, 2, 0.5, 1), _rand_mask(K, 2, 0.3, 2)
+    ea, eb = oracle.expand_mask(part.c, K, a), oracle.expand_mask(part.c, K, b)
+    assert np.array_equal(oracle.expand_mask(part.c, K, a | b), ea | eb)
+    assert np.array_equal(oracle.expand_mask(part.c, K, a & b), ea & eb)
+    valid = synth.pack_bits(np.ones((1, V), dtype=bool))
+    assert np.array_equal(oracle.expand_mask(part.c, K, ~a), ~ea & valid)
+
+
+def test_expand_invariant_under_class_relabelling():
+    V, K = 3001, 97
+    part = synth.zipf_partition(V, K, 1.1, seed=6)
+    perm = rng.permutation(rng.stream_key(5, 5), K)  # new id of class k is perm[k]
+    bits = synth.unpack_bits(_rand_mask(K, 3, 0.4, 9), K)
+    bits2 = np.zeros_like(bits)
+    bits2[:, perm] = bits
+    c2 = perm[part.c].astype(np.int32)
+    assert np.array_equal(oracle.expand_mask(part.c, K, synth.pack_bits(bits)),
+                          oracle.expand_mask(c2, K, synth.pack_bits(bits2)))
+
+
+@pytest.mark.parametrize("maker", ["zipf", "heavy"])
+def test_token_and_its_representative_share_a_bit(maker):
+    # corollary of Theorem 1: feeding the engine r_{c_t} instead of t changes nothing
+    V, K = 20000, 300
+    part = (synth.zipf_partition(V, K, 1.1, seed=8) if maker == "zipf"
+            else synth.heavy_tail_partition(V, K, 0.6, 1.3, seed=8))
+    vm = oracle.expand_mask(part.c, K, _rand_mask(K, 4, 0.2, 3))
+    bits = synth.unpack_bits(vm, V)
+    reps = part.r[part.c]
+    assert np.array_equal(bits, bits[:, reps])
+
+
+@pytest.mark.parametrize("V,K", SHAPES + [(32000, 256)])
+def test_dense_and_class_side_expansion_agree(V, K):
+    K = min(K, V)
+    part = synth.zipf_partition(V, K, 1.1, seed=2)
+    off, tok = oracle.build_csr(part.c, K)
+    assert off[0] == 0 and off[-1] == V
+    assert np.array_equal(np.diff(off), np.bincount(part.c, minlength=K))
+    assert sorted(tok.tolist()) == list(range(V))
+    for k in range(K):
+        seg = tok[off[k]:off[k + 1]]
+        assert np.all(part.c[seg] == k) and np.all(np.diff(seg) > 0)
+    cm = _rand_mask(K, 3, 0.3, V, 4)
+    assert np.array_equal(oracle.expand_mask(part.c, K, cm), oracle.expand_mask_csr(off, tok, V, K, cm))
+
+
+# ---------------------------------------------------------------- mask_logits
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_mask_logits_identities(dtype):
+    V, stride, B = 1003, 1010, 3
+    z0 = synth.logits_normal(B, stride, 1.0, dtype, (1, 2, 3))
+    ones = synth.pack_bits(np.ones((B, V), dtype=bool))
+    z = z0.copy()
+    oracle.mask_logits(z, V, ones)
+    assert np.array_equal(z.view(np.uint8), z0.view(np.uint8))  # all allowed: bit-identical
+    z = z0.copy()
+    oracle.mask_logits(z, V, np.zeros_like(ones))
+    ninf = NEG_INF_F32 if dtype == "f32" else NEG_INF_BF16
+    bits = z.view(np.uint32 if dtype == "f32" else np.uint16)
+    assert np.all(bits[:, :V] == ninf)
+    assert np.array_equal(bits[:, V:], z0.view(bits.dtype)[:, V:])  # beyond V untouched
+    vm = synth.pack_bits(rng.uniform(rng.stream_key(4), B * V).reshape(B, V) < 0.3)
+    z = z0.copy()
+    oracle.mask_logits(z, V, vm)
+    once = z.copy()
+    oracle.mask_logits(z, V, vm)
+    assert np.array_equal(z.view(np.uint8), once.view(np.uint8))  # idempotent
+    bits = once.view(np.uint32 if dtype == "f32" else np.uint16)
+    keep = synth.unpack_bits(vm, V)
+    assert np.array_equal(bits[:, :V][keep], z0.view(bits.dtype)[:, :V][keep])
+    assert np.all(bits[:, :V][~keep] == ninf)
+    assert ((bits[:, :V] == ninf).sum(axis=1) == V - _popcount_rows(vm)).all()
+
+
+# ---------------------------------------------------------------- log-softmax / argmax
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_logsoftmax_reduces_to_library_routine_when_everything_is_allowed(dtype):
+    V, B = 4001, 5
+    z = synth.logits_normal(B, V, 2.0, dtype, (7, 7))
+    ones = synth.pack_bits(np.ones((B, V), dtype=bool))
+    am, lse, lpa, full = oracle.logsoftmax_argmax(z, V, ones, want_full=True)
+    if dtype == "bf16":
+        zt = torch.from_numpy(z.view(np.int16)).view(torch.bfloat16).to(torch.float64)
+    else:
+        zt = torch.from_numpy(z).to(torch.float64)
+    ref = torch.log_softmax(zt, dim=-1).numpy()
+    assert np.allclose(full, ref, rtol=0, atol=1e-10)
+    assert np.allclose(lse, torch.logsumexp(zt, dim=-1).numpy(), rtol=0, atol=1e-10)
+    assert am.tolist() == [int(np.flatnonzero(row == row.max())[0]) for row in zt.numpy()]
+    assert np.allclose(lpa, ref[np.arange(B), am], rtol=0, atol=1e-10)
+
+
+def test_logsoftmax_masked_equals_library_routine_on_the_allowed_subset():
+    V, B = 3000, 4
+    z = synth.logits_normal(B, V, 1.0, "f32", (8, 1))
+    keep = rng.uniform(rng.stream_key(8, 2), B * V).reshape(B, V) < 0.2
+    vm = synth.pack_bits(keep)
+    oracle.mask_logits(z, V, vm)
+    am, lse, lpa, full = oracle.logsoftmax_argmax(z, V, vm, want_full=True)
+    for b in range(B):
+        idx = np.flatnonzero(keep[b])
+        sub = torch.from_numpy(z[b, idx]).to(torch.float64)
+        ref = torch.log_softmax(sub, dim=-1).numpy()
+        assert np.allclose(full[b, idx], ref, rtol=0, atol=1e-10)
+        assert np.all(np.isneginf(full[b, ~keep[b]]))
+        assert am[b] == idx[int(np.argmax(sub.numpy()))]
+        assert abs(np.exp(full[b, idx]).sum() - 1.0) < 1e-9
+
+
+def test_logsoftmax_closed_forms():
+    V = 777
+    for n, a in [(1, 3.5), (7, -2.0), (777, 0.25)]:
+        z = np.full((1, V), a, dtype=np.float32)
+        keep = np.zeros((1, V), dtype=bool)
+        keep[0, rng.permutation(rng.stream_key(n), V)[:n]] = True
+        vm = synth.pack_bits(keep)
+        oracle.mask_logits(z, V, vm)
+        am, lse, lpa, _ = oracle.logsoftmax_argmax(z, V, vm)
+        assert abs(lse[0] - (a + math.log(n))) < 1e-12
+        assert abs(lpa[0] + math.log(n)) < 1e-12
+        assert am[0] == np.flatnonzero(keep[0])[0]  # constant row: lowest allowed id
+
+
+def test_logsoftmax_shift_invariance_and_sign():
+    V, B = 2000, 3
+    z = synth.logits_normal(B, V, 1.0, "f32", (9, 1))
+    vm = synth.pack_bits(rng.uniform(rng.stream_key(9, 2), B * V).reshape(B, V) < 0.5)
+    z2 = (z + np.float32(4.0)).astype(np.float32)
+    oracle.mask_logits(z, V, vm)
+    oracle.mask_logits(z2, V, vm)
+    a1, l1, p1, f1 = oracle.logsoftmax_argmax(z, V, vm, want_full=True)
+    a2, l2, p2, f2 = oracle.logsoftmax_argmax(z2, V, vm, want_full=True)
+    assert np.array_equal(a1, a2)
+    assert np.allclose(l2 - l1, 4.0, atol=1e-5)  # float32 rounding of the shifted inputs
+    fin = np.isfinite(f1)
+    assert np.allclose(f1[fin], f2[fin], atol=1e-5)
+    assert np.all(p1 <= 0.0)
+
+
+def test_argmax_planted_spikes_and_ties():
+    V, K = 5000, 64
+    part = synth.zipf_partition(V, K, 1.1, seed=11)
+    bits = np.zeros((1, K), dtype=bool)
+    bits[0, :20] = True
+    cm = synth.pack_bits(bits)
+    allowed = np.flatnonzero(bits[0][part.c])
+    masked = np.flatnonzero(~bits[0][part.c])
+    z0 = synth.logits_normal(1, V, 1.0, "f32", (12,))
+
+    def run(z):
+        return oracle.decode_step([part], None, cm, z.copy())
+
+    z = z0.copy(); z[0, allowed[37]] = 50.0
+    assert run(z)["argmax"][0] == allowed[37]
+    z = z0.copy(); z[0, allowed[90]] = 50.0; z[0, allowed[12]] = 50.0
+    assert run(z)["argmax"][0] == allowed[12]  # equal maxima: lower id
+    z = z0.copy(); z[0, masked[5]] = 99.0; z[0, allowed[41]] = 50.0
+    out = run(z)
+    assert out["argmax"][0] == allowed[41]  # a spike at a disallowed token is never returned
+    assert synth.unpack_bits(out["vocab_mask"], V)[0, out["argmax"][0]]
+    z = np.full((1, V), -3.0, dtype=np.float32); z[0, allowed[7]] = 0.0; z[0, allowed[3]] = -0.0
+    assert run(z)["argmax"][0] == allowed[3]  # -0.0 == +0.0: a tie, lower id wins
+    brute = max(allowed, key=lambda i: (z0[0, i], -i))
+    assert run(z0)["argmax"][0] == brute
+
+
+def test_degenerate_rows():
+    V, K = 100, 4
+    part = synth.zipf_partition(V, K, 1.1, seed=1)
+    z = synth.logits_normal(2, V, 1.0, "f32", (13,))
+    cm = np.array([[0], [0b10]], dtype=np.uint32)
+    z[1, part.c == 1] = -np.inf  # every allowed logit of row 1 is -inf
+    out = oracle.decode_step([part], None, cm, z, want_full=True)
+    assert out["argmax"][0] == -1 and out["rep"][0] == -1
+    assert np.isneginf(out["lse"][0]) and np.isneginf(out["logp_argmax"][0])
+    assert np.all(np.isneginf(z[0])) and not out["vocab_mask"][0].any()
+    assert out["argmax"][1] == np.flatnonzero(part.c == 1)[0]
+    assert out["rep"][1] == part.r[1]
+    assert np.isneginf(out["lse"][1]) and np.all(np.isneginf(out["logp_full"][1]))
+
+
+# ---------------------------------------------------------------- map_tokens / whole step
+
+def test_map_tokens_algebra():
+    V, K = 9000, 150
+    part = synth.zipf_partition(V, K, 1.1, seed=14)
+    assert np.array_equal(part.c[part.r], np.arange(K))  # c[r_k] = k
+    toks = np.arange(V, dtype=np.int32)
+    m = oracle.map_tokens(part.c, part.r, toks)
+    assert np.array_equal(oracle.map_tokens(part.c, part.r, m), m)  # idempotent
+    assert np.array_equal(part.c[m], part.c)  # stays inside the class
+    assert np.all(m <= toks)  # representative is the lowest id of the class
+    assert oracle.map_tokens(part.c, part.r, np.array([-1, V, V + 5], dtype=np.int32)).tolist() == [-1, -1, -1]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_decode_step_is_the_composition_of_its_steps_and_handles_row_partitions(dtype):
+    V, K, B = 2500, 70, 6
+    parts = [synth.zipf_partition(V, K, 1.1, seed=s) for s in range(3)]
+    row_part = np.array([0, 1, 2, 2, 1, 0], dtype=np.int32)
+    cm = _rand_mask(K, B, 0.3, 15)
+    z0 = synth.logits_normal(B, V, 2.0, dtype, (15,))
+    z = z0.copy()
+    out = oracle.decode_step(parts, row_part, cm, z, want_full=True, threads=3)
+    for b in range(B):
+        p = parts[row_part[b]]
+        vm = oracle.expand_mask(p.c, K, cm[b:b + 1])
+        zb = z0[b:b + 1].copy()
+        oracle.mask_logits(zb, V, vm)
+        am, lse, lpa, full = oracle.logsoftmax_argmax(zb, V, vm, want_full=True)
+        assert np.array_equal(out["vocab_mask"][b:b + 1], vm)
+        assert np.array_equal(z[b:b + 1].view(np.uint8), zb.view(np.uint8))
+        assert out["argmax"][b] == am[0] and out["lse"][b] == lse[0] and out["logp_argmax"][b] == lpa[0]
+        assert np.array_equal(out["logp_full"][b], full[0])
+        assert out["rep"][b] == p.r[p.c[am[0]]]
+
+
+def test_bf16_ties_go_to_the_lowest_id():
+    # bf16 logits over thousands of allowed tokens tie at the maximum routinely
+    V = 128256
+    z = synth.logits_normal(1, V, 2.0, "bf16", (16,))
+    ones = synth.pack_bits(np.ones((1, V), dtype=bool))
+    am, _, _, _ = oracle.logsoftmax_argmax(z, V, ones)
+    f = rng.bf16_bits_to_f32(z[0])
+    assert am[0] == np.flatnonzero(f == f.max())[0]
