@@ -1,0 +1,199 @@
+/*
+ * cfgzip.h - C ABI of the CFGzip decode-step library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the inference-time wrapper of CFGzip (paper Section 3.1,
+ * "Inference", and Figure 1): a grammar engine that works over K equivalence-class
+ * representatives hands over an allow-mask over the classes; the mask is expanded to
+ * the full token vocabulary through the token->class vector c, applied to the
+ * language model's logits, the next token is chosen, and the chosen token is mapped
+ * to the representative r_{c_t} of its class for the engine's next step.
+ *
+ * Conventions shared by every call
+ *   - Bit masks are packed 32-bit words, least-significant bit first: bit j of word w
+ *     stands for index 32*w + j; 1 = allowed. KW = ceil(K/32), VW = ceil(V/32).
+ *     Class-mask bits at index >= K are ignored. Vocab-mask bits at index >= V inside
+ *     word VW-1 are written as 0; words at index >= VW of a row are never touched.
+ *   - "dev" pointers are device memory of the context's GPU, "host" pointers are host
+ *     memory. The caller owns every buffer it passes; the library owns only the
+ *     partition tables and a small scratch area inside the context.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     Per-step calls only enqueue work on `stream`: they never synchronise, never
+ *     allocate, and may be captured into a CUDA graph. Calls that share one context
+ *     share its scratch area, so they must be ordered on one stream (use one context
+ *     per concurrent stream).
+ *   - Every function returns CFGZIP_OK (0) or a negative error code. Argument errors
+ *     are detected on the host before anything is launched. Data errors that only the
+ *     GPU can see (a token id outside [0, V), a row with no allowed class, a row whose
+ *     partition id is not loaded) give a defined output and bump a sticky counter that
+ *     cfgzip_poll_status reads; they never trap.
+ */
+#ifndef CFGZIP_H
+#define CFGZIP_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct cfgzip_ctx cfgzip_ctx; /* opaque: device tables, scratch, sticky status */
+typedef int32_t cfgzip_part_id;       /* small dense id inside one context */
+
+enum { CFGZIP_F32 = 0, CFGZIP_BF16 = 1 };                   /* logit element type */
+enum { CFGZIP_AUTO = 0, CFGZIP_DENSE = 1, CFGZIP_SPARSE = 2 }; /* expansion strategy */
+enum {
+    CFGZIP_OK = 0,
+    CFGZIP_E_ARG = -1,       /* null pointer, negative size, stride too small, unknown enum */
+    CFGZIP_E_RANGE = -2,     /* partition id not loaded, V mismatch, size beyond a limit */
+    CFGZIP_E_PARTITION = -3, /* c / r do not describe a partition (see cfgzip_check_partition) */
+    CFGZIP_E_ALIGN = -4,     /* reserved; unaligned logits are handled by a slower path */
+    CFGZIP_E_CUDA = -5,      /* a CUDA runtime call failed (no device, launch error) */
+    CFGZIP_E_NOMEM = -6      /* device allocation failed, or B exceeds the reserved rows */
+};
+
+/* Human-readable name of a status code; never NULL. */
+const char* cfgzip_status_string(int status);
+
+/*
+ * Create a context on CUDA device `device`. Allocates the scratch area (a few MB)
+ * and row-plan buffers for up to 16384 rows per call (see cfgzip_reserve_rows).
+ * Fails with CFGZIP_E_CUDA when no usable device exists: there is no CPU fallback.
+ */
+int cfgzip_create(int device, cfgzip_ctx** out);
+/* Free every partition and the context. Synchronises the device. */
+int cfgzip_destroy(cfgzip_ctx* ctx);
+/* Grow the per-call row capacity (allocates; call outside the per-step path). */
+int cfgzip_reserve_rows(cfgzip_ctx* ctx, int32_t max_rows);
+
+/*
+ * Host-only check that (c, r) is a partition as Section 3.1 ("Pre-Computation")
+ * defines the two vectors: c[i] in [0, K) for every token, every class non-empty,
+ * r[k] in [0, V) and c[r[k]] == k. Returns CFGZIP_OK or CFGZIP_E_PARTITION /
+ * CFGZIP_E_ARG. Touches no GPU.
+ */
+int cfgzip_check_partition(const int32_t* token_to_class /*host [V]*/, int32_t V,
+                           const int32_t* class_to_rep /*host [K]*/, int32_t K);
+
+/*
+ * Host-only inverse of c: off[k]..off[k+1] delimits, inside tok, the tokens of class
+ * k in ascending id (the class->token lists the sparse path scatters from).
+ * `off` has K+1 entries, `tok` has V. Touches no GPU.
+ */
+int cfgzip_build_class_lists(const int32_t* token_to_class /*host [V]*/, int32_t V, int32_t K,
+                             int32_t* off /*host [K+1]*/, int32_t* tok /*host [V]*/);
+
+/*
+ * Load one tokenizer/grammar partition (Section 3.1: vectors c and r, "cached" once per
+ * tokenizer/CFG pair). Validates as cfgzip_check_partition does, builds the class->token
+ * lists, copies everything to the device on `stream` and waits for the copy. Returns the
+ * new id in *out_id. Not a per-step call.
+ */
+int cfgzip_load_partition(cfgzip_ctx* ctx, const int32_t* token_to_class /*host [V]*/, int32_t V,
+                          const int32_t* class_to_rep /*host [K]*/, int32_t K, void* stream,
+                          cfgzip_part_id* out_id);
+/* Release a partition's device tables (synchronises the device first). */
+int cfgzip_free_partition(cfgzip_ctx* ctx, cfgzip_part_id id);
+
+/*
+ * Row -> partition: `row_part` is NULL (every row uses `part0`) or a dev int32 [B] of
+ * partition ids; all partitions used in one call must have the same V (K may differ;
+ * class_stride_words must cover the largest KW). Rows whose id is not a loaded
+ * partition of that V are skipped (outputs untouched) and counted as bad rows.
+ */
+
+/*
+ * Expand class masks to vocab masks: vocab bit (b, i) = class bit (b, c[i])
+ * (Section 3.1, "Inference": the mask entry applied to token i is m_{c_i}; Figure 1b).
+ *   class_mask : dev uint32 [B, class_stride_words], class_stride_words >= KW
+ *   vocab_mask : dev uint32 [B, vocab_stride_words], vocab_stride_words >= VW (written)
+ *   mode       : CFGZIP_DENSE gathers through c; CFGZIP_SPARSE clears the row and
+ *                scatters the members of each allowed class; CFGZIP_AUTO = dense.
+ */
+int cfgzip_expand_mask(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part,
+                       const uint32_t* class_mask, int64_t class_stride_words, uint32_t* vocab_mask,
+                       int64_t vocab_stride_words, int32_t B, int mode, void* stream);
+
+/*
+ * Apply a vocab mask to logits in place: a disallowed logit becomes -inf, an allowed
+ * one keeps its bits (Section 2.2: "the corresponding logit is set to -inf";
+ * Section 3.1 applies it after the gather).
+ *   logits : dev [B, row_stride_elems] of `dtype`, row_stride_elems >= V; elements at
+ *            index >= V of a row are not touched. 16-byte aligned rows take the
+ *            vectorised path, anything else a scalar one.
+ */
+int cfgzip_mask_logits(cfgzip_ctx* ctx, void* logits, int dtype, int64_t row_stride_elems, int32_t B,
+                       int32_t V, const uint32_t* vocab_mask, int64_t vocab_stride_words, void* stream);
+
+/*
+ * The whole step in one pass over the logits (Section 3.1, "Inference"): expand the
+ * class mask, mask the logits in place, take the greedy choice and the log-softmax
+ * normaliser over the allowed tokens, and map the choice to its representative.
+ *   argmax      : dev int32 [B]; largest allowed logit, ties to the lowest token id,
+ *                 compared as values (-0.0 == +0.0); -1 when nothing is allowed
+ *   rep         : nullable dev int32 [B]; r[c[argmax]] or -1
+ *   lse         : nullable dev float [B]; log sum_{allowed} exp(z_i), fp32 accumulate
+ *   logp_argmax : nullable dev float [B]; z_argmax - lse
+ *   logp_full   : nullable dev float [B, V] (row stride V); z_i - lse, -inf where masked
+ *   vocab_mask  : nullable; as in cfgzip_expand_mask
+ * A row with no allowed token, or whose allowed logits are all -inf, gets lse =
+ * logp_argmax = -inf (the latter still returns the lowest allowed id). +inf and NaN
+ * logits are outside the contract for the reductions (the masking itself still copies
+ * them bit for bit); logits below -1.7e38 count as -inf in the normaliser.
+ */
+int cfgzip_masked_logsoftmax_argmax(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part,
+                                    const uint32_t* class_mask, int64_t class_stride_words, void* logits,
+                                    int dtype, int64_t row_stride_elems, int32_t B, uint32_t* vocab_mask,
+                                    int64_t vocab_stride_words, int32_t* argmax, int32_t* rep,
+                                    float* logp_argmax, float* lse, float* logp_full, int mode,
+                                    void* stream);
+
+/*
+ * Token -> representative of its class, reps[b] = r[c[tokens[b]]] (Section 3.1,
+ * "Inference": the engine is fed r_{c_i} instead of t^(i); Figure 1a). A token id
+ * outside [0, V) gives -1 and counts as a bad token.
+ */
+int cfgzip_map_tokens(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part,
+                      const int32_t* tokens /*dev [B]*/, int32_t* reps /*dev [B]*/, int32_t B,
+                      void* stream);
+
+/*
+ * The same step for callers whose data lives on the host: copies the class masks and
+ * logits (pinned or pageable host memory) to staging buffers owned by the context,
+ * runs cfgzip_masked_logsoftmax_argmax, copies the requested results back and waits
+ * for `stream`. Staging buffers grow on first use (that call allocates).
+ *   logits_host     : host [B, V] of `dtype`, dense rows; left unmodified
+ *   masked_logits   : nullable host [B, V]; receives the masked logits
+ *   vocab_mask_host : nullable host uint32 [B, VW]
+ *   argmax/rep/lse/logp_argmax : nullable host [B]
+ */
+int cfgzip_decode_step_host(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part_host,
+                            const uint32_t* class_mask_host, int64_t class_stride_words,
+                            const void* logits_host, int dtype, int32_t B, void* masked_logits,
+                            uint32_t* vocab_mask_host, int32_t* argmax, int32_t* rep, float* logp_argmax,
+                            float* lse, int mode, void* stream);
+
+/*
+ * Synchronise `stream`, then return and clear the sticky counters: rows that had no
+ * allowed token, token ids out of range in cfgzip_map_tokens, rows skipped for a bad
+ * partition id. Any output pointer may be NULL.
+ */
+int cfgzip_poll_status(cfgzip_ctx* ctx, void* stream, int32_t* n_empty_rows, int32_t* n_bad_tokens,
+                       int32_t* n_bad_rows);
+
+/* Kernels this context has launched so far (monotonic; for launch accounting). */
+int cfgzip_launch_count(cfgzip_ctx* ctx, int64_t* out);
+
+/*
+ * Tuning knobs for benchmarking; defaults are chosen from the device at create time.
+ *   "ctas_per_sm"  target resident thread blocks per SM for the fused kernel (1..16)
+ *   "token_warps"  0 = automatic, else warps side by side along the vocabulary (1..8)
+ *   "row_warps"    0 = automatic, else 1, 2 or 4 row batches handled by separate warps
+ *   "pdl"          1 = launch with programmatic dependent launch (default), 0 = off
+ * Unknown names give CFGZIP_E_ARG.
+ */
+int cfgzip_set_tuning(cfgzip_ctx* ctx, const char* name, int32_t value);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CFGZIP_H */

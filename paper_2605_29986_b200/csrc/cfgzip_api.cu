@@ -1,0 +1,745 @@
+// C ABI of the CFGzip decode-step library: argument checks, partition tables, launch
+// planning. The declarations and their contracts are in include/cfgzip.h.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdint>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "cfgzip.h"
+#include "cfgzip_kernels.cuh"
+
+using namespace cfgzip;
+
+namespace {
+
+struct Part {
+    bool live = false;
+    int32_t V = 0, K = 0, KW = 0, VW = 0;
+    void* block = nullptr;  // one device allocation holding every table of the partition
+    PartDev dev{};
+};
+
+constexpr size_t kPartialSlots = size_t(1) << 18;  // 4 MB of (max, sum, pos) slots
+constexpr int kDefaultRows = 16384;
+
+}  // namespace
+
+struct cfgzip_ctx {
+    int device = 0;
+    int sm_count = 0;
+    int smem_optin = 0;
+    std::vector<Part> parts;
+    PartDev* d_parts = nullptr;
+    Partial* d_partials = nullptr;
+    unsigned int* d_tickets = nullptr;  // reserved_rows entries
+    int32_t* d_status = nullptr;        // 3 counters
+    int32_t* d_group_part = nullptr;
+    int32_t* d_group_rows = nullptr;
+    int32_t* d_n_groups = nullptr;
+    int32_t reserved_rows = 0;
+    int32_t max_groups = 0;
+    // staging for cfgzip_decode_step_host
+    void* st_logits = nullptr;
+    size_t st_logits_bytes = 0;
+    uint32_t* st_cm = nullptr;
+    size_t st_cm_bytes = 0;
+    uint32_t* st_vm = nullptr;
+    size_t st_vm_bytes = 0;
+    int32_t* st_small = nullptr;  // row_part, argmax, rep, lse, logp_argmax: 5 arrays of st_rows
+    int32_t st_rows = 0;
+    int64_t launches = 0;
+    // tuning
+    int32_t ctas_per_sm = 4;
+    int32_t token_warps = 0;
+    int32_t row_warps = 0;
+    int32_t pdl = 1;
+};
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+inline int ceil_div(int64_t a, int64_t b) { return int((a + b - 1) / b); }
+
+template <typename... KArgs, typename... Args>
+int launch(cfgzip_ctx* ctx, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+           Args&&... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = ctx->pdl ? 1 : 0;
+    if (cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...) != cudaSuccess) {
+        cudaGetLastError();
+        return CFGZIP_E_CUDA;
+    }
+    ctx->launches += 1;
+    return CFGZIP_OK;
+}
+
+template <typename K>
+int ensure_smem(K kernel, size_t bytes) {
+    if (bytes <= 48 * 1024) return CFGZIP_OK;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(bytes)) != cudaSuccess) {
+        cudaGetLastError();
+        return CFGZIP_E_CUDA;
+    }
+    return CFGZIP_OK;
+}
+
+int check_partition_host(const int32_t* c, int32_t V, const int32_t* r, int32_t K) {
+    if (!c || !r || V <= 0 || K <= 0 || K > V) return CFGZIP_E_ARG;
+    std::vector<uint8_t> seen(size_t(K), 0);
+    for (int32_t i = 0; i < V; ++i) {
+        if (c[i] < 0 || c[i] >= K) return CFGZIP_E_PARTITION;
+        seen[size_t(c[i])] = 1;
+    }
+    for (int32_t k = 0; k < K; ++k) {
+        if (!seen[size_t(k)]) return CFGZIP_E_PARTITION;
+        if (r[k] < 0 || r[k] >= V || c[r[k]] != k) return CFGZIP_E_PARTITION;
+    }
+    return CFGZIP_OK;
+}
+
+void build_class_lists_host(const int32_t* c, int32_t V, int32_t K, int32_t* off, int32_t* tok) {
+    std::fill(off, off + K + 1, 0);
+    for (int32_t i = 0; i < V; ++i) off[c[i] + 1] += 1;
+    for (int32_t k = 0; k < K; ++k) off[k + 1] += off[k];
+    std::vector<int32_t> cursor(off, off + K);
+    for (int32_t i = 0; i < V; ++i) tok[cursor[size_t(c[i])]++] = i;  // ascending ids inside a class
+}
+
+// Everything a per-step call needs to know about the partitions it may touch.
+struct PartSet {
+    int32_t V = 0, VW = 0, maxK = 0, maxKW = 0, n_live_same_v = 0;
+    bool all_c16 = true;
+};
+
+int resolve_parts(cfgzip_ctx* ctx, cfgzip_part_id part0, bool mixed, PartSet* ps) {
+    if (part0 < 0 || size_t(part0) >= ctx->parts.size() || !ctx->parts[size_t(part0)].live) return CFGZIP_E_RANGE;
+    const Part& p0 = ctx->parts[size_t(part0)];
+    ps->V = p0.V;
+    ps->VW = p0.VW;
+    if (!mixed) {
+        ps->maxK = p0.K;
+        ps->maxKW = p0.KW;
+        ps->n_live_same_v = 1;
+        ps->all_c16 = p0.dev.c16 != nullptr;
+        return CFGZIP_OK;
+    }
+    for (const Part& p : ctx->parts) {
+        if (!p.live || p.V != p0.V) continue;
+        ps->maxK = std::max(ps->maxK, p.K);
+        ps->maxKW = std::max(ps->maxKW, p.KW);
+        ps->n_live_same_v += 1;
+        ps->all_c16 = ps->all_c16 && p.dev.c16 != nullptr;
+    }
+    return CFGZIP_OK;
+}
+
+bool aligned16(const void* p, int64_t row_stride_elems, int elem_size) {
+    return (reinterpret_cast<uintptr_t>(p) & 15u) == 0 && ((row_stride_elems * elem_size) & 15) == 0;
+}
+
+size_t dense_smem_bytes(int table_words, int n_warps) {
+    return size_t(table_words) * 4 + kGroupRows * 4 + size_t(n_warps) * kGroupRows * sizeof(Partial);
+}
+
+// Launch shape of the dense kernels.
+struct DensePlan {
+    int S = 1, per_split = 0, WT = 4, threads = 128, table_words = 0;
+    int n_groups_ub = 1;
+    bool use_plan_kernel = false;
+    bool ok = false;  // false: the dense kernels cannot run this call (generic path instead)
+};
+
+DensePlan plan_dense(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, int units, int unit_chunk,
+                     bool fused) {
+    // units: octets (fused) or 32-token words (expand); unit_chunk: units one warp covers per iteration
+    DensePlan d;
+    d.table_words = (ps.maxKW + 1) * 32;
+    d.use_plan_kernel = mixed;
+    d.n_groups_ub = mixed ? ceil_div(B, kGroupRows) + ps.n_live_same_v : ceil_div(B, kGroupRows);
+    if (!ps.all_c16) return d;
+    if (dense_smem_bytes(d.table_words, 8) > size_t(ctx->smem_optin)) return d;
+    if (mixed && (B > ctx->reserved_rows || d.n_groups_ub > ctx->max_groups)) return d;
+    const int target = ctx->sm_count * ctx->ctas_per_sm;
+    const int n_chunks = ceil_div(units, unit_chunk);
+    const int s0 = std::max(1, target / d.n_groups_ub);
+    int cps = ceil_div(n_chunks, s0);  // chunks per block
+    int WR = 1;
+    if (fused) {
+        WR = ctx->row_warps ? ctx->row_warps : (cps <= 2 ? 4 : 1);
+        if (WR != 1 && WR != 2 && WR != 4) WR = 1;
+        d.WT = ctx->token_warps ? ctx->token_warps : (WR == 4 ? std::min(cps, 2) : (WR == 2 ? 2 : 4));
+        d.WT = std::max(1, std::min(d.WT, 8 / WR));
+        d.threads = d.WT * WR * 32;
+    } else {
+        d.WT = 8;
+        d.threads = 256;
+    }
+    for (;;) {
+        d.S = ceil_div(n_chunks, cps);
+        if (d.S == 1 || !fused || size_t(d.n_groups_ub) * kGroupRows * size_t(d.S) <= kPartialSlots) break;
+        cps *= 2;
+    }
+    if (fused && d.S > 1 && d.n_groups_ub > ctx->reserved_rows) return d;  // tickets
+    d.per_split = cps * unit_chunk;
+    d.ok = true;
+    return d;
+}
+
+int check_step_args(cfgzip_ctx* ctx, const uint32_t* class_mask, int64_t cm_stride, int32_t B, int mode) {
+    if (!ctx || B < 0) return CFGZIP_E_ARG;
+    if (mode != CFGZIP_AUTO && mode != CFGZIP_DENSE && mode != CFGZIP_SPARSE) return CFGZIP_E_ARG;
+    if (B > 0 && (!class_mask || cm_stride <= 0)) return CFGZIP_E_ARG;
+    return CFGZIP_OK;
+}
+
+int run_plan_kernel(cfgzip_ctx* ctx, const int32_t* row_part, int32_t B, int32_t V, const DensePlan& d,
+                    cudaStream_t st) {
+    return launch(ctx, k_plan_rows, dim3(1), dim3(1024), 0, st, (const PartDev*)ctx->d_parts, int(ctx->parts.size()),
+                  row_part, int(B), int(V), d.n_groups_ub, ctx->d_group_part, ctx->d_group_rows, ctx->d_n_groups,
+                  ctx->d_status);
+}
+
+void fill_groups(cfgzip_ctx* ctx, StepArgs& a, const DensePlan& d) {
+    if (d.use_plan_kernel) {
+        a.group_part = ctx->d_group_part;
+        a.group_rows = ctx->d_group_rows;
+        a.n_groups = ctx->d_n_groups;
+    } else {
+        a.group_part = nullptr;
+        a.group_rows = nullptr;
+        a.n_groups = nullptr;
+    }
+    a.S = d.S;
+    a.per_split = d.per_split;
+    a.WT = d.WT;
+    a.table_words = d.table_words;
+}
+
+// Sparse launch shape: S blocks per row, each owning per_split vocab-mask words in shared memory.
+bool plan_sparse(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool fused, int* S, int* per_split) {
+    const int target = ctx->sm_count * ctx->ctas_per_sm;
+    int s = std::max(1, target / std::max(B, 1));
+    s = std::min(s, std::max(1, ps.VW / 256));
+    const int max_words = (ctx->smem_optin - 4096) / 4;
+    for (;;) {
+        *per_split = ((ceil_div(ps.VW, s) + 3) / 4) * 4;
+        if (*per_split <= max_words) break;
+        s *= 2;
+    }
+    *S = ceil_div(ps.VW, *per_split);
+    if (fused && *S > 1) {
+        if (B > ctx->reserved_rows) return false;
+        if (size_t(B) * size_t(*S) > kPartialSlots) {
+            // fall back to one block per row if shared memory allows it
+            *per_split = ((ps.VW + 3) / 4) * 4;
+            *S = 1;
+            if (*per_split > max_words) return false;
+        }
+    }
+    return true;
+}
+
+template <int DT>
+int launch_fused(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, int mode, bool aligned, float* logp_full,
+                 cudaStream_t st) {
+    int rc;
+    if (mode == CFGZIP_SPARSE) {
+        int S, per_split;
+        if (plan_sparse(ctx, ps, a.B, true, &S, &per_split)) {
+            a.S = S;
+            a.per_split = per_split;
+            const size_t smem = size_t(per_split) * 4;
+            auto kern = aligned ? k_step_sparse<DT, true, true> : k_step_sparse<DT, true, false>;
+            if ((rc = ensure_smem(kern, smem)) != CFGZIP_OK) return rc;
+            rc = launch(ctx, kern, dim3(unsigned(a.B) * unsigned(S)), dim3(256), smem, st, a);
+        } else {
+            rc = launch(ctx, k_step_generic<DT, true>, dim3(unsigned(a.B)), dim3(256), 0, st, a);
+        }
+    } else {
+        const DensePlan d = plan_dense(ctx, ps, a.B, mixed, 4 * ps.VW, 32, true);
+        if (d.ok) {
+            if (d.use_plan_kernel && (rc = run_plan_kernel(ctx, a.row_part, a.B, a.V, d, st)) != CFGZIP_OK) return rc;
+            fill_groups(ctx, a, d);
+            const size_t smem = dense_smem_bytes(d.table_words, d.threads / 32);
+            auto kern = aligned ? k_step_dense<DT, true> : k_step_dense<DT, false>;
+            if ((rc = ensure_smem(kern, smem)) != CFGZIP_OK) return rc;
+            rc = launch(ctx, kern, dim3(unsigned(d.n_groups_ub) * unsigned(d.S)), dim3(unsigned(d.threads)), smem, st, a);
+        } else {
+            rc = launch(ctx, k_step_generic<DT, true>, dim3(unsigned(a.B)), dim3(256), 0, st, a);
+        }
+    }
+    if (rc != CFGZIP_OK) return rc;
+    if (logp_full) {
+        const int64_t total = int64_t(a.B) * a.V;
+        const unsigned grid = unsigned(std::min<int64_t>((total + 255) / 256, int64_t(ctx->sm_count) * 16));
+        rc = launch(ctx, k_logp_full<DT>, dim3(grid), dim3(256), 0, st, (const void*)a.logits, a.row_stride, int(a.B),
+                    int(a.V), (const float*)a.lse, logp_full);
+    }
+    return rc;
+}
+
+int grow(void** p, size_t* have, size_t need) {
+    if (need <= *have) return CFGZIP_OK;
+    if (*p) cudaFree(*p);
+    *p = nullptr;
+    *have = 0;
+    if (cudaMalloc(p, need) != cudaSuccess) {
+        cudaGetLastError();
+        return CFGZIP_E_NOMEM;
+    }
+    *have = need;
+    return CFGZIP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* cfgzip_status_string(int status) {
+    switch (status) {
+        case CFGZIP_OK: return "CFGZIP_OK";
+        case CFGZIP_E_ARG: return "CFGZIP_E_ARG: invalid argument";
+        case CFGZIP_E_RANGE: return "CFGZIP_E_RANGE: id or size out of range";
+        case CFGZIP_E_PARTITION: return "CFGZIP_E_PARTITION: c / r do not describe a partition";
+        case CFGZIP_E_ALIGN: return "CFGZIP_E_ALIGN: misaligned buffer";
+        case CFGZIP_E_CUDA: return "CFGZIP_E_CUDA: CUDA runtime error";
+        case CFGZIP_E_NOMEM: return "CFGZIP_E_NOMEM: out of memory or capacity";
+        default: return "CFGZIP: unknown status";
+    }
+}
+
+int cfgzip_check_partition(const int32_t* token_to_class, int32_t V, const int32_t* class_to_rep, int32_t K) {
+    return check_partition_host(token_to_class, V, class_to_rep, K);
+}
+
+int cfgzip_build_class_lists(const int32_t* token_to_class, int32_t V, int32_t K, int32_t* off, int32_t* tok) {
+    if (!token_to_class || !off || !tok || V <= 0 || K <= 0 || K > V) return CFGZIP_E_ARG;
+    for (int32_t i = 0; i < V; ++i)
+        if (token_to_class[i] < 0 || token_to_class[i] >= K) return CFGZIP_E_PARTITION;
+    build_class_lists_host(token_to_class, V, K, off, tok);
+    return CFGZIP_OK;
+}
+
+int cfgzip_reserve_rows(cfgzip_ctx* ctx, int32_t max_rows) {
+    if (!ctx || max_rows <= 0) return CFGZIP_E_ARG;
+    if (max_rows <= ctx->reserved_rows) return CFGZIP_OK;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return CFGZIP_E_CUDA;
+    cudaDeviceSynchronize();
+    cudaFree(ctx->d_tickets);
+    cudaFree(ctx->d_group_part);
+    cudaFree(ctx->d_group_rows);
+    ctx->d_tickets = nullptr;
+    ctx->d_group_part = ctx->d_group_rows = nullptr;
+    ctx->reserved_rows = 0;
+    const int32_t groups = ceil_div(max_rows, kGroupRows) + kMaxParts;
+    const size_t tickets = size_t(std::max(max_rows, groups));
+    if (cudaMalloc(&ctx->d_tickets, tickets * sizeof(unsigned int)) != cudaSuccess ||
+        cudaMalloc(&ctx->d_group_part, size_t(groups) * sizeof(int32_t)) != cudaSuccess ||
+        cudaMalloc(&ctx->d_group_rows, size_t(groups) * kGroupRows * sizeof(int32_t)) != cudaSuccess) {
+        cudaGetLastError();
+        return CFGZIP_E_NOMEM;
+    }
+    cudaMemset(ctx->d_tickets, 0, tickets * sizeof(unsigned int));
+    ctx->reserved_rows = max_rows;
+    ctx->max_groups = groups;
+    return CFGZIP_OK;
+}
+
+int cfgzip_create(int device, cfgzip_ctx** out) {
+    if (!out) return CFGZIP_E_ARG;
+    *out = nullptr;
+    int n = 0;
+    if (cudaGetDeviceCount(&n) != cudaSuccess || device < 0 || device >= n) {
+        cudaGetLastError();
+        return CFGZIP_E_CUDA;
+    }
+    DeviceGuard guard(device);
+    if (!guard.ok) return CFGZIP_E_CUDA;
+    cfgzip_ctx* ctx = new (std::nothrow) cfgzip_ctx();
+    if (!ctx) return CFGZIP_E_NOMEM;
+    ctx->device = device;
+    cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
+    cudaDeviceGetAttribute(&ctx->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+    bool ok = cudaMalloc(&ctx->d_parts, kMaxParts * sizeof(PartDev)) == cudaSuccess &&
+              cudaMalloc(&ctx->d_partials, kPartialSlots * sizeof(Partial)) == cudaSuccess &&
+              cudaMalloc(&ctx->d_status, 4 * sizeof(int32_t)) == cudaSuccess &&
+              cudaMalloc(&ctx->d_n_groups, sizeof(int32_t)) == cudaSuccess;
+    if (ok) {
+        cudaMemset(ctx->d_parts, 0, kMaxParts * sizeof(PartDev));
+        cudaMemset(ctx->d_status, 0, 4 * sizeof(int32_t));
+        cudaMemset(ctx->d_n_groups, 0, sizeof(int32_t));
+        ok = cfgzip_reserve_rows(ctx, kDefaultRows) == CFGZIP_OK;
+    }
+    if (!ok || cudaDeviceSynchronize() != cudaSuccess) {
+        cudaGetLastError();
+        cfgzip_destroy(ctx);
+        return CFGZIP_E_NOMEM;
+    }
+    *out = ctx;
+    return CFGZIP_OK;
+}
+
+int cfgzip_destroy(cfgzip_ctx* ctx) {
+    if (!ctx) return CFGZIP_E_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaDeviceSynchronize();
+    for (Part& p : ctx->parts)
+        if (p.block) cudaFree(p.block);
+    cudaFree(ctx->d_parts);
+    cudaFree(ctx->d_partials);
+    cudaFree(ctx->d_tickets);
+    cudaFree(ctx->d_status);
+    cudaFree(ctx->d_group_part);
+    cudaFree(ctx->d_group_rows);
+    cudaFree(ctx->d_n_groups);
+    cudaFree(ctx->st_logits);
+    cudaFree(ctx->st_cm);
+    cudaFree(ctx->st_vm);
+    cudaFree(ctx->st_small);
+    cudaGetLastError();
+    delete ctx;
+    return CFGZIP_OK;
+}
+
+int cfgzip_load_partition(cfgzip_ctx* ctx, const int32_t* c, int32_t V, const int32_t* r, int32_t K, void* stream,
+                          cfgzip_part_id* out_id) {
+    if (!ctx || !out_id) return CFGZIP_E_ARG;
+    int rc = check_partition_host(c, V, r, K);
+    if (rc != CFGZIP_OK) return rc;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return CFGZIP_E_CUDA;
+    size_t slot = 0;
+    while (slot < ctx->parts.size() && ctx->parts[slot].live) ++slot;
+    if (slot >= size_t(kMaxParts)) return CFGZIP_E_RANGE;
+    if (slot == ctx->parts.size()) ctx->parts.emplace_back();
+
+    Part p;
+    p.V = V;
+    p.K = K;
+    p.KW = ceil_div(K, 32);
+    p.VW = ceil_div(V, 32);
+    const bool has16 = K <= 65535;  // the value K itself is the padding id
+    // host image of the device block: c32 | r | off | tok | c16 (16-byte aligned pieces)
+    auto align4 = [](size_t n) { return (n + 3) & ~size_t(3); };
+    const size_t n_c32 = align4(size_t(V)), n_r = align4(size_t(K)), n_off = align4(size_t(K) + 1), n_tok = align4(size_t(V));
+    const size_t n_c16_words = has16 ? size_t(p.VW) * 16 : 0;  // 32*VW uint16 = 16*VW words
+    std::vector<int32_t> img(n_c32 + n_r + n_off + n_tok + n_c16_words, 0);
+    int32_t* h_c32 = img.data();
+    int32_t* h_r = h_c32 + n_c32;
+    int32_t* h_off = h_r + n_r;
+    int32_t* h_tok = h_off + n_off;
+    uint16_t* h_c16 = reinterpret_cast<uint16_t*>(h_tok + n_tok);
+    std::memcpy(h_c32, c, size_t(V) * 4);
+    std::memcpy(h_r, r, size_t(K) * 4);
+    build_class_lists_host(c, V, K, h_off, h_tok);
+    if (has16) {
+        for (int32_t i = 0; i < V; ++i) h_c16[i] = uint16_t(c[i]);
+        for (int32_t i = V; i < 32 * p.VW; ++i) h_c16[i] = uint16_t(K);
+    }
+    if (cudaMalloc(&p.block, img.size() * 4) != cudaSuccess) {
+        cudaGetLastError();
+        return CFGZIP_E_NOMEM;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t* d = static_cast<int32_t*>(p.block);
+    p.dev.c32 = d;
+    p.dev.r = d + n_c32;
+    p.dev.off = d + n_c32 + n_r;
+    p.dev.tok = d + n_c32 + n_r + n_off;
+    p.dev.c16 = has16 ? reinterpret_cast<const uint16_t*>(d + n_c32 + n_r + n_off + n_tok) : nullptr;
+    p.dev.K = K;
+    p.dev.KW = p.KW;
+    p.dev.V = V;
+    p.dev.live = 1;
+    p.live = true;
+    bool ok = cudaMemcpyAsync(p.block, img.data(), img.size() * 4, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+              cudaMemcpyAsync(ctx->d_parts + slot, &p.dev, sizeof(PartDev), cudaMemcpyHostToDevice, st) == cudaSuccess &&
+              cudaStreamSynchronize(st) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        cudaFree(p.block);
+        return CFGZIP_E_CUDA;
+    }
+    ctx->parts[slot] = p;
+    *out_id = cfgzip_part_id(slot);
+    return CFGZIP_OK;
+}
+
+int cfgzip_free_partition(cfgzip_ctx* ctx, cfgzip_part_id id) {
+    if (!ctx) return CFGZIP_E_ARG;
+    if (id < 0 || size_t(id) >= ctx->parts.size() || !ctx->parts[size_t(id)].live) return CFGZIP_E_RANGE;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return CFGZIP_E_CUDA;
+    cudaDeviceSynchronize();
+    Part& p = ctx->parts[size_t(id)];
+    cudaFree(p.block);
+    p = Part();
+    cudaMemset(ctx->d_parts + id, 0, sizeof(PartDev));
+    cudaDeviceSynchronize();
+    return cudaGetLastError() == cudaSuccess ? CFGZIP_OK : CFGZIP_E_CUDA;
+}
+
+int cfgzip_expand_mask(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part, const uint32_t* class_mask,
+                       int64_t class_stride_words, uint32_t* vocab_mask, int64_t vocab_stride_words, int32_t B,
+                       int mode, void* stream) {
+    int rc = check_step_args(ctx, class_mask, class_stride_words, B, mode);
+    if (rc != CFGZIP_OK) return rc;
+    PartSet ps;
+    const bool mixed = row_part != nullptr;
+    if ((rc = resolve_parts(ctx, part0, mixed, &ps)) != CFGZIP_OK) return rc;
+    if (B == 0) return CFGZIP_OK;
+    if (!vocab_mask || vocab_stride_words < ps.VW || class_stride_words < ps.maxKW) return CFGZIP_E_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return CFGZIP_E_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    StepArgs a{};
+    a.parts = ctx->d_parts;
+    a.part0 = part0;
+    a.n_parts = int32_t(ctx->parts.size());
+    a.row_part = row_part;
+    a.class_mask = class_mask;
+    a.cm_stride = class_stride_words;
+    a.vocab_mask = vocab_mask;
+    a.vm_stride = vocab_stride_words;
+    a.B = B;
+    a.V = ps.V;
+    a.VW = ps.VW;
+    a.partials = ctx->d_partials;
+    a.tickets = ctx->d_tickets;
+    a.status = ctx->d_status;
+    if (mode == CFGZIP_SPARSE) {
+        int S, per_split;
+        if (plan_sparse(ctx, ps, B, false, &S, &per_split)) {
+            a.S = S;
+            a.per_split = per_split;
+            const size_t smem = size_t(per_split) * 4;
+            auto kern = k_step_sparse<kF32, false, false>;
+            if ((rc = ensure_smem(kern, smem)) != CFGZIP_OK) return rc;
+            return launch(ctx, kern, dim3(unsigned(B) * unsigned(S)), dim3(256), smem, st, a);
+        }
+        return launch(ctx, k_step_generic<kF32, false>, dim3(unsigned(B)), dim3(256), 0, st, a);
+    }
+    const DensePlan d = plan_dense(ctx, ps, B, mixed, ps.VW, 8, false);
+    if (!d.ok) return launch(ctx, k_step_generic<kF32, false>, dim3(unsigned(B)), dim3(256), 0, st, a);
+    if (d.use_plan_kernel && (rc = run_plan_kernel(ctx, row_part, B, ps.V, d, st)) != CFGZIP_OK) return rc;
+    fill_groups(ctx, a, d);
+    const size_t smem = dense_smem_bytes(d.table_words, 0);
+    if ((rc = ensure_smem(k_expand_dense, smem)) != CFGZIP_OK) return rc;
+    return launch(ctx, k_expand_dense, dim3(unsigned(d.n_groups_ub) * unsigned(d.S)), dim3(256), smem, st, a);
+}
+
+int cfgzip_mask_logits(cfgzip_ctx* ctx, void* logits, int dtype, int64_t row_stride_elems, int32_t B, int32_t V,
+                       const uint32_t* vocab_mask, int64_t vocab_stride_words, void* stream) {
+    if (!ctx || B < 0 || V <= 0 || (dtype != CFGZIP_F32 && dtype != CFGZIP_BF16)) return CFGZIP_E_ARG;
+    if (B == 0) return CFGZIP_OK;
+    const int VW = ceil_div(V, 32);
+    if (!logits || !vocab_mask || row_stride_elems < V || vocab_stride_words < VW) return CFGZIP_E_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return CFGZIP_E_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int es = dtype == CFGZIP_BF16 ? 2 : 4;
+    const bool al = aligned16(logits, row_stride_elems, es);
+    const int n_octets = ceil_div(V, 8);
+    const int64_t items = int64_t(B) * ceil_div(n_octets, 256 * 4);
+    const unsigned grid = unsigned(std::min<int64_t>(items, int64_t(ctx->sm_count) * 8));
+    if (dtype == CFGZIP_BF16) {
+        auto kern = al ? k_mask_logits<kBF16, true> : k_mask_logits<kBF16, false>;
+        return launch(ctx, kern, dim3(grid), dim3(256), 0, st, logits, row_stride_elems, int(B), int(V), VW, vocab_mask,
+                      vocab_stride_words);
+    }
+    auto kern = al ? k_mask_logits<kF32, true> : k_mask_logits<kF32, false>;
+    return launch(ctx, kern, dim3(grid), dim3(256), 0, st, logits, row_stride_elems, int(B), int(V), VW, vocab_mask,
+                  vocab_stride_words);
+}
+
+int cfgzip_masked_logsoftmax_argmax(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part,
+                                    const uint32_t* class_mask, int64_t class_stride_words, void* logits, int dtype,
+                                    int64_t row_stride_elems, int32_t B, uint32_t* vocab_mask,
+                                    int64_t vocab_stride_words, int32_t* argmax, int32_t* rep, float* logp_argmax,
+                                    float* lse, float* logp_full, int mode, void* stream) {
+    int rc = check_step_args(ctx, class_mask, class_stride_words, B, mode);
+    if (rc != CFGZIP_OK) return rc;
+    if (dtype != CFGZIP_F32 && dtype != CFGZIP_BF16) return CFGZIP_E_ARG;
+    PartSet ps;
+    const bool mixed = row_part != nullptr;
+    if ((rc = resolve_parts(ctx, part0, mixed, &ps)) != CFGZIP_OK) return rc;
+    if (B == 0) return CFGZIP_OK;
+    if (!logits || !argmax || row_stride_elems < ps.V || class_stride_words < ps.maxKW) return CFGZIP_E_ARG;
+    if (vocab_mask && vocab_stride_words < ps.VW) return CFGZIP_E_ARG;
+    if (logp_full && !lse) return CFGZIP_E_ARG;  // the full log-probabilities are formed from lse
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return CFGZIP_E_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    StepArgs a{};
+    a.parts = ctx->d_parts;
+    a.part0 = part0;
+    a.n_parts = int32_t(ctx->parts.size());
+    a.row_part = row_part;
+    a.class_mask = class_mask;
+    a.cm_stride = class_stride_words;
+    a.logits = logits;
+    a.row_stride = row_stride_elems;
+    a.vocab_mask = vocab_mask;
+    a.vm_stride = vocab_stride_words;
+    a.argmax = argmax;
+    a.rep = rep;
+    a.logp_argmax = logp_argmax;
+    a.lse = lse;
+    a.B = B;
+    a.V = ps.V;
+    a.VW = ps.VW;
+    a.partials = ctx->d_partials;
+    a.tickets = ctx->d_tickets;
+    a.status = ctx->d_status;
+    const int es = dtype == CFGZIP_BF16 ? 2 : 4;
+    const bool al = aligned16(logits, row_stride_elems, es);
+    if (dtype == CFGZIP_BF16) return launch_fused<kBF16>(ctx, a, ps, mixed, mode, al, logp_full, st);
+    return launch_fused<kF32>(ctx, a, ps, mixed, mode, al, logp_full, st);
+}
+
+int cfgzip_map_tokens(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part, const int32_t* tokens,
+                      int32_t* reps, int32_t B, void* stream) {
+    if (!ctx || B < 0) return CFGZIP_E_ARG;
+    PartSet ps;
+    int rc = resolve_parts(ctx, part0, row_part != nullptr, &ps);
+    if (rc != CFGZIP_OK) return rc;
+    if (B == 0) return CFGZIP_OK;
+    if (!tokens || !reps) return CFGZIP_E_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return CFGZIP_E_CUDA;
+    return launch(ctx, k_map_tokens, dim3(unsigned(ceil_div(B, 256))), dim3(256), 0, static_cast<cudaStream_t>(stream),
+                  (const PartDev*)ctx->d_parts, int(ctx->parts.size()), int(part0), row_part, tokens, reps, int(B),
+                  int(ps.V), ctx->d_status);
+}
+
+int cfgzip_decode_step_host(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part_host,
+                            const uint32_t* class_mask_host, int64_t class_stride_words, const void* logits_host,
+                            int dtype, int32_t B, void* masked_logits, uint32_t* vocab_mask_host, int32_t* argmax,
+                            int32_t* rep, float* logp_argmax, float* lse, int mode, void* stream) {
+    int rc = check_step_args(ctx, class_mask_host, class_stride_words, B, mode);
+    if (rc != CFGZIP_OK) return rc;
+    if (dtype != CFGZIP_F32 && dtype != CFGZIP_BF16) return CFGZIP_E_ARG;
+    PartSet ps;
+    if ((rc = resolve_parts(ctx, part0, row_part_host != nullptr, &ps)) != CFGZIP_OK) return rc;
+    if (B == 0) return CFGZIP_OK;
+    if (!logits_host || class_stride_words < ps.maxKW) return CFGZIP_E_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return CFGZIP_E_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t es = dtype == CFGZIP_BF16 ? 2 : 4;
+    const size_t logit_bytes = size_t(B) * size_t(ps.V) * es;
+    const size_t cm_bytes = size_t(B) * size_t(class_stride_words) * 4;
+    const size_t vm_bytes = size_t(B) * size_t(ps.VW) * 4;
+    if (logit_bytes > ctx->st_logits_bytes || cm_bytes > ctx->st_cm_bytes || vm_bytes > ctx->st_vm_bytes ||
+        B > ctx->st_rows) {
+        cudaStreamSynchronize(st);
+        if ((rc = grow(&ctx->st_logits, &ctx->st_logits_bytes, logit_bytes)) != CFGZIP_OK) return rc;
+        if ((rc = grow(reinterpret_cast<void**>(&ctx->st_cm), &ctx->st_cm_bytes, cm_bytes)) != CFGZIP_OK) return rc;
+        if ((rc = grow(reinterpret_cast<void**>(&ctx->st_vm), &ctx->st_vm_bytes, vm_bytes)) != CFGZIP_OK) return rc;
+        if (B > ctx->st_rows) {
+            size_t have = size_t(ctx->st_rows) * 20;
+            if ((rc = grow(reinterpret_cast<void**>(&ctx->st_small), &have, size_t(B) * 20)) != CFGZIP_OK) {
+                ctx->st_rows = 0;
+                return rc;
+            }
+            ctx->st_rows = B;
+        }
+    }
+    int32_t* d_rp = ctx->st_small;
+    int32_t* d_am = d_rp + ctx->st_rows;
+    int32_t* d_rep = d_am + ctx->st_rows;
+    float* d_lse = reinterpret_cast<float*>(d_rep + ctx->st_rows);
+    float* d_lpa = d_lse + ctx->st_rows;
+    bool ok = cudaMemcpyAsync(ctx->st_cm, class_mask_host, cm_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess &&
+              cudaMemcpyAsync(ctx->st_logits, logits_host, logit_bytes, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (ok && row_part_host)
+        ok = cudaMemcpyAsync(d_rp, row_part_host, size_t(B) * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        return CFGZIP_E_CUDA;
+    }
+    rc = cfgzip_masked_logsoftmax_argmax(ctx, part0, row_part_host ? d_rp : nullptr, ctx->st_cm, class_stride_words,
+                                         ctx->st_logits, dtype, ps.V, B, vocab_mask_host ? ctx->st_vm : nullptr, ps.VW,
+                                         d_am, d_rep, d_lpa, d_lse, nullptr, mode, stream);
+    if (rc != CFGZIP_OK) return rc;
+    auto back = [&](void* dst, const void* src, size_t n) {
+        if (dst && ok) ok = cudaMemcpyAsync(dst, src, n, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    };
+    back(masked_logits, ctx->st_logits, logit_bytes);
+    back(vocab_mask_host, ctx->st_vm, vm_bytes);
+    back(argmax, d_am, size_t(B) * 4);
+    back(rep, d_rep, size_t(B) * 4);
+    back(lse, d_lse, size_t(B) * 4);
+    back(logp_argmax, d_lpa, size_t(B) * 4);
+    if (!ok || cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return CFGZIP_E_CUDA;
+    }
+    return CFGZIP_OK;
+}
+
+int cfgzip_poll_status(cfgzip_ctx* ctx, void* stream, int32_t* n_empty_rows, int32_t* n_bad_tokens,
+                       int32_t* n_bad_rows) {
+    if (!ctx) return CFGZIP_E_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return CFGZIP_E_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t h[3] = {0, 0, 0};
+    if (cudaMemcpyAsync(h, ctx->d_status, sizeof h, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaMemsetAsync(ctx->d_status, 0, sizeof h, st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return CFGZIP_E_CUDA;
+    }
+    if (n_empty_rows) *n_empty_rows = h[0];
+    if (n_bad_tokens) *n_bad_tokens = h[1];
+    if (n_bad_rows) *n_bad_rows = h[2];
+    return CFGZIP_OK;
+}
+
+int cfgzip_launch_count(cfgzip_ctx* ctx, int64_t* out) {
+    if (!ctx || !out) return CFGZIP_E_ARG;
+    *out = ctx->launches;
+    return CFGZIP_OK;
+}
+
+int cfgzip_set_tuning(cfgzip_ctx* ctx, const char* name, int32_t value) {
+    if (!ctx || !name) return CFGZIP_E_ARG;
+    if (!std::strcmp(name, "ctas_per_sm")) {
+        if (value < 1 || value > 16) return CFGZIP_E_ARG;
+        ctx->ctas_per_sm = value;
+    } else if (!std::strcmp(name, "token_warps")) {
+        if (value < 0 || value > 8) return CFGZIP_E_ARG;
+        ctx->token_warps = value;
+    } else if (!std::strcmp(name, "row_warps")) {
+        if (value != 0 && value != 1 && value != 2 && value != 4) return CFGZIP_E_ARG;
+        ctx->row_warps = value;
+    } else if (!std::strcmp(name, "pdl")) {
+        ctx->pdl = value ? 1 : 0;
+    } else {
+        return CFGZIP_E_ARG;
+    }
+    return CFGZIP_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,224 @@
+// Device-side building blocks shared by the kernels: partition descriptors, the
+// (max, sum-exp, position) partial state and its merge, bit-matrix transposes,
+// and 16-byte "octet" (8 tokens) loads and stores.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace cfgzip {
+
+constexpr int kGroupRows = 32;        // rows that share one bit-sliced class table
+constexpr int kBatchRows = 8;         // rows a warp streams together
+constexpr int kNoPos = 0x7FFFFFFF;    // "no allowed token seen"
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kRefFloor = -1.7e38f; // lowest reference used for exp(z - ref)
+
+enum : int { kF32 = 0, kBF16 = 1 };
+
+// One loaded partition, as the kernels see it (all pointers are device memory).
+struct PartDev {
+    const uint16_t* c16;   // token -> class, padded to 32*VW entries with the value K; null when K > 65535
+    const int32_t* c32;    // token -> class, V entries
+    const int32_t* r;      // class -> representative token, K entries
+    const int32_t* off;    // class -> start in tok, K+1 entries
+    const int32_t* tok;    // tokens grouped by class, ascending inside a class
+    int32_t K;
+    int32_t KW;
+    int32_t V;
+    int32_t live;          // 0 when the slot is free
+};
+
+// Per-row reduction state. m: largest allowed logit seen (-inf if none or all -inf);
+// s: sum of exp(z - max(m, kRefFloor)) over allowed logits; pos: position (octet or
+// token index, ascending with the token id) of the first occurrence of m.
+struct Partial {
+    float m;
+    float s;
+    int pos;
+    int pad;
+};
+
+__device__ __forceinline__ Partial partial_empty() { return Partial{-INFINITY, 0.f, kNoPos, 0}; }
+
+__device__ __forceinline__ float ex2f(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Total order used at every level: larger value wins; equal values: lower position.
+// The sums are brought to the larger reference before they are added.
+__device__ __forceinline__ void partial_merge(float& m, float& s, int& pos, float m2, float s2, int pos2) {
+    const float r1 = fmaxf(m, kRefFloor), r2 = fmaxf(m2, kRefFloor);
+    const float d = r1 - r2;
+    const float e = ex2f(-fabsf(d) * kLog2e);
+    s = d >= 0.f ? fmaf(s2, e, s) : fmaf(s, e, s2);
+    const bool take2 = (m2 > m) || (m2 == m && pos2 < pos);
+    pos = take2 ? pos2 : pos;
+    m = fmaxf(m, m2);
+}
+
+// Butterfly all-reduce of one row's state over the 32 lanes of a warp.
+__device__ __forceinline__ void partial_warp_allreduce(float& m, float& s, int& pos) {
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+        const float m2 = __shfl_xor_sync(0xFFFFFFFFu, m, d);
+        const float s2 = __shfl_xor_sync(0xFFFFFFFFu, s, d);
+        const int p2 = __shfl_xor_sync(0xFFFFFFFFu, pos, d);
+        partial_merge(m, s, pos, m2, s2, p2);
+    }
+}
+
+// 32x32 bit-matrix transpose across a warp: on entry lane r holds row r (bit j = column
+// j); on return lane j holds column j (bit r = row r). Five block-swap stages.
+__device__ __forceinline__ uint32_t warp_transpose32(uint32_t x, int lane) {
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+        // low mask of each 2d-wide bit block: d=16 -> 0x0000FFFF, 8 -> 0x00FF00FF, ...
+        const uint32_t lo = 0xFFFFFFFFu / ((1u << d) + 1u);
+        const uint32_t y = __shfl_xor_sync(0xFFFFFFFFu, x, d);
+        x = (lane & d) ? ((y >> d) & lo) | (x & ~lo) : (x & lo) | ((y & lo) << d);
+    }
+    return x;
+}
+
+// 8x8 bit-matrix transpose held in two registers. On entry byte j of (lo, hi) -- lo holds
+// j = 0..3, hi holds j = 4..7 -- is row j, bit i of that byte is column i. On return byte i
+// is column i with bit j = old row j.
+__host__ __device__ __forceinline__ void transpose8x8(uint32_t& lo, uint32_t& hi) {
+    uint32_t t;
+    // swap the off-diagonal 4x4 blocks (rows 0-3 / cols 4-7 with rows 4-7 / cols 0-3)
+    t = ((lo >> 4) ^ hi) & 0x0F0F0F0Fu;
+    hi ^= t;
+    lo ^= t << 4;
+    // 2x2 blocks inside each 4x4: rows j and j+2 are 16 bits apart inside one register
+    t = (lo ^ (lo >> 14)) & 0x0000CCCCu;
+    lo ^= t ^ (t << 14);
+    t = (hi ^ (hi >> 14)) & 0x0000CCCCu;
+    hi ^= t ^ (t << 14);
+    // single bits inside each 2x2: rows j and j+1 are 8 bits apart
+    t = (lo ^ (lo >> 7)) & 0x00AA00AAu;
+    lo ^= t ^ (t << 7);
+    t = (hi ^ (hi >> 7)) & 0x00AA00AAu;
+    hi ^= t ^ (t << 7);
+}
+
+__device__ __forceinline__ uint32_t neg_inf_bits_f32() { return 0xFF800000u; }
+__device__ __forceinline__ uint32_t neg_inf_bits_bf16x2() { return 0xFF80FF80u; }
+
+// Spread the 4 bits of a nibble to the top bit of the 4 bytes of a word (bit j -> bit 8j+7).
+__device__ __forceinline__ uint32_t nibble_to_byte_msbs(uint32_t nib) { return nib * 0x10204080u; }
+
+// PTX byte permute in its default mode: selector nibble n picks byte (n & 7) of {b, a};
+// with bit 3 of the nibble set, the top bit of that byte is replicated over the result byte.
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+
+// Streaming 16-byte accesses for the logits (read once, written once).
+__device__ __forceinline__ uint4 ld_stream16(const void* p) { return __ldcs(reinterpret_cast<const uint4*>(p)); }
+__device__ __forceinline__ void st_stream16(void* p, uint4 v) { __stcs(reinterpret_cast<uint4*>(p), v); }
+
+// Logit element access by dtype (scalar, for ragged tails and unaligned buffers).
+template <int DT>
+__device__ __forceinline__ float load_elem(const void* base, int64_t idx) {
+    if (DT == kBF16) return __uint_as_float(uint32_t(reinterpret_cast<const uint16_t*>(base)[idx]) << 16);
+    return reinterpret_cast<const float*>(base)[idx];
+}
+template <int DT>
+__device__ __forceinline__ void store_neg_inf(void* base, int64_t idx) {
+    if (DT == kBF16)
+        reinterpret_cast<uint16_t*>(base)[idx] = 0xFF80u;
+    else
+        reinterpret_cast<uint32_t*>(base)[idx] = 0xFF800000u;
+}
+
+// Eight consecutive logits of one row ("octet"), masked by the 8 allow bits in `byte`:
+// the masked values land in f[0..7] and the masked bit patterns in the registers that are
+// stored back. bf16: one 16-byte vector; f32: two.
+template <int DT>
+struct Octet;
+
+template <>
+struct Octet<kBF16> {
+    uint4 v;
+    __device__ __forceinline__ void load(const void* row_base, int o) {
+        v = ld_stream16(reinterpret_cast<const uint16_t*>(row_base) + 8 * int64_t(o));
+    }
+    __device__ __forceinline__ void store(void* row_base, int o) const {
+        st_stream16(reinterpret_cast<uint16_t*>(row_base) + 8 * int64_t(o), v);
+    }
+    __device__ __forceinline__ void fill_neg_inf() { v = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u); }
+    __device__ __forceinline__ void mask(uint32_t byte, float (&f)[8]) {
+        const uint32_t xl = nibble_to_byte_msbs(byte & 0xFu), xh = nibble_to_byte_msbs(byte >> 4);
+        // replicate the top bit of byte 2p / 2p+1 over the low / high half-word
+        const uint32_t m0 = prmt(xl, 0u, 0x9988), m1 = prmt(xl, 0u, 0xBBAA);
+        const uint32_t m2 = prmt(xh, 0u, 0x9988), m3 = prmt(xh, 0u, 0xBBAA);
+        const uint32_t ni = 0xFF80FF80u;
+        v.x = (v.x & m0) | (ni & ~m0);
+        v.y = (v.y & m1) | (ni & ~m1);
+        v.z = (v.z & m2) | (ni & ~m2);
+        v.w = (v.w & m3) | (ni & ~m3);
+        f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xFFFF0000u);
+        f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xFFFF0000u);
+        f[4] = __uint_as_float(v.z << 16); f[5] = __uint_as_float(v.z & 0xFFFF0000u);
+        f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xFFFF0000u);
+    }
+};
+
+template <>
+struct Octet<kF32> {
+    uint4 a, b;
+    __device__ __forceinline__ void load(const void* row_base, int o) {
+        const float* p = reinterpret_cast<const float*>(row_base) + 8 * int64_t(o);
+        a = ld_stream16(p);
+        b = ld_stream16(p + 4);
+    }
+    __device__ __forceinline__ void store(void* row_base, int o) const {
+        float* p = reinterpret_cast<float*>(row_base) + 8 * int64_t(o);
+        st_stream16(p, a);
+        st_stream16(p + 4, b);
+    }
+    __device__ __forceinline__ void fill_neg_inf() {
+        a = make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u);
+        b = a;
+    }
+    __device__ __forceinline__ void mask(uint32_t byte, float (&f)[8]) {
+        const uint32_t xl = nibble_to_byte_msbs(byte & 0xFu), xh = nibble_to_byte_msbs(byte >> 4);
+        const uint32_t ni = 0xFF800000u;
+        uint32_t m;
+        m = prmt(xl, 0u, 0x8888); a.x = (a.x & m) | (ni & ~m);
+        m = prmt(xl, 0u, 0x9999); a.y = (a.y & m) | (ni & ~m);
+        m = prmt(xl, 0u, 0xAAAA); a.z = (a.z & m) | (ni & ~m);
+        m = prmt(xl, 0u, 0xBBBB); a.w = (a.w & m) | (ni & ~m);
+        m = prmt(xh, 0u, 0x8888); b.x = (b.x & m) | (ni & ~m);
+        m = prmt(xh, 0u, 0x9999); b.y = (b.y & m) | (ni & ~m);
+        m = prmt(xh, 0u, 0xAAAA); b.z = (b.z & m) | (ni & ~m);
+        m = prmt(xh, 0u, 0xBBBB); b.w = (b.w & m) | (ni & ~m);
+        f[0] = __uint_as_float(a.x); f[1] = __uint_as_float(a.y);
+        f[2] = __uint_as_float(a.z); f[3] = __uint_as_float(a.w);
+        f[4] = __uint_as_float(b.x); f[5] = __uint_as_float(b.y);
+        f[6] = __uint_as_float(b.z); f[7] = __uint_as_float(b.w);
+    }
+};
+
+// Fold one masked octet into a running per-row state.
+__device__ __forceinline__ void partial_add_octet(float& m, float& s, int& pos, const float (&f)[8], uint32_t byte,
+                                                  int position) {
+    const float vmax = fmaxf(fmaxf(fmaxf(f[0], f[1]), fmaxf(f[2], f[3])), fmaxf(fmaxf(f[4], f[5]), fmaxf(f[6], f[7])));
+    const bool upd = (vmax > m) || (byte != 0u && pos == kNoPos);
+    pos = upd ? position : pos;
+    const float ref_old = fmaxf(m, kRefFloor);
+    m = fmaxf(m, vmax);
+    const float ref = fmaxf(m, kRefFloor);
+    float acc = 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc += ex2f((f[j] - ref) * kLog2e);
+    s = fmaf(s, ex2f((ref_old - ref) * kLog2e), acc);
+}
+
+}  // namespace cfgzip

@@ -1,0 +1,650 @@
+// Kernels of the decode-step path. All of them are bandwidth- or latency-bound
+// scans: no tensor cores. Notation: V tokens, K classes, B rows, VW = ceil(V/32),
+// KW = ceil(K/32); an "octet" is 8 consecutive tokens of one row (16 bytes of bf16,
+// 32 bytes of f32, one byte of vocab mask).
+#pragma once
+
+#include "cfgzip_device.cuh"
+
+namespace cfgzip {
+
+// Arguments of one step (expand / fused), shared by the dense, sparse and generic kernels.
+struct StepArgs {
+    const PartDev* parts;
+    int32_t part0;
+    int32_t n_parts;
+    const int32_t* row_part;    // dev [B] or null
+    // row groups (dense kernels): null = implicit groups of 32 consecutive rows using part0
+    const int32_t* group_part;  // dev [n_groups]
+    const int32_t* group_rows;  // dev [n_groups * 32], -1 = empty slot, valid slots first
+    const int32_t* n_groups;    // dev scalar
+    const uint32_t* class_mask;
+    int64_t cm_stride;
+    void* logits;
+    int64_t row_stride;         // elements
+    uint32_t* vocab_mask;       // nullable
+    int64_t vm_stride;
+    int32_t* argmax;
+    int32_t* rep;
+    float* logp_argmax;
+    float* lse;
+    int32_t B, V, VW;
+    int32_t S;                  // CTAs that share one group (dense) or one row (sparse)
+    int32_t per_split;          // octets (dense) or vocab-mask words (sparse) per CTA
+    int32_t WT;                 // dense: warps side by side along the vocabulary
+    int32_t table_words;        // dense: shared-memory words of the bit-sliced class table
+    Partial* partials;
+    unsigned int* tickets;
+    int32_t* status;            // [0] empty rows, [1] bad tokens, [2] bad rows
+};
+
+__device__ __forceinline__ void pdl_prologue() {
+    // Let the next kernel of the stream start its launch early, then wait until everything
+    // launched before this kernel has completed. Both are no-ops without the launch attribute.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+template <int DT>
+__device__ __forceinline__ float ldcg_elem(const void* base, int64_t idx) {
+    if (DT == kBF16) return __uint_as_float(uint32_t(__ldcg(reinterpret_cast<const unsigned short*>(base) + idx)) << 16);
+    return __ldcg(reinterpret_cast<const float*>(base) + idx);
+}
+
+// Turn a merged row state into the row's outputs. `pos` is an octet index (pos_is_token
+// false: the first allowed token of that octet whose value equals m is the choice) or the
+// token index itself.
+template <int DT>
+__device__ void finalize_row(const StepArgs& a, const PartDev& P, int row, float m, float s, int pos,
+                             bool pos_is_token) {
+    if (row < 0) return;
+    int tok = -1, repv = -1;
+    float lsev = -INFINITY, lpa = -INFINITY;
+    if (pos != kNoPos) {
+        if (pos_is_token) {
+            tok = pos;
+        } else {
+            const uint32_t* cm = a.class_mask + int64_t(row) * a.cm_stride;
+            const void* base = reinterpret_cast<const char*>(a.logits) + int64_t(row) * a.row_stride * (DT == kBF16 ? 2 : 4);
+            for (int j = 0; j < 8 && tok < 0; ++j) {
+                const int t = 8 * pos + j;
+                if (t >= a.V) break;
+                const int k = P.c32[t];
+                if (((cm[k >> 5] >> (k & 31)) & 1u) && ldcg_elem<DT>(base, t) == m) tok = t;
+            }
+        }
+        if (tok >= 0) repv = P.r[P.c32[tok]];
+        if (m > kRefFloor && s > 0.f) {
+            const float l = logf(s);
+            lsev = m + l;
+            lpa = -l;
+        }
+    } else {
+        atomicAdd(a.status + 0, 1);
+    }
+    a.argmax[row] = tok;
+    if (a.rep) a.rep[row] = repv;
+    if (a.lse) a.lse[row] = lsev;
+    if (a.logp_argmax) a.logp_argmax[row] = lpa;
+}
+
+// Eight tokens handled one element at a time: ragged tail of a row, or unaligned logits.
+template <int DT>
+__device__ __noinline__ void octet_scalar(void* row_base, int o, int V, uint32_t byte, float (&f)[8]) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int t = 8 * o + j;
+        f[j] = -INFINITY;
+        if (t < V) {
+            if ((byte >> j) & 1u)
+                f[j] = load_elem<DT>(row_base, t);
+            else
+                store_neg_inf<DT>(row_base, t);
+        }
+    }
+}
+
+// Fill the 32 row slots of group g and return the partition the group uses.
+__device__ __forceinline__ int group_rows_setup(const StepArgs& a, int g, int* s_row, int tid) {
+    if (tid < kGroupRows) {
+        int row;
+        if (a.group_rows) {
+            row = a.group_rows[g * kGroupRows + tid];
+        } else {
+            row = g * kGroupRows + tid;
+            if (row >= a.B) row = -1;
+        }
+        s_row[tid] = row;
+    }
+    return a.group_part ? a.group_part[g] : a.part0;
+}
+
+// Bit-sliced class table of one row group: T[k] bit r = "row slot r allows class k".
+// Entries K .. 32*(KW+1)-1 are zero, so the padding class id K looks up "nobody".
+__device__ __forceinline__ void build_class_table(const StepArgs& a, const PartDev& P, const int* s_row, uint32_t* T,
+                                                  int warp, int lane, int n_warps) {
+    const int row = s_row[lane];
+    const uint32_t* cm = a.class_mask + int64_t(row < 0 ? 0 : row) * a.cm_stride;
+    for (int kw = warp; kw <= P.KW; kw += n_warps) {
+        uint32_t x = 0;
+        if (kw < P.KW && row >= 0) {
+            x = __ldg(cm + kw);
+            if (kw == P.KW - 1 && (P.K & 31)) x &= (1u << (P.K & 31)) - 1u;
+        }
+        T[kw * 32 + lane] = warp_transpose32(x, lane);
+    }
+}
+
+// Allow bits of rows 8*rb .. 8*rb+7 for the 8 tokens of octet o: byte i of (lo, hi)
+// belongs to row 8*rb + i, bit j of it to token 8*o + j.
+__device__ __forceinline__ void octet_allow_bits(const PartDev& P, const uint32_t* T, int o, int rb, bool active,
+                                                 uint32_t& lo, uint32_t& hi) {
+    lo = hi = 0;
+    if (!active) return;
+    const uint4 cv = __ldg(reinterpret_cast<const uint4*>(P.c16) + o);
+    const uint32_t w0 = T[cv.x & 0xFFFFu], w1 = T[cv.x >> 16], w2 = T[cv.y & 0xFFFFu], w3 = T[cv.y >> 16];
+    const uint32_t w4 = T[cv.z & 0xFFFFu], w5 = T[cv.z >> 16], w6 = T[cv.w & 0xFFFFu], w7 = T[cv.w >> 16];
+    const uint32_t sel = uint32_t(rb) | (uint32_t(4 + rb) << 4);  // byte rb of both operands
+    lo = __byte_perm(__byte_perm(w0, w1, sel), __byte_perm(w2, w3, sel), 0x5410);
+    hi = __byte_perm(__byte_perm(w4, w5, sel), __byte_perm(w6, w7, sel), 0x5410);
+    transpose8x8(lo, hi);
+}
+
+// ---------------------------------------------------------------------------------------
+// Fused dense step: expand + mask in place + (max, sum-exp, position) per row.
+// Grid: n_groups * S thread blocks; block (g, split) owns octets [split*per_split, ...) of the
+// 32 rows of group g. Warps are arranged WT (along tokens) x WR (row batches of 8).
+// ---------------------------------------------------------------------------------------
+template <int DT, bool ALIGNED>
+__global__ void __launch_bounds__(256) k_step_dense(const __grid_constant__ StepArgs a) {
+    extern __shared__ __align__(16) uint32_t smem[];
+    uint32_t* T = smem;
+    int* s_row = reinterpret_cast<int*>(T + a.table_words);
+    Partial* red = reinterpret_cast<Partial*>(s_row + kGroupRows);
+    __shared__ int s_last;
+
+    pdl_prologue();
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, n_warps = blockDim.x >> 5;
+    const int g = blockIdx.x / a.S, split = blockIdx.x - g * a.S;
+    if (a.n_groups && g >= __ldg(a.n_groups)) return;
+    const int part = group_rows_setup(a, g, s_row, tid);
+    for (int i = tid; i < n_warps * kGroupRows; i += blockDim.x) red[i] = partial_empty();
+    __syncthreads();
+    const PartDev P = a.parts[part];
+    const int nrow = __popc(__ballot_sync(0xFFFFFFFFu, s_row[lane] >= 0));
+    build_class_table(a, P, s_row, T, warp, lane, n_warps);
+    __syncthreads();
+
+    const int wt = warp % a.WT, wr = warp / a.WT, WR = n_warps / a.WT;
+    const int n_octets = 4 * a.VW, n_full = a.V >> 3;
+    const int o_begin = split * a.per_split;
+    const int o_end = min(o_begin + a.per_split, n_octets);
+    constexpr int ES = DT == kBF16 ? 2 : 4;
+    uint8_t* vm8 = reinterpret_cast<uint8_t*>(a.vocab_mask);
+
+    for (int rb = wr; rb * kBatchRows < nrow; rb += WR) {
+        float m[kBatchRows], s[kBatchRows];
+        int pos[kBatchRows];
+        char* rowp[kBatchRows];
+        uint8_t* vmp[kBatchRows];
+#pragma unroll
+        for (int i = 0; i < kBatchRows; ++i) {
+            m[i] = -INFINITY; s[i] = 0.f; pos[i] = kNoPos;
+            const int row = s_row[min(rb * kBatchRows + i, kGroupRows - 1)];
+            rowp[i] = reinterpret_cast<char*>(a.logits) + int64_t(max(row, 0)) * a.row_stride * ES;
+            vmp[i] = vm8 ? vm8 + int64_t(max(row, 0)) * a.vm_stride * 4 : nullptr;
+        }
+        const int live = min(kBatchRows, nrow - rb * kBatchRows);
+
+        for (int o0 = o_begin + wt * 32; o0 < o_end; o0 += a.WT * 32) {
+            const int o = o0 + lane;
+            const bool active = o < o_end;
+            const bool vec = ALIGNED && o < n_full;
+            Octet<DT> oc[kBatchRows];
+#pragma unroll
+            for (int i = 0; i < kBatchRows; ++i)
+                if (i < live && active && vec) oc[i].load(rowp[i], o);
+            uint32_t lo, hi;
+            octet_allow_bits(P, T, o, rb, active, lo, hi);
+#pragma unroll
+            for (int i = 0; i < kBatchRows; ++i) {
+                if (i < live && active) {
+                    const uint32_t byte = ((i < 4 ? lo : hi) >> (8 * (i & 3))) & 0xFFu;
+                    float f[8];
+                    if (vec) {
+                        oc[i].mask(byte, f);
+                        oc[i].store(rowp[i], o);
+                    } else {
+                        octet_scalar<DT>(rowp[i], o, a.V, byte, f);
+                    }
+                    if (vmp[i]) vmp[i][o] = uint8_t(byte);
+                    partial_add_octet(m[i], s[i], pos[i], f, byte, o);
+                }
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < kBatchRows; ++i) {
+            partial_warp_allreduce(m[i], s[i], pos[i]);
+            if (lane == 0 && i < live) red[warp * kGroupRows + rb * kBatchRows + i] = Partial{m[i], s[i], pos[i], 0};
+        }
+    }
+    __syncthreads();
+
+    // one thread per row slot folds the warps' results
+    float rm = -INFINITY, rs = 0.f;
+    int rpos = kNoPos;
+    if (tid < kGroupRows) {
+        for (int w = 0; w < n_warps; ++w) {
+            const Partial p = red[w * kGroupRows + tid];
+            partial_merge(rm, rs, rpos, p.m, p.s, p.pos);
+        }
+    }
+    if (a.S == 1) {
+        if (tid < kGroupRows) finalize_row<DT>(a, P, s_row[tid], rm, rs, rpos, false);
+        return;
+    }
+    // several blocks share the group: publish, and let the last one to arrive finish the rows
+    if (tid < kGroupRows)
+        a.partials[(int64_t(g) * kGroupRows + tid) * a.S + split] = Partial{rm, rs, rpos, 0};
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_last = (atomicAdd(a.tickets + g, 1u) == unsigned(a.S - 1));
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    for (int j = warp; j < nrow; j += n_warps) {
+        float m2 = -INFINITY, s2 = 0.f;
+        int p2 = kNoPos;
+        const Partial* src = a.partials + (int64_t(g) * kGroupRows + j) * a.S;
+        for (int sp = lane; sp < a.S; sp += 32) {
+            const int4 raw = __ldcg(reinterpret_cast<const int4*>(src + sp));
+            partial_merge(m2, s2, p2, __int_as_float(raw.x), __int_as_float(raw.y), raw.z);
+        }
+        partial_warp_allreduce(m2, s2, p2);
+        if (lane == 0) finalize_row<DT>(a, P, s_row[j], m2, s2, p2, false);
+    }
+    if (tid == 0) a.tickets[g] = 0u;
+}
+
+// ---------------------------------------------------------------------------------------
+// Dense expansion only: lane <-> token, one ballot per row builds the packed word.
+// Same grid and row groups as the fused kernel; per_split counts 32-token words here.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) k_expand_dense(const __grid_constant__ StepArgs a) {
+    extern __shared__ __align__(16) uint32_t smem[];
+    uint32_t* T = smem;
+    int* s_row = reinterpret_cast<int*>(T + a.table_words);
+
+    pdl_prologue();
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, n_warps = blockDim.x >> 5;
+    const int g = blockIdx.x / a.S, split = blockIdx.x - g * a.S;
+    if (a.n_groups && g >= __ldg(a.n_groups)) return;
+    const int part = group_rows_setup(a, g, s_row, tid);
+    __syncthreads();
+    const PartDev P = a.parts[part];
+    const int nrow = __popc(__ballot_sync(0xFFFFFFFFu, s_row[lane] >= 0));
+    build_class_table(a, P, s_row, T, warp, lane, n_warps);
+    __syncthreads();
+
+    const int w_begin = split * a.per_split, w_end = min(w_begin + a.per_split, a.VW);
+    const int my_row = s_row[lane];
+    uint32_t* out = a.vocab_mask + int64_t(max(my_row, 0)) * a.vm_stride;
+    // a warp takes 8 consecutive words (256 tokens) per iteration; lane r ends up holding row r's words
+    for (int w0 = w_begin + warp * 8; w0 < w_end; w0 += n_warps * 8) {
+        uint32_t mine[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int w = w0 + q;
+            uint32_t bits = 0;
+            if (w < w_end) bits = T[P.c16[w * 32 + lane]];  // c16 is padded to 32*VW entries
+            mine[q] = 0;
+            for (int r = 0; r < nrow; ++r) {
+                const uint32_t word = __ballot_sync(0xFFFFFFFFu, (bits >> r) & 1u);
+                if (lane == r) mine[q] = word;
+            }
+        }
+        if (my_row >= 0) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                if (w0 + q < w_end) out[w0 + q] = mine[q];
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Sparse step: one row per block (S blocks per row). The row's vocab bitmask is built in
+// shared memory by scattering the member lists of the allowed classes; then the row is
+// streamed: octets with no allowed token are overwritten with -inf without being read.
+// FUSED = false stops after writing the vocab mask.
+// ---------------------------------------------------------------------------------------
+constexpr int kBigClass = 4096;  // classes at least this large are scattered by the whole block
+constexpr int kBigListCap = 64;
+
+__device__ __forceinline__ int lower_bound_tok(const int32_t* tok, int lo, int hi, int t) {
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(tok + mid) < t) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+
+template <int DT, bool FUSED, bool ALIGNED>
+__global__ void __launch_bounds__(256) k_step_sparse(const __grid_constant__ StepArgs a) {
+    extern __shared__ __align__(16) uint32_t smem[];
+    uint32_t* bits = smem;  // per_split words
+    __shared__ int s_big[kBigListCap];
+    __shared__ int s_nbig;
+    __shared__ int s_last;
+    __shared__ Partial s_red[8];
+
+    pdl_prologue();
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, n_warps = blockDim.x >> 5;
+    const int row = blockIdx.x / a.S, split = blockIdx.x - row * a.S;
+    const int part = a.row_part ? a.row_part[row] : a.part0;
+    if (part < 0 || part >= a.n_parts || !a.parts[part].live || a.parts[part].V != a.V) {
+        if (tid == 0 && split == 0) atomicAdd(a.status + 2, 1);
+        return;
+    }
+    const PartDev P = a.parts[part];
+    const int w_begin = split * a.per_split, w_end = min(w_begin + a.per_split, a.VW);
+    const int t0 = w_begin * 32, t1 = min(w_end * 32, a.V);
+    for (int i = tid; i < a.per_split; i += blockDim.x) bits[i] = 0u;
+    if (tid == 0) s_nbig = 0;
+    __syncthreads();
+
+    const uint32_t* cm = a.class_mask + int64_t(row) * a.cm_stride;
+    for (int kw = warp; kw < P.KW; kw += n_warps) {
+        uint32_t word = __ldg(cm + kw);
+        if (kw == P.KW - 1 && (P.K & 31)) word &= (1u << (P.K & 31)) - 1u;
+        while (word) {
+            const int k = kw * 32 + __ffs(word) - 1;
+            word &= word - 1u;
+            int lo = __ldg(P.off + k), hi = __ldg(P.off + k + 1);
+            if (a.S > 1) {
+                lo = lower_bound_tok(P.tok, lo, hi, t0);
+                hi = lower_bound_tok(P.tok, lo, hi, t1);
+            }
+            if (hi - lo >= kBigClass) {
+                int slot = 0;
+                if (lane == 0) slot = atomicAdd(&s_nbig, 1);
+                slot = __shfl_sync(0xFFFFFFFFu, slot, 0);
+                if (slot < kBigListCap) {
+                    if (lane == 0) s_big[slot] = k;
+                    continue;
+                }
+            }
+            for (int i = lo + lane; i < hi; i += 32) {
+                const int t = __ldg(P.tok + i);
+                atomicOr(bits + ((t >> 5) - w_begin), 1u << (t & 31));
+            }
+        }
+    }
+    __syncthreads();
+    const int nbig = min(s_nbig, kBigListCap);
+    for (int b = 0; b < nbig; ++b) {
+        const int k = s_big[b];
+        int lo = __ldg(P.off + k), hi = __ldg(P.off + k + 1);
+        if (a.S > 1) {
+            lo = lower_bound_tok(P.tok, lo, hi, t0);
+            hi = lower_bound_tok(P.tok, lo, hi, t1);
+        }
+        for (int i = lo + tid; i < hi; i += blockDim.x) {
+            const int t = __ldg(P.tok + i);
+            atomicOr(bits + ((t >> 5) - w_begin), 1u << (t & 31));
+        }
+    }
+    __syncthreads();
+
+    if (a.vocab_mask) {
+        uint32_t* out = a.vocab_mask + int64_t(row) * a.vm_stride;
+        for (int w = w_begin + tid; w < w_end; w += blockDim.x) out[w] = bits[w - w_begin];
+    }
+    if (!FUSED) return;
+
+    constexpr int ES = DT == kBF16 ? 2 : 4;
+    char* rowp = reinterpret_cast<char*>(a.logits) + int64_t(row) * a.row_stride * ES;
+    const uint8_t* bytes = reinterpret_cast<const uint8_t*>(bits);
+    const int o_begin = 4 * w_begin, o_end = 4 * w_end, n_full = a.V >> 3;
+    float m = -INFINITY, s = 0.f;
+    int pos = kNoPos;
+    constexpr int U = 4;
+    for (int ob = o_begin + tid; ob < o_end; ob += U * blockDim.x) {
+        Octet<DT> oc[U];
+        uint32_t byte[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int o = ob + u * blockDim.x;
+            byte[u] = o < o_end ? bytes[o - o_begin] : 0u;
+            if (o < o_end && byte[u] && ALIGNED && o < n_full) oc[u].load(rowp, o);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int o = ob + u * blockDim.x;
+            if (o >= o_end) continue;
+            if (ALIGNED && o < n_full) {
+                if (byte[u] == 0u) {
+                    oc[u].fill_neg_inf();
+                    oc[u].store(rowp, o);
+                } else {
+                    float f[8];
+                    oc[u].mask(byte[u], f);
+                    if (byte[u] != 0xFFu) oc[u].store(rowp, o);
+                    partial_add_octet(m, s, pos, f, byte[u], o);
+                }
+            } else {
+                float f[8];
+                octet_scalar<DT>(rowp, o, a.V, byte[u], f);
+                if (byte[u]) partial_add_octet(m, s, pos, f, byte[u], o);
+            }
+        }
+    }
+    partial_warp_allreduce(m, s, pos);
+    if (lane == 0) s_red[warp] = Partial{m, s, pos, 0};
+    __threadfence();  // the row's masked logits must be visible to whichever block finishes the row
+    __syncthreads();
+    if (tid == 0) {
+        for (int w = 1; w < n_warps; ++w) partial_merge(m, s, pos, s_red[w].m, s_red[w].s, s_red[w].pos);
+        if (a.S == 1) {
+            finalize_row<DT>(a, P, row, m, s, pos, false);
+        } else {
+            a.partials[int64_t(row) * a.S + split] = Partial{m, s, pos, 0};
+            __threadfence();
+            s_last = (atomicAdd(a.tickets + row, 1u) == unsigned(a.S - 1));
+        }
+    }
+    if (a.S == 1) return;
+    __syncthreads();
+    if (!s_last || warp != 0) return;
+    __threadfence();
+    float m2 = -INFINITY, s2 = 0.f;
+    int p2 = kNoPos;
+    for (int sp = lane; sp < a.S; sp += 32) {
+        const int4 raw = __ldcg(reinterpret_cast<const int4*>(a.partials + int64_t(row) * a.S + sp));
+        partial_merge(m2, s2, p2, __int_as_float(raw.x), __int_as_float(raw.y), raw.z);
+    }
+    partial_warp_allreduce(m2, s2, p2);
+    if (lane == 0) {
+        finalize_row<DT>(a, P, row, m2, s2, p2, false);
+        a.tickets[row] = 0u;
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Generic step: one block per row, one token per thread per iteration, no alignment or
+// size requirement (any K, int32 class ids, odd strides). FUSED = false: expansion only.
+// ---------------------------------------------------------------------------------------
+template <int DT, bool FUSED>
+__global__ void __launch_bounds__(256) k_step_generic(const __grid_constant__ StepArgs a) {
+    __shared__ Partial s_red[8];
+    pdl_prologue();
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, n_warps = blockDim.x >> 5;
+    const int row = blockIdx.x;
+    const int part = a.row_part ? a.row_part[row] : a.part0;
+    if (part < 0 || part >= a.n_parts || !a.parts[part].live || a.parts[part].V != a.V) {
+        if (tid == 0) atomicAdd(a.status + 2, 1);
+        return;
+    }
+    const PartDev P = a.parts[part];
+    const uint32_t* cm = a.class_mask + int64_t(row) * a.cm_stride;
+    constexpr int ES = DT == kBF16 ? 2 : 4;
+    char* rowp = FUSED ? reinterpret_cast<char*>(a.logits) + int64_t(row) * a.row_stride * ES : nullptr;
+    uint32_t* out = a.vocab_mask ? a.vocab_mask + int64_t(row) * a.vm_stride : nullptr;
+    float m = -INFINITY, s = 0.f;
+    int pos = kNoPos;
+    for (int w = warp; w < a.VW; w += n_warps) {
+        const int t = w * 32 + lane;
+        bool allowed = false;
+        if (t < a.V) {
+            const int k = __ldg(P.c32 + t);
+            allowed = (__ldg(cm + (k >> 5)) >> (k & 31)) & 1u;
+        }
+        const uint32_t word = __ballot_sync(0xFFFFFFFFu, allowed);
+        if (out && lane == 0) out[w] = word;
+        if (FUSED && t < a.V) {
+            if (allowed) {
+                const float z = load_elem<DT>(rowp, t);
+                const bool upd = (z > m) || pos == kNoPos;
+                pos = upd ? t : pos;
+                const float ref_old = fmaxf(m, kRefFloor);
+                m = fmaxf(m, z);
+                const float ref = fmaxf(m, kRefFloor);
+                s = fmaf(s, ex2f((ref_old - ref) * kLog2e), ex2f((z - ref) * kLog2e));
+            } else {
+                store_neg_inf<DT>(rowp, t);
+            }
+        }
+    }
+    if (!FUSED) return;
+    partial_warp_allreduce(m, s, pos);
+    if (lane == 0) s_red[warp] = Partial{m, s, pos, 0};
+    __syncthreads();
+    if (tid == 0) {
+        for (int w = 1; w < n_warps; ++w) partial_merge(m, s, pos, s_red[w].m, s_red[w].s, s_red[w].pos);
+        finalize_row<DT>(a, P, row, m, s, pos, true);
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Row plan for batches that mix partitions: bucket the rows by partition into groups of
+// up to 32 rows (valid slots first). One block.
+// ---------------------------------------------------------------------------------------
+constexpr int kMaxParts = 256;
+
+__global__ void __launch_bounds__(1024) k_plan_rows(const PartDev* parts, int n_parts, const int32_t* row_part, int B,
+                                                    int V, int max_groups, int32_t* group_part, int32_t* group_rows,
+                                                    int32_t* n_groups, int32_t* status) {
+    __shared__ int cnt[kMaxParts], gbase[kMaxParts + 1], cur[kMaxParts];
+    pdl_prologue();
+    const int tid = threadIdx.x;
+    for (int p = tid; p < kMaxParts; p += blockDim.x) { cnt[p] = 0; cur[p] = 0; }
+    __syncthreads();
+    for (int b = tid; b < B; b += blockDim.x) {
+        const int p = row_part[b];
+        if (p >= 0 && p < n_parts && parts[p].live && parts[p].V == V) atomicAdd(&cnt[p], 1);
+        else atomicAdd(status + 2, 1);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int acc = 0;
+        for (int p = 0; p < n_parts; ++p) { gbase[p] = acc; acc += (cnt[p] + kGroupRows - 1) / kGroupRows; }
+        gbase[n_parts] = acc;
+        *n_groups = acc;
+    }
+    __syncthreads();
+    const int total = gbase[n_parts];
+    for (int i = tid; i < max_groups * kGroupRows; i += blockDim.x) group_rows[i] = -1;
+    for (int p = 0; p < n_parts; ++p)
+        for (int gq = gbase[p] + tid; gq < gbase[p + 1]; gq += blockDim.x) group_part[gq] = p;
+    for (int gq = total + tid; gq < max_groups; gq += blockDim.x) group_part[gq] = 0;
+    __syncthreads();
+    for (int b = tid; b < B; b += blockDim.x) {
+        const int p = row_part[b];
+        if (p >= 0 && p < n_parts && parts[p].live && parts[p].V == V) {
+            const int slot = atomicAdd(&cur[p], 1);
+            group_rows[(gbase[p] + slot / kGroupRows) * kGroupRows + (slot % kGroupRows)] = b;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// mask_logits: apply an existing vocab bitmask in place. Octets whose 8 tokens are all
+// allowed are neither read nor written; octets with none allowed are written without a read.
+// ---------------------------------------------------------------------------------------
+template <int DT, bool ALIGNED>
+__global__ void __launch_bounds__(256) k_mask_logits(void* logits, int64_t row_stride, int B, int V, int VW,
+                                                     const uint32_t* vocab_mask, int64_t vm_stride) {
+    pdl_prologue();
+    constexpr int ES = DT == kBF16 ? 2 : 4;
+    constexpr int U = 4;
+    const int n_octets = (V + 7) >> 3, n_full = V >> 3;
+    const int chunks = (n_octets + blockDim.x * U - 1) / (blockDim.x * U);
+    const int64_t total = int64_t(B) * chunks;
+    const uint8_t* vm8 = reinterpret_cast<const uint8_t*>(vocab_mask);
+    for (int64_t item = blockIdx.x; item < total; item += gridDim.x) {
+        const int row = int(item / chunks), ch = int(item - int64_t(row) * chunks);
+        char* rowp = reinterpret_cast<char*>(logits) + int64_t(row) * row_stride * ES;
+        const uint8_t* vrow = vm8 + int64_t(row) * vm_stride * 4;
+        const int ob = ch * blockDim.x * U + threadIdx.x;
+        Octet<DT> oc[U];
+        uint32_t byte[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int o = ob + u * blockDim.x;
+            byte[u] = 0xFFu;
+            if (o < n_octets) {
+                byte[u] = vrow[o];
+                if (8 * o + 8 > V) byte[u] = (byte[u] | (0xFFu << (V - 8 * o))) & 0xFFu;  // past V: leave alone
+                if (ALIGNED && o < n_full && byte[u] != 0xFFu && byte[u] != 0u) oc[u].load(rowp, o);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int o = ob + u * blockDim.x;
+            if (o >= n_octets || byte[u] == 0xFFu) continue;
+            float f[8];
+            if (ALIGNED && o < n_full) {
+                if (byte[u] == 0u) oc[u].fill_neg_inf(); else oc[u].mask(byte[u], f);
+                oc[u].store(rowp, o);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (8 * o + j < V && !((byte[u] >> j) & 1u)) store_neg_inf<DT>(rowp, 8 * o + j);
+            }
+        }
+    }
+}
+
+// logp_full[b, i] = z'[b, i] - lse[b] from the masked logits (fp32 out, row stride V).
+template <int DT>
+__global__ void __launch_bounds__(256) k_logp_full(const void* logits, int64_t row_stride, int B, int V, const float* lse,
+                                                   float* out) {
+    pdl_prologue();
+    const int64_t total = int64_t(B) * V;
+    for (int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += int64_t(gridDim.x) * blockDim.x) {
+        const int row = int(i / V), t = int(i - int64_t(row) * V);
+        const float l = lse[row];
+        const float z = load_elem<DT>(logits, int64_t(row) * row_stride + t);
+        out[i] = (l == -INFINITY || z == -INFINITY) ? -INFINITY : z - l;
+    }
+}
+
+// reps[b] = r[c[tokens[b]]]
+__global__ void __launch_bounds__(256) k_map_tokens(const PartDev* parts, int n_parts, int part0, const int32_t* row_part,
+                                                    const int32_t* tokens, int32_t* reps, int B, int V_expected,
+                                                    int32_t* status) {
+    pdl_prologue();
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    const int p = row_part ? row_part[b] : part0;
+    if (p < 0 || p >= n_parts || !parts[p].live || parts[p].V != V_expected) {
+        atomicAdd(status + 2, 1);
+        return;
+    }
+    const int t = tokens[b];
+    int rv = -1;
+    if (t >= 0 && t < parts[p].V) rv = parts[p].r[parts[p].c32[t]];
+    else atomicAdd(status + 1, 1);
+    reps[b] = rv;
+}
+
+}  // namespace cfgzip
