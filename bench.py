@@ -147,7 +147,7 @@ class StepRunner:
     """A ring of resident working buffers for one workload and CUDA graphs that run steps over it."""
 
     def __init__(self, cz, torch, device: int, config: int, B: int = None, mode: str = "dense", steps_hint: int = 1000,
-                 unique: int = 8):
+                 unique: int = 8, tune=()):
         self.cz, self.torch = cz, torch
         spec = synth.CONFIGS[config]
         self.w = synth.make_workload(config, B=min(B or spec["B"], 64))  # unique rows; tiled up to B below
@@ -157,6 +157,9 @@ class StepRunner:
         self.VW, self.KW = (self.V + 31) // 32, (self.K + 31) // 32
         self.mode = {"dense": cz.DENSE, "sparse": cz.SPARSE, "auto": cz.AUTO}[mode]
         self.ctx = cz.cfgzip_create(device)
+        for item in tune:
+            name, value = item.split("=")
+            cz.cfgzip_set_tuning(self.ctx, name, int(value))
         self.parts = [cz.cfgzip_load_partition(self.ctx, p.c, p.V, p.r, p.K) for p in self.w.partitions]
         step_bytes = self.B * self.V * self.elem
         ring = max(4, -(-RING_BYTES // step_bytes))
@@ -358,7 +361,8 @@ def run_own(args):
         if dist is not None:
             dist.barrier()
 
-    runner = StepRunner(cz, torch, local_rank, args.workload, B=args.batch, mode=args.mode, steps_hint=args.steps)
+    runner = StepRunner(cz, torch, local_rank, args.workload, B=args.batch, mode=args.mode, steps_hint=args.steps,
+                        tune=args.tune)
     props = torch.cuda.get_device_properties(local_rank)
     sampler = ClockSampler("GPU-" + str(props.uuid))
     seconds, launches = runner.timed(args.steps, args.warmup, barrier, sampler)
@@ -410,7 +414,8 @@ def run_own(args):
     if rank == 0 and world == 1 and not args.no_extras:
         extras = []
         for B in (128, 256, 1024):
-            r2 = StepRunner(cz, torch, local_rank, args.workload, B=B, mode=args.mode, steps_hint=8, unique=2)
+            r2 = StepRunner(cz, torch, local_rank, args.workload, B=B, mode=args.mode, steps_hint=8, unique=2,
+                            tune=args.tune)
             n = 3 * r2.R
             s2, l2 = r2.timed(n, r2.R)
             a2 = r2.alg_bytes() / (s2 / n) / 1e9
@@ -479,6 +484,8 @@ def main():
     ap.add_argument("--batch", type=int, default=None, help="override the workload's row count")
     ap.add_argument("--mode", choices=["dense", "sparse", "auto"], default="dense")
     ap.add_argument("--e2e-steps", type=int, default=200)
+    ap.add_argument("--tune", action="append", default=[], metavar="NAME=VALUE",
+                    help="library tuning knob (see cfgzip_set_tuning); may be repeated")
     ap.add_argument("--no-extras", action="store_true", help="skip the larger-batch sweep")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

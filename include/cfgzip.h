@@ -175,7 +175,9 @@ int cfgzip_decode_step_host(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t
 /*
  * Synchronise `stream`, then return and clear the sticky counters: rows that had no
  * allowed token, token ids out of range in cfgzip_map_tokens, rows skipped for a bad
- * partition id. Any output pointer may be NULL.
+ * partition id. Any output pointer may be NULL. Returns CFGZIP_E_CUDA if a kernel reported
+ * that one of its asynchronous copies never completed (its bounded wait ran out); the
+ * results of that call are then undefined.
  */
 int cfgzip_poll_status(cfgzip_ctx* ctx, void* stream, int32_t* n_empty_rows, int32_t* n_bad_tokens,
                        int32_t* n_bad_rows);
@@ -186,9 +188,13 @@ int cfgzip_launch_count(cfgzip_ctx* ctx, int64_t* out);
 /*
  * Tuning knobs for benchmarking; defaults are chosen from the device at create time.
  *   "ctas_per_sm"  target resident thread blocks per SM for the fused kernel (1..16)
- *   "token_warps"  0 = automatic, else warps side by side along the vocabulary (1..8)
+ *   "token_warps"  0 = automatic, else warps side by side along the vocabulary (1..16)
  *   "row_warps"    0 = automatic, else 1, 2 or 4 row batches handled by separate warps
  *   "pdl"          1 = launch with programmatic dependent launch (default), 0 = off
+ *   "pipeline"     1 = aligned logits stream through per-warp rings of bulk asynchronous copies
+ *                  in shared memory (default), 0 = plain 16-byte loads into registers
+ *   "pipe_warps"   warps per thread block of the pipelined kernel (4, 8, 12 or 16)
+ *   "pipe_depth"   stages per warp of the pipelined kernel (2..8; lowered to fit shared memory)
  * Unknown names give CFGZIP_E_ARG.
  */
 int cfgzip_set_tuning(cfgzip_ctx* ctx, const char* name, int32_t value);

@@ -56,6 +56,9 @@ struct cfgzip_ctx {
     int32_t token_warps = 0;
     int32_t row_warps = 0;
     int32_t pdl = 1;
+    int32_t pipeline = 1;     // bulk-copy pipelined dense kernel for aligned logits
+    int32_t pipe_warps = 8;
+    int32_t pipe_depth = 4;
 };
 
 namespace {
@@ -157,39 +160,87 @@ bool aligned16(const void* p, int64_t row_stride_elems, int elem_size) {
     return (reinterpret_cast<uintptr_t>(p) & 15u) == 0 && ((row_stride_elems * elem_size) & 15) == 0;
 }
 
-size_t dense_smem_bytes(int table_words, int n_warps) {
-    return size_t(table_words) * 4 + kGroupRows * 4 + size_t(n_warps) * kGroupRows * sizeof(Partial);
+size_t dense_smem_bytes(int table_words, int n_warps, int stage_stride) {
+    return size_t(table_words) * 4 + kGroupRows * 4 + size_t(n_warps) * kGroupRows * sizeof(Partial) +
+           size_t(stage_stride) * kGroupRows * 4;
 }
 
 // Launch shape of the dense kernels.
 struct DensePlan {
-    int S = 1, per_split = 0, WT = 4, threads = 128, table_words = 0;
+    int S = 1, per_split = 0, WT = 4, threads = 128, table_words = 0, stage_stride = 0;
+    int depth = 0;       // > 0: pipelined kernel with this many stages per warp
+    size_t smem = 0;
     int n_groups_ub = 1;
     bool use_plan_kernel = false;
     bool ok = false;  // false: the dense kernels cannot run this call (generic path instead)
 };
 
+size_t pipe_smem_bytes(int table_words, int n_warps, int depth, int stage_bytes, int stage_stride) {
+    return size_t(table_words) * 4 + kGroupRows * 4 + size_t(n_warps) * kGroupRows * sizeof(Partial) +
+           ((size_t(n_warps) * depth * 8 + 127) & ~size_t(127)) + size_t(n_warps) * depth * stage_bytes +
+           size_t(stage_stride) * kGroupRows * 4;
+}
+
+// units: octets (fused) or 32-token words (expand); unit_chunk: units one warp covers per iteration.
+// elem_size: bytes per logit when the pipelined kernel may be used (aligned fused call), else 0.
 DensePlan plan_dense(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, int units, int unit_chunk,
-                     bool fused) {
-    // units: octets (fused) or 32-token words (expand); unit_chunk: units one warp covers per iteration
+                     bool fused, int elem_size) {
     DensePlan d;
     d.table_words = (ps.maxKW + 1) * 32;
     d.use_plan_kernel = mixed;
     d.n_groups_ub = mixed ? ceil_div(B, kGroupRows) + ps.n_live_same_v : ceil_div(B, kGroupRows);
     if (!ps.all_c16) return d;
-    if (dense_smem_bytes(d.table_words, 8) > size_t(ctx->smem_optin)) return d;
+    if (dense_smem_bytes(d.table_words, 8, 0) > size_t(ctx->smem_optin) - 2048) return d;
     if (mixed && (B > ctx->reserved_rows || d.n_groups_ub > ctx->max_groups)) return d;
-    const int target = ctx->sm_count * ctx->ctas_per_sm;
+    int ctas_per_sm = ctx->ctas_per_sm;
+    int n_warps = 4;
+    if (fused && elem_size && ctx->pipeline) {
+        const int stage_bytes = 8 * 32 * 8 * elem_size + 512;
+        n_warps = ctx->pipe_warps;
+        int depth = ctx->pipe_depth;
+        const size_t cap = size_t(ctx->smem_optin) - 2048;  // room for the kernels' static shared memory
+        int stride = ps.maxKW | 1;
+        if (pipe_smem_bytes(d.table_words, n_warps, 2, stage_bytes, stride) > cap) stride = 0;
+        while (depth > 2 && pipe_smem_bytes(d.table_words, n_warps, depth, stage_bytes, stride) > cap) --depth;
+        while (n_warps > 4 && pipe_smem_bytes(d.table_words, n_warps, depth, stage_bytes, stride) > cap) n_warps -= 4;
+        const size_t smem = pipe_smem_bytes(d.table_words, n_warps, depth, stage_bytes, stride);
+        if (smem <= cap) {
+            d.depth = depth;
+            d.smem = smem;
+            d.stage_stride = stride;
+            const int fit = std::max(1, int((cap + 1024) / (smem + 1024)));
+            ctas_per_sm = std::min(ctas_per_sm, fit);
+        }
+    }
+    if (!d.depth) {
+        // stage the class masks through shared memory while that keeps a block under 64 KB
+        if (dense_smem_bytes(d.table_words, 8, ps.maxKW | 1) <= 64 * 1024) d.stage_stride = ps.maxKW | 1;
+    }
+    const int target = ctx->sm_count * ctas_per_sm;
     const int n_chunks = ceil_div(units, unit_chunk);
     const int s0 = std::max(1, target / d.n_groups_ub);
     int cps = ceil_div(n_chunks, s0);  // chunks per block
     int WR = 1;
     if (fused) {
-        WR = ctx->row_warps ? ctx->row_warps : (cps <= 2 ? 4 : 1);
-        if (WR != 1 && WR != 2 && WR != 4) WR = 1;
-        d.WT = ctx->token_warps ? ctx->token_warps : (WR == 4 ? std::min(cps, 2) : (WR == 2 ? 2 : 4));
-        d.WT = std::max(1, std::min(d.WT, 8 / WR));
+        if (d.depth) {
+            WR = ctx->row_warps ? ctx->row_warps : (cps * 4 <= n_warps ? 4 : (cps * 2 <= n_warps ? 2 : 1));
+            if (WR != 1 && WR != 2 && WR != 4) WR = 1;
+            d.WT = ctx->token_warps ? ctx->token_warps : n_warps / WR;
+            d.WT = std::max(1, std::min(d.WT, 16 / WR));
+            cps = ceil_div(cps, d.WT) * d.WT;  // every warp of a block gets the same number of chunks
+        } else {
+            WR = ctx->row_warps ? ctx->row_warps : (cps <= 2 ? 4 : 1);
+            if (WR != 1 && WR != 2 && WR != 4) WR = 1;
+            d.WT = ctx->token_warps ? ctx->token_warps : (WR == 4 ? std::min(cps, 2) : (WR == 2 ? 2 : 4));
+            d.WT = std::max(1, std::min(d.WT, 8 / WR));
+        }
         d.threads = d.WT * WR * 32;
+        if (d.depth) {
+            // the ring was sized for n_warps; recompute for the warps actually launched
+            const int stage_bytes = 8 * 32 * 8 * elem_size + 512;
+            d.smem = pipe_smem_bytes(d.table_words, d.threads / 32, d.depth, stage_bytes, d.stage_stride);
+            if (d.smem > size_t(ctx->smem_optin) - 2048) return d;
+        }
     } else {
         d.WT = 8;
         d.threads = 256;
@@ -201,6 +252,7 @@ DensePlan plan_dense(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, 
     }
     if (fused && d.S > 1 && d.n_groups_ub > ctx->reserved_rows) return d;  // tickets
     d.per_split = cps * unit_chunk;
+    if (!d.depth) d.smem = dense_smem_bytes(d.table_words, fused ? d.threads / 32 : 0, d.stage_stride);
     d.ok = true;
     return d;
 }
@@ -233,6 +285,9 @@ void fill_groups(cfgzip_ctx* ctx, StepArgs& a, const DensePlan& d) {
     a.per_split = d.per_split;
     a.WT = d.WT;
     a.table_words = d.table_words;
+    a.stage_stride = d.stage_stride;
+    a.depth = d.depth;
+    a.p0 = ctx->parts[size_t(a.part0)].dev;
 }
 
 // Sparse launch shape: S blocks per row, each owning per_split vocab-mask words in shared memory.
@@ -240,7 +295,7 @@ bool plan_sparse(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool fused, int*
     const int target = ctx->sm_count * ctx->ctas_per_sm;
     int s = std::max(1, target / std::max(B, 1));
     s = std::min(s, std::max(1, ps.VW / 256));
-    const int max_words = (ctx->smem_optin - 4096) / 4;
+    const int max_words = (ctx->smem_optin - 8192) / 4;
     for (;;) {
         *per_split = ((ceil_div(ps.VW, s) + 3) / 4) * 4;
         if (*per_split <= max_words) break;
@@ -263,27 +318,35 @@ template <int DT>
 int launch_fused(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, int mode, bool aligned, float* logp_full,
                  cudaStream_t st) {
     int rc;
-    if (mode == CFGZIP_SPARSE) {
+    if (!aligned) {
+        // rows off the 16-byte grid: the per-row kernel with element-wise accesses
+        rc = launch(ctx, k_step_generic<DT, true>, dim3(unsigned(a.B)), dim3(256), 0, st, a);
+    } else if (mode == CFGZIP_SPARSE) {
         int S, per_split;
         if (plan_sparse(ctx, ps, a.B, true, &S, &per_split)) {
             a.S = S;
             a.per_split = per_split;
             const size_t smem = size_t(per_split) * 4;
-            auto kern = aligned ? k_step_sparse<DT, true, true> : k_step_sparse<DT, true, false>;
+            auto kern = k_step_sparse<DT, true>;
             if ((rc = ensure_smem(kern, smem)) != CFGZIP_OK) return rc;
             rc = launch(ctx, kern, dim3(unsigned(a.B) * unsigned(S)), dim3(256), smem, st, a);
         } else {
             rc = launch(ctx, k_step_generic<DT, true>, dim3(unsigned(a.B)), dim3(256), 0, st, a);
         }
     } else {
-        const DensePlan d = plan_dense(ctx, ps, a.B, mixed, 4 * ps.VW, 32, true);
+        const DensePlan d = plan_dense(ctx, ps, a.B, mixed, 4 * ps.VW, 32, true, DT == kBF16 ? 2 : 4);
         if (d.ok) {
             if (d.use_plan_kernel && (rc = run_plan_kernel(ctx, a.row_part, a.B, a.V, d, st)) != CFGZIP_OK) return rc;
             fill_groups(ctx, a, d);
-            const size_t smem = dense_smem_bytes(d.table_words, d.threads / 32);
-            auto kern = aligned ? k_step_dense<DT, true> : k_step_dense<DT, false>;
-            if ((rc = ensure_smem(kern, smem)) != CFGZIP_OK) return rc;
-            rc = launch(ctx, kern, dim3(unsigned(d.n_groups_ub) * unsigned(d.S)), dim3(unsigned(d.threads)), smem, st, a);
+            const dim3 grid(unsigned(d.n_groups_ub) * unsigned(d.S)), block{unsigned(d.threads)};
+            if (d.depth) {
+                if ((rc = ensure_smem(k_step_dense_pipe<DT>, d.smem)) != CFGZIP_OK) return rc;
+                rc = launch(ctx, k_step_dense_pipe<DT>, grid, block, d.smem, st, a);
+            } else {
+                auto kern = k_step_dense<DT>;
+                if ((rc = ensure_smem(kern, d.smem)) != CFGZIP_OK) return rc;
+                rc = launch(ctx, kern, grid, block, d.smem, st, a);
+            }
         } else {
             rc = launch(ctx, k_step_generic<DT, true>, dim3(unsigned(a.B)), dim3(256), 0, st, a);
         }
@@ -534,19 +597,18 @@ int cfgzip_expand_mask(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row
             a.S = S;
             a.per_split = per_split;
             const size_t smem = size_t(per_split) * 4;
-            auto kern = k_step_sparse<kF32, false, false>;
+            auto kern = k_step_sparse<kF32, false>;
             if ((rc = ensure_smem(kern, smem)) != CFGZIP_OK) return rc;
             return launch(ctx, kern, dim3(unsigned(B) * unsigned(S)), dim3(256), smem, st, a);
         }
         return launch(ctx, k_step_generic<kF32, false>, dim3(unsigned(B)), dim3(256), 0, st, a);
     }
-    const DensePlan d = plan_dense(ctx, ps, B, mixed, ps.VW, 8, false);
+    const DensePlan d = plan_dense(ctx, ps, B, mixed, ps.VW, 8, false, 0);
     if (!d.ok) return launch(ctx, k_step_generic<kF32, false>, dim3(unsigned(B)), dim3(256), 0, st, a);
     if (d.use_plan_kernel && (rc = run_plan_kernel(ctx, row_part, B, ps.V, d, st)) != CFGZIP_OK) return rc;
     fill_groups(ctx, a, d);
-    const size_t smem = dense_smem_bytes(d.table_words, 0);
-    if ((rc = ensure_smem(k_expand_dense, smem)) != CFGZIP_OK) return rc;
-    return launch(ctx, k_expand_dense, dim3(unsigned(d.n_groups_ub) * unsigned(d.S)), dim3(256), smem, st, a);
+    if ((rc = ensure_smem(k_expand_dense, d.smem)) != CFGZIP_OK) return rc;
+    return launch(ctx, k_expand_dense, dim3(unsigned(d.n_groups_ub) * unsigned(d.S)), dim3(256), d.smem, st, a);
 }
 
 int cfgzip_mask_logits(cfgzip_ctx* ctx, void* logits, int dtype, int64_t row_stride_elems, int32_t B, int32_t V,
@@ -705,7 +767,7 @@ int cfgzip_poll_status(cfgzip_ctx* ctx, void* stream, int32_t* n_empty_rows, int
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return CFGZIP_E_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    int32_t h[3] = {0, 0, 0};
+    int32_t h[4] = {0, 0, 0, 0};
     if (cudaMemcpyAsync(h, ctx->d_status, sizeof h, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
         cudaMemsetAsync(ctx->d_status, 0, sizeof h, st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) {
         cudaGetLastError();
@@ -714,7 +776,7 @@ int cfgzip_poll_status(cfgzip_ctx* ctx, void* stream, int32_t* n_empty_rows, int
     if (n_empty_rows) *n_empty_rows = h[0];
     if (n_bad_tokens) *n_bad_tokens = h[1];
     if (n_bad_rows) *n_bad_rows = h[2];
-    return CFGZIP_OK;
+    return h[3] ? CFGZIP_E_CUDA : CFGZIP_OK;  // h[3]: asynchronous copies that never completed
 }
 
 int cfgzip_launch_count(cfgzip_ctx* ctx, int64_t* out) {
@@ -729,13 +791,21 @@ int cfgzip_set_tuning(cfgzip_ctx* ctx, const char* name, int32_t value) {
         if (value < 1 || value > 16) return CFGZIP_E_ARG;
         ctx->ctas_per_sm = value;
     } else if (!std::strcmp(name, "token_warps")) {
-        if (value < 0 || value > 8) return CFGZIP_E_ARG;
+        if (value < 0 || value > 16) return CFGZIP_E_ARG;
         ctx->token_warps = value;
     } else if (!std::strcmp(name, "row_warps")) {
         if (value != 0 && value != 1 && value != 2 && value != 4) return CFGZIP_E_ARG;
         ctx->row_warps = value;
     } else if (!std::strcmp(name, "pdl")) {
         ctx->pdl = value ? 1 : 0;
+    } else if (!std::strcmp(name, "pipeline")) {
+        ctx->pipeline = value ? 1 : 0;
+    } else if (!std::strcmp(name, "pipe_warps")) {
+        if (value != 4 && value != 8 && value != 12 && value != 16) return CFGZIP_E_ARG;
+        ctx->pipe_warps = value;
+    } else if (!std::strcmp(name, "pipe_depth")) {
+        if (value < 2 || value > 8) return CFGZIP_E_ARG;
+        ctx->pipe_depth = value;
     } else {
         return CFGZIP_E_ARG;
     }

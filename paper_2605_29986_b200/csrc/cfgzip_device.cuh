@@ -149,6 +149,9 @@ struct Octet<kBF16> {
     __device__ __forceinline__ void load(const void* row_base, int o) {
         v = ld_stream16(reinterpret_cast<const uint16_t*>(row_base) + 8 * int64_t(o));
     }
+    __device__ __forceinline__ void load_shared(const char* stage_row, int lane) {
+        v = *reinterpret_cast<const uint4*>(stage_row + lane * 16);
+    }
     __device__ __forceinline__ void store(void* row_base, int o) const {
         st_stream16(reinterpret_cast<uint16_t*>(row_base) + 8 * int64_t(o), v);
     }
@@ -178,6 +181,10 @@ struct Octet<kF32> {
         a = ld_stream16(p);
         b = ld_stream16(p + 4);
     }
+    __device__ __forceinline__ void load_shared(const char* stage_row, int lane) {
+        a = *reinterpret_cast<const uint4*>(stage_row + lane * 32);
+        b = *reinterpret_cast<const uint4*>(stage_row + lane * 32 + 16);
+    }
     __device__ __forceinline__ void store(void* row_base, int o) const {
         float* p = reinterpret_cast<float*>(row_base) + 8 * int64_t(o);
         st_stream16(p, a);
@@ -206,19 +213,85 @@ struct Octet<kF32> {
     }
 };
 
-// Fold one masked octet into a running per-row state.
-__device__ __forceinline__ void partial_add_octet(float& m, float& s, int& pos, const float (&f)[8], uint32_t byte,
-                                                  int position) {
-    const float vmax = fmaxf(fmaxf(fmaxf(f[0], f[1]), fmaxf(f[2], f[3])), fmaxf(fmaxf(f[4], f[5]), fmaxf(f[6], f[7])));
-    const bool upd = (vmax > m) || (byte != 0u && pos == kNoPos);
-    pos = upd ? position : pos;
-    const float ref_old = fmaxf(m, kRefFloor);
-    m = fmaxf(m, vmax);
-    const float ref = fmaxf(m, kRefFloor);
-    float acc = 0.f;
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
+// Running state of one row inside one thread. The sum is kept relative to a reference that
+// only moves when a value overtakes it by more than kRefSlack (so the common case is one
+// fused multiply-add and one ex2 per logit): s = sum 2^(z*log2e + nrl), nrl = -(ref*log2e).
+// pos is the position (octet index) of the first octet whose maximum is the row maximum m.
+constexpr float kRefSlack = 57.7f;  // in powers of two: 40 nats
+struct RowAcc {
+    float m, s, nrl;
+    int pos;
+    __device__ __forceinline__ void init() {
+        m = -INFINITY;
+        s = 0.f;
+        nrl = -(kRefFloor * kLog2e);
+        pos = kNoPos;
+    }
+    __device__ __forceinline__ void add_octet(const float (&f)[8], int position) {
+        const float vmax = fmax3(fmax3(f[0], f[1], f[2]), fmax3(f[3], f[4], f[5]), fmaxf(f[6], f[7]));
+        pos = vmax > m ? position : pos;
+        m = fmaxf(m, vmax);
+        if (fmaf(vmax, kLog2e, nrl) > kRefSlack) {  // rare: move the reference up to vmax
+            const float n2 = -(vmax * kLog2e);
+            s *= ex2f(n2 - nrl);
+            nrl = n2;
+        }
+        float acc = 0.f;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) acc += ex2f((f[j] - ref) * kLog2e);
-    s = fmaf(s, ex2f((ref_old - ref) * kLog2e), acc);
+        for (int j = 0; j < 8; ++j) acc += ex2f(fmaf(f[j], kLog2e, nrl));
+        s += acc;
+    }
+    // Bring the sum to the convention of Partial: relative to max(m, kRefFloor).
+    __device__ __forceinline__ Partial to_partial() const {
+        // nothing finite seen: the reference never moved off the floor and the sum is empty
+        if (!(m > kRefFloor)) return Partial{m, 0.f, pos, 0};
+        return Partial{m, s * ex2f(-fmaf(m, kLog2e, nrl)), pos, 0};
+    }
+};
+
+// ---- mbarrier + bulk asynchronous copy (global -> shared) wrappers, CTA scope ----------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_init_fence() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// One bounded attempt: returns true once the phase with the given parity has completed.
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(2000u)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait (about half a second at most); false means the copy never arrived.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    for (int it = 0; it < 250000; ++it)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+// size and both addresses are multiples of 16 bytes
+__device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_u32(dst_smem)),
+                 "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
 }
 
 }  // namespace cfgzip

@@ -33,9 +33,12 @@ struct StepArgs {
     int32_t per_split;          // octets (dense) or vocab-mask words (sparse) per CTA
     int32_t WT;                 // dense: warps side by side along the vocabulary
     int32_t table_words;        // dense: shared-memory words of the bit-sliced class table
+    int32_t stage_stride;       // dense: words per row of the class-mask staging area, 0 = no staging
+    int32_t depth;              // pipelined dense kernel: stages per warp
+    PartDev p0;                 // descriptor of part0 (saves a dependent load when rows do not mix partitions)
     Partial* partials;
     unsigned int* tickets;
-    int32_t* status;            // [0] empty rows, [1] bad tokens, [2] bad rows
+    int32_t* status;            // [0] empty rows, [1] bad tokens, [2] bad rows, [3] copies that never arrived
 };
 
 __device__ __forceinline__ void pdl_prologue() {
@@ -88,9 +91,17 @@ __device__ void finalize_row(const StepArgs& a, const PartDev& P, int row, float
     if (a.logp_argmax) a.logp_argmax[row] = lpa;
 }
 
+// Same for a whole warp whose lanes all hold the row's merged state (octet position): lanes
+// 0..7 test the 8 tokens of the winning octet side by side. A row without a position either
+// allows nothing or holds only -inf at its allowed tokens: the class lists give its lowest
+// allowed token. Needs first_allowed_share / write_row_outputs (defined below).
+template <int DT>
+__device__ __forceinline__ void warp_finalize_row(const StepArgs& a, const PartDev& P, int row, float m, float s,
+                                                  int pos, int lane);
+
 // Eight tokens handled one element at a time: ragged tail of a row, or unaligned logits.
 template <int DT>
-__device__ __noinline__ void octet_scalar(void* row_base, int o, int V, uint32_t byte, float (&f)[8]) {
+__device__ __forceinline__ void octet_scalar(void* row_base, int o, int V, uint32_t byte, float (&f)[8]) {
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         const int t = 8 * o + j;
@@ -119,29 +130,72 @@ __device__ __forceinline__ int group_rows_setup(const StepArgs& a, int g, int* s
     return a.group_part ? a.group_part[g] : a.part0;
 }
 
-// Bit-sliced class table of one row group: T[k] bit r = "row slot r allows class k".
-// Entries K .. 32*(KW+1)-1 are zero, so the padding class id K looks up "nobody".
-__device__ __forceinline__ void build_class_table(const StepArgs& a, const PartDev& P, const int* s_row, uint32_t* T,
+// Copy the class-mask rows of the group's 32 row slots to shared memory (`stage`, rows
+// stage_stride words apart). A warp takes one row at a time with coalesced loads, four rows
+// and two 32-word spans per pass, so up to eight loads per thread are in flight together.
+__device__ __forceinline__ void stage_class_masks(const StepArgs& a, const PartDev& P, const int* s_row, uint32_t* stage,
                                                   int warp, int lane, int n_warps) {
-    const int row = s_row[lane];
-    const uint32_t* cm = a.class_mask + int64_t(row < 0 ? 0 : row) * a.cm_stride;
-    for (int kw = warp; kw <= P.KW; kw += n_warps) {
-        uint32_t x = 0;
-        if (kw < P.KW && row >= 0) {
-            x = __ldg(cm + kw);
-            if (kw == P.KW - 1 && (P.K & 31)) x &= (1u << (P.K & 31)) - 1u;
+    for (int r0 = warp; r0 < kGroupRows; r0 += 4 * n_warps) {
+        for (int kw0 = lane; kw0 < P.KW; kw0 += 64) {
+            uint32_t v[4][2];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int r = r0 + q * n_warps;
+                const int row = r < kGroupRows ? s_row[r] : -1;
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int kw = kw0 + 32 * u;
+                    v[q][u] = (row >= 0 && kw < P.KW) ? __ldg(a.class_mask + int64_t(row) * a.cm_stride + kw) : 0u;
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int r = r0 + q * n_warps;
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int kw = kw0 + 32 * u;
+                    if (r < kGroupRows && kw < P.KW) stage[r * a.stage_stride + kw] = v[q][u];
+                }
+            }
         }
-        T[kw * 32 + lane] = warp_transpose32(x, lane);
     }
 }
 
-// Allow bits of rows 8*rb .. 8*rb+7 for the 8 tokens of octet o: byte i of (lo, hi)
-// belongs to row 8*rb + i, bit j of it to token 8*o + j.
-__device__ __forceinline__ void octet_allow_bits(const PartDev& P, const uint32_t* T, int o, int rb, bool active,
-                                                 uint32_t& lo, uint32_t& hi) {
+// Bit-sliced class table of one row group: T[k] bit r = "row slot r allows class k".
+// Entries K .. 32*(KW+1)-1 are zero, so the padding class id K looks up "nobody".
+// With a staging area (filled by stage_class_masks, then a block barrier) the 32x32 bit
+// blocks are read from shared memory; stage_stride is odd, so those column reads hit 32
+// banks. Without one, each lane reads its row's words from global memory, eight at a time.
+__device__ __forceinline__ void build_class_table(const StepArgs& a, const PartDev& P, const int* s_row, uint32_t* T,
+                                                  const uint32_t* stage, int warp, int lane, int n_warps) {
+    const uint32_t tail = (P.K & 31) ? (1u << (P.K & 31)) - 1u : 0xFFFFFFFFu;
+    const int row = s_row[lane];
+    const uint32_t* cm = a.class_mask + int64_t(row < 0 ? 0 : row) * a.cm_stride;
+    constexpr int U = 4;
+    for (int kw0 = warp; kw0 <= P.KW; kw0 += n_warps * U) {
+        uint32_t x[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int kw = kw0 + u * n_warps;
+            x[u] = 0u;
+            if (kw < P.KW && row >= 0) x[u] = a.stage_stride ? stage[lane * a.stage_stride + kw] : __ldg(cm + kw);
+            if (kw == P.KW - 1) x[u] &= tail;
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int kw = kw0 + u * n_warps;
+            const uint32_t t = warp_transpose32(x[u], lane);  // independent chains: their shuffles overlap
+            if (kw <= P.KW) T[kw * 32 + lane] = t;
+        }
+    }
+}
+
+// Allow bits of rows 8*rb .. 8*rb+7 for the 8 tokens whose class ids are packed in cv:
+// byte i of (lo, hi) belongs to row 8*rb + i, bit j of it to token j of the octet.
+__device__ __forceinline__ void octet_allow_bits(const uint4& cv, const uint32_t* T, int rb, bool active, uint32_t& lo,
+                                                 uint32_t& hi) {
     lo = hi = 0;
     if (!active) return;
-    const uint4 cv = __ldg(reinterpret_cast<const uint4*>(P.c16) + o);
     const uint32_t w0 = T[cv.x & 0xFFFFu], w1 = T[cv.x >> 16], w2 = T[cv.y & 0xFFFFu], w3 = T[cv.y >> 16];
     const uint32_t w4 = T[cv.z & 0xFFFFu], w5 = T[cv.z >> 16], w6 = T[cv.w & 0xFFFFu], w7 = T[cv.w >> 16];
     const uint32_t sel = uint32_t(rb) | (uint32_t(4 + rb) << 4);  // byte rb of both operands
@@ -150,87 +204,88 @@ __device__ __forceinline__ void octet_allow_bits(const PartDev& P, const uint32_
     transpose8x8(lo, hi);
 }
 
-// ---------------------------------------------------------------------------------------
-// Fused dense step: expand + mask in place + (max, sum-exp, position) per row.
-// Grid: n_groups * S thread blocks; block (g, split) owns octets [split*per_split, ...) of the
-// 32 rows of group g. Warps are arranged WT (along tokens) x WR (row batches of 8).
-// ---------------------------------------------------------------------------------------
-template <int DT, bool ALIGNED>
-__global__ void __launch_bounds__(256) k_step_dense(const __grid_constant__ StepArgs a) {
-    extern __shared__ __align__(16) uint32_t smem[];
-    uint32_t* T = smem;
-    int* s_row = reinterpret_cast<int*>(T + a.table_words);
-    Partial* red = reinterpret_cast<Partial*>(s_row + kGroupRows);
-    __shared__ int s_last;
-
-    pdl_prologue();
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, n_warps = blockDim.x >> 5;
-    const int g = blockIdx.x / a.S, split = blockIdx.x - g * a.S;
-    if (a.n_groups && g >= __ldg(a.n_groups)) return;
-    const int part = group_rows_setup(a, g, s_row, tid);
-    for (int i = tid; i < n_warps * kGroupRows; i += blockDim.x) red[i] = partial_empty();
-    __syncthreads();
-    const PartDev P = a.parts[part];
-    const int nrow = __popc(__ballot_sync(0xFFFFFFFFu, s_row[lane] >= 0));
-    build_class_table(a, P, s_row, T, warp, lane, n_warps);
-    __syncthreads();
-
-    const int wt = warp % a.WT, wr = warp / a.WT, WR = n_warps / a.WT;
-    const int n_octets = 4 * a.VW, n_full = a.V >> 3;
-    const int o_begin = split * a.per_split;
-    const int o_end = min(o_begin + a.per_split, n_octets);
-    constexpr int ES = DT == kBF16 ? 2 : 4;
-    uint8_t* vm8 = reinterpret_cast<uint8_t*>(a.vocab_mask);
-
-    for (int rb = wr; rb * kBatchRows < nrow; rb += WR) {
-        float m[kBatchRows], s[kBatchRows];
-        int pos[kBatchRows];
-        char* rowp[kBatchRows];
-        uint8_t* vmp[kBatchRows];
-#pragma unroll
-        for (int i = 0; i < kBatchRows; ++i) {
-            m[i] = -INFINITY; s[i] = 0.f; pos[i] = kNoPos;
-            const int row = s_row[min(rb * kBatchRows + i, kGroupRows - 1)];
-            rowp[i] = reinterpret_cast<char*>(a.logits) + int64_t(max(row, 0)) * a.row_stride * ES;
-            vmp[i] = vm8 ? vm8 + int64_t(max(row, 0)) * a.vm_stride * 4 : nullptr;
-        }
-        const int live = min(kBatchRows, nrow - rb * kBatchRows);
-
-        for (int o0 = o_begin + wt * 32; o0 < o_end; o0 += a.WT * 32) {
-            const int o = o0 + lane;
-            const bool active = o < o_end;
-            const bool vec = ALIGNED && o < n_full;
-            Octet<DT> oc[kBatchRows];
-#pragma unroll
-            for (int i = 0; i < kBatchRows; ++i)
-                if (i < live && active && vec) oc[i].load(rowp[i], o);
-            uint32_t lo, hi;
-            octet_allow_bits(P, T, o, rb, active, lo, hi);
-#pragma unroll
-            for (int i = 0; i < kBatchRows; ++i) {
-                if (i < live && active) {
-                    const uint32_t byte = ((i < 4 ? lo : hi) >> (8 * (i & 3))) & 0xFFu;
-                    float f[8];
-                    if (vec) {
-                        oc[i].mask(byte, f);
-                        oc[i].store(rowp[i], o);
-                    } else {
-                        octet_scalar<DT>(rowp[i], o, a.V, byte, f);
-                    }
-                    if (vmp[i]) vmp[i][o] = uint8_t(byte);
-                    partial_add_octet(m[i], s[i], pos[i], f, byte, o);
-                }
-            }
-        }
-#pragma unroll
-        for (int i = 0; i < kBatchRows; ++i) {
-            partial_warp_allreduce(m[i], s[i], pos[i]);
-            if (lane == 0 && i < live) red[warp * kGroupRows + rb * kBatchRows + i] = Partial{m[i], s[i], pos[i], 0};
+// Lowest allowed token of a row, found from the class side: the first member of every allowed
+// class (the member lists are ascending), minimum over the classes this caller looks at
+// (words l, l+n, ... of the class mask). Returns (token << 32) | representative, ~0 if none.
+// Only rows whose allowed logits are all -inf (or that allow nothing) come here.
+__device__ __forceinline__ unsigned long long first_allowed_share(const StepArgs& a, const PartDev& P, int row, int l,
+                                                                  int n) {
+    unsigned long long best = ~0ull;
+    const uint32_t* cm = a.class_mask + int64_t(row) * a.cm_stride;
+    for (int kw = l; kw < P.KW; kw += n) {
+        uint32_t w = cm[kw];
+        if (kw == P.KW - 1 && (P.K & 31)) w &= (1u << (P.K & 31)) - 1u;
+        while (w) {
+            const int k = kw * 32 + __ffs(w) - 1;
+            w &= w - 1u;
+            const unsigned long long cand =
+                (static_cast<unsigned long long>(P.tok[P.off[k]]) << 32) | static_cast<unsigned int>(P.r[k]);
+            best = cand < best ? cand : best;
         }
     }
-    __syncthreads();
+    return best;
+}
 
-    // one thread per row slot folds the warps' results
+__device__ __forceinline__ void write_row_outputs(const StepArgs& a, int row, float m, float s, unsigned long long pick) {
+    int tok = -1, repv = -1;
+    float lsev = -INFINITY, lpa = -INFINITY;
+    if (pick != ~0ull) {
+        tok = int(pick >> 32);
+        repv = int(pick & 0xFFFFFFFFull);
+        if (m > kRefFloor && s > 0.f) {
+            const float l = logf(s);
+            lsev = m + l;
+            lpa = -l;
+        }
+    } else {
+        atomicAdd(a.status + 0, 1);
+    }
+    a.argmax[row] = tok;
+    if (a.rep) a.rep[row] = repv;
+    if (a.lse) a.lse[row] = lsev;
+    if (a.logp_argmax) a.logp_argmax[row] = lpa;
+}
+
+template <int DT>
+__device__ __forceinline__ void warp_finalize_row(const StepArgs& a, const PartDev& P, int row, float m, float s,
+                                                  int pos, int lane) {
+    unsigned long long cand = ~0ull;
+    if (pos == kNoPos) {
+        cand = first_allowed_share(a, P, row, lane, 32);
+    } else {
+        const int t = 8 * pos + lane;
+        if (lane < 8 && t < a.V) {
+            const float z = ldcg_elem<DT>(reinterpret_cast<const char*>(a.logits) + int64_t(row) * a.row_stride * (DT == kBF16 ? 2 : 4), t);
+            const int k = P.c32[t];
+            const uint32_t word = a.class_mask[int64_t(row) * a.cm_stride + (k >> 5)];
+            const int repv = P.r[k];
+            if (((word >> (k & 31)) & 1u) && z == m) cand = (static_cast<unsigned long long>(t) << 32) | static_cast<unsigned int>(repv);
+        }
+    }
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+        const unsigned long long other = __shfl_xor_sync(0xFFFFFFFFu, cand, d);
+        cand = other < cand ? other : cand;
+    }
+    if (lane == 0) write_row_outputs(a, row, m, s, cand);
+}
+
+// Shared-memory scratch of the end of a dense block.
+struct DenseTail {
+    int last;
+    Partial fin[kGroupRows];
+    unsigned long long pick[kGroupRows];  // (token id << 32) | representative of the best match
+};
+
+// End of a dense block: every warp has left the states of the rows it streamed in
+// red[warp][row slot]. Fold them, publish / collect across the S blocks of the group, then
+// turn each complete row state into the row's outputs.
+template <int DT>
+__device__ __forceinline__ void dense_block_tail(const StepArgs& a, const PartDev& P, int g, int split, const int* s_row,
+                                                 int nrow, Partial* red, DenseTail& tl) {
+    constexpr int ES = DT == kBF16 ? 2 : 4;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, n_warps = blockDim.x >> 5;
+    __syncthreads();
     float rm = -INFINITY, rs = 0.f;
     int rpos = kNoPos;
     if (tid < kGroupRows) {
@@ -239,31 +294,373 @@ __global__ void __launch_bounds__(256) k_step_dense(const __grid_constant__ Step
             partial_merge(rm, rs, rpos, p.m, p.s, p.pos);
         }
     }
-    if (a.S == 1) {
-        if (tid < kGroupRows) finalize_row<DT>(a, P, s_row[tid], rm, rs, rpos, false);
-        return;
-    }
-    // several blocks share the group: publish, and let the last one to arrive finish the rows
-    if (tid < kGroupRows)
-        a.partials[(int64_t(g) * kGroupRows + tid) * a.S + split] = Partial{rm, rs, rpos, 0};
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) s_last = (atomicAdd(a.tickets + g, 1u) == unsigned(a.S - 1));
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    for (int j = warp; j < nrow; j += n_warps) {
-        float m2 = -INFINITY, s2 = 0.f;
-        int p2 = kNoPos;
-        const Partial* src = a.partials + (int64_t(g) * kGroupRows + j) * a.S;
-        for (int sp = lane; sp < a.S; sp += 32) {
-            const int4 raw = __ldcg(reinterpret_cast<const int4*>(src + sp));
-            partial_merge(m2, s2, p2, __int_as_float(raw.x), __int_as_float(raw.y), raw.z);
+    if (a.S > 1) {
+        // several blocks share the group: publish, and let the last one to arrive finish the rows
+        if (tid < kGroupRows)
+            a.partials[(int64_t(g) * a.S + split) * kGroupRows + tid] = Partial{rm, rs, rpos, 0};
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) tl.last = (atomicAdd(a.tickets + g, 1u) == unsigned(a.S - 1));
+        __syncthreads();
+        if (!tl.last) return;
+        __threadfence();
+        // every thread folds a strided share of the S published states of its row slot
+        const Partial* src = a.partials + int64_t(g) * a.S * kGroupRows + lane;
+        rm = -INFINITY; rs = 0.f; rpos = kNoPos;
+#pragma unroll 8
+        for (int sp = warp; sp < a.S; sp += n_warps) {
+            const int4 raw = __ldcg(reinterpret_cast<const int4*>(src + sp * kGroupRows));
+            partial_merge(rm, rs, rpos, __int_as_float(raw.x), __int_as_float(raw.y), raw.z);
         }
-        partial_warp_allreduce(m2, s2, p2);
-        if (lane == 0) finalize_row<DT>(a, P, s_row[j], m2, s2, p2, false);
+        red[warp * kGroupRows + lane] = Partial{rm, rs, rpos, 0};
+        __syncthreads();
+        rm = -INFINITY; rs = 0.f; rpos = kNoPos;
+        if (tid < kGroupRows) {
+            for (int w = 0; w < n_warps; ++w) {
+                const Partial p = red[w * kGroupRows + tid];
+                partial_merge(rm, rs, rpos, p.m, p.s, p.pos);
+            }
+        }
+        if (tid == 0) a.tickets[g] = 0u;
     }
-    if (tid == 0) a.tickets[g] = 0u;
+    // rows are complete: 8 threads per row look at the 8 tokens of the winning octet at once and
+    // fetch each candidate's representative alongside, so nothing is left to load afterwards
+    if (tid < kGroupRows) {
+        tl.fin[tid] = Partial{rm, rs, rpos, 0};
+        tl.pick[tid] = ~0ull;
+    }
+    __syncthreads();
+    for (int idx = tid; idx < nrow * 8; idx += blockDim.x) {
+        const int j = idx >> 3;
+        const Partial p = tl.fin[j];
+        const int row = s_row[j];
+        if (p.pos == kNoPos) {
+            const unsigned long long cand = first_allowed_share(a, P, row, idx & 7, 8);
+            if (cand != ~0ull) atomicMin(tl.pick + j, cand);
+            continue;
+        }
+        const int t = 8 * p.pos + (idx & 7);
+        if (t < a.V) {
+            const float z = ldcg_elem<DT>(reinterpret_cast<const char*>(a.logits) + int64_t(row) * a.row_stride * ES, t);
+            const int k = P.c32[t];
+            const uint32_t word = a.class_mask[int64_t(row) * a.cm_stride + (k >> 5)];
+            const int repv = P.r[k];
+            if (((word >> (k & 31)) & 1u) && z == p.m)
+                atomicMin(tl.pick + j, (static_cast<unsigned long long>(t) << 32) | static_cast<unsigned int>(repv));
+        }
+    }
+    __syncthreads();
+    if (tid < nrow) write_row_outputs(a, s_row[tid], tl.fin[tid].m, tl.fin[tid].s, tl.pick[tid]);
+}
+
+// One whole-vector octet of one row: mask, write back, note the vocab-mask byte, fold into the
+// row state.
+template <int DT>
+__device__ __forceinline__ void dense_octet_row(Octet<DT>& oc, char* rowp, uint8_t* vmp, int o, uint32_t byte,
+                                                RowAcc& acc) {
+    float f[8];
+    oc.mask(byte, f);
+    oc.store(rowp, o);
+    if (vmp) vmp[o] = uint8_t(byte);
+    acc.add_octet(f, o);
+}
+
+// The octets past the last whole vector of a row (the ragged one when V is not a multiple of
+// 8, and the padding octets up to the end of the last vocab-mask word): at most four, taken
+// by lanes 0..3 of one warp per row batch, element by element.
+template <int DT>
+__device__ __forceinline__ void dense_tail_octets(const StepArgs& a, const PartDev& P, const uint32_t* T, int rb, int live,
+                                                  int o_first, int o_end, int lane, char* const (&rowp)[kBatchRows],
+                                                  uint8_t* const (&vmp)[kBatchRows], RowAcc (&acc)[kBatchRows]) {
+    const int o = o_first + lane;
+    const bool active = o < o_end;
+    uint4 cv = make_uint4(0, 0, 0, 0);
+    if (active) cv = __ldg(reinterpret_cast<const uint4*>(P.c16) + o);
+    uint32_t lo, hi;
+    octet_allow_bits(cv, T, rb, active, lo, hi);
+#pragma unroll
+    for (int i = 0; i < kBatchRows; ++i) {
+        if (i < live && active) {
+            const uint32_t byte = ((i < 4 ? lo : hi) >> (8 * (i & 3))) & 0xFFu;
+            float f[8];
+            octet_scalar<DT>(rowp[i], o, a.V, byte, f);
+            if (vmp[i]) vmp[i][o] = uint8_t(byte);
+            acc[i].add_octet(f, o);
+        }
+    }
+}
+
+// Reduce the 8 row states of a warp over its 32 lanes and leave them in red_warp[8*rb + i].
+// Recursive halving: lanes first trade half of their rows with the lane 16 away and fold the
+// half they keep, then 2 of 4 with the lane 8 away, then 1 of 2; two butterfly steps finish
+// the single row left (nine folds instead of forty).
+__device__ __forceinline__ void warp_rows_to_red(RowAcc (&acc)[kBatchRows], int live, Partial* red_warp, int rb, int lane) {
+    Partial p[kBatchRows];
+#pragma unroll
+    for (int i = 0; i < kBatchRows; ++i) p[i] = acc[i].to_partial();
+#pragma unroll
+    for (int half = 4; half >= 1; half >>= 1) {
+        const int d = 4 * half;  // 16, 8, 4
+        const bool up = lane & d;
+#pragma unroll
+        for (int k = 0; k < half; ++k) {
+            const Partial keep = up ? p[k + half] : p[k];
+            const Partial send = up ? p[k] : p[k + half];
+            const float m2 = __shfl_xor_sync(0xFFFFFFFFu, send.m, d);
+            const float s2 = __shfl_xor_sync(0xFFFFFFFFu, send.s, d);
+            const int p2 = __shfl_xor_sync(0xFFFFFFFFu, send.pos, d);
+            p[k] = keep;
+            partial_merge(p[k].m, p[k].s, p[k].pos, m2, s2, p2);
+        }
+    }
+#pragma unroll
+    for (int d = 2; d >= 1; d >>= 1) {
+        const float m2 = __shfl_xor_sync(0xFFFFFFFFu, p[0].m, d);
+        const float s2 = __shfl_xor_sync(0xFFFFFFFFu, p[0].s, d);
+        const int p2 = __shfl_xor_sync(0xFFFFFFFFu, p[0].pos, d);
+        partial_merge(p[0].m, p[0].s, p[0].pos, m2, s2, p2);
+    }
+    const int i = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);  // the row this lane ended with
+    if ((lane & 3) == 0 && i < live) red_warp[rb * kBatchRows + i] = p[0];  // a warp visits a row batch once
+}
+
+// ---------------------------------------------------------------------------------------
+// Fused dense step, register version: expand + mask in place + (max, sum-exp, position) per
+// row, logits fetched with 16-byte loads straight into registers (rows 16-byte aligned).
+// Grid: n_groups * S thread blocks; block (g, split) owns octets [split*per_split, ...) of the
+// 32 rows of group g. Warps are arranged WT (along tokens) x WR (row batches of 8).
+// ---------------------------------------------------------------------------------------
+template <int DT>
+__global__ void __launch_bounds__(256) k_step_dense(const __grid_constant__ StepArgs a) {
+    extern __shared__ __align__(128) uint32_t smem[];
+    uint32_t* T = smem;
+    int* s_row = reinterpret_cast<int*>(T + a.table_words);
+    Partial* red = reinterpret_cast<Partial*>(s_row + kGroupRows);
+    uint32_t* stage = reinterpret_cast<uint32_t*>(red + (blockDim.x >> 5) * kGroupRows);
+    __shared__ DenseTail tl;
+
+    pdl_prologue();
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, n_warps = blockDim.x >> 5;
+    const int g = blockIdx.x / a.S, split = blockIdx.x - g * a.S;
+    if (a.n_groups && g >= __ldg(a.n_groups)) return;
+    const int part = group_rows_setup(a, g, s_row, tid);
+    for (int i = tid; i < n_warps * kGroupRows; i += blockDim.x) red[i] = partial_empty();
+    __syncthreads();
+    const PartDev P = a.group_part ? a.parts[part] : a.p0;
+    const int nrow = __popc(__ballot_sync(0xFFFFFFFFu, s_row[lane] >= 0));
+    if (a.stage_stride) {
+        stage_class_masks(a, P, s_row, stage, warp, lane, n_warps);
+        __syncthreads();
+    }
+    build_class_table(a, P, s_row, T, stage, warp, lane, n_warps);
+    __syncthreads();
+
+    const int wt = warp % a.WT, wr = warp / a.WT, WR = n_warps / a.WT;
+    const int n_octets = 4 * a.VW, n_full = a.V >> 3;
+    const int o_begin = split * a.per_split;
+    const int o_end = min(o_begin + a.per_split, n_octets);
+    const int o_vec_end = min(o_end, n_full);
+    constexpr int ES = DT == kBF16 ? 2 : 4;
+    uint8_t* vm8 = reinterpret_cast<uint8_t*>(a.vocab_mask);
+
+    for (int rb = wr; rb * kBatchRows < nrow; rb += WR) {
+        RowAcc acc[kBatchRows];
+        char* rowp[kBatchRows];
+        uint8_t* vmp[kBatchRows];
+#pragma unroll
+        for (int i = 0; i < kBatchRows; ++i) {
+            acc[i].init();
+            const int row = s_row[min(rb * kBatchRows + i, kGroupRows - 1)];
+            rowp[i] = reinterpret_cast<char*>(a.logits) + int64_t(max(row, 0)) * a.row_stride * ES;
+            vmp[i] = vm8 ? vm8 + int64_t(max(row, 0)) * a.vm_stride * 4 : nullptr;
+        }
+        const int live = min(kBatchRows, nrow - rb * kBatchRows);
+
+        for (int o0 = o_begin + wt * 32; o0 < o_vec_end; o0 += a.WT * 32) {
+            const int o = o0 + lane;
+            const bool active = o < o_vec_end;
+            Octet<DT> oc[kBatchRows];
+#pragma unroll
+            for (int i = 0; i < kBatchRows; ++i)
+                if (i < live && active) oc[i].load(rowp[i], o);
+            uint32_t lo, hi;
+            uint4 cv = make_uint4(0, 0, 0, 0);
+            if (active) cv = __ldg(reinterpret_cast<const uint4*>(P.c16) + o);
+            octet_allow_bits(cv, T, rb, active, lo, hi);
+#pragma unroll
+            for (int i = 0; i < kBatchRows; ++i) {
+                if (i < live && active) {
+                    const uint32_t byte = ((i < 4 ? lo : hi) >> (8 * (i & 3))) & 0xFFu;
+                    dense_octet_row<DT>(oc[i], rowp[i], vmp[i], o, byte, acc[i]);
+                }
+            }
+        }
+        if (wt == 0 && o_end > n_full)
+            dense_tail_octets<DT>(a, P, T, rb, live, max(o_begin, n_full), o_end, lane, rowp, vmp, acc);
+        warp_rows_to_red(acc, live, red + warp * kGroupRows, rb, lane);
+    }
+    dense_block_tail<DT>(a, P, g, split, s_row, nrow, red, tl);
+}
+
+// ---------------------------------------------------------------------------------------
+// Fused dense step, pipelined version. Same decomposition as above, but the logits reach the
+// SM through bulk asynchronous copies: every warp runs its own ring of `depth` stages in
+// shared memory, each stage holding 32 octets of 8 rows plus the 32 octets of class ids,
+// filled by copies that lane 0 issues `depth` work items ahead and that signal an mbarrier.
+// The first copies are started before the class table is built. The lanes read their 16
+// bytes per row from shared memory, so no registers wait on memory and the copies of later
+// items overlap the arithmetic of this one. Masked logits go back with 16-byte stores.
+// ---------------------------------------------------------------------------------------
+template <int DT>
+struct PipeGeom {
+    static constexpr int kOctetBytes = DT == kBF16 ? 16 : 32;
+    static constexpr int kRowBytes = 32 * kOctetBytes;                   // one row of a stage
+    static constexpr int kStageBytes = kBatchRows * kRowBytes + 32 * 16;  // + class ids of 32 octets
+};
+
+template <int DT>
+__global__ void __launch_bounds__(512) k_step_dense_pipe(const __grid_constant__ StepArgs a) {
+    using G = PipeGeom<DT>;
+    extern __shared__ __align__(128) uint32_t smem[];
+    uint32_t* T = smem;
+    int* s_row = reinterpret_cast<int*>(T + a.table_words);
+    Partial* red = reinterpret_cast<Partial*>(s_row + kGroupRows);
+    const int n_warps = blockDim.x >> 5;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(red + n_warps * kGroupRows);  // n_warps * depth
+    char* ring = reinterpret_cast<char*>(bars) + ((n_warps * a.depth * 8 + 127) & ~127);  // keeps 128-byte alignment
+    uint32_t* stage = reinterpret_cast<uint32_t*>(ring + size_t(n_warps) * a.depth * G::kStageBytes);
+    __shared__ DenseTail tl;
+
+    pdl_prologue();
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int g = blockIdx.x / a.S, split = blockIdx.x - g * a.S;
+    if (a.n_groups && g >= __ldg(a.n_groups)) return;
+    const int part = group_rows_setup(a, g, s_row, tid);
+    for (int i = tid; i < n_warps * kGroupRows; i += blockDim.x) red[i] = partial_empty();
+    __syncthreads();
+    const PartDev P = a.group_part ? a.parts[part] : a.p0;
+    const int nrow = __popc(__ballot_sync(0xFFFFFFFFu, s_row[lane] >= 0));
+
+    const int wt = warp % a.WT, wr = warp / a.WT, WR = n_warps / a.WT;
+    const int n_octets = 4 * a.VW, n_full = a.V >> 3;
+    const int o_begin = split * a.per_split;
+    const int o_end = min(o_begin + a.per_split, n_octets);
+    const int o_vec_end = min(o_end, n_full);
+    constexpr int ES = DT == kBF16 ? 2 : 4;
+    uint8_t* vm8 = reinterpret_cast<uint8_t*>(a.vocab_mask);
+    char* my_ring = ring + size_t(warp) * a.depth * G::kStageBytes;
+    uint64_t* bar = bars + warp * a.depth;
+
+    // this warp's work items: row batches rb = wr, wr+WR, ... (outer) x chunks of 32 whole-vector octets (inner)
+    const int first_chunk = o_begin + wt * 32;
+    const int chunk_step = a.WT * 32;
+    const int n_chunks = first_chunk < o_vec_end ? (o_vec_end - first_chunk + chunk_step - 1) / chunk_step : 0;
+    const int n_rb = (nrow > wr * kBatchRows) ? ((nrow - wr * kBatchRows + WR * kBatchRows - 1) / (WR * kBatchRows)) : 0;
+    const int n_items = n_chunks * n_rb;
+
+    auto issue = [&](int n) {  // lane 0 only: start the copies of work item n into slot n % depth
+        const int rb = wr + (n / n_chunks) * WR;
+        const int o0 = first_chunk + (n % n_chunks) * chunk_step;
+        const int slot = n % a.depth;
+        char* dst = my_ring + size_t(slot) * G::kStageBytes;
+        const int live = min(kBatchRows, nrow - rb * kBatchRows);
+        const uint32_t nvec = uint32_t(min(o_vec_end - o0, 32));  // >= 1 by construction of the chunk list
+        const uint32_t row_bytes = nvec * G::kOctetBytes;
+        mbar_expect_tx(bar + slot, uint32_t(live) * row_bytes + nvec * 16u);
+        bulk_g2s(dst + kBatchRows * G::kRowBytes, reinterpret_cast<const char*>(P.c16) + size_t(o0) * 16, nvec * 16u, bar + slot);
+        for (int i = 0; i < live; ++i) {
+            const int row = s_row[rb * kBatchRows + i];
+            bulk_g2s(dst + i * G::kRowBytes,
+                     reinterpret_cast<const char*>(a.logits) + (int64_t(row) * a.row_stride * ES + int64_t(o0) * 8 * ES), row_bytes,
+                     bar + slot);
+        }
+    };
+
+    if (lane == 0) {
+        for (int d = 0; d < a.depth; ++d) mbar_init(bar + d, 1);
+        mbar_init_fence();
+        for (int n = 0; n < min(a.depth, n_items); ++n) issue(n);  // in flight while the table is built
+    }
+    if (a.stage_stride) {
+        stage_class_masks(a, P, s_row, stage, warp, lane, n_warps);
+        __syncthreads();
+    }
+    build_class_table(a, P, s_row, T, stage, warp, lane, n_warps);
+    __syncthreads();
+
+    bool failed = false;
+    int n = 0;
+    for (int rbi = 0; rbi < n_rb && !failed; ++rbi) {
+        const int rb = wr + rbi * WR;
+        RowAcc acc[kBatchRows];
+        char* rowp[kBatchRows];
+        uint8_t* vmp[kBatchRows];
+#pragma unroll
+        for (int i = 0; i < kBatchRows; ++i) {
+            acc[i].init();
+            const int row = s_row[min(rb * kBatchRows + i, kGroupRows - 1)];
+            rowp[i] = reinterpret_cast<char*>(a.logits) + int64_t(max(row, 0)) * a.row_stride * ES;
+            vmp[i] = vm8 ? vm8 + int64_t(max(row, 0)) * a.vm_stride * 4 : nullptr;
+        }
+        const int live = min(kBatchRows, nrow - rb * kBatchRows);
+        for (int ci = 0; ci < n_chunks; ++ci, ++n) {
+            const int slot = n % a.depth;
+            const bool arrived = mbar_wait(bar + slot, uint32_t(n / a.depth) & 1u);
+            if (!__all_sync(0xFFFFFFFFu, arrived)) {
+                failed = true;
+                break;
+            }
+            const char* src = my_ring + size_t(slot) * G::kStageBytes;
+            const int o = first_chunk + ci * chunk_step + lane;
+            const bool active = o < o_vec_end;
+            uint4 cv = make_uint4(0, 0, 0, 0);
+            if (active) cv = *reinterpret_cast<const uint4*>(src + kBatchRows * G::kRowBytes + lane * 16);
+            uint32_t lo, hi;
+            octet_allow_bits(cv, T, rb, active, lo, hi);
+#pragma unroll
+            for (int i = 0; i < kBatchRows; ++i) {
+                if (i < live && active) {
+                    Octet<DT> oc;
+                    oc.load_shared(src + i * G::kRowBytes, lane);
+                    const uint32_t byte = ((i < 4 ? lo : hi) >> (8 * (i & 3))) & 0xFFu;
+                    dense_octet_row<DT>(oc, rowp[i], vmp[i], o, byte, acc[i]);
+                }
+            }
+            __syncwarp();  // every lane has its data out of the slot before it is refilled
+            if (lane == 0 && n + a.depth < n_items) issue(n + a.depth);
+        }
+        if (failed) break;
+        if (wt == 0 && o_end > n_full)
+            dense_tail_octets<DT>(a, P, T, rb, live, max(o_begin, n_full), o_end, lane, rowp, vmp, acc);
+        warp_rows_to_red(acc, live, red + warp * kGroupRows, rb, lane);
+    }
+    // a warp without whole-vector chunks may still own the tail octets of its row batches
+    if (n_chunks == 0 && wt == 0 && o_end > n_full) {
+        for (int rb = wr; rb * kBatchRows < nrow; rb += WR) {
+            RowAcc acc[kBatchRows];
+            char* rowp[kBatchRows];
+            uint8_t* vmp[kBatchRows];
+#pragma unroll
+            for (int i = 0; i < kBatchRows; ++i) {
+                acc[i].init();
+                const int row = s_row[min(rb * kBatchRows + i, kGroupRows - 1)];
+                rowp[i] = reinterpret_cast<char*>(a.logits) + int64_t(max(row, 0)) * a.row_stride * ES;
+                vmp[i] = vm8 ? vm8 + int64_t(max(row, 0)) * a.vm_stride * 4 : nullptr;
+            }
+            const int live = min(kBatchRows, nrow - rb * kBatchRows);
+            dense_tail_octets<DT>(a, P, T, rb, live, max(o_begin, n_full), o_end, lane, rowp, vmp, acc);
+            warp_rows_to_red(acc, live, red + warp * kGroupRows, rb, lane);
+        }
+    }
+    if (failed) {
+        // a copy never arrived: flag it, give the copies still in flight the same bounded time to land
+        // (they target this block's shared memory), and let the block leave without results
+        if (lane == 0) {
+            atomicAdd(a.status + 3, 1);
+            for (int k = n; k < min(n + a.depth, n_items); ++k) mbar_wait(bar + k % a.depth, uint32_t(k / a.depth) & 1u);
+        }
+    }
+    dense_block_tail<DT>(a, P, g, split, s_row, nrow, red, tl);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -271,9 +668,10 @@ __global__ void __launch_bounds__(256) k_step_dense(const __grid_constant__ Step
 // Same grid and row groups as the fused kernel; per_split counts 32-token words here.
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) k_expand_dense(const __grid_constant__ StepArgs a) {
-    extern __shared__ __align__(16) uint32_t smem[];
+    extern __shared__ __align__(128) uint32_t smem[];
     uint32_t* T = smem;
     int* s_row = reinterpret_cast<int*>(T + a.table_words);
+    uint32_t* stage = reinterpret_cast<uint32_t*>(s_row + kGroupRows);
 
     pdl_prologue();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, n_warps = blockDim.x >> 5;
@@ -281,9 +679,13 @@ __global__ void __launch_bounds__(256) k_expand_dense(const __grid_constant__ St
     if (a.n_groups && g >= __ldg(a.n_groups)) return;
     const int part = group_rows_setup(a, g, s_row, tid);
     __syncthreads();
-    const PartDev P = a.parts[part];
+    const PartDev P = a.group_part ? a.parts[part] : a.p0;
     const int nrow = __popc(__ballot_sync(0xFFFFFFFFu, s_row[lane] >= 0));
-    build_class_table(a, P, s_row, T, warp, lane, n_warps);
+    if (a.stage_stride) {
+        stage_class_masks(a, P, s_row, stage, warp, lane, n_warps);
+        __syncthreads();
+    }
+    build_class_table(a, P, s_row, T, stage, warp, lane, n_warps);
     __syncthreads();
 
     const int w_begin = split * a.per_split, w_end = min(w_begin + a.per_split, a.VW);
@@ -328,9 +730,9 @@ __device__ __forceinline__ int lower_bound_tok(const int32_t* tok, int lo, int h
     return lo;
 }
 
-template <int DT, bool FUSED, bool ALIGNED>
+template <int DT, bool FUSED>
 __global__ void __launch_bounds__(256) k_step_sparse(const __grid_constant__ StepArgs a) {
-    extern __shared__ __align__(16) uint32_t smem[];
+    extern __shared__ __align__(128) uint32_t smem[];
     uint32_t* bits = smem;  // per_split words
     __shared__ int s_big[kBigListCap];
     __shared__ int s_nbig;
@@ -405,48 +807,60 @@ __global__ void __launch_bounds__(256) k_step_sparse(const __grid_constant__ Ste
     char* rowp = reinterpret_cast<char*>(a.logits) + int64_t(row) * a.row_stride * ES;
     const uint8_t* bytes = reinterpret_cast<const uint8_t*>(bits);
     const int o_begin = 4 * w_begin, o_end = 4 * w_end, n_full = a.V >> 3;
-    float m = -INFINITY, s = 0.f;
-    int pos = kNoPos;
+    const int o_vec_end = min(o_end, n_full);
+    RowAcc acc;
+    acc.init();
     constexpr int U = 4;
-    for (int ob = o_begin + tid; ob < o_end; ob += U * blockDim.x) {
+    for (int ob = o_begin + tid; ob < o_vec_end; ob += U * blockDim.x) {
         Octet<DT> oc[U];
         uint32_t byte[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int o = ob + u * blockDim.x;
-            byte[u] = o < o_end ? bytes[o - o_begin] : 0u;
-            if (o < o_end && byte[u] && ALIGNED && o < n_full) oc[u].load(rowp, o);
+            byte[u] = o < o_vec_end ? bytes[o - o_begin] : 0u;
+            if (byte[u]) oc[u].load(rowp, o);  // octets without an allowed token are never read
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int o = ob + u * blockDim.x;
-            if (o >= o_end) continue;
-            if (ALIGNED && o < n_full) {
-                if (byte[u] == 0u) {
-                    oc[u].fill_neg_inf();
-                    oc[u].store(rowp, o);
-                } else {
-                    float f[8];
-                    oc[u].mask(byte[u], f);
-                    if (byte[u] != 0xFFu) oc[u].store(rowp, o);
-                    partial_add_octet(m, s, pos, f, byte[u], o);
-                }
+            if (o >= o_vec_end) continue;
+            if (byte[u] == 0u) {
+                oc[u].fill_neg_inf();
+                oc[u].store(rowp, o);
             } else {
                 float f[8];
-                octet_scalar<DT>(rowp, o, a.V, byte[u], f);
-                if (byte[u]) partial_add_octet(m, s, pos, f, byte[u], o);
+                oc[u].mask(byte[u], f);
+                if (byte[u] != 0xFFu) oc[u].store(rowp, o);
+                acc.add_octet(f, o);
             }
         }
     }
+    // octets past the last whole vector (ragged end of the row, padding of the last mask word)
+    if (o_end > n_full) {
+        const int o = max(o_begin, n_full) + tid;
+        if (o < o_end) {
+            float f[8];
+            const uint32_t byte = bytes[o - o_begin];
+            octet_scalar<DT>(rowp, o, a.V, byte, f);
+            if (byte) acc.add_octet(f, o);
+        }
+    }
+    const Partial mine = acc.to_partial();
+    float m = mine.m, s = mine.s;
+    int pos = mine.pos;
     partial_warp_allreduce(m, s, pos);
     if (lane == 0) s_red[warp] = Partial{m, s, pos, 0};
     __threadfence();  // the row's masked logits must be visible to whichever block finishes the row
     __syncthreads();
-    if (tid == 0) {
-        for (int w = 1; w < n_warps; ++w) partial_merge(m, s, pos, s_red[w].m, s_red[w].s, s_red[w].pos);
+    if (warp == 0) {
+        if (lane == 0)
+            for (int w = 1; w < n_warps; ++w) partial_merge(m, s, pos, s_red[w].m, s_red[w].s, s_red[w].pos);
         if (a.S == 1) {
-            finalize_row<DT>(a, P, row, m, s, pos, false);
-        } else {
+            m = __shfl_sync(0xFFFFFFFFu, m, 0);
+            s = __shfl_sync(0xFFFFFFFFu, s, 0);
+            pos = __shfl_sync(0xFFFFFFFFu, pos, 0);
+            warp_finalize_row<DT>(a, P, row, m, s, pos, lane);
+        } else if (lane == 0) {
             a.partials[int64_t(row) * a.S + split] = Partial{m, s, pos, 0};
             __threadfence();
             s_last = (atomicAdd(a.tickets + row, 1u) == unsigned(a.S - 1));
@@ -463,10 +877,8 @@ __global__ void __launch_bounds__(256) k_step_sparse(const __grid_constant__ Ste
         partial_merge(m2, s2, p2, __int_as_float(raw.x), __int_as_float(raw.y), raw.z);
     }
     partial_warp_allreduce(m2, s2, p2);
-    if (lane == 0) {
-        finalize_row<DT>(a, P, row, m2, s2, p2, false);
-        a.tickets[row] = 0u;
-    }
+    warp_finalize_row<DT>(a, P, row, m2, s2, p2, lane);
+    if (lane == 0) a.tickets[row] = 0u;
 }
 
 // ---------------------------------------------------------------------------------------

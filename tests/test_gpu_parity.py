@@ -134,20 +134,27 @@ def test_fused_several_tiles_and_ragged_tail(V, stride, dtype, mode):
     assert np.all(got["vocab_mask"][:, (V + 31) // 32:] == 0x5A5A5A5A)
 
 
-@pytest.mark.parametrize("ctas,tw,rw", [(1, 0, 0), (4, 1, 4), (4, 2, 4), (8, 2, 2), (16, 4, 1), (2, 8, 1)])
-def test_fused_launch_shapes_agree(ctas, tw, rw):
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("knobs", [
+    dict(pipeline=0, ctas_per_sm=1), dict(pipeline=0, ctas_per_sm=4, token_warps=1, row_warps=4),
+    dict(pipeline=0, ctas_per_sm=8, token_warps=2, row_warps=2), dict(pipeline=0, ctas_per_sm=2, token_warps=8, row_warps=1),
+    dict(pipeline=1), dict(pipeline=1, pipe_warps=4, pipe_depth=2), dict(pipeline=1, pipe_warps=16, pipe_depth=3),
+    dict(pipeline=1, pipe_warps=8, pipe_depth=8, ctas_per_sm=1), dict(pipeline=1, token_warps=2, row_warps=4),
+    dict(pipeline=1, token_warps=1, row_warps=2, ctas_per_sm=16), dict(pipeline=1, pipe_warps=16, token_warps=16, row_warps=1),
+])
+def test_fused_launch_shapes_agree(knobs, dtype):
     V, K, B = 50000, 700, 40
     part = synth.zipf_partition(V, K, 1.1, seed=6)
     cm = _mask(K, B, 0.1, 3)
-    z = synth.logits_normal(B, V, 2.0, "bf16", (33,))
+    z = synth.logits_normal(B, V, 2.0, dtype, (33,))
     want = oracle_step([part], None, cm, z, V)
     with Ctx([part]) as ctx:
-        cz.cfgzip_set_tuning(ctx.h, "ctas_per_sm", ctas)
-        cz.cfgzip_set_tuning(ctx.h, "token_warps", tw)
-        cz.cfgzip_set_tuning(ctx.h, "row_warps", rw)
+        for name, value in knobs.items():
+            cz.cfgzip_set_tuning(ctx.h, name, value)
         for pdl in (1, 0):
             cz.cfgzip_set_tuning(ctx.h, "pdl", pdl)
-            compare_step(run_fused(ctx, None, cm, z, V), want, V, "ctas=%d tw=%d rw=%d pdl=%d" % (ctas, tw, rw, pdl))
+            compare_step(run_fused(ctx, None, cm, z, V), want, V, "%r pdl=%d" % (knobs, pdl))
+        assert cz.cfgzip_poll_status(ctx.h) == (0, 0, 0)
 
 
 @pytest.mark.parametrize("mode", [cz.DENSE, cz.SPARSE])
