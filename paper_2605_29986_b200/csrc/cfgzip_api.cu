@@ -1,5 +1,6 @@
 // C ABI of the CFGzip decode-step library: argument checks, partition tables, launch
 // planning. The declarations and their contracts are in include/cfgzip.h.
+#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include <algorithm>
@@ -56,7 +57,12 @@ struct cfgzip_ctx {
     int32_t token_warps = 0;
     int32_t row_warps = 0;
     int32_t pdl = 1;
+    // cuTensorMapEncodeTiled, looked up through the runtime (no link against the driver library)
+    CUresult (*encode_tiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                             const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                             CUtensorMapL2promotion, CUtensorMapFloatOOBfill) = nullptr;
     int32_t pipeline = 1;     // bulk-copy pipelined dense kernel for aligned logits
+    int32_t tensor_map = 1;   // tiled 2-D copies for row batches that are consecutive rows
     int32_t pipe_warps = 8;
     int32_t pipe_depth = 4;
 };
@@ -340,8 +346,24 @@ int launch_fused(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, in
             fill_groups(ctx, a, d);
             const dim3 grid(unsigned(d.n_groups_ub) * unsigned(d.S)), block{unsigned(d.threads)};
             if (d.depth) {
-                if ((rc = ensure_smem(k_step_dense_pipe<DT>, d.smem)) != CFGZIP_OK) return rc;
-                rc = launch(ctx, k_step_dense_pipe<DT>, grid, block, d.smem, st, a);
+                // rows of a batch are consecutive unless the plan kernel regrouped them: then one tiled
+                // 2-D copy (box 256 elements x 8 rows) brings a whole batch
+                CUtensorMap tmap;
+                std::memset(&tmap, 0, sizeof tmap);
+                bool tiled = false;
+                if (!d.use_plan_kernel && ctx->tensor_map && ctx->encode_tiled && a.V >= 256) {
+                    const cuuint64_t dims[2] = {cuuint64_t(a.V), cuuint64_t(a.B)};
+                    const cuuint64_t strides[1] = {cuuint64_t(a.row_stride) * (DT == kBF16 ? 2 : 4)};
+                    const cuuint32_t box[2] = {256, 8};
+                    const cuuint32_t estr[2] = {1, 1};
+                    tiled = ctx->encode_tiled(&tmap, DT == kBF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+                                              2, a.logits, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                              CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+                }
+                auto kern = tiled ? k_step_dense_pipe<DT, true> : k_step_dense_pipe<DT, false>;
+                if ((rc = ensure_smem(kern, d.smem)) != CFGZIP_OK) return rc;
+                rc = launch(ctx, kern, grid, block, d.smem, st, a, tmap);
             } else {
                 auto kern = k_step_dense<DT>;
                 if ((rc = ensure_smem(kern, d.smem)) != CFGZIP_OK) return rc;
@@ -444,6 +466,15 @@ int cfgzip_create(int device, cfgzip_ctx** out) {
     ctx->device = device;
     cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
     cudaDeviceGetAttribute(&ctx->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+    {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            ctx->encode_tiled = reinterpret_cast<decltype(ctx->encode_tiled)>(fn);
+        else
+            cudaGetLastError();
+    }
     bool ok = cudaMalloc(&ctx->d_parts, kMaxParts * sizeof(PartDev)) == cudaSuccess &&
               cudaMalloc(&ctx->d_partials, kPartialSlots * sizeof(Partial)) == cudaSuccess &&
               cudaMalloc(&ctx->d_status, 4 * sizeof(int32_t)) == cudaSuccess &&
@@ -800,6 +831,8 @@ int cfgzip_set_tuning(cfgzip_ctx* ctx, const char* name, int32_t value) {
         ctx->pdl = value ? 1 : 0;
     } else if (!std::strcmp(name, "pipeline")) {
         ctx->pipeline = value ? 1 : 0;
+    } else if (!std::strcmp(name, "tensor_map")) {
+        ctx->tensor_map = value ? 1 : 0;
     } else if (!std::strcmp(name, "pipe_warps")) {
         if (value != 4 && value != 8 && value != 12 && value != 16) return CFGZIP_E_ARG;
         ctx->pipe_warps = value;

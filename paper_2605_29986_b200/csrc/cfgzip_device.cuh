@@ -286,6 +286,15 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
+// Tiled 2-D copy through a tensor map: box of (x .. x+boxDim0) elements by (y .. y+boxDim1) rows.
+// x times the element size must be a multiple of 16 bytes; out-of-range parts are zero-filled.
+__device__ __forceinline__ void tma_g2s_2d(void* dst_smem, const void* tensor_map, int x, int y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+            smem_u32(dst_smem)),
+        "l"(tensor_map), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
 // size and both addresses are multiples of 16 bytes
 __device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(

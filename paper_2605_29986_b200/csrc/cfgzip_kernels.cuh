@@ -4,6 +4,8 @@
 // 32 bytes of f32, one byte of vocab mask).
 #pragma once
 
+#include <cuda.h>
+
 #include "cfgzip_device.cuh"
 
 namespace cfgzip {
@@ -518,8 +520,33 @@ struct PipeGeom {
     static constexpr int kStageBytes = kBatchRows * kRowBytes + 32 * 16;  // + class ids of 32 octets
 };
 
-template <int DT>
-__global__ void __launch_bounds__(512) k_step_dense_pipe(const __grid_constant__ StepArgs a) {
+// One work item of a warp: 32 octets of the 8 rows of a batch, read from the stage `src`.
+// FULL: all 8 rows live and all 32 lanes inside the whole-vector range (no per-row tests).
+template <int DT, bool FULL>
+__device__ __forceinline__ void pipe_consume_item(const char* src, const uint32_t* T, int rb, int live, bool active,
+                                                  int o, int lane, char* const (&rowp)[kBatchRows],
+                                                  uint8_t* const (&vmp)[kBatchRows], RowAcc (&acc)[kBatchRows]) {
+    using G = PipeGeom<DT>;
+    uint4 cv = make_uint4(0, 0, 0, 0);
+    if (FULL || active) cv = *reinterpret_cast<const uint4*>(src + kBatchRows * G::kRowBytes + lane * 16);
+    uint32_t lo, hi;
+    octet_allow_bits(cv, T, rb, FULL || active, lo, hi);
+#pragma unroll
+    for (int i = 0; i < kBatchRows; ++i) {
+        if (FULL || (i < live && active)) {
+            Octet<DT> oc;
+            oc.load_shared(src + i * G::kRowBytes, lane);
+            const uint32_t byte = ((i < 4 ? lo : hi) >> (8 * (i & 3))) & 0xFFu;
+            dense_octet_row<DT>(oc, rowp[i], vmp[i], o, byte, acc[i]);
+        }
+    }
+}
+
+// TMAP: the 8 rows of a batch are consecutive rows of the logits matrix and arrive as one
+// tiled 2-D copy through `tmap` (box = 256 elements x 8 rows); otherwise one bulk copy per row.
+template <int DT, bool TMAP>
+__global__ void __launch_bounds__(512) k_step_dense_pipe(const __grid_constant__ StepArgs a,
+                                                         const __grid_constant__ CUtensorMap tmap) {
     using G = PipeGeom<DT>;
     extern __shared__ __align__(128) uint32_t smem[];
     uint32_t* T = smem;
@@ -541,6 +568,7 @@ __global__ void __launch_bounds__(512) k_step_dense_pipe(const __grid_constant__
     const PartDev P = a.group_part ? a.parts[part] : a.p0;
     const int nrow = __popc(__ballot_sync(0xFFFFFFFFu, s_row[lane] >= 0));
 
+    const int depth = a.depth;
     const int wt = warp % a.WT, wr = warp / a.WT, WR = n_warps / a.WT;
     const int n_octets = 4 * a.VW, n_full = a.V >> 3;
     const int o_begin = split * a.per_split;
@@ -548,8 +576,8 @@ __global__ void __launch_bounds__(512) k_step_dense_pipe(const __grid_constant__
     const int o_vec_end = min(o_end, n_full);
     constexpr int ES = DT == kBF16 ? 2 : 4;
     uint8_t* vm8 = reinterpret_cast<uint8_t*>(a.vocab_mask);
-    char* my_ring = ring + size_t(warp) * a.depth * G::kStageBytes;
-    uint64_t* bar = bars + warp * a.depth;
+    char* my_ring = ring + size_t(warp) * depth * G::kStageBytes;
+    uint64_t* bar = bars + warp * depth;
 
     // this warp's work items: row batches rb = wr, wr+WR, ... (outer) x chunks of 32 whole-vector octets (inner)
     const int first_chunk = o_begin + wt * 32;
@@ -558,28 +586,36 @@ __global__ void __launch_bounds__(512) k_step_dense_pipe(const __grid_constant__
     const int n_rb = (nrow > wr * kBatchRows) ? ((nrow - wr * kBatchRows + WR * kBatchRows - 1) / (WR * kBatchRows)) : 0;
     const int n_items = n_chunks * n_rb;
 
-    auto issue = [&](int n) {  // lane 0 only: start the copies of work item n into slot n % depth
-        const int rb = wr + (n / n_chunks) * WR;
-        const int o0 = first_chunk + (n % n_chunks) * chunk_step;
-        const int slot = n % a.depth;
-        char* dst = my_ring + size_t(slot) * G::kStageBytes;
-        const int live = min(kBatchRows, nrow - rb * kBatchRows);
+    // producer cursor (meaningful in lane 0): next item to start, kept without divisions
+    int p_n = 0, p_ci = 0, p_rb = wr, p_slot = 0;
+    auto issue_next = [&]() {
+        const int o0 = first_chunk + p_ci * chunk_step;
+        char* dst = my_ring + size_t(p_slot) * G::kStageBytes;
         const uint32_t nvec = uint32_t(min(o_vec_end - o0, 32));  // >= 1 by construction of the chunk list
-        const uint32_t row_bytes = nvec * G::kOctetBytes;
-        mbar_expect_tx(bar + slot, uint32_t(live) * row_bytes + nvec * 16u);
-        bulk_g2s(dst + kBatchRows * G::kRowBytes, reinterpret_cast<const char*>(P.c16) + size_t(o0) * 16, nvec * 16u, bar + slot);
-        for (int i = 0; i < live; ++i) {
-            const int row = s_row[rb * kBatchRows + i];
-            bulk_g2s(dst + i * G::kRowBytes,
-                     reinterpret_cast<const char*>(a.logits) + (int64_t(row) * a.row_stride * ES + int64_t(o0) * 8 * ES), row_bytes,
-                     bar + slot);
+        if (TMAP) {
+            mbar_expect_tx(bar + p_slot, uint32_t(kBatchRows * G::kRowBytes) + nvec * 16u);
+            tma_g2s_2d(dst, &tmap, o0 * 8, s_row[p_rb * kBatchRows], bar + p_slot);
+        } else {
+            const int live = min(kBatchRows, nrow - p_rb * kBatchRows);
+            const uint32_t row_bytes = nvec * G::kOctetBytes;
+            mbar_expect_tx(bar + p_slot, uint32_t(live) * row_bytes + nvec * 16u);
+            for (int i = 0; i < live; ++i) {
+                const int row = s_row[p_rb * kBatchRows + i];
+                bulk_g2s(dst + i * G::kRowBytes,
+                         reinterpret_cast<const char*>(a.logits) + (int64_t(row) * a.row_stride * ES + int64_t(o0) * 8 * ES),
+                         row_bytes, bar + p_slot);
+            }
         }
+        bulk_g2s(dst + kBatchRows * G::kRowBytes, reinterpret_cast<const char*>(P.c16) + size_t(o0) * 16, nvec * 16u, bar + p_slot);
+        ++p_n;
+        if (++p_slot == depth) p_slot = 0;
+        if (++p_ci == n_chunks) { p_ci = 0; p_rb += WR; }
     };
 
     if (lane == 0) {
-        for (int d = 0; d < a.depth; ++d) mbar_init(bar + d, 1);
+        for (int d = 0; d < depth; ++d) mbar_init(bar + d, 1);
         mbar_init_fence();
-        for (int n = 0; n < min(a.depth, n_items); ++n) issue(n);  // in flight while the table is built
+        while (p_n < min(depth, n_items)) issue_next();  // in flight while the table is built
     }
     if (a.stage_stride) {
         stage_class_masks(a, P, s_row, stage, warp, lane, n_warps);
@@ -589,9 +625,10 @@ __global__ void __launch_bounds__(512) k_step_dense_pipe(const __grid_constant__
     __syncthreads();
 
     bool failed = false;
-    int n = 0;
-    for (int rbi = 0; rbi < n_rb && !failed; ++rbi) {
-        const int rb = wr + rbi * WR;
+    int slot = 0;
+    uint32_t phase = 0;
+    int consumed = 0;
+    for (int rb = wr; rb * kBatchRows < nrow && !failed; rb += WR) {
         RowAcc acc[kBatchRows];
         char* rowp[kBatchRows];
         uint8_t* vmp[kBatchRows];
@@ -603,61 +640,37 @@ __global__ void __launch_bounds__(512) k_step_dense_pipe(const __grid_constant__
             vmp[i] = vm8 ? vm8 + int64_t(max(row, 0)) * a.vm_stride * 4 : nullptr;
         }
         const int live = min(kBatchRows, nrow - rb * kBatchRows);
-        for (int ci = 0; ci < n_chunks; ++ci, ++n) {
-            const int slot = n % a.depth;
-            const bool arrived = mbar_wait(bar + slot, uint32_t(n / a.depth) & 1u);
+        for (int o0 = first_chunk; o0 < o_vec_end; o0 += chunk_step) {
+            const bool arrived = mbar_wait(bar + slot, phase);
             if (!__all_sync(0xFFFFFFFFu, arrived)) {
                 failed = true;
                 break;
             }
             const char* src = my_ring + size_t(slot) * G::kStageBytes;
-            const int o = first_chunk + ci * chunk_step + lane;
-            const bool active = o < o_vec_end;
-            uint4 cv = make_uint4(0, 0, 0, 0);
-            if (active) cv = *reinterpret_cast<const uint4*>(src + kBatchRows * G::kRowBytes + lane * 16);
-            uint32_t lo, hi;
-            octet_allow_bits(cv, T, rb, active, lo, hi);
-#pragma unroll
-            for (int i = 0; i < kBatchRows; ++i) {
-                if (i < live && active) {
-                    Octet<DT> oc;
-                    oc.load_shared(src + i * G::kRowBytes, lane);
-                    const uint32_t byte = ((i < 4 ? lo : hi) >> (8 * (i & 3))) & 0xFFu;
-                    dense_octet_row<DT>(oc, rowp[i], vmp[i], o, byte, acc[i]);
-                }
-            }
+            const int o = o0 + lane;
+            if (live == kBatchRows && o0 + 32 <= o_vec_end)
+                pipe_consume_item<DT, true>(src, T, rb, live, true, o, lane, rowp, vmp, acc);
+            else
+                pipe_consume_item<DT, false>(src, T, rb, live, o < o_vec_end, o, lane, rowp, vmp, acc);
+            ++consumed;
+            if (++slot == depth) { slot = 0; phase ^= 1u; }
             __syncwarp();  // every lane has its data out of the slot before it is refilled
-            if (lane == 0 && n + a.depth < n_items) issue(n + a.depth);
+            if (lane == 0 && p_n < n_items) issue_next();
         }
         if (failed) break;
         if (wt == 0 && o_end > n_full)
             dense_tail_octets<DT>(a, P, T, rb, live, max(o_begin, n_full), o_end, lane, rowp, vmp, acc);
         warp_rows_to_red(acc, live, red + warp * kGroupRows, rb, lane);
     }
-    // a warp without whole-vector chunks may still own the tail octets of its row batches
-    if (n_chunks == 0 && wt == 0 && o_end > n_full) {
-        for (int rb = wr; rb * kBatchRows < nrow; rb += WR) {
-            RowAcc acc[kBatchRows];
-            char* rowp[kBatchRows];
-            uint8_t* vmp[kBatchRows];
-#pragma unroll
-            for (int i = 0; i < kBatchRows; ++i) {
-                acc[i].init();
-                const int row = s_row[min(rb * kBatchRows + i, kGroupRows - 1)];
-                rowp[i] = reinterpret_cast<char*>(a.logits) + int64_t(max(row, 0)) * a.row_stride * ES;
-                vmp[i] = vm8 ? vm8 + int64_t(max(row, 0)) * a.vm_stride * 4 : nullptr;
-            }
-            const int live = min(kBatchRows, nrow - rb * kBatchRows);
-            dense_tail_octets<DT>(a, P, T, rb, live, max(o_begin, n_full), o_end, lane, rowp, vmp, acc);
-            warp_rows_to_red(acc, live, red + warp * kGroupRows, rb, lane);
-        }
-    }
     if (failed) {
         // a copy never arrived: flag it, give the copies still in flight the same bounded time to land
         // (they target this block's shared memory), and let the block leave without results
         if (lane == 0) {
             atomicAdd(a.status + 3, 1);
-            for (int k = n; k < min(n + a.depth, n_items); ++k) mbar_wait(bar + k % a.depth, uint32_t(k / a.depth) & 1u);
+            for (int k = consumed; k < p_n; ++k) {
+                mbar_wait(bar + slot, phase);
+                if (++slot == depth) { slot = 0; phase ^= 1u; }
+            }
         }
     }
     dense_block_tail<DT>(a, P, g, split, s_row, nrow, red, tl);

@@ -138,7 +138,7 @@ def test_fused_several_tiles_and_ragged_tail(V, stride, dtype, mode):
 @pytest.mark.parametrize("knobs", [
     dict(pipeline=0, ctas_per_sm=1), dict(pipeline=0, ctas_per_sm=4, token_warps=1, row_warps=4),
     dict(pipeline=0, ctas_per_sm=8, token_warps=2, row_warps=2), dict(pipeline=0, ctas_per_sm=2, token_warps=8, row_warps=1),
-    dict(pipeline=1), dict(pipeline=1, pipe_warps=4, pipe_depth=2), dict(pipeline=1, pipe_warps=16, pipe_depth=3),
+    dict(pipeline=1), dict(pipeline=1, tensor_map=0), dict(pipeline=1, pipe_warps=4, pipe_depth=2), dict(pipeline=1, pipe_warps=16, pipe_depth=3),
     dict(pipeline=1, pipe_warps=8, pipe_depth=8, ctas_per_sm=1), dict(pipeline=1, token_warps=2, row_warps=4),
     dict(pipeline=1, token_warps=1, row_warps=2, ctas_per_sm=16), dict(pipeline=1, pipe_warps=16, token_warps=16, row_warps=1),
 ])
