@@ -195,7 +195,7 @@ int cfgzip_launch_count(cfgzip_ctx* ctx, int64_t* out);
  *                  in shared memory (default), 0 = plain 16-byte loads into registers
  *   "tensor_map"   1 = a batch of 8 consecutive rows arrives as one tiled 2-D copy through a
  *                  tensor map (default), 0 = one bulk copy per row
- *   "pipe_warps"   warps per thread block of the pipelined kernel (4, 8, 12 or 16)
+ *   "pipe_warps"   warps per thread block of the pipelined kernel (1..16)
  *   "pipe_depth"   stages per warp of the pipelined kernel (2..8; lowered to fit shared memory)
  * Unknown names give CFGZIP_E_ARG.
  */

@@ -175,6 +175,7 @@ size_t dense_smem_bytes(int table_words, int n_warps, int stage_stride) {
 struct DensePlan {
     int S = 1, per_split = 0, WT = 4, threads = 128, table_words = 0, stage_stride = 0;
     int depth = 0;       // > 0: pipelined kernel with this many stages per warp
+    int ctas_per_sm = 1; // blocks per SM the launch was sized for
     size_t smem = 0;
     int n_groups_ub = 1;
     bool use_plan_kernel = false;
@@ -208,7 +209,7 @@ DensePlan plan_dense(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, 
         int stride = ps.maxKW | 1;
         if (pipe_smem_bytes(d.table_words, n_warps, 2, stage_bytes, stride) > cap) stride = 0;
         while (depth > 2 && pipe_smem_bytes(d.table_words, n_warps, depth, stage_bytes, stride) > cap) --depth;
-        while (n_warps > 4 && pipe_smem_bytes(d.table_words, n_warps, depth, stage_bytes, stride) > cap) n_warps -= 4;
+        while (n_warps > 4 && pipe_smem_bytes(d.table_words, n_warps, depth, stage_bytes, stride) > cap) n_warps -= 2;
         const size_t smem = pipe_smem_bytes(d.table_words, n_warps, depth, stage_bytes, stride);
         if (smem <= cap) {
             d.depth = depth;
@@ -222,6 +223,7 @@ DensePlan plan_dense(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, 
         // stage the class masks through shared memory while that keeps a block under 64 KB
         if (dense_smem_bytes(d.table_words, 8, ps.maxKW | 1) <= 64 * 1024) d.stage_stride = ps.maxKW | 1;
     }
+    d.ctas_per_sm = ctas_per_sm;
     const int target = ctx->sm_count * ctas_per_sm;
     const int n_chunks = ceil_div(units, unit_chunk);
     const int s0 = std::max(1, target / d.n_groups_ub);
@@ -229,8 +231,10 @@ DensePlan plan_dense(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, 
     int WR = 1;
     if (fused) {
         if (d.depth) {
-            WR = ctx->row_warps ? ctx->row_warps : (cps * 4 <= n_warps ? 4 : (cps * 2 <= n_warps ? 2 : 1));
-            if (WR != 1 && WR != 2 && WR != 4) WR = 1;
+            // one row batch per warp where the warp count allows: a warp then reduces its rows once
+            WR = ctx->row_warps ? ctx->row_warps : (n_warps % 4 == 0 ? 4 : (n_warps % 2 == 0 ? 2 : 1));
+            while (WR > 1 && (WR - 1) * kBatchRows >= std::min<int>(B, kGroupRows)) WR >>= 1;
+            if ((WR != 1 && WR != 2 && WR != 4) || n_warps % WR) WR = 1;
             d.WT = ctx->token_warps ? ctx->token_warps : n_warps / WR;
             d.WT = std::max(1, std::min(d.WT, 16 / WR));
             cps = ceil_div(cps, d.WT) * d.WT;  // every warp of a block gets the same number of chunks
@@ -351,7 +355,8 @@ int launch_fused(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, in
                 CUtensorMap tmap;
                 std::memset(&tmap, 0, sizeof tmap);
                 bool tiled = false;
-                if (!d.use_plan_kernel && ctx->tensor_map && ctx->encode_tiled && a.V >= 256) {
+                if (!d.use_plan_kernel && ctx->tensor_map && ctx->encode_tiled && a.V >= 256 &&
+                    a.row_stride * (DT == kBF16 ? 2 : 4) < (int64_t(1) << 32) && a.vm_stride * 4 < (int64_t(1) << 32)) {
                     const cuuint64_t dims[2] = {cuuint64_t(a.V), cuuint64_t(a.B)};
                     const cuuint64_t strides[1] = {cuuint64_t(a.row_stride) * (DT == kBF16 ? 2 : 4)};
                     const cuuint32_t box[2] = {256, 8};
@@ -361,7 +366,13 @@ int launch_fused(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, in
                                               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
                 }
-                auto kern = tiled ? k_step_dense_pipe<DT, true> : k_step_dense_pipe<DT, false>;
+                void (*kern)(StepArgs, CUtensorMap);
+                if (d.threads <= 256 && d.ctas_per_sm >= 3)
+                    kern = tiled ? k_step_dense_pipe<DT, true, 256, 3> : k_step_dense_pipe<DT, false, 256, 3>;
+                else if (d.threads <= 320 && d.ctas_per_sm >= 2)
+                    kern = tiled ? k_step_dense_pipe<DT, true, 320, 2> : k_step_dense_pipe<DT, false, 320, 2>;
+                else
+                    kern = tiled ? k_step_dense_pipe<DT, true, 512, 1> : k_step_dense_pipe<DT, false, 512, 1>;
                 if ((rc = ensure_smem(kern, d.smem)) != CFGZIP_OK) return rc;
                 rc = launch(ctx, kern, grid, block, d.smem, st, a, tmap);
             } else {
@@ -834,7 +845,7 @@ int cfgzip_set_tuning(cfgzip_ctx* ctx, const char* name, int32_t value) {
     } else if (!std::strcmp(name, "tensor_map")) {
         ctx->tensor_map = value ? 1 : 0;
     } else if (!std::strcmp(name, "pipe_warps")) {
-        if (value != 4 && value != 8 && value != 12 && value != 16) return CFGZIP_E_ARG;
+        if (value < 1 || value > 16) return CFGZIP_E_ARG;
         ctx->pipe_warps = value;
     } else if (!std::strcmp(name, "pipe_depth")) {
         if (value < 2 || value > 8) return CFGZIP_E_ARG;

@@ -155,6 +155,7 @@ struct Octet<kBF16> {
     __device__ __forceinline__ void store(void* row_base, int o) const {
         st_stream16(reinterpret_cast<uint16_t*>(row_base) + 8 * int64_t(o), v);
     }
+    __device__ __forceinline__ void store_at(void* p) const { st_stream16(p, v); }
     __device__ __forceinline__ void fill_neg_inf() { v = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u); }
     __device__ __forceinline__ void mask(uint32_t byte, float (&f)[8]) {
         const uint32_t xl = nibble_to_byte_msbs(byte & 0xFu), xh = nibble_to_byte_msbs(byte >> 4);
@@ -190,6 +191,10 @@ struct Octet<kF32> {
         st_stream16(p, a);
         st_stream16(p + 4, b);
     }
+    __device__ __forceinline__ void store_at(void* p) const {
+        st_stream16(p, a);
+        st_stream16(reinterpret_cast<char*>(p) + 16, b);
+    }
     __device__ __forceinline__ void fill_neg_inf() {
         a = make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u);
         b = a;
@@ -219,6 +224,32 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
     return d;
 }
 
+// Packed pairs of floats (sm_100 has two-wide fp32 multiply-add and add).
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
+    unsigned long long p;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(p) : "f"(lo), "f"(hi));
+    return p;
+}
+__device__ __forceinline__ void unpack2(unsigned long long p, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(p));
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b) {
+    unsigned long long d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// base + i * stride with a 32-bit stride in one wide multiply-add
+__device__ __forceinline__ char* ptr_mad(char* base, uint32_t i, uint32_t stride) {
+    unsigned long long r;
+    asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(r) : "r"(i), "r"(stride), "l"(reinterpret_cast<unsigned long long>(base)));
+    return reinterpret_cast<char*>(r);
+}
+
 // Running state of one row inside one thread. The sum is kept relative to a reference that
 // only moves when a value overtakes it by more than kRefSlack (so the common case is one
 // fused multiply-add and one ex2 per logit): s = sum 2^(z*log2e + nrl), nrl = -(ref*log2e).
@@ -242,10 +273,18 @@ struct RowAcc {
             s *= ex2f(n2 - nrl);
             nrl = n2;
         }
-        float acc = 0.f;
+        const unsigned long long l2 = pack2(kLog2e, kLog2e), n2p = pack2(nrl, nrl);
+        float e[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) acc += ex2f(fmaf(f[j], kLog2e, nrl));
-        s += acc;
+        for (int j = 0; j < 8; j += 2) {
+            float t0, t1;
+            unpack2(fma2(pack2(f[j], f[j + 1]), l2, n2p), t0, t1);
+            e[j] = ex2f(t0);
+            e[j + 1] = ex2f(t1);
+        }
+        float a0, a1;
+        unpack2(add2(add2(pack2(e[0], e[1]), pack2(e[2], e[3])), add2(pack2(e[4], e[5]), pack2(e[6], e[7]))), a0, a1);
+        s += a0 + a1;
     }
     // Bring the sum to the convention of Partial: relative to max(m, kRefFloor).
     __device__ __forceinline__ Partial to_partial() const {

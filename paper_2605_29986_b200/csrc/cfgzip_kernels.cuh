@@ -520,11 +520,20 @@ struct PipeGeom {
     static constexpr int kStageBytes = kBatchRows * kRowBytes + 32 * 16;  // + class ids of 32 octets
 };
 
+// Where the rows of a batch live. With consecutive rows (CONSEC) the address of row i is one
+// wide multiply-add from the batch's base; otherwise each row has its own base pointer.
+struct BatchAddr {
+    char* item_base;      // CONSEC: logits of row 0 of the batch at this lane's octet
+    uint8_t* vm_item;     // CONSEC: vocab-mask byte of row 0 at this lane's octet (or null)
+    uint32_t row_bytes;   // CONSEC: bytes between rows of the logits
+    uint32_t vm_bytes;    // CONSEC: bytes between rows of the vocab mask
+};
+
 // One work item of a warp: 32 octets of the 8 rows of a batch, read from the stage `src`.
 // FULL: all 8 rows live and all 32 lanes inside the whole-vector range (no per-row tests).
-template <int DT, bool FULL>
+template <int DT, bool FULL, bool CONSEC>
 __device__ __forceinline__ void pipe_consume_item(const char* src, const uint32_t* T, int rb, int live, bool active,
-                                                  int o, int lane, char* const (&rowp)[kBatchRows],
+                                                  int o, int lane, const BatchAddr& ba, char* const (&rowp)[kBatchRows],
                                                   uint8_t* const (&vmp)[kBatchRows], RowAcc (&acc)[kBatchRows]) {
     using G = PipeGeom<DT>;
     uint4 cv = make_uint4(0, 0, 0, 0);
@@ -537,15 +546,26 @@ __device__ __forceinline__ void pipe_consume_item(const char* src, const uint32_
             Octet<DT> oc;
             oc.load_shared(src + i * G::kRowBytes, lane);
             const uint32_t byte = ((i < 4 ? lo : hi) >> (8 * (i & 3))) & 0xFFu;
-            dense_octet_row<DT>(oc, rowp[i], vmp[i], o, byte, acc[i]);
+            float f[8];
+            oc.mask(byte, f);
+            if (CONSEC) {
+                oc.store_at(ptr_mad(ba.item_base, i, ba.row_bytes));
+                if (ba.vm_item) *ptr_mad(reinterpret_cast<char*>(ba.vm_item), i, ba.vm_bytes) = char(byte);
+            } else {
+                oc.store(rowp[i], o);
+                if (vmp[i]) vmp[i][o] = uint8_t(byte);
+            }
+            acc[i].add_octet(f, o);
         }
     }
 }
 
 // TMAP: the 8 rows of a batch are consecutive rows of the logits matrix and arrive as one
 // tiled 2-D copy through `tmap` (box = 256 elements x 8 rows); otherwise one bulk copy per row.
-template <int DT, bool TMAP>
-__global__ void __launch_bounds__(512) k_step_dense_pipe(const __grid_constant__ StepArgs a,
+// LBT / MINB: launch bounds (threads per block, blocks per SM) the variant is compiled for; they set
+// the register budget: (512, 1) 128 registers, (320, 2) 96, (256, 3) 80.
+template <int DT, bool TMAP, int LBT, int MINB>
+__global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_constant__ StepArgs a,
                                                          const __grid_constant__ CUtensorMap tmap) {
     using G = PipeGeom<DT>;
     extern __shared__ __align__(128) uint32_t smem[];
@@ -635,11 +655,21 @@ __global__ void __launch_bounds__(512) k_step_dense_pipe(const __grid_constant__
 #pragma unroll
         for (int i = 0; i < kBatchRows; ++i) {
             acc[i].init();
-            const int row = s_row[min(rb * kBatchRows + i, kGroupRows - 1)];
-            rowp[i] = reinterpret_cast<char*>(a.logits) + int64_t(max(row, 0)) * a.row_stride * ES;
-            vmp[i] = vm8 ? vm8 + int64_t(max(row, 0)) * a.vm_stride * 4 : nullptr;
+            rowp[i] = nullptr;
+            vmp[i] = nullptr;
+            if (!TMAP) {
+                const int row = s_row[min(rb * kBatchRows + i, kGroupRows - 1)];
+                rowp[i] = reinterpret_cast<char*>(a.logits) + int64_t(max(row, 0)) * a.row_stride * ES;
+                vmp[i] = vm8 ? vm8 + int64_t(max(row, 0)) * a.vm_stride * 4 : nullptr;
+            }
         }
         const int live = min(kBatchRows, nrow - rb * kBatchRows);
+        const int row0 = max(s_row[rb * kBatchRows], 0);
+        char* const base0 = reinterpret_cast<char*>(a.logits) + int64_t(row0) * a.row_stride * ES;
+        uint8_t* const vm0 = vm8 ? vm8 + int64_t(row0) * a.vm_stride * 4 : nullptr;
+        BatchAddr ba;
+        ba.row_bytes = uint32_t(a.row_stride * ES);
+        ba.vm_bytes = uint32_t(a.vm_stride * 4);
         for (int o0 = first_chunk; o0 < o_vec_end; o0 += chunk_step) {
             const bool arrived = mbar_wait(bar + slot, phase);
             if (!__all_sync(0xFFFFFFFFu, arrived)) {
@@ -648,18 +678,28 @@ __global__ void __launch_bounds__(512) k_step_dense_pipe(const __grid_constant__
             }
             const char* src = my_ring + size_t(slot) * G::kStageBytes;
             const int o = o0 + lane;
+            ba.item_base = base0 + size_t(o) * G::kOctetBytes;
+            ba.vm_item = vm0 ? vm0 + o : nullptr;
             if (live == kBatchRows && o0 + 32 <= o_vec_end)
-                pipe_consume_item<DT, true>(src, T, rb, live, true, o, lane, rowp, vmp, acc);
+                pipe_consume_item<DT, true, TMAP>(src, T, rb, live, true, o, lane, ba, rowp, vmp, acc);
             else
-                pipe_consume_item<DT, false>(src, T, rb, live, o < o_vec_end, o, lane, rowp, vmp, acc);
+                pipe_consume_item<DT, false, TMAP>(src, T, rb, live, o < o_vec_end, o, lane, ba, rowp, vmp, acc);
             ++consumed;
             if (++slot == depth) { slot = 0; phase ^= 1u; }
             __syncwarp();  // every lane has its data out of the slot before it is refilled
             if (lane == 0 && p_n < n_items) issue_next();
         }
         if (failed) break;
-        if (wt == 0 && o_end > n_full)
+        if (wt == 0 && o_end > n_full) {
+            if (TMAP) {
+#pragma unroll
+                for (int i = 0; i < kBatchRows; ++i) {
+                    rowp[i] = ptr_mad(base0, i, ba.row_bytes);
+                    vmp[i] = vm0 ? reinterpret_cast<uint8_t*>(ptr_mad(reinterpret_cast<char*>(vm0), i, ba.vm_bytes)) : nullptr;
+                }
+            }
             dense_tail_octets<DT>(a, P, T, rb, live, max(o_begin, n_full), o_end, lane, rowp, vmp, acc);
+        }
         warp_rows_to_red(acc, live, red + warp * kGroupRows, rb, lane);
     }
     if (failed) {
