@@ -182,6 +182,44 @@ int cfgzip_decode_step_host(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t
 int cfgzip_poll_status(cfgzip_ctx* ctx, void* stream, int32_t* n_empty_rows, int32_t* n_bad_tokens,
                        int32_t* n_bad_rows);
 
+/*
+ * The fused step for callers that are not allowed to allocate device memory. (The paper has
+ * no counterpart for this call; it exists for integration reasons only.)
+ *
+ * Everything above needs a context, and creating one or loading a partition calls
+ * cudaMalloc. Some hosts of this library cannot do that at the point where they need the
+ * step: a plugin that runs inside another runtime's memory pool and must not grow the
+ * process's device footprint behind its back, code running inside a region where the CUDA
+ * allocator is off limits, or a job whose memory budget was fixed at start-up. This entry
+ * point takes no context and calls no allocating routine. The token->class and
+ * class->representative vectors are DEVICE arrays the caller already holds, and the only
+ * memory the call uses beyond its arguments is a fixed scratch array compiled into the
+ * library (about 1 MiB; every GPU that loads the library carries a copy until the process
+ * exits).
+ *
+ *   token_to_class : dev int32 [V]; an id outside [0, K) makes that token disallowed
+ *   class_to_rep   : dev int32 [K]
+ *   other arguments and all results as in cfgzip_masked_logsoftmax_argmax (no logp_full, no
+ *   row partitions, no sticky counters; rows may have any alignment)
+ *
+ * Limits and rules
+ *   - B <= 1024 rows per call; more gives CFGZIP_E_RANGE and nothing is launched.
+ *   - It runs on the CURRENT device of the calling thread. The first call on each device asks
+ *     the runtime for the address of that device's copy of the scratch array; make that first
+ *     call outside any stream capture.
+ *   - All calls on one GPU share the scratch array, whatever their stream. It is not cleared
+ *     between calls except for the per-row tickets, which every call zeroes on `stream` before
+ *     its kernel. Two calls that can overlap on the GPU (different streams, no dependency)
+ *     race on it and give wrong results: order them.
+ *   - It is slower than the context-based call (one token per thread, no shared-memory
+ *     tables); use it where allocation is impossible, not as the default.
+ */
+int cfgzip_step_noalloc(const int32_t* token_to_class /*dev [V]*/, int32_t V,
+                        const int32_t* class_to_rep /*dev [K]*/, int32_t K, const uint32_t* class_mask,
+                        int64_t class_stride_words, void* logits, int dtype, int64_t row_stride_elems,
+                        int32_t B, uint32_t* vocab_mask, int64_t vocab_stride_words, int32_t* argmax,
+                        int32_t* rep, float* logp_argmax, float* lse, void* stream);
+
 /* Kernels this context has launched so far (monotonic; for launch accounting). */
 int cfgzip_launch_count(cfgzip_ctx* ctx, int64_t* out);
 

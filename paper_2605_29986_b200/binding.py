@@ -34,6 +34,8 @@ _SIGNATURES = {
     "cfgzip_map_tokens": (_int, [_vp, _i32, _vp, _vp, _vp, _i32, _vp]),
     "cfgzip_decode_step_host": (_int, [_vp, _i32, _vp, _vp, _i64, _vp, _int, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _int,
                                        _vp]),
+    "cfgzip_step_noalloc": (_int, [_vp, _i32, _vp, _i32, _vp, _i64, _vp, _int, _i64, _i32, _vp, _i64, _vp, _vp, _vp, _vp,
+                                   _vp]),
     "cfgzip_poll_status": (_int, [_vp, _vp, ctypes.POINTER(_i32), ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
     "cfgzip_launch_count": (_int, [_vp, ctypes.POINTER(_i64)]),
     "cfgzip_set_tuning": (_int, [_vp, ctypes.c_char_p, _i32]),
@@ -165,6 +167,19 @@ def cfgzip_decode_step_host(ctx: int, part0: int, row_part_host, class_mask_host
         ctx, part0, _ptr(row_part_host), _ptr(class_mask_host), class_stride_words, _ptr(logits_host), dtype, B,
         _ptr(masked_logits), _ptr(vocab_mask_host), _ptr(argmax), _ptr(rep), _ptr(logp_argmax), _ptr(lse), mode,
         _stream(stream)), "cfgzip_decode_step_host")
+
+
+def cfgzip_step_noalloc(token_to_class, V: int, class_to_rep, K: int, class_mask, class_stride_words: int, logits,
+                        dtype: int, row_stride_elems: int, B: int, vocab_mask, vocab_stride_words: int, argmax,
+                        rep=None, logp_argmax=None, lse=None, stream=None) -> None:
+    """The fused step without a context and without any allocation (device-resident c and r, built-in scratch).
+
+    For hosts that may not call cudaMalloc where they need the step. At most 1024 rows; runs on the
+    current device; calls that could overlap on one GPU must be ordered by the caller."""
+    _check(load_library().cfgzip_step_noalloc(
+        _ptr(token_to_class), V, _ptr(class_to_rep), K, _ptr(class_mask), class_stride_words, _ptr(logits), dtype,
+        row_stride_elems, B, _ptr(vocab_mask), vocab_stride_words, _ptr(argmax), _ptr(rep), _ptr(logp_argmax),
+        _ptr(lse), _stream(stream)), "cfgzip_step_noalloc")
 
 
 def cfgzip_poll_status(ctx: int, stream=None) -> Tuple[int, int, int]:

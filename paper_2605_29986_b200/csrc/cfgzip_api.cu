@@ -6,6 +6,7 @@
 #include <algorithm>
 #include <cstdint>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -27,6 +28,15 @@ constexpr size_t kPartialSlots = size_t(1) << 18;  // 4 MB of (max, sum, pos) sl
 constexpr int kDefaultRows = 16384;
 
 }  // namespace
+
+// Scratch of cfgzip_step_noalloc: lives in the library image, one copy on every GPU that loads it.
+constexpr int kNoAllocMaxRows = 1024;
+constexpr int kNoAllocMaxSplits = 64;
+struct NoAllocScratch {
+    Partial partials[kNoAllocMaxRows * kNoAllocMaxSplits];  // 1 MiB
+    unsigned int tickets[kNoAllocMaxRows];                  // 4 KiB
+};
+static __device__ __align__(256) NoAllocScratch g_noalloc_scratch;
 
 struct cfgzip_ctx {
     int device = 0;
@@ -857,3 +867,87 @@ int cfgzip_set_tuning(cfgzip_ctx* ctx, const char* name, int32_t value) {
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// cfgzip_step_noalloc: see include/cfgzip.h. In host code `g_noalloc_scratch` is only a handle
+// for the runtime; the device address of each GPU's copy is asked for once per device.
+// ---------------------------------------------------------------------------------------------
+namespace {
+constexpr int kMaxDevices = 64;
+struct NoAllocDevice {
+    NoAllocScratch* scratch = nullptr;
+    int sm_count = 0;
+};
+NoAllocDevice g_noalloc_dev[kMaxDevices];
+std::mutex g_noalloc_mutex;
+}  // namespace
+
+extern "C" int cfgzip_step_noalloc(const int32_t* token_to_class, int32_t V, const int32_t* class_to_rep, int32_t K,
+                                   const uint32_t* class_mask, int64_t class_stride_words, void* logits, int dtype,
+                                   int64_t row_stride_elems, int32_t B, uint32_t* vocab_mask, int64_t vocab_stride_words,
+                                   int32_t* argmax, int32_t* rep, float* logp_argmax, float* lse, void* stream) {
+    if (V <= 0 || K <= 0 || K > V || B < 0 || (dtype != CFGZIP_F32 && dtype != CFGZIP_BF16)) return CFGZIP_E_ARG;
+    if (B == 0) return CFGZIP_OK;
+    if (B > kNoAllocMaxRows) return CFGZIP_E_RANGE;  // more rows than the built-in scratch has tickets for
+    const int VW = ceil_div(V, 32), KW = ceil_div(K, 32);
+    if (!token_to_class || !class_to_rep || !class_mask || !logits || !argmax) return CFGZIP_E_ARG;
+    if (class_stride_words < KW || row_stride_elems < V || (vocab_mask && vocab_stride_words < VW)) return CFGZIP_E_ARG;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        cudaGetLastError();
+        return CFGZIP_E_CUDA;
+    }
+    NoAllocDevice nd;
+    {
+        std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+        if (!g_noalloc_dev[dev].scratch) {
+            // first call on this GPU (it is the current device): ask where its copy of the array lives
+            NoAllocScratch* ptr = nullptr;
+            int sms = 0;
+            if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_noalloc_scratch) != cudaSuccess || !ptr ||
+                cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+                cudaGetLastError();
+                return CFGZIP_E_CUDA;
+            }
+            g_noalloc_dev[dev].scratch = ptr;
+            g_noalloc_dev[dev].sm_count = sms;
+        }
+        nd = g_noalloc_dev[dev];
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the array keeps whatever the last call left: the tickets must read zero when the kernel starts
+    if (cudaMemsetAsync(nd.scratch->tickets, 0, sizeof(unsigned int) * size_t(B), st) != cudaSuccess) {
+        cudaGetLastError();
+        return CFGZIP_E_CUDA;
+    }
+    RowSplitArgs a{};
+    a.c = token_to_class;
+    a.r = class_to_rep;
+    a.V = V;
+    a.K = K;
+    a.VW = VW;
+    a.class_mask = class_mask;
+    a.cm_stride = class_stride_words;
+    a.logits = logits;
+    a.row_stride = row_stride_elems;
+    a.vocab_mask = vocab_mask;
+    a.vm_stride = vocab_stride_words;
+    a.argmax = argmax;
+    a.rep = rep;
+    a.logp_argmax = logp_argmax;
+    a.lse = lse;
+    a.B = B;
+    int S = std::max(1, (4 * nd.sm_count) / B);
+    S = std::min(S, std::min(kNoAllocMaxSplits, std::max(1, VW / 64)));
+    a.words_per_split = ceil_div(VW, S);
+    a.S = ceil_div(VW, a.words_per_split);
+    a.partials = nd.scratch->partials;
+    a.tickets = nd.scratch->tickets;
+    const dim3 grid(unsigned(B) * unsigned(a.S)), block(256);
+    if (dtype == CFGZIP_BF16)
+        k_step_rowsplit<kBF16><<<grid, block, 0, st>>>(a);
+    else
+        k_step_rowsplit<kF32><<<grid, block, 0, st>>>(a);
+    if (cudaGetLastError() != cudaSuccess) return CFGZIP_E_CUDA;
+    return CFGZIP_OK;
+}

@@ -990,6 +990,110 @@ __global__ void __launch_bounds__(256) k_step_generic(const __grid_constant__ St
 }
 
 // ---------------------------------------------------------------------------------------
+// Row-split step on caller-provided tables: the per-row kernel above, with each row shared by
+// S blocks that meet through a scratch area of (max, sum-exp, token) states and one ticket
+// per row, exactly as the sparse kernel's blocks do. It touches no context: token->class and
+// class->representative vectors, masks, logits and outputs all come from the caller, the
+// scratch area from whoever launches it.
+// ---------------------------------------------------------------------------------------
+struct RowSplitArgs {
+    const int32_t* c;   // dev [V]
+    const int32_t* r;   // dev [K]
+    int32_t V, K, VW;
+    const uint32_t* class_mask;
+    int64_t cm_stride;
+    void* logits;
+    int64_t row_stride;
+    uint32_t* vocab_mask;  // nullable
+    int64_t vm_stride;
+    int32_t* argmax;
+    int32_t* rep;          // nullable
+    float* logp_argmax;    // nullable
+    float* lse;            // nullable
+    int32_t B, S, words_per_split;
+    Partial* partials;     // [B * S]
+    unsigned int* tickets; // [B], zero on entry, left zero
+};
+
+template <int DT>
+__global__ void __launch_bounds__(256) k_step_rowsplit(const __grid_constant__ RowSplitArgs a) {
+    __shared__ Partial s_red[8];
+    __shared__ int s_last;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, n_warps = blockDim.x >> 5;
+    const int row = blockIdx.x / a.S, split = blockIdx.x - row * a.S;
+    const uint32_t* cm = a.class_mask + int64_t(row) * a.cm_stride;
+    constexpr int ES = DT == kBF16 ? 2 : 4;
+    char* rowp = reinterpret_cast<char*>(a.logits) + int64_t(row) * a.row_stride * ES;
+    uint32_t* out = a.vocab_mask ? a.vocab_mask + int64_t(row) * a.vm_stride : nullptr;
+    const int w_begin = split * a.words_per_split, w_end = min(w_begin + a.words_per_split, a.VW);
+    float m = -INFINITY, s = 0.f;
+    int pos = kNoPos;
+    for (int w = w_begin + warp; w < w_end; w += n_warps) {
+        const int t = w * 32 + lane;
+        bool allowed = false;
+        if (t < a.V) {
+            const int k = __ldg(a.c + t);
+            if (k >= 0 && k < a.K) allowed = (__ldg(cm + (k >> 5)) >> (k & 31)) & 1u;  // ids out of range: not allowed
+        }
+        const uint32_t word = __ballot_sync(0xFFFFFFFFu, allowed);
+        if (out && lane == 0) out[w] = word;
+        if (t < a.V) {
+            if (allowed) {
+                const float z = load_elem<DT>(rowp, t);
+                const bool upd = (z > m) || pos == kNoPos;
+                pos = upd ? t : pos;
+                const float ref_old = fmaxf(m, kRefFloor);
+                m = fmaxf(m, z);
+                const float ref = fmaxf(m, kRefFloor);
+                s = fmaf(s, ex2f((ref_old - ref) * kLog2e), ex2f((z - ref) * kLog2e));
+            } else {
+                store_neg_inf<DT>(rowp, t);
+            }
+        }
+    }
+    partial_warp_allreduce(m, s, pos);
+    if (lane == 0) s_red[warp] = Partial{m, s, pos, 0};
+    __syncthreads();
+    if (warp != 0) return;
+    if (lane == 0)
+        for (int w = 1; w < n_warps; ++w) partial_merge(m, s, pos, s_red[w].m, s_red[w].s, s_red[w].pos);
+    if (a.S > 1) {
+        if (lane == 0) {
+            a.partials[int64_t(row) * a.S + split] = Partial{m, s, pos, 0};
+            __threadfence();
+            s_last = (atomicAdd(a.tickets + row, 1u) == unsigned(a.S - 1));
+        }
+        __syncwarp();
+        if (!s_last) return;
+        __threadfence();
+        m = -INFINITY; s = 0.f; pos = kNoPos;
+        for (int sp = lane; sp < a.S; sp += 32) {
+            const int4 raw = __ldcg(reinterpret_cast<const int4*>(a.partials + int64_t(row) * a.S + sp));
+            partial_merge(m, s, pos, __int_as_float(raw.x), __int_as_float(raw.y), raw.z);
+        }
+        partial_warp_allreduce(m, s, pos);
+        if (lane == 0) a.tickets[row] = 0u;
+    }
+    if (lane != 0) return;
+    int tok = -1, repv = -1;
+    float lsev = -INFINITY, lpa = -INFINITY;
+    if (pos != kNoPos) {
+        tok = pos;
+        const int k = a.c[tok];
+        repv = a.r[k];
+        if (m > kRefFloor && s > 0.f) {
+            const float l = logf(s);
+            lsev = m + l;
+            lpa = -l;
+        }
+    }
+    a.argmax[row] = tok;
+    if (a.rep) a.rep[row] = repv;
+    if (a.lse) a.lse[row] = lsev;
+    if (a.logp_argmax) a.logp_argmax[row] = lpa;
+}
+
+// ---------------------------------------------------------------------------------------
 // Row plan for batches that mix partitions: bucket the rows by partition into groups of
 // up to 32 rows (valid slots first). One block.
 // ---------------------------------------------------------------------------------------
