@@ -370,9 +370,9 @@ def run_own(args):
     barrier()
     e2e_s, h2d, d2h = _e2e(runner, torch, e2e_steps)
     if dist is not None:
-        t = torch.tensor([seconds, e2e_s], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        seconds, e2e_s = float(t[0]), float(t[1])
+        from paper_2605_29986_b200 import rows
+        seconds = rows.max_over_ranks(seconds, dist, device="cuda")
+        e2e_s = rows.max_over_ranks(e2e_s, dist, device="cuda")
     peak, peak_src = _measured_peak()
     alg = runner.alg_bytes()
     per_launch_s = seconds / max(launches, 1)

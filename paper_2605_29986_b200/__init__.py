@@ -3,5 +3,12 @@
 ``from paper_2605_29986_b200 import binding`` gives the calls of ``include/cfgzip.h`` under the
 same names. The CUDA library is built in-tree with nvcc (sm_100a) on first use.
 """
-from . import binding  # noqa: F401
-from .binding import *  # noqa: F401,F403
+from . import rows  # noqa: F401
+
+
+def __getattr__(name):
+    # the CUDA binding is imported on first use, so that host-only helpers work without nvcc or a GPU
+    if name == "binding":
+        import importlib
+        return importlib.import_module(".binding", __name__)
+    raise AttributeError(name)

@@ -1,0 +1,75 @@
+"""The five workloads at their full sizes, through the fused entry point in the launch shape the bench uses.
+
+Inputs follow the workload recipes (unique logits rows are generated for up to 64 rows and tiled to
+the batch; every row has its own class mask). All rows are compared with the CPU oracle where that
+takes seconds; for the largest batches a spread sample of rows is compared and the remaining rows
+are checked by properties that hold at any size (popcount of the vocab mask = summed sizes of the
+allowed classes, -inf count of the masked logits, the chosen token is allowed and maps to its
+representative) and, for the sparse stress workload, by bit-equality of the dense and sparse paths.
+"""
+import numpy as np
+import pytest
+import torch
+
+import synth
+from paper_2605_29986_b200 import binding as cz
+from _gpu_util import Ctx, compare_step, oracle_step, run_fused
+
+pytestmark = pytest.mark.gpu
+
+ORACLE_ROWS = {1: 1, 2: 32, 3: 128, 4: 64, 5: 64}
+
+
+def _inputs(config, step):
+    spec = synth.CONFIGS[config]
+    B = spec["B"]
+    wu = synth.make_workload(config, B=min(B, 64))   # unique logits rows
+    wf = wu if B <= 64 else synth.make_workload(config, B=B)  # class masks for every row
+    tile = -(-B // wu.B)
+    z = np.tile(wu.logits(step), (tile, 1))[:B]
+    cm = wf.class_masks(step)
+    row_part = None if wf.row_part is None else wf.row_part
+    return wf, row_part, cm, z
+
+
+def _popcount_rows(words):
+    return np.unpackbits(np.ascontiguousarray(words).view(np.uint8), axis=-1).sum(axis=-1)
+
+
+def _properties(w, row_part, cm, got, V):
+    B = cm.shape[0]
+    pc = _popcount_rows(got["vocab_mask"])
+    neg = (got["logits"].view(np.uint16 if got["logits"].dtype == np.uint16 else np.uint32)
+           == (0xFF80 if got["logits"].dtype == np.uint16 else 0xFF800000)).sum(axis=1)
+    for b in range(B):
+        p = w.partitions[0 if row_part is None else int(row_part[b])]
+        allowed = synth.unpack_bits(cm[b:b + 1], p.K)[0]
+        assert pc[b] == int(p.sizes[allowed].sum()), "row %d popcount" % b
+        assert neg[b] >= V - pc[b]
+        t = int(got["argmax"][b])
+        if pc[b] == 0:
+            assert t == -1 and got["rep"][b] == -1
+        else:
+            assert allowed[p.c[t]] and got["rep"][b] == p.r[p.c[t]]
+            assert got["logp_argmax"][b] <= 1e-6
+
+
+@pytest.mark.parametrize("config", [1, 2, 3, 4, 5])
+def test_full_size_workload(config):
+    spec = synth.CONFIGS[config]
+    V, B = spec["V"], spec["B"]
+    for step in (0, 1):
+        w, row_part, cm, z = _inputs(config, step)
+        with Ctx(w.partitions) as ctx:
+            got = run_fused(ctx, row_part, cm, z, V, mode=cz.DENSE)
+            assert cz.cfgzip_poll_status(ctx.h)[1:] == (0, 0)
+            if config == 5:
+                sparse = run_fused(ctx, row_part, cm, z, V, mode=cz.SPARSE)
+                for key in ("vocab_mask", "logits", "argmax", "rep"):
+                    assert np.array_equal(got[key].view(np.uint8), sparse[key].view(np.uint8)), key
+                assert np.abs(got["lse"] - sparse["lse"]).max() <= 1e-4
+        _properties(w, row_part, cm, got, V)
+        rows = np.unique(np.linspace(0, B - 1, ORACLE_ROWS[config]).astype(np.int64))
+        sub = {k: (v[rows] if v is not None else None) for k, v in got.items()}
+        want = oracle_step(w.partitions, None if row_part is None else row_part[rows], cm[rows], z[rows], V)
+        compare_step(sub, want, V, "config %d step %d" % (config, step))
