@@ -148,6 +148,7 @@ void build_class_lists_host(const int32_t* c, int32_t V, int32_t K, int32_t* off
 struct PartSet {
     int32_t V = 0, VW = 0, maxK = 0, maxKW = 0, n_live_same_v = 0;
     bool all_c16 = true;
+    bool all_kw_mult4 = true;
 };
 
 int resolve_parts(cfgzip_ctx* ctx, cfgzip_part_id part0, bool mixed, PartSet* ps) {
@@ -160,6 +161,7 @@ int resolve_parts(cfgzip_ctx* ctx, cfgzip_part_id part0, bool mixed, PartSet* ps
         ps->maxKW = p0.KW;
         ps->n_live_same_v = 1;
         ps->all_c16 = p0.dev.c16 != nullptr;
+        ps->all_kw_mult4 = (p0.KW % 4) == 0;
         return CFGZIP_OK;
     }
     for (const Part& p : ctx->parts) {
@@ -168,6 +170,7 @@ int resolve_parts(cfgzip_ctx* ctx, cfgzip_part_id part0, bool mixed, PartSet* ps
         ps->maxKW = std::max(ps->maxKW, p.KW);
         ps->n_live_same_v += 1;
         ps->all_c16 = ps->all_c16 && p.dev.c16 != nullptr;
+        ps->all_kw_mult4 = ps->all_kw_mult4 && (p.KW % 4) == 0;
     }
     return CFGZIP_OK;
 }
@@ -185,6 +188,7 @@ size_t dense_smem_bytes(int table_words, int n_warps, int stage_stride) {
 struct DensePlan {
     int S = 1, per_split = 0, WT = 4, threads = 128, table_words = 0, stage_stride = 0;
     int depth = 0;       // > 0: pipelined kernel with this many stages per warp
+    int cm_bulk = 0;     // pipelined kernel: class masks staged by bulk copies
     int ctas_per_sm = 1; // blocks per SM the launch was sized for
     size_t smem = 0;
     int n_groups_ub = 1;
@@ -198,10 +202,10 @@ size_t pipe_smem_bytes(int table_words, int n_warps, int depth, int stage_bytes,
            size_t(stage_stride) * kGroupRows * 4;
 }
 
+// Launch shape of the register-based dense kernels.
 // units: octets (fused) or 32-token words (expand); unit_chunk: units one warp covers per iteration.
-// elem_size: bytes per logit when the pipelined kernel may be used (aligned fused call), else 0.
 DensePlan plan_dense(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, int units, int unit_chunk,
-                     bool fused, int elem_size) {
+                     bool fused) {
     DensePlan d;
     d.table_words = (ps.maxKW + 1) * 32;
     d.use_plan_kernel = mixed;
@@ -209,30 +213,9 @@ DensePlan plan_dense(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, 
     if (!ps.all_c16) return d;
     if (dense_smem_bytes(d.table_words, 8, 0) > size_t(ctx->smem_optin) - 2048) return d;
     if (mixed && (B > ctx->reserved_rows || d.n_groups_ub > ctx->max_groups)) return d;
-    int ctas_per_sm = ctx->ctas_per_sm;
-    int n_warps = 4;
-    if (fused && elem_size && ctx->pipeline) {
-        const int stage_bytes = 8 * 32 * 8 * elem_size + 512;
-        n_warps = ctx->pipe_warps;
-        int depth = ctx->pipe_depth;
-        const size_t cap = size_t(ctx->smem_optin) - 2048;  // room for the kernels' static shared memory
-        int stride = ps.maxKW | 1;
-        if (pipe_smem_bytes(d.table_words, n_warps, 2, stage_bytes, stride) > cap) stride = 0;
-        while (depth > 2 && pipe_smem_bytes(d.table_words, n_warps, depth, stage_bytes, stride) > cap) --depth;
-        while (n_warps > 4 && pipe_smem_bytes(d.table_words, n_warps, depth, stage_bytes, stride) > cap) n_warps -= 2;
-        const size_t smem = pipe_smem_bytes(d.table_words, n_warps, depth, stage_bytes, stride);
-        if (smem <= cap) {
-            d.depth = depth;
-            d.smem = smem;
-            d.stage_stride = stride;
-            const int fit = std::max(1, int((cap + 1024) / (smem + 1024)));
-            ctas_per_sm = std::min(ctas_per_sm, fit);
-        }
-    }
-    if (!d.depth) {
-        // stage the class masks through shared memory while that keeps a block under 64 KB
-        if (dense_smem_bytes(d.table_words, 8, ps.maxKW | 1) <= 64 * 1024) d.stage_stride = ps.maxKW | 1;
-    }
+    const int ctas_per_sm = ctx->ctas_per_sm;
+    // stage the class masks through shared memory while that keeps a block under 64 KB
+    if (dense_smem_bytes(d.table_words, 8, ps.maxKW | 1) <= 64 * 1024) d.stage_stride = ps.maxKW | 1;
     d.ctas_per_sm = ctas_per_sm;
     const int target = ctx->sm_count * ctas_per_sm;
     const int n_chunks = ceil_div(units, unit_chunk);
@@ -240,27 +223,11 @@ DensePlan plan_dense(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, 
     int cps = ceil_div(n_chunks, s0);  // chunks per block
     int WR = 1;
     if (fused) {
-        if (d.depth) {
-            // one row batch per warp where the warp count allows: a warp then reduces its rows once
-            WR = ctx->row_warps ? ctx->row_warps : (n_warps % 4 == 0 ? 4 : (n_warps % 2 == 0 ? 2 : 1));
-            while (WR > 1 && (WR - 1) * kBatchRows >= std::min<int>(B, kGroupRows)) WR >>= 1;
-            if ((WR != 1 && WR != 2 && WR != 4) || n_warps % WR) WR = 1;
-            d.WT = ctx->token_warps ? ctx->token_warps : n_warps / WR;
-            d.WT = std::max(1, std::min(d.WT, 16 / WR));
-            cps = ceil_div(cps, d.WT) * d.WT;  // every warp of a block gets the same number of chunks
-        } else {
-            WR = ctx->row_warps ? ctx->row_warps : (cps <= 2 ? 4 : 1);
-            if (WR != 1 && WR != 2 && WR != 4) WR = 1;
-            d.WT = ctx->token_warps ? ctx->token_warps : (WR == 4 ? std::min(cps, 2) : (WR == 2 ? 2 : 4));
-            d.WT = std::max(1, std::min(d.WT, 8 / WR));
-        }
+        WR = ctx->row_warps ? ctx->row_warps : (cps <= 2 ? 4 : 1);
+        if (WR != 1 && WR != 2 && WR != 4) WR = 1;
+        d.WT = ctx->token_warps ? ctx->token_warps : (WR == 4 ? std::min(cps, 2) : (WR == 2 ? 2 : 4));
+        d.WT = std::max(1, std::min(d.WT, 8 / WR));
         d.threads = d.WT * WR * 32;
-        if (d.depth) {
-            // the ring was sized for n_warps; recompute for the warps actually launched
-            const int stage_bytes = 8 * 32 * 8 * elem_size + 512;
-            d.smem = pipe_smem_bytes(d.table_words, d.threads / 32, d.depth, stage_bytes, d.stage_stride);
-            if (d.smem > size_t(ctx->smem_optin) - 2048) return d;
-        }
     } else {
         d.WT = 8;
         d.threads = 256;
@@ -272,7 +239,62 @@ DensePlan plan_dense(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, 
     }
     if (fused && d.S > 1 && d.n_groups_ub > ctx->reserved_rows) return d;  // tickets
     d.per_split = cps * unit_chunk;
-    if (!d.depth) d.smem = dense_smem_bytes(d.table_words, fused ? d.threads / 32 : 0, d.stage_stride);
+    d.smem = dense_smem_bytes(d.table_words, fused ? d.threads / 32 : 0, d.stage_stride);
+    d.ok = true;
+    return d;
+}
+
+// Launch shape of the pipelined fused kernel. A block takes per_split octets (any number, not only
+// whole 32-octet chunks) of one row group, so that the blocks of a step fill the SMs evenly.
+DensePlan plan_pipe(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, int elem_size, bool cm_bulk_ok) {
+    DensePlan d;
+    d.table_words = (ps.maxKW + 1) * 32;
+    d.use_plan_kernel = mixed;
+    d.n_groups_ub = mixed ? ceil_div(B, kGroupRows) + ps.n_live_same_v : ceil_div(B, kGroupRows);
+    if (!ps.all_c16 || !ctx->pipeline) return d;
+    if (mixed && (B > ctx->reserved_rows || d.n_groups_ub > ctx->max_groups)) return d;
+    const int stage_bytes = 8 * 32 * 8 * elem_size + 512;
+    const size_t cap = size_t(ctx->smem_optin) - 2048;  // room for the kernel's static shared memory
+    int n_warps = ctx->pipe_warps, depth = ctx->pipe_depth;
+    d.cm_bulk = cm_bulk_ok && ps.all_kw_mult4;
+    int stride = d.cm_bulk ? ps.maxKW + (ps.maxKW % 8 == 0 ? 4 : 8) : (ps.maxKW | 1);
+    if (pipe_smem_bytes(d.table_words, n_warps, 2, stage_bytes, stride) > cap) {
+        stride = 0;
+        d.cm_bulk = 0;
+    }
+    while (depth > 2 && pipe_smem_bytes(d.table_words, n_warps, depth, stage_bytes, stride) > cap) --depth;
+    while (n_warps > 4 && pipe_smem_bytes(d.table_words, n_warps, depth, stage_bytes, stride) > cap) n_warps -= 2;
+    size_t smem = pipe_smem_bytes(d.table_words, n_warps, depth, stage_bytes, stride);
+    if (smem > cap) return d;
+    d.depth = depth;
+    d.stage_stride = stride;
+    const int fit = std::max(1, int((cap + 1024) / (smem + 1024)));
+    d.ctas_per_sm = std::min(ctx->ctas_per_sm, fit);
+    const int target = ctx->sm_count * d.ctas_per_sm;
+    const int n_oct = 4 * ps.VW;
+    const int s0 = std::max(1, target / d.n_groups_ub);
+    int per = std::max(32, ceil_div(n_oct, s0));
+    // Warps go side by side along the vocabulary first (long contiguous runs per row are kind to
+    // DRAM); only when a block has fewer 32-octet chunks than warps do warps split the row batches.
+    const int chunks = ceil_div(per, 32);
+    int WR = ctx->row_warps;
+    if (!WR) {
+        WR = 1;
+        while (WR < 4 && chunks * WR * 2 <= n_warps) WR <<= 1;
+    }
+    while (WR > 1 && (WR - 1) * kBatchRows >= std::min<int>(B, kGroupRows)) WR >>= 1;
+    if ((WR != 1 && WR != 2 && WR != 4)) WR = 1;
+    d.WT = ctx->token_warps ? ctx->token_warps : n_warps / WR;
+    d.WT = std::max(1, std::min(std::min(d.WT, 16 / WR), chunks));
+    d.threads = d.WT * WR * 32;
+    for (;;) {
+        d.S = ceil_div(n_oct, per);
+        if (d.S == 1 || size_t(d.n_groups_ub) * kGroupRows * size_t(d.S) <= kPartialSlots) break;
+        per *= 2;
+    }
+    if (d.S > 1 && d.n_groups_ub > ctx->reserved_rows) return d;  // tickets
+    d.per_split = per;
+    d.smem = pipe_smem_bytes(d.table_words, d.threads / 32, d.depth, stage_bytes, d.stage_stride);
     d.ok = true;
     return d;
 }
@@ -307,6 +329,7 @@ void fill_groups(cfgzip_ctx* ctx, StepArgs& a, const DensePlan& d) {
     a.table_words = d.table_words;
     a.stage_stride = d.stage_stride;
     a.depth = d.depth;
+    a.cm_bulk = d.cm_bulk;
     a.p0 = ctx->parts[size_t(a.part0)].dev;
 }
 
@@ -354,7 +377,9 @@ int launch_fused(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, in
             rc = launch(ctx, k_step_generic<DT, true>, dim3(unsigned(a.B)), dim3(256), 0, st, a);
         }
     } else {
-        const DensePlan d = plan_dense(ctx, ps, a.B, mixed, 4 * ps.VW, 32, true, DT == kBF16 ? 2 : 4);
+        const bool cm_bulk_ok = (reinterpret_cast<uintptr_t>(a.class_mask) & 15u) == 0 && (a.cm_stride & 3) == 0;
+        DensePlan d = plan_pipe(ctx, ps, a.B, mixed, DT == kBF16 ? 2 : 4, cm_bulk_ok);
+        if (!d.ok) d = plan_dense(ctx, ps, a.B, mixed, 4 * ps.VW, 32, true);
         if (d.ok) {
             if (d.use_plan_kernel && (rc = run_plan_kernel(ctx, a.row_part, a.B, a.V, d, st)) != CFGZIP_OK) return rc;
             fill_groups(ctx, a, d);
@@ -655,7 +680,7 @@ int cfgzip_expand_mask(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row
         }
         return launch(ctx, k_step_generic<kF32, false>, dim3(unsigned(B)), dim3(256), 0, st, a);
     }
-    const DensePlan d = plan_dense(ctx, ps, B, mixed, ps.VW, 8, false, 0);
+    const DensePlan d = plan_dense(ctx, ps, B, mixed, ps.VW, 8, false);
     if (!d.ok) return launch(ctx, k_step_generic<kF32, false>, dim3(unsigned(B)), dim3(256), 0, st, a);
     if (d.use_plan_kernel && (rc = run_plan_kernel(ctx, row_part, B, ps.V, d, st)) != CFGZIP_OK) return rc;
     fill_groups(ctx, a, d);

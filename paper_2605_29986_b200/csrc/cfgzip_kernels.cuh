@@ -37,6 +37,7 @@ struct StepArgs {
     int32_t table_words;        // dense: shared-memory words of the bit-sliced class table
     int32_t stage_stride;       // dense: words per row of the class-mask staging area, 0 = no staging
     int32_t depth;              // pipelined dense kernel: stages per warp
+    int32_t cm_bulk;            // pipelined dense kernel: class-mask rows are fetched by bulk copies (16-byte aligned rows)
     PartDev p0;                 // descriptor of part0 (saves a dependent load when rows do not mix partitions)
     Partial* partials;
     unsigned int* tickets;
@@ -192,6 +193,25 @@ __device__ __forceinline__ void build_class_table(const StepArgs& a, const PartD
     }
 }
 
+// The same table from a staging area whose rows are 16-byte aligned and stage_stride (a
+// multiple of 4, with stage_stride/4 odd) words apart: a lane reads four words of its row at
+// once, which spreads the eight lanes of a quarter warp over all 32 banks.
+__device__ __forceinline__ void build_class_table_quads(const StepArgs& a, const PartDev& P, const int* s_row, uint32_t* T,
+                                                        const uint32_t* stage, int warp, int lane, int n_warps) {
+    const uint32_t tail = (P.K & 31) ? (1u << (P.K & 31)) - 1u : 0xFFFFFFFFu;
+    const bool have = s_row[lane] >= 0;
+    for (int q = warp; 4 * q < P.KW; q += n_warps) {  // KW is a multiple of 4 here
+        uint4 x = make_uint4(0, 0, 0, 0);
+        if (have) x = *reinterpret_cast<const uint4*>(stage + lane * a.stage_stride + 4 * q);
+        if (4 * q + 4 == P.KW) x.w &= tail;
+        const uint32_t t0 = warp_transpose32(x.x, lane), t1 = warp_transpose32(x.y, lane);
+        const uint32_t t2 = warp_transpose32(x.z, lane), t3 = warp_transpose32(x.w, lane);
+        uint32_t* dst = T + (4 * q) * 32 + lane;
+        dst[0] = t0; dst[32] = t1; dst[64] = t2; dst[96] = t3;
+    }
+    if (warp == 0) T[P.KW * 32 + lane] = 0u;  // the padding class
+}
+
 // Allow bits of rows 8*rb .. 8*rb+7 for the 8 tokens whose class ids are packed in cv:
 // byte i of (lo, hi) belongs to row 8*rb + i, bit j of it to token j of the octet.
 __device__ __forceinline__ void octet_allow_bits(const uint4& cv, const uint32_t* T, int rb, bool active, uint32_t& lo,
@@ -279,6 +299,27 @@ struct DenseTail {
     unsigned long long pick[kGroupRows];  // (token id << 32) | representative of the best match
 };
 
+// Fold red[w][row] over the warps w of a block into fin[row] with shuffle trees: the states of
+// one row sit in neighbouring lanes (a power-of-two group), so log2(warps) fold steps suffice.
+__device__ __forceinline__ void fold_red_rows(const Partial* red, int n_warps, Partial* fin) {
+    int group = 1;
+    while (group < n_warps) group <<= 1;  // 1, 2, 4, 8 or 16 lanes per row
+    const int tid = threadIdx.x;
+    for (int base = 0; base < kGroupRows * group; base += blockDim.x) {  // same trip count for every warp
+        const int q = base + tid;
+        const int row = q / group, w = q & (group - 1);
+        Partial p = partial_empty();
+        if (row < kGroupRows && w < n_warps) p = red[w * kGroupRows + row];
+        for (int d = group >> 1; d >= 1; d >>= 1) {
+            const float m2 = __shfl_xor_sync(0xFFFFFFFFu, p.m, d);
+            const float s2 = __shfl_xor_sync(0xFFFFFFFFu, p.s, d);
+            const int p2 = __shfl_xor_sync(0xFFFFFFFFu, p.pos, d);
+            partial_merge(p.m, p.s, p.pos, m2, s2, p2);
+        }
+        if (row < kGroupRows && w == 0) fin[row] = p;
+    }
+}
+
 // End of a dense block: every warp has left the states of the rows it streamed in
 // red[warp][row slot]. Fold them, publish / collect across the S blocks of the group, then
 // turn each complete row state into the row's outputs.
@@ -288,50 +329,40 @@ __device__ __forceinline__ void dense_block_tail(const StepArgs& a, const PartDe
     constexpr int ES = DT == kBF16 ? 2 : 4;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, n_warps = blockDim.x >> 5;
     __syncthreads();
-    float rm = -INFINITY, rs = 0.f;
-    int rpos = kNoPos;
-    if (tid < kGroupRows) {
-        for (int w = 0; w < n_warps; ++w) {
-            const Partial p = red[w * kGroupRows + tid];
-            partial_merge(rm, rs, rpos, p.m, p.s, p.pos);
-        }
-    }
+    fold_red_rows(red, n_warps, tl.fin);
     if (a.S > 1) {
         // several blocks share the group: publish, and let the last one to arrive finish the rows
-        if (tid < kGroupRows)
-            a.partials[(int64_t(g) * a.S + split) * kGroupRows + tid] = Partial{rm, rs, rpos, 0};
+        __syncthreads();
+        if (tid < kGroupRows) a.partials[(int64_t(g) * a.S + split) * kGroupRows + tid] = tl.fin[tid];
         __threadfence();
         __syncthreads();
         if (tid == 0) tl.last = (atomicAdd(a.tickets + g, 1u) == unsigned(a.S - 1));
         __syncthreads();
         if (!tl.last) return;
         __threadfence();
-        // every thread folds a strided share of the S published states of its row slot
+        // every thread folds a strided share of the S published states of its row slot (two chains, so
+        // that the folds of one hide behind the other's)
         const Partial* src = a.partials + int64_t(g) * a.S * kGroupRows + lane;
-        rm = -INFINITY; rs = 0.f; rpos = kNoPos;
+        float m0 = -INFINITY, s0 = 0.f, m1 = -INFINITY, s1 = 0.f;
+        int p0 = kNoPos, p1 = kNoPos;
 #pragma unroll 8
-        for (int sp = warp; sp < a.S; sp += n_warps) {
-            const int4 raw = __ldcg(reinterpret_cast<const int4*>(src + sp * kGroupRows));
-            partial_merge(rm, rs, rpos, __int_as_float(raw.x), __int_as_float(raw.y), raw.z);
+        for (int sp = warp; sp < a.S; sp += 2 * n_warps) {
+            const int4 ra = __ldcg(reinterpret_cast<const int4*>(src + sp * kGroupRows));
+            int4 rb = make_int4(__float_as_int(-INFINITY), 0, kNoPos, 0);
+            if (sp + n_warps < a.S) rb = __ldcg(reinterpret_cast<const int4*>(src + (sp + n_warps) * kGroupRows));
+            partial_merge(m0, s0, p0, __int_as_float(ra.x), __int_as_float(ra.y), ra.z);
+            partial_merge(m1, s1, p1, __int_as_float(rb.x), __int_as_float(rb.y), rb.z);
         }
-        red[warp * kGroupRows + lane] = Partial{rm, rs, rpos, 0};
+        partial_merge(m0, s0, p0, m1, s1, p1);
+        red[warp * kGroupRows + lane] = Partial{m0, s0, p0, 0};
         __syncthreads();
-        rm = -INFINITY; rs = 0.f; rpos = kNoPos;
-        if (tid < kGroupRows) {
-            for (int w = 0; w < n_warps; ++w) {
-                const Partial p = red[w * kGroupRows + tid];
-                partial_merge(rm, rs, rpos, p.m, p.s, p.pos);
-            }
-        }
+        fold_red_rows(red, n_warps, tl.fin);
         if (tid == 0) a.tickets[g] = 0u;
     }
+    if (tid < kGroupRows) tl.pick[tid] = ~0ull;
+    __syncthreads();
     // rows are complete: 8 threads per row look at the 8 tokens of the winning octet at once and
     // fetch each candidate's representative alongside, so nothing is left to load afterwards
-    if (tid < kGroupRows) {
-        tl.fin[tid] = Partial{rm, rs, rpos, 0};
-        tl.pick[tid] = ~0ull;
-    }
-    __syncthreads();
     for (int idx = tid; idx < nrow * 8; idx += blockDim.x) {
         const int j = idx >> 3;
         const Partial p = tl.fin[j];
@@ -577,6 +608,7 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
     char* ring = reinterpret_cast<char*>(bars) + ((n_warps * a.depth * 8 + 127) & ~127);  // keeps 128-byte alignment
     uint32_t* stage = reinterpret_cast<uint32_t*>(ring + size_t(n_warps) * a.depth * G::kStageBytes);
     __shared__ DenseTail tl;
+    __shared__ uint64_t cm_bar;
 
     pdl_prologue();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -634,17 +666,37 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
 
     if (lane == 0) {
         for (int d = 0; d < depth; ++d) mbar_init(bar + d, 1);
+        if (warp == 0) mbar_init(&cm_bar, 1);
         mbar_init_fence();
+    }
+    if (a.cm_bulk) {
+        __syncthreads();  // the class-mask barrier is initialised for everybody
+        if (warp == 0) {
+            // one bulk copy per row of the group, issued side by side by the lanes of one warp
+            if (lane == 0) mbar_expect_tx(&cm_bar, uint32_t(nrow) * uint32_t(P.KW) * 4u);
+            __syncwarp();
+            const int row = s_row[lane];
+            if (row >= 0)
+                bulk_g2s(stage + lane * a.stage_stride, a.class_mask + int64_t(row) * a.cm_stride, uint32_t(P.KW) * 4u, &cm_bar);
+        }
+    }
+    if (lane == 0)
         while (p_n < min(depth, n_items)) issue_next();  // in flight while the table is built
-    }
-    if (a.stage_stride) {
-        stage_class_masks(a, P, s_row, stage, warp, lane, n_warps);
-        __syncthreads();
-    }
-    build_class_table(a, P, s_row, T, stage, warp, lane, n_warps);
-    __syncthreads();
-
     bool failed = false;
+    if (a.cm_bulk) {
+        if (!mbar_wait(&cm_bar, 0)) failed = true;
+        build_class_table_quads(a, P, s_row, T, stage, warp, lane, n_warps);
+    } else {
+        if (a.stage_stride) {
+            stage_class_masks(a, P, s_row, stage, warp, lane, n_warps);
+            __syncthreads();
+        }
+        build_class_table(a, P, s_row, T, stage, warp, lane, n_warps);
+    }
+    __syncthreads();
+    if (__any_sync(0xFFFFFFFFu, failed) && lane == 0) atomicAdd(a.status + 3, 1);  // class masks never arrived
+    failed = false;
+
     int slot = 0;
     uint32_t phase = 0;
     int consumed = 0;
