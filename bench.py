@@ -44,7 +44,7 @@ RING_MAX_BYTES = 24 << 30
 # DRAM traffic of the dominant kernel per launch (dram__bytes_read.sum + dram__bytes_write.sum
 # from one ncu capture), keyed by workload; valid only for the kernel sources whose digest is
 # recorded with it. None until a capture of the current sources exists.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {"cfg2_B32_dense": {"digest": "a4c5b8e2590868fc", "bytes_per_launch": 8565333}}
 
 
 def _kernel_digest() -> str:
@@ -403,7 +403,8 @@ def run_own(args):
                         "logp_argmax out; synchronised every step"},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": traffic, "peak_source": "of " + peak_src, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                     "algorithmic_bytes_per_launch": alg, "kernel": "k_step_%s" % args.mode},
+                     "algorithmic_bytes_per_launch": alg,
+                     "kernel": "k_step_dense_pipe" if args.mode != "sparse" else "k_step_sparse"},
         "clocks": sampler.summary(),
         "paper_context": "paper reports no timing of this path; its speedups (up to two orders of magnitude in grammar-engine "
                          "latency, up to 7.5x end to end) are for 1x H100 + Xeon Gold 6430 x16 threads, precision unstated",
