@@ -228,12 +228,14 @@ int cfgzip_launch_count(cfgzip_ctx* ctx, int64_t* out);
  *   "ctas_per_sm"  target resident thread blocks per SM for the fused kernel (1..16)
  *   "token_warps"  0 = automatic, else warps side by side along the vocabulary (1..16)
  *   "row_warps"    0 = automatic, else 1, 2 or 4 row batches handled by separate warps
- *   "pdl"          1 = launch with programmatic dependent launch (default), 0 = off
+ *   "pdl"          1 = programmatic dependent launch where it pays (steps under 48 MB of logits;
+ *                  default), 0 = never, 2 = always
  *   "pipeline"     1 = aligned logits stream through per-warp rings of bulk asynchronous copies
  *                  in shared memory (default), 0 = plain 16-byte loads into registers
  *   "tensor_map"   1 = a batch of 8 consecutive rows arrives as one tiled 2-D copy through a
  *                  tensor map (default), 0 = one bulk copy per row
  *   "pipe_warps"   warps per thread block of the pipelined kernel (1..16)
+ *   "waves"        thread blocks launched per resident block slot of the pipelined kernel (1..16)
  *   "pipe_depth"   stages per warp of the pipelined kernel (2..8; lowered to fit shared memory)
  * Unknown names give CFGZIP_E_ARG.
  */

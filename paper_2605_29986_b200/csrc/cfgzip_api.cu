@@ -67,6 +67,7 @@ struct cfgzip_ctx {
     int32_t token_warps = 0;
     int32_t row_warps = 0;
     int32_t pdl = 1;
+    bool pdl_now = true;      // set per call: programmatic dependent launch only pays for short kernels
     // cuTensorMapEncodeTiled, looked up through the runtime (no link against the driver library)
     CUresult (*encode_tiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -75,6 +76,7 @@ struct cfgzip_ctx {
     int32_t tensor_map = 1;   // tiled 2-D copies for row batches that are consecutive rows
     int32_t pipe_warps = 8;
     int32_t pipe_depth = 4;
+    int32_t waves = 1;        // pipelined kernel: blocks launched per resident block slot
 };
 
 namespace {
@@ -103,7 +105,7 @@ int launch(cfgzip_ctx* ctx, void (*kernel)(KArgs...), dim3 grid, dim3 block, siz
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = ctx->pdl ? 1 : 0;
+    cfg.numAttrs = (ctx->pdl == 2 || (ctx->pdl && ctx->pdl_now)) ? 1 : 0;
     if (cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...) != cudaSuccess) {
         cudaGetLastError();
         return CFGZIP_E_CUDA;
@@ -270,7 +272,7 @@ DensePlan plan_pipe(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, i
     d.stage_stride = stride;
     const int fit = std::max(1, int((cap + 1024) / (smem + 1024)));
     d.ctas_per_sm = std::min(ctx->ctas_per_sm, fit);
-    const int target = ctx->sm_count * d.ctas_per_sm;
+    const int target = ctx->sm_count * d.ctas_per_sm * ctx->waves;
     const int n_oct = 4 * ps.VW;
     const int s0 = std::max(1, target / d.n_groups_ub);
     int per = std::max(32, ceil_div(n_oct, s0));
@@ -753,8 +755,13 @@ int cfgzip_masked_logsoftmax_argmax(cfgzip_ctx* ctx, cfgzip_part_id part0, const
     a.status = ctx->d_status;
     const int es = dtype == CFGZIP_BF16 ? 2 : 4;
     const bool al = aligned16(logits, row_stride_elems, es);
-    if (dtype == CFGZIP_BF16) return launch_fused<kBF16>(ctx, a, ps, mixed, mode, al, logp_full, st);
-    return launch_fused<kF32>(ctx, a, ps, mixed, mode, al, logp_full, st);
+    // measured: early launch of the next kernel helps steps of a few tens of microseconds and costs
+    // several percent on long ones
+    ctx->pdl_now = int64_t(B) * ps.V * es < (int64_t(48) << 20);
+    rc = dtype == CFGZIP_BF16 ? launch_fused<kBF16>(ctx, a, ps, mixed, mode, al, logp_full, st)
+                              : launch_fused<kF32>(ctx, a, ps, mixed, mode, al, logp_full, st);
+    ctx->pdl_now = true;
+    return rc;
 }
 
 int cfgzip_map_tokens(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part, const int32_t* tokens,
@@ -874,7 +881,8 @@ int cfgzip_set_tuning(cfgzip_ctx* ctx, const char* name, int32_t value) {
         if (value != 0 && value != 1 && value != 2 && value != 4) return CFGZIP_E_ARG;
         ctx->row_warps = value;
     } else if (!std::strcmp(name, "pdl")) {
-        ctx->pdl = value ? 1 : 0;
+        if (value < 0 || value > 2) return CFGZIP_E_ARG;
+        ctx->pdl = value;
     } else if (!std::strcmp(name, "pipeline")) {
         ctx->pipeline = value ? 1 : 0;
     } else if (!std::strcmp(name, "tensor_map")) {
@@ -882,6 +890,9 @@ int cfgzip_set_tuning(cfgzip_ctx* ctx, const char* name, int32_t value) {
     } else if (!std::strcmp(name, "pipe_warps")) {
         if (value < 1 || value > 16) return CFGZIP_E_ARG;
         ctx->pipe_warps = value;
+    } else if (!std::strcmp(name, "waves")) {
+        if (value < 1 || value > 16) return CFGZIP_E_ARG;
+        ctx->waves = value;
     } else if (!std::strcmp(name, "pipe_depth")) {
         if (value < 2 || value > 8) return CFGZIP_E_ARG;
         ctx->pipe_depth = value;

@@ -243,6 +243,13 @@ __device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigne
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
+// One byte to global memory. Written as an explicit global store so that the compiler does not
+// have to order it against shared-memory accesses (a pointer that comes out of inline assembly is
+// generic to it); nothing in a kernel reads these bytes back.
+__device__ __forceinline__ void st_global_u8(void* p, uint32_t v) {
+    asm volatile("st.global.u8 [%0], %1;" ::"l"(p), "r"(v));
+}
+
 // base + i * stride with a 32-bit stride in one wide multiply-add
 __device__ __forceinline__ char* ptr_mad(char* base, uint32_t i, uint32_t stride) {
     unsigned long long r;

@@ -581,7 +581,7 @@ __device__ __forceinline__ void pipe_consume_item(const char* src, const uint32_
             oc.mask(byte, f);
             if (CONSEC) {
                 oc.store_at(ptr_mad(ba.item_base, i, ba.row_bytes));
-                if (ba.vm_item) *ptr_mad(reinterpret_cast<char*>(ba.vm_item), i, ba.vm_bytes) = char(byte);
+                if (ba.vm_item) st_global_u8(ptr_mad(reinterpret_cast<char*>(ba.vm_item), i, ba.vm_bytes), byte);
             } else {
                 oc.store(rowp[i], o);
                 if (vmp[i]) vmp[i][o] = uint8_t(byte);
