@@ -182,7 +182,7 @@ bool aligned16(const void* p, int64_t row_stride_elems, int elem_size) {
 }
 
 size_t dense_smem_bytes(int table_words, int n_warps, int stage_stride) {
-    return size_t(table_words) * 4 + kGroupRows * 4 + size_t(n_warps) * kGroupRows * sizeof(Partial) +
+    return size_t(table_words) * 4 + kGroupRows * 4 + size_t(n_warps + 1) * kGroupRows * sizeof(Partial) +
            size_t(stage_stride) * kGroupRows * 4;
 }
 
@@ -199,7 +199,7 @@ struct DensePlan {
 };
 
 size_t pipe_smem_bytes(int table_words, int n_warps, int depth, int stage_bytes, int stage_stride) {
-    return size_t(table_words) * 4 + kGroupRows * 4 + size_t(n_warps) * kGroupRows * sizeof(Partial) +
+    return size_t(table_words) * 4 + kGroupRows * 4 + size_t(n_warps + 1) * kGroupRows * sizeof(Partial) +
            ((size_t(n_warps) * depth * 8 + 127) & ~size_t(127)) + size_t(n_warps) * depth * stage_bytes +
            size_t(stage_stride) * kGroupRows * 4;
 }
@@ -274,7 +274,9 @@ DensePlan plan_pipe(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, i
     d.ctas_per_sm = std::min(ctx->ctas_per_sm, fit);
     const int target = ctx->sm_count * d.ctas_per_sm * ctx->waves;
     const int n_oct = 4 * ps.VW;
-    const int s0 = std::max(1, target / d.n_groups_ub);
+    // blocks of groups that turn out not to exist leave at once, so size the split for the fewest
+    // groups the batch can have
+    const int s0 = std::max(1, target / ceil_div(B, kGroupRows));
     int per = std::max(32, ceil_div(n_oct, s0));
     // Warps go side by side along the vocabulary first (long contiguous runs per row are kind to
     // DRAM); only when a block has fewer 32-octet chunks than warps do warps split the row batches.

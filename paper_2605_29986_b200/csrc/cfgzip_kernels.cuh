@@ -299,6 +299,42 @@ struct DenseTail {
     unsigned long long pick[kGroupRows];  // (token id << 32) | representative of the best match
 };
 
+// The octets past the last whole vector of a row (the ragged one when V is not a multiple of
+// 8, and the padding octets up to the end of the last vocab-mask word): at most four per row.
+// One warp takes them after the streaming loop, lane r = row slot r, token by token straight
+// from the class-id vector and the row's class mask (compact code, run by one block per group).
+template <int DT>
+__device__ __forceinline__ Partial dense_tail_octets(const StepArgs& a, const PartDev& P, int row, int o_first, int o_end) {
+    constexpr int ES = DT == kBF16 ? 2 : 4;
+    float m = -INFINITY, s = 0.f;
+    int pos = kNoPos;
+    if (row < 0) return Partial{m, s, pos, 0};
+    const uint32_t* cm = a.class_mask + int64_t(row) * a.cm_stride;
+    char* rowp = reinterpret_cast<char*>(a.logits) + int64_t(row) * a.row_stride * ES;
+    uint8_t* vmp = a.vocab_mask ? reinterpret_cast<uint8_t*>(a.vocab_mask) + int64_t(row) * a.vm_stride * 4 : nullptr;
+    for (int o = o_first; o < o_end; ++o) {
+        uint32_t byte = 0;
+        for (int j = 0; j < 8; ++j) {
+            const int t = 8 * o + j;
+            if (t >= a.V) break;
+            const int k = P.c32[t];
+            if ((cm[k >> 5] >> (k & 31)) & 1u) {
+                byte |= 1u << j;
+                const float z = load_elem<DT>(rowp, t);
+                if (z > m) pos = o;
+                const float ref_old = fmaxf(m, kRefFloor);
+                m = fmaxf(m, z);
+                const float ref = fmaxf(m, kRefFloor);
+                s = fmaf(s, ex2f((ref_old - ref) * kLog2e), ex2f((z - ref) * kLog2e));
+            } else {
+                store_neg_inf<DT>(rowp, t);
+            }
+        }
+        if (vmp) vmp[o] = uint8_t(byte);
+    }
+    return Partial{m, s, pos, 0};
+}
+
 // Fold red[w][row] over the warps w of a block into fin[row] with shuffle trees: the states of
 // one row sit in neighbouring lanes (a power-of-two group), so log2(warps) fold steps suffice.
 __device__ __forceinline__ void fold_red_rows(const Partial* red, int n_warps, Partial* fin) {
@@ -325,11 +361,14 @@ __device__ __forceinline__ void fold_red_rows(const Partial* red, int n_warps, P
 // turn each complete row state into the row's outputs.
 template <int DT>
 __device__ __forceinline__ void dense_block_tail(const StepArgs& a, const PartDev& P, int g, int split, const int* s_row,
-                                                 int nrow, Partial* red, DenseTail& tl) {
+                                                 int nrow, Partial* red, DenseTail& tl, int tail_first, int tail_end) {
     constexpr int ES = DT == kBF16 ? 2 : 4;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, n_warps = blockDim.x >> 5;
+    // the block that owns the end of the vocabulary also takes the octets past the last whole vector;
+    // their row states go to the extra slot red[n_warps]
+    if (warp == 0 && tail_end > tail_first) red[n_warps * kGroupRows + lane] = dense_tail_octets<DT>(a, P, s_row[lane], tail_first, tail_end);
     __syncthreads();
-    fold_red_rows(red, n_warps, tl.fin);
+    fold_red_rows(red, n_warps + 1, tl.fin);
     if (a.S > 1) {
         // several blocks share the group: publish, and let the last one to arrive finish the rows
         __syncthreads();
@@ -398,31 +437,6 @@ __device__ __forceinline__ void dense_octet_row(Octet<DT>& oc, char* rowp, uint8
     acc.add_octet(f, o);
 }
 
-// The octets past the last whole vector of a row (the ragged one when V is not a multiple of
-// 8, and the padding octets up to the end of the last vocab-mask word): at most four, taken
-// by lanes 0..3 of one warp per row batch, element by element.
-template <int DT>
-__device__ __forceinline__ void dense_tail_octets(const StepArgs& a, const PartDev& P, const uint32_t* T, int rb, int live,
-                                                  int o_first, int o_end, int lane, char* const (&rowp)[kBatchRows],
-                                                  uint8_t* const (&vmp)[kBatchRows], RowAcc (&acc)[kBatchRows]) {
-    const int o = o_first + lane;
-    const bool active = o < o_end;
-    uint4 cv = make_uint4(0, 0, 0, 0);
-    if (active) cv = __ldg(reinterpret_cast<const uint4*>(P.c16) + o);
-    uint32_t lo, hi;
-    octet_allow_bits(cv, T, rb, active, lo, hi);
-#pragma unroll
-    for (int i = 0; i < kBatchRows; ++i) {
-        if (i < live && active) {
-            const uint32_t byte = ((i < 4 ? lo : hi) >> (8 * (i & 3))) & 0xFFu;
-            float f[8];
-            octet_scalar<DT>(rowp[i], o, a.V, byte, f);
-            if (vmp[i]) vmp[i][o] = uint8_t(byte);
-            acc[i].add_octet(f, o);
-        }
-    }
-}
-
 // Reduce the 8 row states of a warp over its 32 lanes and leave them in red_warp[8*rb + i].
 // Recursive halving: lanes first trade half of their rows with the lane 16 away and fold the
 // half they keep, then 2 of 4 with the lane 8 away, then 1 of 2; two butterfly steps finish
@@ -469,7 +483,7 @@ __global__ void __launch_bounds__(256) k_step_dense(const __grid_constant__ Step
     uint32_t* T = smem;
     int* s_row = reinterpret_cast<int*>(T + a.table_words);
     Partial* red = reinterpret_cast<Partial*>(s_row + kGroupRows);
-    uint32_t* stage = reinterpret_cast<uint32_t*>(red + (blockDim.x >> 5) * kGroupRows);
+    uint32_t* stage = reinterpret_cast<uint32_t*>(red + ((blockDim.x >> 5) + 1) * kGroupRows);
     __shared__ DenseTail tl;
 
     pdl_prologue();
@@ -477,7 +491,7 @@ __global__ void __launch_bounds__(256) k_step_dense(const __grid_constant__ Step
     const int g = blockIdx.x / a.S, split = blockIdx.x - g * a.S;
     if (a.n_groups && g >= __ldg(a.n_groups)) return;
     const int part = group_rows_setup(a, g, s_row, tid);
-    for (int i = tid; i < n_warps * kGroupRows; i += blockDim.x) red[i] = partial_empty();
+    for (int i = tid; i < (n_warps + 1) * kGroupRows; i += blockDim.x) red[i] = partial_empty();
     __syncthreads();
     const PartDev P = a.group_part ? a.parts[part] : a.p0;
     const int nrow = __popc(__ballot_sync(0xFFFFFFFFu, s_row[lane] >= 0));
@@ -528,11 +542,9 @@ __global__ void __launch_bounds__(256) k_step_dense(const __grid_constant__ Step
                 }
             }
         }
-        if (wt == 0 && o_end > n_full)
-            dense_tail_octets<DT>(a, P, T, rb, live, max(o_begin, n_full), o_end, lane, rowp, vmp, acc);
         warp_rows_to_red(acc, live, red + warp * kGroupRows, rb, lane);
     }
-    dense_block_tail<DT>(a, P, g, split, s_row, nrow, red, tl);
+    dense_block_tail<DT>(a, P, g, split, s_row, nrow, red, tl, max(o_begin, n_full), o_end);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -604,7 +616,7 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
     int* s_row = reinterpret_cast<int*>(T + a.table_words);
     Partial* red = reinterpret_cast<Partial*>(s_row + kGroupRows);
     const int n_warps = blockDim.x >> 5;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(red + n_warps * kGroupRows);  // n_warps * depth
+    uint64_t* bars = reinterpret_cast<uint64_t*>(red + (n_warps + 1) * kGroupRows);  // n_warps * depth
     char* ring = reinterpret_cast<char*>(bars) + ((n_warps * a.depth * 8 + 127) & ~127);  // keeps 128-byte alignment
     uint32_t* stage = reinterpret_cast<uint32_t*>(ring + size_t(n_warps) * a.depth * G::kStageBytes);
     __shared__ DenseTail tl;
@@ -615,7 +627,7 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
     const int g = blockIdx.x / a.S, split = blockIdx.x - g * a.S;
     if (a.n_groups && g >= __ldg(a.n_groups)) return;
     const int part = group_rows_setup(a, g, s_row, tid);
-    for (int i = tid; i < n_warps * kGroupRows; i += blockDim.x) red[i] = partial_empty();
+    for (int i = tid; i < (n_warps + 1) * kGroupRows; i += blockDim.x) red[i] = partial_empty();
     __syncthreads();
     const PartDev P = a.group_part ? a.parts[part] : a.p0;
     const int nrow = __popc(__ballot_sync(0xFFFFFFFFu, s_row[lane] >= 0));
@@ -742,16 +754,6 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
             if (lane == 0 && p_n < n_items) issue_next();
         }
         if (failed) break;
-        if (wt == 0 && o_end > n_full) {
-            if (TMAP) {
-#pragma unroll
-                for (int i = 0; i < kBatchRows; ++i) {
-                    rowp[i] = ptr_mad(base0, i, ba.row_bytes);
-                    vmp[i] = vm0 ? reinterpret_cast<uint8_t*>(ptr_mad(reinterpret_cast<char*>(vm0), i, ba.vm_bytes)) : nullptr;
-                }
-            }
-            dense_tail_octets<DT>(a, P, T, rb, live, max(o_begin, n_full), o_end, lane, rowp, vmp, acc);
-        }
         warp_rows_to_red(acc, live, red + warp * kGroupRows, rb, lane);
     }
     if (failed) {
@@ -765,7 +767,7 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
             }
         }
     }
-    dense_block_tail<DT>(a, P, g, split, s_row, nrow, red, tl);
+    dense_block_tail<DT>(a, P, g, split, s_row, nrow, red, tl, max(o_begin, n_full), o_end);
 }
 
 // ---------------------------------------------------------------------------------------
