@@ -392,7 +392,8 @@ def run_own(args):
             "rows_per_gpu": runner.B, "global_rows": world * runner.B,
             "l2": "inputs larger than L2: ring of %d working buffers (%.2f GB), refilled with unmasked logits before the "
                   "timed region" % (runner.R, runner.R * runner.B * runner.V * runner.elem / 1e9),
-            "launch": "CUDA graph of %d steps replayed; one kernel per step" % min(runner.R, args.steps),
+            "launch": "CUDA graph of %d steps replayed; %.0f kernels per step (streaming pass + per-row finalize)" % (
+                min(runner.R, args.steps), launches / max(args.steps, 1)),
             "parallelism": "rows sharded over %d GPU(s), no collective on the path" % world,
         },
         "us_per_step": seconds / args.steps * 1e6,

@@ -182,8 +182,8 @@ bool aligned16(const void* p, int64_t row_stride_elems, int elem_size) {
 }
 
 size_t dense_smem_bytes(int table_words, int n_warps, int stage_stride) {
-    return size_t(table_words) * 4 + kGroupRows * 4 + size_t(n_warps + 1) * kGroupRows * sizeof(Partial) +
-           size_t(stage_stride) * kGroupRows * 4;
+    (void)n_warps;
+    return size_t(table_words) * 4 + kGroupRows * 4 + size_t(stage_stride) * kGroupRows * 4;
 }
 
 // Launch shape of the dense kernels.
@@ -199,8 +199,7 @@ struct DensePlan {
 };
 
 size_t pipe_smem_bytes(int table_words, int n_warps, int depth, int stage_bytes, int stage_stride) {
-    return size_t(table_words) * 4 + kGroupRows * 4 + size_t(n_warps + 1) * kGroupRows * sizeof(Partial) +
-           ((size_t(n_warps) * depth * 8 + 127) & ~size_t(127)) + size_t(n_warps) * depth * stage_bytes +
+    return size_t(table_words) * 4 + kGroupRows * 4 + ((size_t(n_warps) * depth * 8 + 127) & ~size_t(127)) + size_t(n_warps) * depth * stage_bytes +
            size_t(stage_stride) * kGroupRows * 4;
 }
 
@@ -236,10 +235,10 @@ DensePlan plan_dense(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, 
     }
     for (;;) {
         d.S = ceil_div(n_chunks, cps);
-        if (d.S == 1 || !fused || size_t(d.n_groups_ub) * kGroupRows * size_t(d.S) <= kPartialSlots) break;
+        if (!fused || size_t(d.n_groups_ub) * kGroupRows * (size_t(d.S) * d.WT + 1) <= kPartialSlots) break;
+        if (cps >= n_chunks) return d;
         cps *= 2;
     }
-    if (fused && d.S > 1 && d.n_groups_ub > ctx->reserved_rows) return d;  // tickets
     d.per_split = cps * unit_chunk;
     d.smem = dense_smem_bytes(d.table_words, fused ? d.threads / 32 : 0, d.stage_stride);
     d.ok = true;
@@ -293,10 +292,10 @@ DensePlan plan_pipe(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, i
     d.threads = d.WT * WR * 32;
     for (;;) {
         d.S = ceil_div(n_oct, per);
-        if (d.S == 1 || size_t(d.n_groups_ub) * kGroupRows * size_t(d.S) <= kPartialSlots) break;
+        if (size_t(d.n_groups_ub) * kGroupRows * (size_t(d.S) * d.WT + 1) <= kPartialSlots) break;
+        if (per >= n_oct) return d;
         per *= 2;
     }
-    if (d.S > 1 && d.n_groups_ub > ctx->reserved_rows) return d;  // tickets
     d.per_split = per;
     d.smem = pipe_smem_bytes(d.table_words, d.threads / 32, d.depth, stage_bytes, d.stage_stride);
     d.ok = true;
@@ -334,6 +333,7 @@ void fill_groups(cfgzip_ctx* ctx, StepArgs& a, const DensePlan& d) {
     a.stage_stride = d.stage_stride;
     a.depth = d.depth;
     a.cm_bulk = d.cm_bulk;
+    a.slots = d.S * d.WT + 1;
     a.p0 = ctx->parts[size_t(a.part0)].dev;
 }
 
@@ -419,6 +419,9 @@ int launch_fused(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, in
                 if ((rc = ensure_smem(kern, d.smem)) != CFGZIP_OK) return rc;
                 rc = launch(ctx, kern, grid, block, d.smem, st, a);
             }
+            // second kernel: one block per row folds the published states and writes the results
+            if (rc == CFGZIP_OK)
+                rc = launch(ctx, k_finalize_rows<DT>, dim3(unsigned(d.n_groups_ub) * kGroupRows), dim3(128), 0, st, a);
         } else {
             rc = launch(ctx, k_step_generic<DT, true>, dim3(unsigned(a.B)), dim3(256), 0, st, a);
         }

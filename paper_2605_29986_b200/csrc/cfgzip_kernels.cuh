@@ -32,6 +32,7 @@ struct StepArgs {
     float* lse;
     int32_t B, V, VW;
     int32_t S;                  // CTAs that share one group (dense) or one row (sparse)
+    int32_t slots;              // dense: published states per row (S * WT + 1)
     int32_t per_split;          // octets (dense) or vocab-mask words (sparse) per CTA
     int32_t WT;                 // dense: warps side by side along the vocabulary
     int32_t table_words;        // dense: shared-memory words of the bit-sliced class table
@@ -292,13 +293,6 @@ __device__ __forceinline__ void warp_finalize_row(const StepArgs& a, const PartD
     if (lane == 0) write_row_outputs(a, row, m, s, cand);
 }
 
-// Shared-memory scratch of the end of a dense block.
-struct DenseTail {
-    int last;
-    Partial fin[kGroupRows];
-    unsigned long long pick[kGroupRows];  // (token id << 32) | representative of the best match
-};
-
 // The octets past the last whole vector of a row (the ragged one when V is not a multiple of
 // 8, and the padding octets up to the end of the last vocab-mask word): at most four per row.
 // One warp takes them after the streaming loop, lane r = row slot r, token by token straight
@@ -335,94 +329,64 @@ __device__ __forceinline__ Partial dense_tail_octets(const StepArgs& a, const Pa
     return Partial{m, s, pos, 0};
 }
 
-// Fold red[w][row] over the warps w of a block into fin[row] with shuffle trees: the states of
-// one row sit in neighbouring lanes (a power-of-two group), so log2(warps) fold steps suffice.
-__device__ __forceinline__ void fold_red_rows(const Partial* red, int n_warps, Partial* fin) {
-    int group = 1;
-    while (group < n_warps) group <<= 1;  // 1, 2, 4, 8 or 16 lanes per row
-    const int tid = threadIdx.x;
-    for (int base = 0; base < kGroupRows * group; base += blockDim.x) {  // same trip count for every warp
-        const int q = base + tid;
-        const int row = q / group, w = q & (group - 1);
-        Partial p = partial_empty();
-        if (row < kGroupRows && w < n_warps) p = red[w * kGroupRows + row];
-        for (int d = group >> 1; d >= 1; d >>= 1) {
-            const float m2 = __shfl_xor_sync(0xFFFFFFFFu, p.m, d);
-            const float s2 = __shfl_xor_sync(0xFFFFFFFFu, p.s, d);
-            const int p2 = __shfl_xor_sync(0xFFFFFFFFu, p.pos, d);
-            partial_merge(p.m, p.s, p.pos, m2, s2, p2);
-        }
-        if (row < kGroupRows && w == 0) fin[row] = p;
-    }
+// Where the (max, sum-exp, position) states of a row go: every warp that streamed a row batch
+// publishes one state per row in its own slot, slot = split * WT + wt, and the block that owns the
+// end of the vocabulary adds the state of the octets past the last whole vector in the last
+// slot. a.slots = S * WT + 1 states per row, rows of a group side by side.
+__device__ __forceinline__ Partial* row_slots(const StepArgs& a, int g, int row_slot) {
+    return a.partials + (int64_t(g) * kGroupRows + row_slot) * a.slots;
 }
 
-// End of a dense block: every warp has left the states of the rows it streamed in
-// red[warp][row slot]. Fold them, publish / collect across the S blocks of the group, then
-// turn each complete row state into the row's outputs.
+// After the streaming loop of a dense block: the warp that is told to (warp 0 of the block that
+// owns the end of the vocabulary) handles the tail octets, lane r = row slot r.
 template <int DT>
-__device__ __forceinline__ void dense_block_tail(const StepArgs& a, const PartDev& P, int g, int split, const int* s_row,
-                                                 int nrow, Partial* red, DenseTail& tl, int tail_first, int tail_end) {
-    constexpr int ES = DT == kBF16 ? 2 : 4;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, n_warps = blockDim.x >> 5;
-    // the block that owns the end of the vocabulary also takes the octets past the last whole vector;
-    // their row states go to the extra slot red[n_warps]
-    if (warp == 0 && tail_end > tail_first) red[n_warps * kGroupRows + lane] = dense_tail_octets<DT>(a, P, s_row[lane], tail_first, tail_end);
-    __syncthreads();
-    fold_red_rows(red, n_warps + 1, tl.fin);
-    if (a.S > 1) {
-        // several blocks share the group: publish, and let the last one to arrive finish the rows
-        __syncthreads();
-        if (tid < kGroupRows) a.partials[(int64_t(g) * a.S + split) * kGroupRows + tid] = tl.fin[tid];
-        __threadfence();
-        __syncthreads();
-        if (tid == 0) tl.last = (atomicAdd(a.tickets + g, 1u) == unsigned(a.S - 1));
-        __syncthreads();
-        if (!tl.last) return;
-        __threadfence();
-        // every thread folds a strided share of the S published states of its row slot (two chains, so
-        // that the folds of one hide behind the other's)
-        const Partial* src = a.partials + int64_t(g) * a.S * kGroupRows + lane;
-        float m0 = -INFINITY, s0 = 0.f, m1 = -INFINITY, s1 = 0.f;
-        int p0 = kNoPos, p1 = kNoPos;
-#pragma unroll 8
-        for (int sp = warp; sp < a.S; sp += 2 * n_warps) {
-            const int4 ra = __ldcg(reinterpret_cast<const int4*>(src + sp * kGroupRows));
-            int4 rb = make_int4(__float_as_int(-INFINITY), 0, kNoPos, 0);
-            if (sp + n_warps < a.S) rb = __ldcg(reinterpret_cast<const int4*>(src + (sp + n_warps) * kGroupRows));
-            partial_merge(m0, s0, p0, __int_as_float(ra.x), __int_as_float(ra.y), ra.z);
-            partial_merge(m1, s1, p1, __int_as_float(rb.x), __int_as_float(rb.y), rb.z);
-        }
-        partial_merge(m0, s0, p0, m1, s1, p1);
-        red[warp * kGroupRows + lane] = Partial{m0, s0, p0, 0};
-        __syncthreads();
-        fold_red_rows(red, n_warps, tl.fin);
-        if (tid == 0) a.tickets[g] = 0u;
+__device__ __forceinline__ void publish_tail_octets(const StepArgs& a, const PartDev& P, int g, const int* s_row, int lane,
+                                                    int tail_first, int tail_end) {
+    const Partial p = dense_tail_octets<DT>(a, P, s_row[lane], tail_first, tail_end);
+    if (s_row[lane] >= 0) row_slots(a, g, lane)[a.slots - 1] = p;
+}
+
+// ---------------------------------------------------------------------------------------
+// Second kernel of a dense step: one block per (group, row slot). Folds the row's published
+// states, finds the winning token among the 8 tokens of the winning octet (8 lanes side by side,
+// each fetching its candidate's representative as well) and writes the row's results.
+// ---------------------------------------------------------------------------------------
+template <int DT>
+__global__ void __launch_bounds__(128) k_finalize_rows(const __grid_constant__ StepArgs a) {
+    __shared__ Partial s_red[4];
+    pdl_prologue();
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int g = blockIdx.x / kGroupRows, j = blockIdx.x - g * kGroupRows;
+    if (a.n_groups && g >= __ldg(a.n_groups)) return;
+    int row;
+    if (a.group_rows) {
+        row = a.group_rows[g * kGroupRows + j];
+    } else {
+        row = g * kGroupRows + j;
+        if (row >= a.B) row = -1;
     }
-    if (tid < kGroupRows) tl.pick[tid] = ~0ull;
-    __syncthreads();
-    // rows are complete: 8 threads per row look at the 8 tokens of the winning octet at once and
-    // fetch each candidate's representative alongside, so nothing is left to load afterwards
-    for (int idx = tid; idx < nrow * 8; idx += blockDim.x) {
-        const int j = idx >> 3;
-        const Partial p = tl.fin[j];
-        const int row = s_row[j];
-        if (p.pos == kNoPos) {
-            const unsigned long long cand = first_allowed_share(a, P, row, idx & 7, 8);
-            if (cand != ~0ull) atomicMin(tl.pick + j, cand);
-            continue;
-        }
-        const int t = 8 * p.pos + (idx & 7);
-        if (t < a.V) {
-            const float z = ldcg_elem<DT>(reinterpret_cast<const char*>(a.logits) + int64_t(row) * a.row_stride * ES, t);
-            const int k = P.c32[t];
-            const uint32_t word = a.class_mask[int64_t(row) * a.cm_stride + (k >> 5)];
-            const int repv = P.r[k];
-            if (((word >> (k & 31)) & 1u) && z == p.m)
-                atomicMin(tl.pick + j, (static_cast<unsigned long long>(t) << 32) | static_cast<unsigned int>(repv));
-        }
+    if (row < 0) return;
+    const PartDev P = a.group_part ? a.parts[a.group_part[g]] : a.p0;
+    const Partial* src = row_slots(a, g, j);
+    // two independent fold chains per thread, then a shuffle tree and a 4-way fold
+    float m0 = -INFINITY, s0 = 0.f, m1 = -INFINITY, s1 = 0.f;
+    int p0 = kNoPos, p1 = kNoPos;
+#pragma unroll 2
+    for (int sp = tid; sp < a.slots; sp += 256) {
+        const int4 ra = __ldcg(reinterpret_cast<const int4*>(src + sp));
+        int4 rb = make_int4(__float_as_int(-INFINITY), 0, kNoPos, 0);
+        if (sp + 128 < a.slots) rb = __ldcg(reinterpret_cast<const int4*>(src + sp + 128));
+        partial_merge(m0, s0, p0, __int_as_float(ra.x), __int_as_float(ra.y), ra.z);
+        partial_merge(m1, s1, p1, __int_as_float(rb.x), __int_as_float(rb.y), rb.z);
     }
+    partial_merge(m0, s0, p0, m1, s1, p1);
+    partial_warp_allreduce(m0, s0, p0);
+    if (lane == 0) s_red[warp] = Partial{m0, s0, p0, 0};
     __syncthreads();
-    if (tid < nrow) write_row_outputs(a, s_row[tid], tl.fin[tid].m, tl.fin[tid].s, tl.pick[tid]);
+    if (warp != 0) return;
+#pragma unroll
+    for (int w = 1; w < 4; ++w) partial_merge(m0, s0, p0, s_red[w].m, s_red[w].s, s_red[w].pos);
+    warp_finalize_row<DT>(a, P, row, m0, s0, p0, lane);
 }
 
 // One whole-vector octet of one row: mask, write back, note the vocab-mask byte, fold into the
@@ -437,11 +401,12 @@ __device__ __forceinline__ void dense_octet_row(Octet<DT>& oc, char* rowp, uint8
     acc.add_octet(f, o);
 }
 
-// Reduce the 8 row states of a warp over its 32 lanes and leave them in red_warp[8*rb + i].
+// Reduce the 8 row states of a warp over its 32 lanes and publish them in the warp's slot of each row.
 // Recursive halving: lanes first trade half of their rows with the lane 16 away and fold the
 // half they keep, then 2 of 4 with the lane 8 away, then 1 of 2; two butterfly steps finish
 // the single row left (nine folds instead of forty).
-__device__ __forceinline__ void warp_rows_to_red(RowAcc (&acc)[kBatchRows], int live, Partial* red_warp, int rb, int lane) {
+__device__ __forceinline__ void warp_rows_publish(const StepArgs& a, RowAcc (&acc)[kBatchRows], int live, int g, int slot,
+                                                  int rb, int lane) {
     Partial p[kBatchRows];
 #pragma unroll
     for (int i = 0; i < kBatchRows; ++i) p[i] = acc[i].to_partial();
@@ -468,7 +433,7 @@ __device__ __forceinline__ void warp_rows_to_red(RowAcc (&acc)[kBatchRows], int 
         partial_merge(p[0].m, p[0].s, p[0].pos, m2, s2, p2);
     }
     const int i = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);  // the row this lane ended with
-    if ((lane & 3) == 0 && i < live) red_warp[rb * kBatchRows + i] = p[0];  // a warp visits a row batch once
+    if ((lane & 3) == 0 && i < live) row_slots(a, g, rb * kBatchRows + i)[slot] = p[0];
 }
 
 // ---------------------------------------------------------------------------------------
@@ -482,16 +447,13 @@ __global__ void __launch_bounds__(256) k_step_dense(const __grid_constant__ Step
     extern __shared__ __align__(128) uint32_t smem[];
     uint32_t* T = smem;
     int* s_row = reinterpret_cast<int*>(T + a.table_words);
-    Partial* red = reinterpret_cast<Partial*>(s_row + kGroupRows);
-    uint32_t* stage = reinterpret_cast<uint32_t*>(red + ((blockDim.x >> 5) + 1) * kGroupRows);
-    __shared__ DenseTail tl;
+    uint32_t* stage = reinterpret_cast<uint32_t*>(s_row + kGroupRows);
 
     pdl_prologue();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, n_warps = blockDim.x >> 5;
     const int g = blockIdx.x / a.S, split = blockIdx.x - g * a.S;
     if (a.n_groups && g >= __ldg(a.n_groups)) return;
     const int part = group_rows_setup(a, g, s_row, tid);
-    for (int i = tid; i < (n_warps + 1) * kGroupRows; i += blockDim.x) red[i] = partial_empty();
     __syncthreads();
     const PartDev P = a.group_part ? a.parts[part] : a.p0;
     const int nrow = __popc(__ballot_sync(0xFFFFFFFFu, s_row[lane] >= 0));
@@ -542,9 +504,10 @@ __global__ void __launch_bounds__(256) k_step_dense(const __grid_constant__ Step
                 }
             }
         }
-        warp_rows_to_red(acc, live, red + warp * kGroupRows, rb, lane);
+        warp_rows_publish(a, acc, live, g, split * a.WT + wt, rb, lane);
     }
-    dense_block_tail<DT>(a, P, g, split, s_row, nrow, red, tl, max(o_begin, n_full), o_end);
+    // the block that reaches the end of the vocabulary takes the octets past the last whole vector
+    if (warp == 0 && o_end == n_octets) publish_tail_octets<DT>(a, P, g, s_row, lane, max(o_begin, n_full), o_end);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -614,12 +577,10 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
     extern __shared__ __align__(128) uint32_t smem[];
     uint32_t* T = smem;
     int* s_row = reinterpret_cast<int*>(T + a.table_words);
-    Partial* red = reinterpret_cast<Partial*>(s_row + kGroupRows);
     const int n_warps = blockDim.x >> 5;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(red + (n_warps + 1) * kGroupRows);  // n_warps * depth
+    uint64_t* bars = reinterpret_cast<uint64_t*>(s_row + kGroupRows);  // n_warps * depth
     char* ring = reinterpret_cast<char*>(bars) + ((n_warps * a.depth * 8 + 127) & ~127);  // keeps 128-byte alignment
     uint32_t* stage = reinterpret_cast<uint32_t*>(ring + size_t(n_warps) * a.depth * G::kStageBytes);
-    __shared__ DenseTail tl;
     __shared__ uint64_t cm_bar;
 
     pdl_prologue();
@@ -627,7 +588,6 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
     const int g = blockIdx.x / a.S, split = blockIdx.x - g * a.S;
     if (a.n_groups && g >= __ldg(a.n_groups)) return;
     const int part = group_rows_setup(a, g, s_row, tid);
-    for (int i = tid; i < (n_warps + 1) * kGroupRows; i += blockDim.x) red[i] = partial_empty();
     __syncthreads();
     const PartDev P = a.group_part ? a.parts[part] : a.p0;
     const int nrow = __popc(__ballot_sync(0xFFFFFFFFu, s_row[lane] >= 0));
@@ -754,7 +714,7 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
             if (lane == 0 && p_n < n_items) issue_next();
         }
         if (failed) break;
-        warp_rows_to_red(acc, live, red + warp * kGroupRows, rb, lane);
+        warp_rows_publish(a, acc, live, g, split * a.WT + wt, rb, lane);
     }
     if (failed) {
         // a copy never arrived: flag it, give the copies still in flight the same bounded time to land
@@ -767,7 +727,8 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
             }
         }
     }
-    dense_block_tail<DT>(a, P, g, split, s_row, nrow, red, tl, max(o_begin, n_full), o_end);
+    // the block that reaches the end of the vocabulary takes the octets past the last whole vector
+    if (warp == 0 && o_end == n_octets) publish_tail_octets<DT>(a, P, g, s_row, lane, max(o_begin, n_full), o_end);
 }
 
 // ---------------------------------------------------------------------------------------
