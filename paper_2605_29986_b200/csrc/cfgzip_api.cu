@@ -421,7 +421,7 @@ int launch_fused(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, in
             }
             // second kernel: one block per row folds the published states and writes the results
             if (rc == CFGZIP_OK)
-                rc = launch(ctx, k_finalize_rows<DT>, dim3(unsigned(d.n_groups_ub) * kGroupRows), dim3(128), 0, st, a);
+                rc = launch(ctx, k_finalize_rows<DT>, dim3(unsigned(d.n_groups_ub) * kGroupRows), dim3(kFinalizeThreads), 0, st, a);
         } else {
             rc = launch(ctx, k_step_generic<DT, true>, dim3(unsigned(a.B)), dim3(256), 0, st, a);
         }

@@ -351,9 +351,11 @@ __device__ __forceinline__ void publish_tail_octets(const StepArgs& a, const Par
 // states, finds the winning token among the 8 tokens of the winning octet (8 lanes side by side,
 // each fetching its candidate's representative as well) and writes the row's results.
 // ---------------------------------------------------------------------------------------
+constexpr int kFinalizeThreads = 256;
+
 template <int DT>
-__global__ void __launch_bounds__(128) k_finalize_rows(const __grid_constant__ StepArgs a) {
-    __shared__ Partial s_red[4];
+__global__ void __launch_bounds__(kFinalizeThreads) k_finalize_rows(const __grid_constant__ StepArgs a) {
+    __shared__ Partial s_red[kFinalizeThreads / 32];
     pdl_prologue();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = blockIdx.x / kGroupRows, j = blockIdx.x - g * kGroupRows;
@@ -368,16 +370,22 @@ __global__ void __launch_bounds__(128) k_finalize_rows(const __grid_constant__ S
     if (row < 0) return;
     const PartDev P = a.group_part ? a.parts[a.group_part[g]] : a.p0;
     const Partial* src = row_slots(a, g, j);
-    // two independent fold chains per thread, then a shuffle tree and a 4-way fold
+    // each thread fetches up to four states in one batch (all loads in flight together), folds them
+    // as two independent chains; then a shuffle tree and a fold over the warps
     float m0 = -INFINITY, s0 = 0.f, m1 = -INFINITY, s1 = 0.f;
     int p0 = kNoPos, p1 = kNoPos;
-#pragma unroll 2
-    for (int sp = tid; sp < a.slots; sp += 256) {
-        const int4 ra = __ldcg(reinterpret_cast<const int4*>(src + sp));
-        int4 rb = make_int4(__float_as_int(-INFINITY), 0, kNoPos, 0);
-        if (sp + 128 < a.slots) rb = __ldcg(reinterpret_cast<const int4*>(src + sp + 128));
-        partial_merge(m0, s0, p0, __int_as_float(ra.x), __int_as_float(ra.y), ra.z);
-        partial_merge(m1, s1, p1, __int_as_float(rb.x), __int_as_float(rb.y), rb.z);
+    for (int base = 0; base < a.slots; base += 4 * kFinalizeThreads) {
+        int4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int sp = base + u * kFinalizeThreads + tid;
+            v[u] = make_int4(__float_as_int(-INFINITY), 0, kNoPos, 0);
+            if (sp < a.slots) v[u] = __ldcg(reinterpret_cast<const int4*>(src + sp));
+        }
+        partial_merge(m0, s0, p0, __int_as_float(v[0].x), __int_as_float(v[0].y), v[0].z);
+        partial_merge(m1, s1, p1, __int_as_float(v[1].x), __int_as_float(v[1].y), v[1].z);
+        partial_merge(m0, s0, p0, __int_as_float(v[2].x), __int_as_float(v[2].y), v[2].z);
+        partial_merge(m1, s1, p1, __int_as_float(v[3].x), __int_as_float(v[3].y), v[3].z);
     }
     partial_merge(m0, s0, p0, m1, s1, p1);
     partial_warp_allreduce(m0, s0, p0);
@@ -385,7 +393,7 @@ __global__ void __launch_bounds__(128) k_finalize_rows(const __grid_constant__ S
     __syncthreads();
     if (warp != 0) return;
 #pragma unroll
-    for (int w = 1; w < 4; ++w) partial_merge(m0, s0, p0, s_red[w].m, s_red[w].s, s_red[w].pos);
+    for (int w = 1; w < kFinalizeThreads / 32; ++w) partial_merge(m0, s0, p0, s_red[w].m, s_red[w].s, s_red[w].pos);
     warp_finalize_row<DT>(a, P, row, m0, s0, p0, lane);
 }
 
