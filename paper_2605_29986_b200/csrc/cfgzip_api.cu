@@ -74,8 +74,8 @@ struct cfgzip_ctx {
                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill) = nullptr;
     int32_t pipeline = 1;     // bulk-copy pipelined dense kernel for aligned logits
     int32_t tensor_map = 1;   // tiled 2-D copies for row batches that are consecutive rows
-    int32_t pipe_warps = 8;
-    int32_t pipe_depth = 4;
+    int32_t pipe_warps = 16;
+    int32_t pipe_depth = 2;
     int32_t waves = 1;        // pipelined kernel: blocks launched per resident block slot
 };
 

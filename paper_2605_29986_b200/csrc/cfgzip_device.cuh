@@ -12,7 +12,6 @@ constexpr int kGroupRows = 32;        // rows that share one bit-sliced class ta
 constexpr int kBatchRows = 8;         // rows a warp streams together
 constexpr int kNoPos = 0x7FFFFFFF;    // "no allowed token seen"
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRefFloor = -1.7e38f; // lowest reference used for exp(z - ref)
 
 enum : int { kF32 = 0, kBF16 = 1 };
@@ -104,9 +103,6 @@ __host__ __device__ __forceinline__ void transpose8x8(uint32_t& lo, uint32_t& hi
     t = (hi ^ (hi >> 7)) & 0x00AA00AAu;
     hi ^= t ^ (t << 7);
 }
-
-__device__ __forceinline__ uint32_t neg_inf_bits_f32() { return 0xFF800000u; }
-__device__ __forceinline__ uint32_t neg_inf_bits_bf16x2() { return 0xFF80FF80u; }
 
 // Spread the 4 bits of a nibble to the top bit of the 4 bytes of a word (bit j -> bit 8j+7).
 __device__ __forceinline__ uint32_t nibble_to_byte_msbs(uint32_t nib) { return nib * 0x10204080u; }
