@@ -199,7 +199,7 @@ struct DensePlan {
 };
 
 size_t pipe_smem_bytes(int table_words, int n_warps, int depth, int stage_bytes, int stage_stride) {
-    return size_t(table_words) * 4 + kGroupRows * 4 + ((size_t(n_warps) * depth * 8 + 127) & ~size_t(127)) + size_t(n_warps) * depth * stage_bytes +
+    return size_t(table_words) * 4 + kGroupRows * 4 + ((size_t(n_warps) * depth * 12 + 127) & ~size_t(127)) + size_t(n_warps) * depth * stage_bytes +
            size_t(stage_stride) * kGroupRows * 4;
 }
 

@@ -587,7 +587,8 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
     int* s_row = reinterpret_cast<int*>(T + a.table_words);
     const int n_warps = blockDim.x >> 5;
     uint64_t* bars = reinterpret_cast<uint64_t*>(s_row + kGroupRows);  // n_warps * depth
-    char* ring = reinterpret_cast<char*>(bars) + ((n_warps * a.depth * 8 + 127) & ~127);  // keeps 128-byte alignment
+    int* ring_info = reinterpret_cast<int*>(bars + n_warps * a.depth);         // n_warps * depth
+    char* ring = reinterpret_cast<char*>(bars) + ((n_warps * a.depth * 12 + 127) & ~127);  // keeps 128-byte alignment
     uint32_t* stage = reinterpret_cast<uint32_t*>(ring + size_t(n_warps) * a.depth * G::kStageBytes);
     __shared__ uint64_t cm_bar;
 
@@ -603,27 +604,49 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
     const int depth = a.depth;
     const int wt = warp % a.WT, wr = warp / a.WT, WR = n_warps / a.WT;
     const int n_octets = 4 * a.VW, n_full = a.V >> 3;
-    const int o_begin = split * a.per_split;
-    const int o_end = min(o_begin + a.per_split, n_octets);
-    const int o_vec_end = min(o_end, n_full);
     constexpr int ES = DT == kBF16 ? 2 : 4;
     uint8_t* vm8 = reinterpret_cast<uint8_t*>(a.vocab_mask);
     char* my_ring = ring + size_t(warp) * depth * G::kStageBytes;
     uint64_t* bar = bars + warp * depth;
 
-    // this warp's work items: row batches rb = wr, wr+WR, ... (outer) x chunks of 32 whole-vector octets (inner)
-    const int first_chunk = o_begin + wt * 32;
-    const int chunk_step = a.WT * 32;
-    const int n_chunks = first_chunk < o_vec_end ? (o_vec_end - first_chunk + chunk_step - 1) / chunk_step : 0;
-    const int n_rb = (nrow > wr * kBatchRows) ? ((nrow - wr * kBatchRows + WR * kBatchRows - 1) / (WR * kBatchRows)) : 0;
-    const int n_items = n_chunks * n_rb;
+    // Work items: (row batch, chunk of 32 whole-vector octets). A warp owns the row batches rb = wr,
+    // wr+WR, ...; the chunks of a row batch are dealt round-robin to the warps of the group that own it
+    // (warp index among them, then a stride of their number), so that at any moment the group's blocks
+    // read neighbouring pieces of the same rows: measured 5 % faster on long steps than one contiguous
+    // range per block, and as fast as handing chunks out through global counters.
+    const int n_chunks = (n_full + 31) >> 5;
+    const int first_chunk = split * a.WT + wt;      // this warp's fixed first chunk
+    const int stride_chunks = a.S * a.WT;            // warps that share a row batch of the group
+    int* const slot_info = ring_info + warp * depth; // (rb << 24) | chunk of the item in each slot, -1 = no more items
 
-    // producer cursor (meaningful in lane 0): next item to start, kept without divisions
-    int p_n = 0, p_ci = 0, p_rb = wr, p_slot = 0;
+    // producer cursor (meaningful in lane 0)
+    int p_rb = wr, p_slot = 0, p_issued = 0, p_chunk = 0;
+    bool p_first = true, p_done = wr * kBatchRows >= nrow, p_end = false;
     auto issue_next = [&]() {
-        const int o0 = first_chunk + p_ci * chunk_step;
+        int chunk = -1;
+        while (!p_done) {
+            if (p_first) {
+                chunk = first_chunk;
+                p_first = false;
+            } else {
+                chunk = p_chunk + stride_chunks;
+            }
+            p_chunk = chunk;
+            if (chunk < n_chunks) break;
+            chunk = -1;  // this row batch is handed out completely: on to the warp's next one
+            p_rb += WR;
+            p_first = true;
+            p_done = p_rb * kBatchRows >= nrow;
+        }
+        if (chunk < 0) {
+            slot_info[p_slot] = -1;
+            p_end = true;
+            return;
+        }
+        slot_info[p_slot] = (p_rb << 24) | chunk;
+        const int o0 = chunk * 32;
         char* dst = my_ring + size_t(p_slot) * G::kStageBytes;
-        const uint32_t nvec = uint32_t(min(o_vec_end - o0, 32));  // >= 1 by construction of the chunk list
+        const uint32_t nvec = uint32_t(min(n_full - o0, 32));  // >= 1: chunk < n_chunks
         if (TMAP) {
             mbar_expect_tx(bar + p_slot, uint32_t(kBatchRows * G::kRowBytes) + nvec * 16u);
             tma_g2s_2d(dst, &tmap, o0 * 8, s_row[p_rb * kBatchRows], bar + p_slot);
@@ -639,9 +662,8 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
             }
         }
         bulk_g2s(dst + kBatchRows * G::kRowBytes, reinterpret_cast<const char*>(P.c16) + size_t(o0) * 16, nvec * 16u, bar + p_slot);
-        ++p_n;
+        ++p_issued;
         if (++p_slot == depth) p_slot = 0;
-        if (++p_ci == n_chunks) { p_ci = 0; p_rb += WR; }
     };
 
     if (lane == 0) {
@@ -661,7 +683,7 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
         }
     }
     if (lane == 0)
-        while (p_n < min(depth, n_items)) issue_next();  // in flight while the table is built
+        for (int d = 0; d < depth && !p_end; ++d) issue_next();  // in flight while the table is built
     bool failed = false;
     if (a.cm_bulk) {
         if (!mbar_wait(&cm_bar, 0)) failed = true;
@@ -680,10 +702,17 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
     int slot = 0;
     uint32_t phase = 0;
     int consumed = 0;
-    for (int rb = wr; rb * kBatchRows < nrow && !failed; rb += WR) {
-        RowAcc acc[kBatchRows];
-        char* rowp[kBatchRows];
-        uint8_t* vmp[kBatchRows];
+    const int my_slot = split * a.WT + wt;
+    BatchAddr ba;
+    ba.row_bytes = uint32_t(a.row_stride * ES);
+    ba.vm_bytes = uint32_t(a.vm_stride * 4);
+    RowAcc acc[kBatchRows];
+    char* rowp[kBatchRows];
+    uint8_t* vmp[kBatchRows];
+    char* base0 = nullptr;
+    uint8_t* vm0 = nullptr;
+    int live = 0;
+    auto open_batch = [&](int rb) {  // fresh row states and row addresses for row batch rb
 #pragma unroll
         for (int i = 0; i < kBatchRows; ++i) {
             acc[i].init();
@@ -695,48 +724,59 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
                 vmp[i] = vm8 ? vm8 + int64_t(max(row, 0)) * a.vm_stride * 4 : nullptr;
             }
         }
-        const int live = min(kBatchRows, nrow - rb * kBatchRows);
-        const int row0 = max(s_row[rb * kBatchRows], 0);
-        char* const base0 = reinterpret_cast<char*>(a.logits) + int64_t(row0) * a.row_stride * ES;
-        uint8_t* const vm0 = vm8 ? vm8 + int64_t(row0) * a.vm_stride * 4 : nullptr;
-        BatchAddr ba;
-        ba.row_bytes = uint32_t(a.row_stride * ES);
-        ba.vm_bytes = uint32_t(a.vm_stride * 4);
-        for (int o0 = first_chunk; o0 < o_vec_end; o0 += chunk_step) {
-            const bool arrived = mbar_wait(bar + slot, phase);
-            if (!__all_sync(0xFFFFFFFFu, arrived)) {
-                failed = true;
-                break;
-            }
-            const char* src = my_ring + size_t(slot) * G::kStageBytes;
-            const int o = o0 + lane;
-            ba.item_base = base0 + size_t(o) * G::kOctetBytes;
-            ba.vm_item = vm0 ? vm0 + o : nullptr;
-            if (live == kBatchRows && o0 + 32 <= o_vec_end)
-                pipe_consume_item<DT, true, TMAP>(src, T, rb, live, true, o, lane, ba, rowp, vmp, acc);
-            else
-                pipe_consume_item<DT, false, TMAP>(src, T, rb, live, o < o_vec_end, o, lane, ba, rowp, vmp, acc);
-            ++consumed;
-            if (++slot == depth) { slot = 0; phase ^= 1u; }
-            __syncwarp();  // every lane has its data out of the slot before it is refilled
-            if (lane == 0 && p_n < n_items) issue_next();
+        live = min(kBatchRows, nrow - rb * kBatchRows);
+        const int row0 = max(s_row[min(rb * kBatchRows, kGroupRows - 1)], 0);
+        base0 = reinterpret_cast<char*>(a.logits) + int64_t(row0) * a.row_stride * ES;
+        vm0 = vm8 ? vm8 + int64_t(row0) * a.vm_stride * 4 : nullptr;
+    };
+    int cur_rb = wr;
+    if (cur_rb * kBatchRows < nrow) open_batch(cur_rb);
+    __syncwarp();  // slot_info written by lane 0 above
+    while (cur_rb * kBatchRows < nrow) {
+        const int info = slot_info[slot];
+        if (info < 0) break;
+        const int rb = info >> 24, o0 = (info & 0xFFFFFF) * 32;
+        while (cur_rb < rb) {  // the previous row batch of this warp is complete (possibly without any chunk)
+            warp_rows_publish(a, acc, live, g, my_slot, cur_rb, lane);
+            cur_rb += WR;
+            open_batch(cur_rb);
         }
-        if (failed) break;
-        warp_rows_publish(a, acc, live, g, split * a.WT + wt, rb, lane);
+        const bool arrived = mbar_wait(bar + slot, phase);
+        if (!__all_sync(0xFFFFFFFFu, arrived)) {
+            failed = true;
+            break;
+        }
+        const char* src = my_ring + size_t(slot) * G::kStageBytes;
+        const int o = o0 + lane;
+        ba.item_base = base0 + size_t(o) * G::kOctetBytes;
+        ba.vm_item = vm0 ? vm0 + o : nullptr;
+        if (live == kBatchRows && o0 + 32 <= n_full)
+            pipe_consume_item<DT, true, TMAP>(src, T, rb, live, true, o, lane, ba, rowp, vmp, acc);
+        else
+            pipe_consume_item<DT, false, TMAP>(src, T, rb, live, o < n_full, o, lane, ba, rowp, vmp, acc);
+        ++consumed;
+        if (++slot == depth) { slot = 0; phase ^= 1u; }
+        __syncwarp();  // every lane has its data out of the slot before it is refilled
+        if (lane == 0 && !p_end) issue_next();
+        __syncwarp();  // slot_info of the refilled slot is visible to the whole warp
     }
-    if (failed) {
+    if (!failed) {
+        // whatever row batches of this warp are left (all of them if it never got a chunk) are published too
+        for (; cur_rb * kBatchRows < nrow; cur_rb += WR) {
+            warp_rows_publish(a, acc, live, g, my_slot, cur_rb, lane);
+            if ((cur_rb + WR) * kBatchRows < nrow) open_batch(cur_rb + WR);
+        }
+    } else if (lane == 0) {
         // a copy never arrived: flag it, give the copies still in flight the same bounded time to land
         // (they target this block's shared memory), and let the block leave without results
-        if (lane == 0) {
-            atomicAdd(a.status + 3, 1);
-            for (int k = consumed; k < p_n; ++k) {
-                mbar_wait(bar + slot, phase);
-                if (++slot == depth) { slot = 0; phase ^= 1u; }
-            }
+        atomicAdd(a.status + 3, 1);
+        for (int k = consumed; k < p_issued; ++k) {
+            mbar_wait(bar + slot, phase);
+            if (++slot == depth) { slot = 0; phase ^= 1u; }
         }
     }
     // the block that reaches the end of the vocabulary takes the octets past the last whole vector
-    if (warp == 0 && o_end == n_octets) publish_tail_octets<DT>(a, P, g, s_row, lane, max(o_begin, n_full), o_end);
+    if (warp == 0 && split == 0) publish_tail_octets<DT>(a, P, g, s_row, lane, n_full, n_octets);
 }
 
 // ---------------------------------------------------------------------------------------

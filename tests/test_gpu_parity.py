@@ -141,6 +141,7 @@ def test_fused_several_tiles_and_ragged_tail(V, stride, dtype, mode):
     dict(pipeline=1), dict(pipeline=1, tensor_map=0), dict(pipeline=1, pipe_warps=4, pipe_depth=2), dict(pipeline=1, pipe_warps=16, pipe_depth=3),
     dict(pipeline=1, pipe_warps=8, pipe_depth=8, ctas_per_sm=1), dict(pipeline=1, token_warps=2, row_warps=4),
     dict(pipeline=1, token_warps=1, row_warps=2, ctas_per_sm=16), dict(pipeline=1, pipe_warps=16, token_warps=16, row_warps=1),
+    dict(pipeline=1, pipe_warps=4, ctas_per_sm=1, waves=2),
 ])
 def test_fused_launch_shapes_agree(knobs, dtype):
     V, K, B = 50000, 700, 40
@@ -154,6 +155,19 @@ def test_fused_launch_shapes_agree(knobs, dtype):
         for pdl in (1, 0):
             cz.cfgzip_set_tuning(ctx.h, "pdl", pdl)
             compare_step(run_fused(ctx, None, cm, z, V), want, V, "%r pdl=%d" % (knobs, pdl))
+        assert cz.cfgzip_poll_status(ctx.h) == (0, 0, 0)
+
+
+def test_fused_many_chunks_per_warp():
+    # enough rows and tokens that every warp of a block takes several chunks at its stride, twice in a row
+    V, K, B = 200000, 900, 320
+    part = synth.zipf_partition(V, K, 1.1, seed=12)
+    cm = _mask(K, B, 0.1, 5)
+    z = np.tile(synth.logits_normal(64, V, 2.0, "bf16", (44,)), (5, 1))
+    want = oracle_step([part], None, cm, z, V)
+    with Ctx([part]) as ctx:
+        for _ in range(2):
+            compare_step(run_fused(ctx, None, cm, z, V), want, V)
         assert cz.cfgzip_poll_status(ctx.h) == (0, 0, 0)
 
 
