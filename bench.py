@@ -147,8 +147,9 @@ class StepRunner:
     """A ring of resident working buffers for one workload and CUDA graphs that run steps over it."""
 
     def __init__(self, cz, torch, device: int, config: int, B: int = None, mode: str = "dense", steps_hint: int = 1000,
-                 unique: int = 8, tune=()):
+                 unique: int = 8, tune=(), unfused: bool = False):
         self.cz, self.torch = cz, torch
+        self.unfused = unfused  # separate expand + mask calls instead of the fused step (no reductions)
         spec = synth.CONFIGS[config]
         self.w = synth.make_workload(config, B=min(B or spec["B"], 64))  # unique rows; tiled up to B below
         self.B = B or spec["B"]
@@ -207,6 +208,12 @@ class StepRunner:
 
     def call(self, j: int, stream):
         cz = self.cz
+        if self.unfused:
+            cz.cfgzip_expand_mask(self.ctx, self.parts[0], self.row_part, self.cm[j], self.KW, self.vm[j], self.VW,
+                                  self.B, self.mode, stream)
+            cz.cfgzip_mask_logits(self.ctx, self.work[j], cz.BF16 if self.dtype == "bf16" else cz.F32, self.V, self.B,
+                                  self.V, self.vm[j], self.VW, stream)
+            return
         cz.cfgzip_masked_logsoftmax_argmax(
             self.ctx, self.parts[0], self.row_part, self.cm[j], self.KW, self.work[j],
             cz.BF16 if self.dtype == "bf16" else cz.F32, self.V, self.B, self.vm[j], self.VW, self.am[j], self.rep[j],
@@ -425,6 +432,25 @@ def run_own(args):
                            "frac_of_measured": a2 / peak, "ring": r2.R})
             r2.close()
         line["larger_batches"] = extras
+        # the same masking through the two separate calls (expand, then mask; no normaliser, argmax or map):
+        # the vocab mask is written and read back, so it moves more bytes for less work
+        r3 = StepRunner(cz, torch, local_rank, args.workload, B=args.batch, mode=args.mode, steps_hint=256, unique=2,
+                        tune=args.tune, unfused=True)
+        n = 2 * r3.R
+        s3, l3 = r3.timed(n, r3.R)
+        line["unfused_expand_then_mask"] = {"us_per_step": s3 / n * 1e6, "launches_per_step": l3 / n}
+        r3.close()
+        # sparse-mask stress workload (1-5 allowed classes per row): gather path against class-list scatter path
+        pair = {}
+        for mode in ("dense", "sparse"):
+            r4 = StepRunner(cz, torch, local_rank, 5, mode=mode, steps_hint=4, unique=1, tune=args.tune)
+            n = 4 * r4.R
+            s4, _ = r4.timed(n, r4.R)
+            pair[mode + "_us_per_step"] = s4 / n * 1e6
+            pair["dense_algorithmic_gbs_" + mode] = r4.alg_bytes() / (s4 / n) / 1e9
+            r4.close()
+        pair["workload"] = "cfg5 sparse-stress: V=128256 K=512 B=1024 f32"
+        line["sparse_vs_dense"] = pair
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
