@@ -241,6 +241,19 @@ int cfgzip_launch_count(cfgzip_ctx* ctx, int64_t* out);
  */
 int cfgzip_set_tuning(cfgzip_ctx* ctx, const char* name, int32_t value);
 
+/*
+ * Host-only: the launch shape the library would choose for a fused dense step on a device with
+ * `sm_count` SMs and `smem_optin` bytes of opt-in shared memory per block (default tuning). For
+ * tests of the planner; touches no GPU. out[0] kernel kind (2 pipelined, 1 register, 0 per-row),
+ * [1] row groups (upper bound), [2] blocks per group S, [3] octets per block (register kernel),
+ * [4] warps along tokens, [5] threads per block, [6] stages per warp, [7] dynamic shared memory
+ * bytes, [8] class-table words, [9] staging stride, [10] class masks by bulk copy, [11] published
+ * states per row, [12] sparse path: blocks per row (0 = per-row kernel), [13] sparse path: mask
+ * words per block, [14] capacity of the state scratch, [15] blocks per SM the launch is sized for.
+ */
+int cfgzip_plan_query(int32_t sm_count, int32_t smem_optin, int32_t V, int32_t K, int32_t B, int dtype,
+                      int32_t n_partitions, int32_t aligned_class_masks, int32_t out[16]);
+
 #ifdef __cplusplus
 }
 #endif

@@ -39,6 +39,7 @@ _SIGNATURES = {
     "cfgzip_poll_status": (_int, [_vp, _vp, ctypes.POINTER(_i32), ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
     "cfgzip_launch_count": (_int, [_vp, ctypes.POINTER(_i64)]),
     "cfgzip_set_tuning": (_int, [_vp, ctypes.c_char_p, _i32]),
+    "cfgzip_plan_query": (_int, [_i32, _i32, _i32, _i32, _i32, _int, _i32, _i32, ctypes.POINTER(_i32)]),
 }
 
 EXPORTED_SYMBOLS = tuple(_SIGNATURES)
@@ -198,3 +199,16 @@ def cfgzip_launch_count(ctx: int) -> int:
 
 def cfgzip_set_tuning(ctx: int, name: str, value: int) -> None:
     _check(load_library().cfgzip_set_tuning(ctx, name.encode(), value), "cfgzip_set_tuning")
+
+
+PLAN_FIELDS = ("kind", "groups", "S", "octets_per_block", "token_warps", "threads", "depth", "smem_bytes", "table_words",
+               "stage_stride", "cm_bulk", "states_per_row", "sparse_S", "sparse_words", "state_capacity", "ctas_per_sm")
+
+
+def cfgzip_plan_query(sm_count: int, smem_optin: int, V: int, K: int, B: int, dtype: int, n_partitions: int = 1,
+                      aligned_class_masks: bool = True) -> dict:
+    """Launch shape the library would pick for a fused dense step (host-only, no GPU)."""
+    out = (_i32 * 16)()
+    _check(load_library().cfgzip_plan_query(sm_count, smem_optin, V, K, B, dtype, n_partitions,
+                                            1 if aligned_class_masks else 0, out), "cfgzip_plan_query")
+    return dict(zip(PLAN_FIELDS, list(out)))

@@ -259,7 +259,10 @@ DensePlan plan_pipe(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, i
     int n_warps = ctx->pipe_warps, depth = ctx->pipe_depth;
     d.cm_bulk = cm_bulk_ok && ps.all_kw_mult4;
     int stride = d.cm_bulk ? ps.maxKW + (ps.maxKW % 8 == 0 ? 4 : 8) : (ps.maxKW | 1);
+    // a staged class-mask fetch is worth giving up warps for (down to 8) when the class table is large
+    while (n_warps > 8 && pipe_smem_bytes(d.table_words, n_warps, 2, stage_bytes, stride) > cap) n_warps -= 4;
     if (pipe_smem_bytes(d.table_words, n_warps, 2, stage_bytes, stride) > cap) {
+        n_warps = ctx->pipe_warps;
         stride = 0;
         d.cm_bulk = 0;
     }
@@ -990,5 +993,44 @@ extern "C" int cfgzip_step_noalloc(const int32_t* token_to_class, int32_t V, con
     else
         k_step_rowsplit<kF32><<<grid, block, 0, st>>>(a);
     if (cudaGetLastError() != cudaSuccess) return CFGZIP_E_CUDA;
+    return CFGZIP_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host-only view of the launch planner, for tests: no GPU is touched. See include/cfgzip.h.
+// ---------------------------------------------------------------------------------------------
+extern "C" int cfgzip_plan_query(int32_t sm_count, int32_t smem_optin, int32_t V, int32_t K, int32_t B, int dtype,
+                                 int32_t n_partitions, int32_t aligned_class_masks, int32_t out[16]) {
+    if (!out || sm_count <= 0 || smem_optin <= 0 || V <= 0 || K <= 0 || K > V || B <= 0 || n_partitions <= 0 ||
+        (dtype != CFGZIP_F32 && dtype != CFGZIP_BF16))
+        return CFGZIP_E_ARG;
+    cfgzip_ctx fake;  // plain host object: the planners read its limits and tuning fields only
+    fake.sm_count = sm_count;
+    fake.smem_optin = smem_optin;
+    fake.reserved_rows = kDefaultRows;
+    fake.max_groups = ceil_div(kDefaultRows, kGroupRows) + kMaxParts;
+    PartSet ps;
+    ps.V = V;
+    ps.VW = ceil_div(V, 32);
+    ps.maxK = K;
+    ps.maxKW = ceil_div(K, 32);
+    ps.n_live_same_v = n_partitions;
+    ps.all_c16 = K <= 65535;
+    ps.all_kw_mult4 = (ps.maxKW % 4) == 0;
+    const bool mixed = n_partitions > 1;
+    const int es = dtype == CFGZIP_BF16 ? 2 : 4;
+    DensePlan d = plan_pipe(&fake, ps, B, mixed, es, aligned_class_masks != 0);
+    int kind = 2;  // pipelined
+    if (!d.ok) {
+        d = plan_dense(&fake, ps, B, mixed, 4 * ps.VW, 32, true);
+        kind = 1;  // register kernel
+    }
+    if (!d.ok) kind = 0;  // per-row kernel
+    int sp_S = 0, sp_per = 0;
+    const bool sparse_ok = plan_sparse(&fake, ps, B, true, &sp_S, &sp_per);
+    const int32_t vals[16] = {kind, d.n_groups_ub, d.S, d.per_split, d.WT, d.threads, d.depth, int32_t(d.smem),
+                              d.table_words, d.stage_stride, d.cm_bulk, d.S * d.WT + 1, sparse_ok ? sp_S : 0,
+                              sparse_ok ? sp_per : 0, int32_t(kPartialSlots), d.ctas_per_sm};
+    std::memcpy(out, vals, sizeof vals);
     return CFGZIP_OK;
 }
