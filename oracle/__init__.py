@@ -38,7 +38,8 @@ def _load():
     if _lib is None:
         _lib = ctypes.CDLL(build())
         for name in ("oracle_expand_mask", "oracle_build_csr", "oracle_expand_mask_csr", "oracle_mask_logits",
-                     "oracle_logsoftmax_argmax", "oracle_map_tokens", "oracle_decode_step"):
+                     "oracle_logsoftmax_argmax", "oracle_map_tokens", "oracle_decode_step", "oracle_sample",
+                     "oracle_sample_step"):
             getattr(_lib, name).restype = None
     return _lib
 
@@ -119,6 +120,24 @@ def logsoftmax_argmax(logits: np.ndarray, V: int, vocab_mask, want_full: bool = 
     return argmax, lse, lpa, full
 
 
+def sample(logits: np.ndarray, V: int, vocab_mask, inv_temperature: float, u, want_cdf: bool = False):
+    """(token int32 [B], lse f64 [B], logp_token f64 [B], cdf f64 [B,V] or None) from masked logits and
+    one uniform number per row: inverse CDF of the tempered distribution in token-id order."""
+    assert logits.flags.c_contiguous and logits.ndim == 2
+    vocab_mask = _u32(vocab_mask)
+    B = logits.shape[0]
+    u = np.ascontiguousarray(u, dtype=np.float64)
+    assert u.shape == (B,)
+    token = np.empty(B, dtype=np.int32)
+    lse = np.empty(B, dtype=np.float64)
+    lpt = np.empty(B, dtype=np.float64)
+    cdf = np.empty((B, V), dtype=np.float64) if want_cdf else None
+    _load().oracle_sample(_p(logits), ctypes.c_int(_dtype_code(logits)), ctypes.c_int64(logits.shape[1]),
+                          ctypes.c_int32(B), ctypes.c_int32(V), _p(vocab_mask), ctypes.c_int64(vocab_mask.shape[1]),
+                          ctypes.c_double(inv_temperature), _p(u), _p(token), _p(lse), _p(lpt), _p(cdf))
+    return token, lse, lpt, cdf
+
+
 def map_tokens(c, r, tokens) -> np.ndarray:
     c, r, tokens = _i32(c), _i32(r), _i32(tokens)
     reps = np.empty(len(tokens), dtype=np.int32)
@@ -176,3 +195,43 @@ def decode_step(partitions: Sequence, row_part, class_mask, logits: np.ndarray, 
         with ThreadPoolExecutor(max_workers=threads) as ex:
             list(ex.map(run, chunks))
     return dict(vocab_mask=vm, argmax=am, rep=rp, lse=lse, logp_argmax=lpa, logp_full=full)
+
+
+def sample_step(partitions: Sequence, row_part, class_mask, logits: np.ndarray, inv_temperature: float, u,
+                want_cdf: bool = False, threads: int = 1):
+    """One full sampling step: expand, mask (in place on ``logits``), sample by inverse CDF at the given
+    temperature with one uniform number per row, map the sampled token to its representative.
+    Returns dict(vocab_mask, token, rep, lse, logp_token, cdf)."""
+    assert logits.flags.c_contiguous and logits.ndim == 2
+    class_mask = _u32(class_mask)
+    B = logits.shape[0]
+    V = len(partitions[0].c)
+    cs = [_i32(p.c) for p in partitions]
+    rs = [_i32(p.r) for p in partitions]
+    u = np.ascontiguousarray(u, dtype=np.float64)
+    vm = np.empty((B, (V + 31) // 32), dtype=np.uint32)
+    tok = np.empty(B, dtype=np.int32)
+    rp = np.empty(B, dtype=np.int32)
+    lse = np.empty(B, dtype=np.float64)
+    lpt = np.empty(B, dtype=np.float64)
+    cdf = np.empty((B, V), dtype=np.float64) if want_cdf else None
+    part_of = np.zeros(B, dtype=np.int64) if row_part is None else np.asarray(row_part, dtype=np.int64)
+    lib = _load()
+
+    def run(rows: List[int]):
+        for b in rows:
+            p = int(part_of[b])
+            lib.oracle_sample_step(
+                _p(cs[p]), _p(rs[p]), ctypes.c_int32(V), ctypes.c_int32(int(partitions[p].K)), _p(class_mask[b:b + 1]),
+                ctypes.c_int64(class_mask.shape[1]), _p(logits[b:b + 1]), ctypes.c_int(_dtype_code(logits)),
+                ctypes.c_int64(logits.shape[1]), ctypes.c_int32(1), _p(vm[b:b + 1]), ctypes.c_int64(vm.shape[1]),
+                ctypes.c_double(inv_temperature), _p(u[b:b + 1]), _p(tok[b:b + 1]), _p(rp[b:b + 1]), _p(lse[b:b + 1]),
+                _p(lpt[b:b + 1]), _p(cdf[b:b + 1]) if cdf is not None else None)
+
+    if threads <= 1 or B == 1:
+        run(list(range(B)))
+    else:
+        chunks = [list(range(t, B, threads)) for t in range(threads)]
+        with ThreadPoolExecutor(max_workers=threads) as ex:
+            list(ex.map(run, chunks))
+    return dict(vocab_mask=vm, token=tok, rep=rp, lse=lse, logp_token=lpt, cdf=cdf)

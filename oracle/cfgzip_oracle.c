@@ -21,6 +21,11 @@
  *   - a row with nothing allowed yields argmax = rep = -1 and -inf log
  *     quantities; a row whose allowed logits are all -inf yields the lowest
  *     allowed token id and -inf log quantities.
+ *   - sampling (Section 3.1 says a token "is sampled from the next-token
+ *     distribution", Section 4 fixes the temperature, neither names the
+ *     sampler): p_i = exp(z_i/T) / sum_{allowed j} exp(z_j/T); the uniform
+ *     number u in [0,1) is an input; the chosen token is the lowest id whose
+ *     cumulative probability, taken in token-id order, exceeds u.
  *
  * Parity pins: every function here is pinned by tests/test_oracle_pins.py
  * (closed forms, invariants, a library log-softmax, brute force); nothing in
@@ -189,4 +194,68 @@ void oracle_decode_step(const int32_t* c, const int32_t* r, int32_t V, int32_t K
     oracle_logsoftmax_argmax(logits, dtype, row_stride_elems, B, V, vocab_mask, vocab_stride_words, argmax, lse,
                              logp_argmax, logp_full);
     oracle_map_tokens(c, r, V, K, argmax, rep, B);
+}
+
+/*
+ * Sampling from the tempered distribution over the allowed tokens (Section 3.1,
+ * "Inference": the next token is sampled from the next-token distribution; Section 4:
+ * temperature T, 0.2 in the paper's runs), from logits that are already masked.
+ *   p_i      = exp(z_i / T) / sum_{allowed j} exp(z_j / T)          (0 where masked)
+ *   token    = min { i : sum_{j <= i} p_j > u },  u in [0,1) given per row
+ *              (if rounding leaves no such i, the last token with p_i > 0)
+ *   lse      = log sum_{allowed} exp(z_i / T)
+ *   logp_tok = z_token / T - lse
+ * cdf (nullable, [B, V] doubles, row stride V) receives sum_{j <= i} p_j so that a test can
+ * see how close u lies to a boundary. Degenerate rows as for the greedy choice: nothing
+ * allowed -> token -1; all allowed logits -inf -> lowest allowed id; both with -inf logs.
+ */
+void oracle_sample(const void* logits, int dtype, int64_t row_stride_elems, int32_t B, int32_t V,
+                   const uint32_t* vocab_mask, int64_t vocab_stride_words, double inv_temperature,
+                   const double* u, int32_t* token, double* lse, double* logp_token, double* cdf) {
+    for (int32_t b = 0; b < B; ++b) {
+        const uint32_t* v = vocab_mask + (int64_t)b * vocab_stride_words;
+        int64_t base = (int64_t)b * row_stride_elems;
+        int32_t first = -1;
+        double M = -INFINITY;
+        for (int32_t i = 0; i < V; ++i) {
+            if (!get_bit(v, i)) continue;
+            if (first < 0) first = i;
+            double z = (double)load_logit(logits, dtype, base + i);
+            if (z > M) M = z;
+        }
+        int finite = first >= 0 && M > -INFINITY;
+        double S = 0.0;
+        if (finite)
+            for (int32_t i = 0; i < V; ++i)
+                if (get_bit(v, i)) S += exp(((double)load_logit(logits, dtype, base + i) - M) * inv_temperature);
+        int32_t pick = finite ? -1 : first, last_pos = -1;
+        double run = 0.0;
+        for (int32_t i = 0; i < V; ++i) {
+            double w = 0.0;
+            if (finite && get_bit(v, i)) w = exp(((double)load_logit(logits, dtype, base + i) - M) * inv_temperature);
+            run += w;
+            if (w > 0.0) last_pos = i;
+            if (finite && pick < 0 && run > u[b] * S) pick = i;
+            if (cdf) cdf[(int64_t)b * V + i] = finite ? run / S : 0.0;
+        }
+        if (finite && pick < 0) pick = last_pos;
+        token[b] = pick;
+        lse[b] = finite ? M * inv_temperature + log(S) : -INFINITY;
+        logp_token[b] = finite ? ((double)load_logit(logits, dtype, base + pick) - M) * inv_temperature - log(S) : -INFINITY;
+    }
+}
+
+/*
+ * One whole sampling step for rows that share one partition: expand, mask, sample, map the
+ * sampled token to its representative (the order of Section 3.1, "Inference").
+ */
+void oracle_sample_step(const int32_t* c, const int32_t* r, int32_t V, int32_t K, const uint32_t* class_mask,
+                        int64_t class_stride_words, void* logits, int dtype, int64_t row_stride_elems, int32_t B,
+                        uint32_t* vocab_mask, int64_t vocab_stride_words, double inv_temperature, const double* u,
+                        int32_t* token, int32_t* rep, double* lse, double* logp_token, double* cdf) {
+    oracle_expand_mask(c, V, K, class_mask, class_stride_words, vocab_mask, vocab_stride_words, B);
+    oracle_mask_logits(logits, dtype, row_stride_elems, B, V, vocab_mask, vocab_stride_words);
+    oracle_sample(logits, dtype, row_stride_elems, B, V, vocab_mask, vocab_stride_words, inv_temperature, u, token, lse,
+                  logp_token, cdf);
+    oracle_map_tokens(c, r, V, K, token, rep, B);
 }

@@ -17,7 +17,7 @@ import numpy as np
 from . import rng
 
 # stream purposes
-_P_RANKS, _P_SHUFFLE, _P_MASK, _P_LOGITS, _P_SPIKES, _P_DENSITY, _P_NCLS = 1, 2, 3, 4, 5, 6, 7
+_P_RANKS, _P_SHUFFLE, _P_MASK, _P_LOGITS, _P_SPIKES, _P_DENSITY, _P_NCLS, _P_UNIFORM = 1, 2, 3, 4, 5, 6, 7, 8
 
 
 @dataclass
@@ -204,6 +204,12 @@ class Workload:
         """Fresh [B, V] logits for decode step ``step`` (float32, or uint16 bf16 bit patterns)."""
         return logits_normal(self.B, self.V, self.spec["sigma"], self.dtype,
                              (rng.SEED_BASE, self.config, step), spikes=self.spec.get("spikes", 0))
+
+    def uniforms(self, step: int) -> np.ndarray:
+        """float32 [B] in [0, 1): the one random number per row that a sampling step consumes."""
+        key = rng.stream_key(rng.SEED_BASE, self.config, _P_UNIFORM, step)
+        u = (rng.u64(key, self.B) >> np.uint64(40)).astype(np.float32) * np.float32(2.0 ** -24)  # 24 bits: exact in float32
+        return u
 
     def partition_of_row(self, b: int) -> Partition:
         return self.partitions[0 if self.row_part is None else int(self.row_part[b])]

@@ -340,3 +340,151 @@ def test_bf16_ties_go_to_the_lowest_id():
     am, _, _, _ = oracle.logsoftmax_argmax(z, V, ones)
     f = rng.bf16_bits_to_f32(z[0])
     assert am[0] == np.flatnonzero(f == f.max())[0]
+
+
+# ---------------------------------------------------------------- sampling (inverse CDF at a temperature)
+
+def _full_mask(V):
+    return synth.pack_bits(np.ones((1, V), dtype=bool))
+
+
+def test_sample_hand_worked_example():
+    # allowed tokens 0, 2, 3, 5 with weights 1 : 2 : 3 : 4 (logits = their logs), tokens 1 and 4 masked
+    w = np.array([1.0, 7.0, 2.0, 3.0, 9.0, 4.0])
+    z = np.log(w).astype(np.float32)[None, :]
+    vm = synth.pack_bits(np.array([[1, 0, 1, 1, 0, 1]], dtype=bool))
+    oracle.mask_logits(z, 6, vm)
+    # cumulative probabilities over the allowed tokens: 0.1, 0.3, 0.6, 1.0
+    for u, want in [(0.0, 0), (0.05, 0), (0.15, 2), (0.29, 2), (0.31, 3), (0.59, 3), (0.61, 5), (0.999999, 5)]:
+        tok, lse, lpt, cdf = oracle.sample(z.copy(), 6, vm, 1.0, [u], want_cdf=True)
+        assert tok.tolist() == [want], (u, tok)
+        assert abs(lse[0] - math.log(10.0)) < 1e-6
+        assert abs(lpt[0] - math.log(w[want] / 10.0)) < 1e-6
+        assert np.allclose(cdf[0], [0.1, 0.1, 0.3, 0.6, 0.6, 1.0], atol=1e-7)
+    # temperature 1/2 squares the weights: 1 : 4 : 9 : 16 -> cumulative 1/30, 5/30, 14/30, 1
+    for u, want in [(0.03, 0), (0.04, 2), (0.16, 2), (0.17, 3), (0.46, 3), (0.47, 5)]:
+        tok, lse, lpt, _ = oracle.sample(z.copy(), 6, vm, 2.0, [u])
+        assert tok.tolist() == [want], (u, tok)
+        assert abs(lse[0] - math.log(30.0)) < 1e-5
+        assert abs(lpt[0] - math.log(w[want] ** 2 / 30.0)) < 1e-5
+
+
+def test_sample_equal_logits_closed_form():
+    # n equal allowed logits: token = the floor(u*n)-th allowed one, lse = a/T + log n, logp = -log n
+    V, n = 1000, 37
+    allowed = np.sort(rng.permutation(rng.stream_key(5, 1), V)[:n])
+    bits = np.zeros((1, V), dtype=bool)
+    bits[0, allowed] = True
+    vm = synth.pack_bits(bits)
+    z = np.full((1, V), 1.5, dtype=np.float32)
+    oracle.mask_logits(z, V, vm)
+    for u in [0.0, 0.013, 0.25, 0.5, 0.77, 0.99]:
+        tok, lse, lpt, _ = oracle.sample(z.copy(), V, vm, 4.0, [u])
+        assert tok[0] == allowed[int(u * n)]
+        assert abs(lse[0] - (1.5 * 4.0 + math.log(n))) < 1e-12 and abs(lpt[0] + math.log(n)) < 1e-12
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_sample_matches_library_cumsum_search(dtype):
+    # away from its boundaries the inverse CDF is numpy's searchsorted on the cumulative softmax of the allowed subset
+    V, K, B = 3000, 40, 6
+    part = synth.zipf_partition(V, K, 1.1, seed=9)
+    cm = _rand_mask(K, B, 0.3, 77)
+    z = synth.logits_normal(B, V, 2.0, dtype, (4, 4))
+    vm = oracle.expand_mask(part.c, K, cm)
+    oracle.mask_logits(z, V, vm)
+    zf = rng.bf16_bits_to_f32(z.reshape(-1)).reshape(B, V) if dtype == "bf16" else z
+    for inv_t in (1.0, 5.0):
+        for trial in range(5):
+            u = rng.uniform(rng.stream_key(8, trial), B)
+            tok, lse, lpt, _ = oracle.sample(z.copy(), V, vm, inv_t, u)
+            for b in range(B):
+                idx = np.flatnonzero(synth.unpack_bits(vm[b:b + 1], V)[0])
+                p = torch.softmax(torch.from_numpy(zf[b, idx].astype(np.float64)) * inv_t, dim=0).numpy()
+                cdf = np.cumsum(p)
+                j = int(np.searchsorted(cdf, u[b], side="right"))
+                if min(abs(cdf - u[b])) < 1e-9:
+                    continue  # on a boundary: rounding order decides
+                assert tok[b] == idx[j]
+                assert abs(lpt[b] - math.log(p[j])) < 1e-9
+                want_lse = torch.logsumexp(torch.from_numpy(zf[b, idx].astype(np.float64)) * inv_t, dim=0).item()
+                assert abs(lse[b] - want_lse) < 1e-9
+
+
+def test_sample_stratified_uniforms_reproduce_the_distribution():
+    # N evenly spaced u hit token i between N*p_i - 1 and N*p_i + 1 times: a property of any inverse CDF,
+    # so a wrong sum, order or normalisation anywhere shows up as a wrong count
+    V, N = 50, 20000
+    z = (rng.normal_f32(rng.stream_key(6, 6), V, 1.5))[None, :].astype(np.float32)
+    bits = np.ones((1, V), dtype=bool)
+    bits[0, ::7] = False
+    vm = synth.pack_bits(bits)
+    oracle.mask_logits(z, V, vm)
+    inv_t = 1.0 / 0.7
+    p = np.where(bits[0], np.exp((z[0].astype(np.float64) - z[0][bits[0]].max()) * inv_t), 0.0)
+    p /= p.sum()
+    us = (np.arange(N) + 0.5) / N
+    zz = np.repeat(z, N, axis=0)
+    vv = np.repeat(vm, N, axis=0)
+    tok, _, _, _ = oracle.sample(zz, V, vv, inv_t, us)
+    counts = np.bincount(tok, minlength=V)
+    assert np.all(np.abs(counts - N * p) <= 1.0 + 1e-6)
+    assert counts[::7].sum() == 0  # a masked token is never drawn
+    assert np.all(np.diff(tok) >= 0)  # monotone in u
+
+
+def test_sample_temperature_identities():
+    V = 400
+    z = rng.normal_f32(rng.stream_key(6, 7), V, 1.0)[None, :].astype(np.float32)
+    vm = _full_mask(V)
+    u = rng.uniform(rng.stream_key(6, 8), 64)
+    zz, vv = np.repeat(z, 64, axis=0), np.repeat(vm, 64, axis=0)
+    # halving the temperature = doubling the logits (exact in float32)
+    t_a, lse_a, lp_a, _ = oracle.sample(zz.copy(), V, vv, 2.0, u)
+    t_b, lse_b, lp_b, _ = oracle.sample((2.0 * zz).astype(np.float32), V, vv, 1.0, u)
+    assert np.array_equal(t_a, t_b) and np.allclose(lse_a, lse_b, atol=1e-12) and np.allclose(lp_a, lp_b, atol=1e-12)
+    # T = 1: lse is the greedy path's lse, and a cold distribution collapses onto the argmax
+    am, lse_g, _, _ = oracle.logsoftmax_argmax(zz.copy(), V, vv)
+    _, lse_1, _, _ = oracle.sample(zz.copy(), V, vv, 1.0, u)
+    assert np.allclose(lse_1, lse_g, atol=1e-12)
+    t_cold, _, lp_cold, _ = oracle.sample(zz.copy(), V, vv, 1000.0, np.minimum(u, 0.999))
+    assert np.array_equal(t_cold, am) and np.all(lp_cold > -1e-3)
+    # adding a constant to the row moves lse by constant/T and nothing else (logits on a 1/64 grid: the shift is exact)
+    zq = (np.round(zz * 64.0) / 64.0).astype(np.float32)
+    t_q, lse_q, lp_q, _ = oracle.sample(zq.copy(), V, vv, 2.0, u)
+    t_s, lse_s, lp_s, _ = oracle.sample((zq + np.float32(4.0)).astype(np.float32), V, vv, 2.0, u)
+    assert np.array_equal(t_s, t_q) and np.allclose(lse_s, lse_q + 8.0, atol=1e-12) and np.allclose(lp_s, lp_q, atol=1e-12)
+
+
+def test_sample_degenerate_rows_and_last_token():
+    V = 70
+    z = np.zeros((3, V), dtype=np.float32)
+    bits = np.zeros((3, V), dtype=bool)
+    bits[1, [5, 40]] = True
+    bits[2, [3, 66]] = True
+    z[1, [5, 40]] = -np.inf          # allowed, but both -inf
+    vm = synth.pack_bits(bits)
+    oracle.mask_logits(z, V, vm)
+    tok, lse, lpt, cdf = oracle.sample(z, V, vm, 1.0, [0.5, 0.5, 0.999999999], want_cdf=True)
+    assert tok.tolist() == [-1, 5, 66]
+    assert np.isneginf(lse[:2]).all() and np.isneginf(lpt[:2]).all()
+    assert abs(lse[2] - math.log(2.0)) < 1e-12 and cdf[2, 66] == 1.0 and cdf[2, 3] == 0.5
+
+
+def test_sample_step_is_the_composition_of_its_steps():
+    w = synth.make_workload(4, B=16, V=5000, K=300)
+    cm, z, u = w.class_masks(0), w.logits(0), w.uniforms(0)
+    assert u.dtype == np.float32 and np.all((u >= 0) & (u < 1))
+    z1 = z.copy()
+    out = oracle.sample_step(w.partitions, w.row_part, cm, z1, 5.0, u, threads=2)
+    for b in range(w.B):
+        p = w.partition_of_row(b)
+        vm = oracle.expand_mask(p.c, p.K, cm[b:b + 1])
+        zb = z[b:b + 1].copy()
+        oracle.mask_logits(zb, w.V, vm)
+        tok, lse, lpt, _ = oracle.sample(zb, w.V, vm, 5.0, u[b:b + 1])
+        assert np.array_equal(vm[0], out["vocab_mask"][b]) and np.array_equal(zb[0], z1[b])
+        assert tok[0] == out["token"][b] and lse[0] == out["lse"][b] and lpt[0] == out["logp_token"][b]
+        assert oracle.map_tokens(p.c, p.r, tok)[0] == out["rep"][b]
+        t = int(tok[0])
+        assert (int(vm[0, t // 32]) >> (t % 32)) & 1 == 1
