@@ -147,9 +147,10 @@ class StepRunner:
     """A ring of resident working buffers for one workload and CUDA graphs that run steps over it."""
 
     def __init__(self, cz, torch, device: int, config: int, B: int = None, mode: str = "dense", steps_hint: int = 1000,
-                 unique: int = 8, tune=(), unfused: bool = False, ring: int = 0):
+                 unique: int = 8, tune=(), unfused: bool = False, ring: int = 0, inv_temperature: float = 0.0):
         self.cz, self.torch = cz, torch
         self.unfused = unfused  # separate expand + mask calls instead of the fused step (no reductions)
+        self.inv_temperature = inv_temperature  # > 0: the sampling step (cfgzip_masked_sample) instead of the greedy one
         spec = synth.CONFIGS[config]
         self.w = synth.make_workload(config, B=min(B or spec["B"], 64))  # unique rows; tiled up to B below
         self.B = B or spec["B"]
@@ -194,6 +195,10 @@ class StepRunner:
         self.rep = torch.empty_like(self.am)
         self.lse = torch.empty((self.R, self.B), dtype=torch.float32, device="cuda")
         self.lpa = torch.empty_like(self.lse)
+        self.u = None
+        if inv_temperature > 0:
+            us = np.stack([np.tile(self.w.uniforms(j), tile)[: self.B] for j in range(self.R)])
+            self.u = torch.from_numpy(us).cuda()
         self.stream = torch.cuda.Stream()
         self.graphs = {}
         self.launches = {}
@@ -218,6 +223,12 @@ class StepRunner:
                                   self.B, self.mode, stream)
             cz.cfgzip_mask_logits(self.ctx, self.work[j], cz.BF16 if self.dtype == "bf16" else cz.F32, self.V, self.B,
                                   self.V, self.vm[j], self.VW, stream)
+            return
+        if self.u is not None:
+            cz.cfgzip_masked_sample(
+                self.ctx, self.parts[0], self.row_part, self.cm[j], self.KW, self.work[j],
+                cz.BF16 if self.dtype == "bf16" else cz.F32, self.V, self.B, self.vm[j], self.VW, self.u[j],
+                self.inv_temperature, self.am[j], self.rep[j], self.lpa[j], self.lse[j], self.mode, stream)
             return
         cz.cfgzip_masked_logsoftmax_argmax(
             self.ctx, self.parts[0], self.row_part, self.cm[j], self.KW, self.work[j],
@@ -456,6 +467,17 @@ def run_own(args):
         s3, l3 = r3.timed(n, r3.R)
         line["unfused_expand_then_mask"] = {"us_per_step": s3 / n * 1e6, "launches_per_step": l3 / n}
         r3.close()
+        # the sampling step (inverse CDF at the paper's temperature 0.2, one uniform number per row) on the same workload
+        samp = []
+        for B in (args.batch or synth.CONFIGS[args.workload]["B"], 1024):
+            r6 = StepRunner(cz, torch, local_rank, args.workload, B=B, mode=args.mode, steps_hint=64, unique=2,
+                            tune=args.tune, inv_temperature=5.0)
+            n = 3 * r6.R
+            s6, l6 = r6.timed(n, r6.R)
+            samp.append({"B": B, "us_per_step": s6 / n * 1e6, "launches_per_step": l6 / n,
+                         "frac_of_measured": r6.alg_bytes() / (s6 / n) / 1e9 / peak})
+            r6.close()
+        line["sampling_step_T0.2"] = samp
         # the same step on two buffers that stay in the 126 MB L2: NOT an HBM figure, only the latency floor
         r5 = StepRunner(cz, torch, local_rank, args.workload, B=args.batch, mode=args.mode, steps_hint=2, unique=2,
                         tune=args.tune, ring=2)

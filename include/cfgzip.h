@@ -148,6 +148,31 @@ int cfgzip_masked_logsoftmax_argmax(cfgzip_ctx* ctx, cfgzip_part_id part0, const
                                     void* stream);
 
 /*
+ * The same pass with the token SAMPLED instead of taken greedily (Section 3.1, "Inference": a
+ * token "is sampled from the next-token distribution"; Section 4: temperature 0.2 in the paper's
+ * runs). The paper names no sampler; this one is the inverse CDF in token-id order:
+ *   p_i   = exp(z_i / T) / sum_{allowed j} exp(z_j / T),  1/T = inv_temperature > 0 (at most 1e6)
+ *   token = the lowest token id i with sum_{j <= i} p_j > u[b]
+ * with ONE uniform number per row supplied by the caller (the library draws no random numbers).
+ *   u          : dev float [B], values in [0, 1)
+ *   token      : dev int32 [B]; -1 when nothing is allowed
+ *   rep        : nullable dev int32 [B]; r[c[token]] or -1
+ *   lse        : nullable dev float [B]; log sum_{allowed} exp(z_i / T)
+ *   logp_token : nullable dev float [B]; z_token / T - lse
+ *   logits, vocab_mask, class masks, row_part: as in cfgzip_masked_logsoftmax_argmax; the logits
+ *                are masked in place and NOT scaled by 1/T
+ *   mode       : CFGZIP_AUTO or CFGZIP_DENSE (CFGZIP_SPARSE gives CFGZIP_E_ARG)
+ * The sums are accumulated in fp32 in a fixed order, so the result is deterministic; where u lies
+ * within rounding (about 1e-6) of a boundary of the exact CDF the neighbouring token may come out.
+ * A row whose allowed logits are all -inf yields the lowest allowed id with lse = logp_token = -inf.
+ */
+int cfgzip_masked_sample(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part,
+                         const uint32_t* class_mask, int64_t class_stride_words, void* logits, int dtype,
+                         int64_t row_stride_elems, int32_t B, uint32_t* vocab_mask,
+                         int64_t vocab_stride_words, const float* u, float inv_temperature, int32_t* token,
+                         int32_t* rep, float* logp_token, float* lse, int mode, void* stream);
+
+/*
  * Token -> representative of its class, reps[b] = r[c[tokens[b]]] (Section 3.1,
  * "Inference": the engine is fed r_{c_i} instead of t^(i); Figure 1a). A token id
  * outside [0, V) gives -1 and counts as a bad token.

@@ -31,6 +31,8 @@ _SIGNATURES = {
     "cfgzip_mask_logits": (_int, [_vp, _vp, _int, _i64, _i32, _i32, _vp, _i64, _vp]),
     "cfgzip_masked_logsoftmax_argmax": (_int, [_vp, _i32, _vp, _vp, _i64, _vp, _int, _i64, _i32, _vp, _i64, _vp, _vp,
                                                _vp, _vp, _vp, _int, _vp]),
+    "cfgzip_masked_sample": (_int, [_vp, _i32, _vp, _vp, _i64, _vp, _int, _i64, _i32, _vp, _i64, _vp, ctypes.c_float, _vp,
+                                    _vp, _vp, _vp, _int, _vp]),
     "cfgzip_map_tokens": (_int, [_vp, _i32, _vp, _vp, _vp, _i32, _vp]),
     "cfgzip_decode_step_host": (_int, [_vp, _i32, _vp, _vp, _i64, _vp, _int, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _int,
                                        _vp]),
@@ -154,6 +156,15 @@ def cfgzip_masked_logsoftmax_argmax(ctx: int, part0: int, row_part, class_mask, 
         ctx, part0, _ptr(row_part), _ptr(class_mask), class_stride_words, _ptr(logits), dtype, row_stride_elems, B,
         _ptr(vocab_mask), vocab_stride_words, _ptr(argmax), _ptr(rep), _ptr(logp_argmax), _ptr(lse), _ptr(logp_full),
         mode, _stream(stream)), "cfgzip_masked_logsoftmax_argmax")
+
+
+def cfgzip_masked_sample(ctx: int, part0: int, row_part, class_mask, class_stride_words: int, logits, dtype: int,
+                         row_stride_elems: int, B: int, vocab_mask, vocab_stride_words: int, u, inv_temperature: float,
+                         token, rep=None, logp_token=None, lse=None, mode: int = AUTO, stream=None) -> None:
+    _check(load_library().cfgzip_masked_sample(
+        ctx, part0, _ptr(row_part), _ptr(class_mask), class_stride_words, _ptr(logits), dtype, row_stride_elems, B,
+        _ptr(vocab_mask), vocab_stride_words, _ptr(u), inv_temperature, _ptr(token), _ptr(rep), _ptr(logp_token),
+        _ptr(lse), mode, _stream(stream)), "cfgzip_masked_sample")
 
 
 def cfgzip_map_tokens(ctx: int, part0: int, row_part, tokens, reps, B: int, stream=None) -> None:

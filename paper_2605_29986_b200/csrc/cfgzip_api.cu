@@ -364,6 +364,42 @@ bool plan_sparse(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool fused, int*
     return true;
 }
 
+// The pipelined streaming kernel for a planned step (d.depth > 0; `a` filled by fill_groups).
+template <int DT>
+int launch_pipe(cfgzip_ctx* ctx, const StepArgs& a, const DensePlan& d, dim3 grid, dim3 block, cudaStream_t st) {
+    int rc;
+    // rows of a batch are consecutive unless the plan kernel regrouped them: then one tiled
+    // 2-D copy (box 256 elements x 8 rows) brings a whole batch
+    CUtensorMap tmap;
+    std::memset(&tmap, 0, sizeof tmap);
+    bool tiled = false;
+    if (!d.use_plan_kernel && ctx->tensor_map && ctx->encode_tiled && a.V >= 256 &&
+        a.row_stride * (DT == kBF16 ? 2 : 4) < (int64_t(1) << 32) && a.vm_stride * 4 < (int64_t(1) << 32)) {
+        const cuuint64_t dims[2] = {cuuint64_t(a.V), cuuint64_t(a.B)};
+        const cuuint64_t strides[1] = {cuuint64_t(a.row_stride) * (DT == kBF16 ? 2 : 4)};
+        const cuuint32_t box[2] = {256, 8};
+        const cuuint32_t estr[2] = {1, 1};
+        tiled = ctx->encode_tiled(&tmap, DT == kBF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
+                                  2, a.logits, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                  CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    }
+    void (*kern)(StepArgs, CUtensorMap);
+    const bool tempered = a.u != nullptr;  // only a sampling step has a temperature
+#define CFGZIP_PIPE_VARIANT(LBT, MINB)                                                                              \
+    (tempered ? (tiled ? k_step_dense_pipe<DT, true, LBT, MINB, true> : k_step_dense_pipe<DT, false, LBT, MINB, true>) \
+              : (tiled ? k_step_dense_pipe<DT, true, LBT, MINB, false> : k_step_dense_pipe<DT, false, LBT, MINB, false>))
+    if (d.threads <= 256 && d.ctas_per_sm >= 3)
+        kern = CFGZIP_PIPE_VARIANT(256, 3);
+    else if (d.threads <= 320 && d.ctas_per_sm >= 2)
+        kern = CFGZIP_PIPE_VARIANT(320, 2);
+    else
+        kern = CFGZIP_PIPE_VARIANT(512, 1);
+#undef CFGZIP_PIPE_VARIANT
+    if ((rc = ensure_smem(kern, d.smem)) != CFGZIP_OK) return rc;
+    return launch(ctx, kern, grid, block, d.smem, st, a, tmap);
+}
+
 template <int DT>
 int launch_fused(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, int mode, bool aligned, float* logp_full,
                  cudaStream_t st) {
@@ -392,31 +428,7 @@ int launch_fused(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, in
             fill_groups(ctx, a, d);
             const dim3 grid(unsigned(d.n_groups_ub) * unsigned(d.S)), block{unsigned(d.threads)};
             if (d.depth) {
-                // rows of a batch are consecutive unless the plan kernel regrouped them: then one tiled
-                // 2-D copy (box 256 elements x 8 rows) brings a whole batch
-                CUtensorMap tmap;
-                std::memset(&tmap, 0, sizeof tmap);
-                bool tiled = false;
-                if (!d.use_plan_kernel && ctx->tensor_map && ctx->encode_tiled && a.V >= 256 &&
-                    a.row_stride * (DT == kBF16 ? 2 : 4) < (int64_t(1) << 32) && a.vm_stride * 4 < (int64_t(1) << 32)) {
-                    const cuuint64_t dims[2] = {cuuint64_t(a.V), cuuint64_t(a.B)};
-                    const cuuint64_t strides[1] = {cuuint64_t(a.row_stride) * (DT == kBF16 ? 2 : 4)};
-                    const cuuint32_t box[2] = {256, 8};
-                    const cuuint32_t estr[2] = {1, 1};
-                    tiled = ctx->encode_tiled(&tmap, DT == kBF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32,
-                                              2, a.logits, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                              CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-                                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-                }
-                void (*kern)(StepArgs, CUtensorMap);
-                if (d.threads <= 256 && d.ctas_per_sm >= 3)
-                    kern = tiled ? k_step_dense_pipe<DT, true, 256, 3> : k_step_dense_pipe<DT, false, 256, 3>;
-                else if (d.threads <= 320 && d.ctas_per_sm >= 2)
-                    kern = tiled ? k_step_dense_pipe<DT, true, 320, 2> : k_step_dense_pipe<DT, false, 320, 2>;
-                else
-                    kern = tiled ? k_step_dense_pipe<DT, true, 512, 1> : k_step_dense_pipe<DT, false, 512, 1>;
-                if ((rc = ensure_smem(kern, d.smem)) != CFGZIP_OK) return rc;
-                rc = launch(ctx, kern, grid, block, d.smem, st, a, tmap);
+                rc = launch_pipe<DT>(ctx, a, d, grid, block, st);
             } else {
                 auto kern = k_step_dense<DT>;
                 if ((rc = ensure_smem(kern, d.smem)) != CFGZIP_OK) return rc;
@@ -437,6 +449,40 @@ int launch_fused(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, in
                     int(a.V), (const float*)a.lse, logp_full);
     }
     return rc;
+}
+
+// A sampling step: the streaming kernel leaves the states of a row in token order, the sampling kernel
+// (one block per row) draws the token. Rows off the 16-byte grid, and shapes the pipelined kernel does not
+// take, go through the per-row kernel, whose single state per row stands for the whole row.
+template <int DT>
+int launch_sample(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, bool aligned, cudaStream_t st) {
+    int rc;
+    DensePlan d;
+    if (aligned) {
+        const bool cm_bulk_ok = (reinterpret_cast<uintptr_t>(a.class_mask) & 15u) == 0 && (a.cm_stride & 3) == 0;
+        d = plan_pipe(ctx, ps, a.B, mixed, DT == kBF16 ? 2 : 4, cm_bulk_ok);
+    }
+    if (d.ok && d.depth) {
+        if (d.use_plan_kernel && (rc = run_plan_kernel(ctx, a.row_part, a.B, a.V, d, st)) != CFGZIP_OK) return rc;
+        fill_groups(ctx, a, d);
+        const int n_chunks = ((ps.V >> 3) + 31) >> 5;
+        a.run_chunks = std::max(1, ceil_div(n_chunks, d.S * d.WT));
+        a.tail_state = 1;
+        const dim3 grid(unsigned(d.n_groups_ub) * unsigned(d.S)), block{unsigned(d.threads)};
+        if ((rc = launch_pipe<DT>(ctx, a, d, grid, block, st)) != CFGZIP_OK) return rc;
+        return launch(ctx, k_sample_rows<DT>, dim3(unsigned(d.n_groups_ub) * kGroupRows), dim3(kSampleThreads), 0, st, a, 1);
+    }
+    if (size_t(a.B) > kPartialSlots) return CFGZIP_E_NOMEM;
+    a.group_part = nullptr;
+    a.group_rows = nullptr;
+    a.n_groups = nullptr;
+    a.slots = 1;
+    a.run_chunks = ceil_div(ps.V, 256);
+    a.tail_state = 0;
+    a.p0 = ctx->parts[size_t(a.part0)].dev;
+    if ((rc = launch(ctx, k_step_generic<DT, true>, dim3(unsigned(a.B)), dim3(256), 0, st, a)) != CFGZIP_OK) return rc;
+    return launch(ctx, k_sample_rows<DT>, dim3(unsigned(ceil_div(a.B, kGroupRows)) * kGroupRows), dim3(kSampleThreads), 0, st,
+                  a, aligned ? 1 : 0);
 }
 
 int grow(void** p, size_t* have, size_t need) {
@@ -678,6 +724,8 @@ int cfgzip_expand_mask(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row
     a.partials = ctx->d_partials;
     a.tickets = ctx->d_tickets;
     a.status = ctx->d_status;
+    a.scale = kLog2e;
+    a.inv_t = 1.f;
     if (mode == CFGZIP_SPARSE) {
         int S, per_split;
         if (plan_sparse(ctx, ps, B, false, &S, &per_split)) {
@@ -761,6 +809,8 @@ int cfgzip_masked_logsoftmax_argmax(cfgzip_ctx* ctx, cfgzip_part_id part0, const
     a.partials = ctx->d_partials;
     a.tickets = ctx->d_tickets;
     a.status = ctx->d_status;
+    a.scale = kLog2e;
+    a.inv_t = 1.f;
     const int es = dtype == CFGZIP_BF16 ? 2 : 4;
     const bool al = aligned16(logits, row_stride_elems, es);
     // measured: early launch of the next kernel helps steps of a few tens of microseconds and costs
@@ -768,6 +818,56 @@ int cfgzip_masked_logsoftmax_argmax(cfgzip_ctx* ctx, cfgzip_part_id part0, const
     ctx->pdl_now = int64_t(B) * ps.V * es < (int64_t(48) << 20);
     rc = dtype == CFGZIP_BF16 ? launch_fused<kBF16>(ctx, a, ps, mixed, mode, al, logp_full, st)
                               : launch_fused<kF32>(ctx, a, ps, mixed, mode, al, logp_full, st);
+    ctx->pdl_now = true;
+    return rc;
+}
+
+int cfgzip_masked_sample(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part, const uint32_t* class_mask,
+                         int64_t class_stride_words, void* logits, int dtype, int64_t row_stride_elems, int32_t B,
+                         uint32_t* vocab_mask, int64_t vocab_stride_words, const float* u, float inv_temperature,
+                         int32_t* token, int32_t* rep, float* logp_token, float* lse, int mode, void* stream) {
+    int rc = check_step_args(ctx, class_mask, class_stride_words, B, mode);
+    if (rc != CFGZIP_OK) return rc;
+    if (dtype != CFGZIP_F32 && dtype != CFGZIP_BF16) return CFGZIP_E_ARG;
+    if (mode == CFGZIP_SPARSE) return CFGZIP_E_ARG;  // the class-list kernel does not leave its states in token order
+    if (!(inv_temperature > 0.f) || !(inv_temperature <= 1e6f)) return CFGZIP_E_ARG;
+    PartSet ps;
+    const bool mixed = row_part != nullptr;
+    if ((rc = resolve_parts(ctx, part0, mixed, &ps)) != CFGZIP_OK) return rc;
+    if (B == 0) return CFGZIP_OK;
+    if (!logits || !token || !u || row_stride_elems < ps.V || class_stride_words < ps.maxKW) return CFGZIP_E_ARG;
+    if (vocab_mask && vocab_stride_words < ps.VW) return CFGZIP_E_ARG;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return CFGZIP_E_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    StepArgs a{};
+    a.parts = ctx->d_parts;
+    a.part0 = part0;
+    a.n_parts = int32_t(ctx->parts.size());
+    a.row_part = row_part;
+    a.class_mask = class_mask;
+    a.cm_stride = class_stride_words;
+    a.logits = logits;
+    a.row_stride = row_stride_elems;
+    a.vocab_mask = vocab_mask;
+    a.vm_stride = vocab_stride_words;
+    a.argmax = token;
+    a.rep = rep;
+    a.logp_argmax = logp_token;
+    a.lse = lse;
+    a.B = B;
+    a.V = ps.V;
+    a.VW = ps.VW;
+    a.partials = ctx->d_partials;
+    a.tickets = ctx->d_tickets;
+    a.status = ctx->d_status;
+    a.scale = kLog2e * inv_temperature;
+    a.inv_t = inv_temperature;
+    a.u = u;
+    const int es = dtype == CFGZIP_BF16 ? 2 : 4;
+    const bool al = aligned16(logits, row_stride_elems, es);
+    ctx->pdl_now = int64_t(B) * ps.V * es < (int64_t(48) << 20);
+    rc = dtype == CFGZIP_BF16 ? launch_sample<kBF16>(ctx, a, ps, mixed, al, st) : launch_sample<kF32>(ctx, a, ps, mixed, al, st);
     ctx->pdl_now = true;
     return rc;
 }

@@ -48,11 +48,13 @@ __device__ __forceinline__ float ex2f(float x) {
 }
 
 // Total order used at every level: larger value wins; equal values: lower position.
-// The sums are brought to the larger reference before they are added.
-__device__ __forceinline__ void partial_merge(float& m, float& s, int& pos, float m2, float s2, int pos2) {
+// The sums are brought to the larger reference before they are added. `scale` is log2(e) / T:
+// the sums are of exp(z / T) (T = 1 everywhere except in a sampling step).
+__device__ __forceinline__ void partial_merge(float& m, float& s, int& pos, float m2, float s2, int pos2,
+                                              float scale = kLog2e) {
     const float r1 = fmaxf(m, kRefFloor), r2 = fmaxf(m2, kRefFloor);
     const float d = r1 - r2;
-    const float e = ex2f(-fabsf(d) * kLog2e);
+    const float e = ex2f(-fabsf(d) * scale);
     s = d >= 0.f ? fmaf(s2, e, s) : fmaf(s, e, s2);
     const bool take2 = (m2 > m) || (m2 == m && pos2 < pos);
     pos = take2 ? pos2 : pos;
@@ -60,13 +62,13 @@ __device__ __forceinline__ void partial_merge(float& m, float& s, int& pos, floa
 }
 
 // Butterfly all-reduce of one row's state over the 32 lanes of a warp.
-__device__ __forceinline__ void partial_warp_allreduce(float& m, float& s, int& pos) {
+__device__ __forceinline__ void partial_warp_allreduce(float& m, float& s, int& pos, float scale = kLog2e) {
 #pragma unroll
     for (int d = 16; d >= 1; d >>= 1) {
         const float m2 = __shfl_xor_sync(0xFFFFFFFFu, m, d);
         const float s2 = __shfl_xor_sync(0xFFFFFFFFu, s, d);
         const int p2 = __shfl_xor_sync(0xFFFFFFFFu, pos, d);
-        partial_merge(m, s, pos, m2, s2, p2);
+        partial_merge(m, s, pos, m2, s2, p2, scale);
     }
 }
 
@@ -255,8 +257,9 @@ __device__ __forceinline__ char* ptr_mad(char* base, uint32_t i, uint32_t stride
 
 // Running state of one row inside one thread. The sum is kept relative to a reference that
 // only moves when a value overtakes it by more than kRefSlack (so the common case is one
-// fused multiply-add and one ex2 per logit): s = sum 2^(z*log2e + nrl), nrl = -(ref*log2e).
-// pos is the position (octet index) of the first octet whose maximum is the row maximum m.
+// fused multiply-add and one ex2 per logit): s = sum 2^(z*scale + nrl), nrl = -(ref*scale), with
+// scale = log2(e) / T. pos is the position (octet index) of the first octet whose maximum is the
+// row maximum m.
 constexpr float kRefSlack = 57.7f;  // in powers of two: 40 nats
 struct RowAcc {
     float m, s, nrl;
@@ -267,16 +270,16 @@ struct RowAcc {
         nrl = -(kRefFloor * kLog2e);
         pos = kNoPos;
     }
-    __device__ __forceinline__ void add_octet(const float (&f)[8], int position) {
+    __device__ __forceinline__ void add_octet(const float (&f)[8], int position, float scale = kLog2e) {
         const float vmax = fmax3(fmax3(f[0], f[1], f[2]), fmax3(f[3], f[4], f[5]), fmaxf(f[6], f[7]));
         pos = vmax > m ? position : pos;
         m = fmaxf(m, vmax);
-        if (fmaf(vmax, kLog2e, nrl) > kRefSlack) {  // rare: move the reference up to vmax
-            const float n2 = -(vmax * kLog2e);
+        if (fmaf(vmax, scale, nrl) > kRefSlack) {  // rare: move the reference up to vmax
+            const float n2 = -(vmax * scale);
             s *= ex2f(n2 - nrl);
             nrl = n2;
         }
-        const unsigned long long l2 = pack2(kLog2e, kLog2e), n2p = pack2(nrl, nrl);
+        const unsigned long long l2 = pack2(scale, scale), n2p = pack2(nrl, nrl);
         float e[8];
 #pragma unroll
         for (int j = 0; j < 8; j += 2) {
@@ -290,10 +293,10 @@ struct RowAcc {
         s += a0 + a1;
     }
     // Bring the sum to the convention of Partial: relative to max(m, kRefFloor).
-    __device__ __forceinline__ Partial to_partial() const {
+    __device__ __forceinline__ Partial to_partial(float scale = kLog2e) const {
         // nothing finite seen: the reference never moved off the floor and the sum is empty
         if (!(m > kRefFloor)) return Partial{m, 0.f, pos, 0};
-        return Partial{m, s * ex2f(-fmaf(m, kLog2e, nrl)), pos, 0};
+        return Partial{m, s * ex2f(-fmaf(m, scale, nrl)), pos, 0};
     }
 };
 

@@ -39,6 +39,12 @@ struct StepArgs {
     int32_t stage_stride;       // dense: words per row of the class-mask staging area, 0 = no staging
     int32_t depth;              // pipelined dense kernel: stages per warp
     int32_t cm_bulk;            // pipelined dense kernel: class-mask rows are fetched by bulk copies (16-byte aligned rows)
+    int32_t run_chunks;         // sampling step: every warp slot of the pipelined kernel takes one contiguous run of this
+                                // many chunks, so that the published states of a row follow the token order
+    int32_t tail_state;         // sampling kernel: the last state of a row stands for the octets past the last whole vector
+    float scale;                // log2(e) / temperature: the sums are of exp(z / T); log2(e) in a greedy step
+    float inv_t;                // 1 / temperature
+    const float* u;             // sampling step: dev [B] uniform numbers in [0, 1), else null
     PartDev p0;                 // descriptor of part0 (saves a dependent load when rows do not mix partitions)
     Partial* partials;
     unsigned int* tickets;
@@ -298,7 +304,8 @@ __device__ __forceinline__ void warp_finalize_row(const StepArgs& a, const PartD
 // One warp takes them after the streaming loop, lane r = row slot r, token by token straight
 // from the class-id vector and the row's class mask (compact code, run by one block per group).
 template <int DT>
-__device__ __forceinline__ Partial dense_tail_octets(const StepArgs& a, const PartDev& P, int row, int o_first, int o_end) {
+__device__ __forceinline__ Partial dense_tail_octets(const StepArgs& a, const PartDev& P, int row, int o_first, int o_end,
+                                                     float scale) {
     constexpr int ES = DT == kBF16 ? 2 : 4;
     float m = -INFINITY, s = 0.f;
     int pos = kNoPos;
@@ -319,7 +326,7 @@ __device__ __forceinline__ Partial dense_tail_octets(const StepArgs& a, const Pa
                 const float ref_old = fmaxf(m, kRefFloor);
                 m = fmaxf(m, z);
                 const float ref = fmaxf(m, kRefFloor);
-                s = fmaf(s, ex2f((ref_old - ref) * kLog2e), ex2f((z - ref) * kLog2e));
+                s = fmaf(s, ex2f((ref_old - ref) * scale), ex2f((z - ref) * scale));
             } else {
                 store_neg_inf<DT>(rowp, t);
             }
@@ -341,8 +348,8 @@ __device__ __forceinline__ Partial* row_slots(const StepArgs& a, int g, int row_
 // owns the end of the vocabulary) handles the tail octets, lane r = row slot r.
 template <int DT>
 __device__ __forceinline__ void publish_tail_octets(const StepArgs& a, const PartDev& P, int g, const int* s_row, int lane,
-                                                    int tail_first, int tail_end) {
-    const Partial p = dense_tail_octets<DT>(a, P, s_row[lane], tail_first, tail_end);
+                                                    int tail_first, int tail_end, float scale = kLog2e) {
+    const Partial p = dense_tail_octets<DT>(a, P, s_row[lane], tail_first, tail_end, scale);
     if (s_row[lane] >= 0) row_slots(a, g, lane)[a.slots - 1] = p;
 }
 
@@ -414,10 +421,10 @@ __device__ __forceinline__ void dense_octet_row(Octet<DT>& oc, char* rowp, uint8
 // half they keep, then 2 of 4 with the lane 8 away, then 1 of 2; two butterfly steps finish
 // the single row left (nine folds instead of forty).
 __device__ __forceinline__ void warp_rows_publish(const StepArgs& a, RowAcc (&acc)[kBatchRows], int live, int g, int slot,
-                                                  int rb, int lane) {
+                                                  int rb, int lane, float scale = kLog2e) {
     Partial p[kBatchRows];
 #pragma unroll
-    for (int i = 0; i < kBatchRows; ++i) p[i] = acc[i].to_partial();
+    for (int i = 0; i < kBatchRows; ++i) p[i] = acc[i].to_partial(scale);
 #pragma unroll
     for (int half = 4; half >= 1; half >>= 1) {
         const int d = 4 * half;  // 16, 8, 4
@@ -430,7 +437,7 @@ __device__ __forceinline__ void warp_rows_publish(const StepArgs& a, RowAcc (&ac
             const float s2 = __shfl_xor_sync(0xFFFFFFFFu, send.s, d);
             const int p2 = __shfl_xor_sync(0xFFFFFFFFu, send.pos, d);
             p[k] = keep;
-            partial_merge(p[k].m, p[k].s, p[k].pos, m2, s2, p2);
+            partial_merge(p[k].m, p[k].s, p[k].pos, m2, s2, p2, scale);
         }
     }
 #pragma unroll
@@ -438,7 +445,7 @@ __device__ __forceinline__ void warp_rows_publish(const StepArgs& a, RowAcc (&ac
         const float m2 = __shfl_xor_sync(0xFFFFFFFFu, p[0].m, d);
         const float s2 = __shfl_xor_sync(0xFFFFFFFFu, p[0].s, d);
         const int p2 = __shfl_xor_sync(0xFFFFFFFFu, p[0].pos, d);
-        partial_merge(p[0].m, p[0].s, p[0].pos, m2, s2, p2);
+        partial_merge(p[0].m, p[0].s, p[0].pos, m2, s2, p2, scale);
     }
     const int i = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);  // the row this lane ended with
     if ((lane & 3) == 0 && i < live) row_slots(a, g, rb * kBatchRows + i)[slot] = p[0];
@@ -548,7 +555,7 @@ struct BatchAddr {
 template <int DT, bool FULL, bool CONSEC>
 __device__ __forceinline__ void pipe_consume_item(const char* src, const uint32_t* T, int rb, int live, bool active,
                                                   int o, int lane, const BatchAddr& ba, char* const (&rowp)[kBatchRows],
-                                                  uint8_t* const (&vmp)[kBatchRows], RowAcc (&acc)[kBatchRows]) {
+                                                  uint8_t* const (&vmp)[kBatchRows], RowAcc (&acc)[kBatchRows], float scale) {
     using G = PipeGeom<DT>;
     uint4 cv = make_uint4(0, 0, 0, 0);
     if (FULL || active) cv = *reinterpret_cast<const uint4*>(src + kBatchRows * G::kRowBytes + lane * 16);
@@ -569,7 +576,7 @@ __device__ __forceinline__ void pipe_consume_item(const char* src, const uint32_
                 oc.store(rowp[i], o);
                 if (vmp[i]) vmp[i][o] = uint8_t(byte);
             }
-            acc[i].add_octet(f, o);
+            acc[i].add_octet(f, o, scale);
         }
     }
 }
@@ -577,8 +584,9 @@ __device__ __forceinline__ void pipe_consume_item(const char* src, const uint32_
 // TMAP: the 8 rows of a batch are consecutive rows of the logits matrix and arrive as one
 // tiled 2-D copy through `tmap` (box = 256 elements x 8 rows); otherwise one bulk copy per row.
 // LBT / MINB: launch bounds (threads per block, blocks per SM) the variant is compiled for; they set
-// the register budget: (512, 1) 128 registers, (320, 2) 96, (256, 3) 80.
-template <int DT, bool TMAP, int LBT, int MINB>
+// the register budget: (512, 1) 128 registers, (320, 2) 96, (256, 3) 80. TEMPERED: the sums are of
+// exp(z / T) with the step's temperature (sampling steps); otherwise T = 1 is compiled in.
+template <int DT, bool TMAP, int LBT, int MINB, bool TEMPERED>
 __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_constant__ StepArgs a,
                                                          const __grid_constant__ CUtensorMap tmap) {
     using G = PipeGeom<DT>;
@@ -593,6 +601,7 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
     __shared__ uint64_t cm_bar;
 
     pdl_prologue();
+    const float scale = TEMPERED ? a.scale : kLog2e;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = blockIdx.x / a.S, split = blockIdx.x - g * a.S;
     if (a.n_groups && g >= __ldg(a.n_groups)) return;
@@ -614,9 +623,12 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
     // (warp index among them, then a stride of their number), so that at any moment the group's blocks
     // read neighbouring pieces of the same rows: measured 5 % faster on long steps than one contiguous
     // range per block, and as fast as handing chunks out through global counters.
+    // In a sampling step (TEMPERED) the states of a row must follow the token order: every warp slot then
+    // takes one contiguous run of run_chunks chunks instead.
     const int n_chunks = (n_full + 31) >> 5;
-    const int first_chunk = split * a.WT + wt;      // this warp's fixed first chunk
-    const int stride_chunks = a.S * a.WT;            // warps that share a row batch of the group
+    const int first_chunk = TEMPERED ? (split * a.WT + wt) * a.run_chunks : split * a.WT + wt;  // this warp's first chunk
+    const int stride_chunks = TEMPERED ? 1 : a.S * a.WT;  // round-robin: warps that share a row batch of the group
+    const int chunk_end = TEMPERED ? min(first_chunk + a.run_chunks, n_chunks) : n_chunks;
     int* const slot_info = ring_info + warp * depth; // (rb << 24) | chunk of the item in each slot, -1 = no more items
 
     // producer cursor (meaningful in lane 0)
@@ -632,7 +644,7 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
                 chunk = p_chunk + stride_chunks;
             }
             p_chunk = chunk;
-            if (chunk < n_chunks) break;
+            if (chunk < chunk_end) break;
             chunk = -1;  // this row batch is handed out completely: on to the warp's next one
             p_rb += WR;
             p_first = true;
@@ -737,7 +749,7 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
         if (info < 0) break;
         const int rb = info >> 24, o0 = (info & 0xFFFFFF) * 32;
         while (cur_rb < rb) {  // the previous row batch of this warp is complete (possibly without any chunk)
-            warp_rows_publish(a, acc, live, g, my_slot, cur_rb, lane);
+            warp_rows_publish(a, acc, live, g, my_slot, cur_rb, lane, scale);
             cur_rb += WR;
             open_batch(cur_rb);
         }
@@ -751,9 +763,9 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
         ba.item_base = base0 + size_t(o) * G::kOctetBytes;
         ba.vm_item = vm0 ? vm0 + o : nullptr;
         if (live == kBatchRows && o0 + 32 <= n_full)
-            pipe_consume_item<DT, true, TMAP>(src, T, rb, live, true, o, lane, ba, rowp, vmp, acc);
+            pipe_consume_item<DT, true, TMAP>(src, T, rb, live, true, o, lane, ba, rowp, vmp, acc, scale);
         else
-            pipe_consume_item<DT, false, TMAP>(src, T, rb, live, o < n_full, o, lane, ba, rowp, vmp, acc);
+            pipe_consume_item<DT, false, TMAP>(src, T, rb, live, o < n_full, o, lane, ba, rowp, vmp, acc, scale);
         ++consumed;
         if (++slot == depth) { slot = 0; phase ^= 1u; }
         __syncwarp();  // every lane has its data out of the slot before it is refilled
@@ -763,7 +775,7 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
     if (!failed) {
         // whatever row batches of this warp are left (all of them if it never got a chunk) are published too
         for (; cur_rb * kBatchRows < nrow; cur_rb += WR) {
-            warp_rows_publish(a, acc, live, g, my_slot, cur_rb, lane);
+            warp_rows_publish(a, acc, live, g, my_slot, cur_rb, lane, scale);
             if ((cur_rb + WR) * kBatchRows < nrow) open_batch(cur_rb + WR);
         }
     } else if (lane == 0) {
@@ -776,7 +788,7 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
         }
     }
     // the block that reaches the end of the vocabulary takes the octets past the last whole vector
-    if (warp == 0 && split == 0) publish_tail_octets<DT>(a, P, g, s_row, lane, n_full, n_octets);
+    if (warp == 0 && split == 0) publish_tail_octets<DT>(a, P, g, s_row, lane, n_full, n_octets, scale);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -1036,19 +1048,220 @@ __global__ void __launch_bounds__(256) k_step_generic(const __grid_constant__ St
                 const float ref_old = fmaxf(m, kRefFloor);
                 m = fmaxf(m, z);
                 const float ref = fmaxf(m, kRefFloor);
-                s = fmaf(s, ex2f((ref_old - ref) * kLog2e), ex2f((z - ref) * kLog2e));
+                s = fmaf(s, ex2f((ref_old - ref) * a.scale), ex2f((z - ref) * a.scale));
             } else {
                 store_neg_inf<DT>(rowp, t);
             }
         }
     }
     if (!FUSED) return;
-    partial_warp_allreduce(m, s, pos);
+    partial_warp_allreduce(m, s, pos, a.scale);
     if (lane == 0) s_red[warp] = Partial{m, s, pos, 0};
     __syncthreads();
     if (tid == 0) {
-        for (int w = 1; w < n_warps; ++w) partial_merge(m, s, pos, s_red[w].m, s_red[w].s, s_red[w].pos);
-        finalize_row<DT>(a, P, row, m, s, pos, true);
+        for (int w = 1; w < n_warps; ++w) partial_merge(m, s, pos, s_red[w].m, s_red[w].s, s_red[w].pos, a.scale);
+        if (a.u)
+            a.partials[row] = Partial{m, s, pos, 0};  // a sampling step: the sampling kernel takes it from here
+        else
+            finalize_row<DT>(a, P, row, m, s, pos, true);
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Second kernel of a sampling step: one block per row draws the row's token from the tempered
+// distribution over its allowed tokens by inverse CDF in token order, with the row's uniform number
+// u: the lowest token whose cumulative weight exceeds u times the total. The states the streaming
+// kernel published stand for consecutive runs of tokens (state k: chunks [k * run_chunks,
+// (k+1) * run_chunks) of 256 tokens; with tail_state the last one: the tokens past the last whole
+// vector), so the block first scans the states for the run that holds the crossing, then re-reads
+// the masked logits of that run only and scans them. All sums are taken in a fixed order.
+// ---------------------------------------------------------------------------------------
+constexpr int kSampleThreads = 256;
+
+// Exclusive prefix sum of one value per thread over the block, in thread order; total to everybody.
+__device__ __forceinline__ float block_exclusive_scan(float v, float* s_warp, float& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    float inc = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const float up = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+        if (lane >= d) inc += up;
+    }
+    __syncthreads();  // s_warp may still be read from an earlier call
+    if (lane == 31) s_warp[warp] = inc;
+    __syncthreads();
+    float before = 0.f, all = 0.f;
+#pragma unroll
+    for (int w = 0; w < kSampleThreads / 32; ++w) {
+        const float t = s_warp[w];
+        if (w < warp) before += t;
+        all += t;
+    }
+    total = all;
+    return before + inc - v;
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kSampleThreads) k_sample_rows(const __grid_constant__ StepArgs a, int aligned) {
+    __shared__ float s_warp[kSampleThreads / 32];
+    __shared__ int s_pick, s_last;
+    __shared__ float s_base;
+    pdl_prologue();
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int g = blockIdx.x / kGroupRows, j = blockIdx.x - g * kGroupRows;
+    if (a.n_groups && g >= __ldg(a.n_groups)) return;
+    int row;
+    if (a.group_rows) {
+        row = a.group_rows[g * kGroupRows + j];
+    } else {
+        row = g * kGroupRows + j;
+        if (row >= a.B) row = -1;
+    }
+    if (row < 0) return;
+    PartDev P = a.p0;
+    if (a.group_part) {
+        P = a.parts[a.group_part[g]];
+    } else if (a.row_part) {
+        const int part = a.row_part[row];
+        if (part < 0 || part >= a.n_parts || !a.parts[part].live || a.parts[part].V != a.V) return;  // counted by the step kernel
+        P = a.parts[part];
+    }
+    const Partial* src = row_slots(a, g, j);
+    const int n_states = a.slots;
+    const int per = (n_states + kSampleThreads - 1) / kSampleThreads;  // consecutive states per thread
+    const int k0 = tid * per, k1 = min(k0 + per, n_states);
+
+    // the row maximum
+    float M = -INFINITY;
+    for (int k = k0; k < k1; ++k) M = fmaxf(M, __ldcg(&src[k].m));
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, d));
+    if (lane == 0) s_warp[warp] = M;
+    if (tid == 0) { s_pick = kNoPos; s_last = -1; }
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < kSampleThreads / 32; ++w) M = fmaxf(M, s_warp[w]);
+    if (!(M > kRefFloor)) {
+        // nothing allowed, or only -inf allowed: the lowest allowed token (if any) and -inf logs
+        if (warp == 0) {
+            unsigned long long cand = first_allowed_share(a, P, row, lane, 32);
+#pragma unroll
+            for (int d = 16; d >= 1; d >>= 1) {
+                const unsigned long long other = __shfl_xor_sync(0xFFFFFFFFu, cand, d);
+                cand = other < cand ? other : cand;
+            }
+            if (lane == 0) write_row_outputs(a, row, -INFINITY, 0.f, cand);
+        }
+        return;
+    }
+
+    // weights of the states relative to M, their exclusive prefix sums in token order, the total
+    float mine = 0.f;
+    for (int k = k0; k < k1; ++k) {
+        const int4 raw = __ldcg(reinterpret_cast<const int4*>(src + k));
+        mine += __int_as_float(raw.y) * ex2f((fmaxf(__int_as_float(raw.x), kRefFloor) - M) * a.scale);
+    }
+    float total;
+    const float front = block_exclusive_scan(mine, s_warp, total);  // weight in front of this thread's states
+    const float tau = __ldg(a.u + row) * total;
+    auto weight = [&](int k) {
+        const int4 raw = __ldcg(reinterpret_cast<const int4*>(src + k));
+        return __int_as_float(raw.y) * ex2f((fmaxf(__int_as_float(raw.x), kRefFloor) - M) * a.scale);
+    };
+    float run = front;
+    for (int k = k0; k < k1; ++k) {
+        const float w = weight(k);
+        if (w > 0.f) {
+            atomicMax(&s_last, k);
+            if (run + w > tau) {
+                atomicMin(&s_pick, k);
+                break;
+            }
+        }
+        run += w;
+    }
+    __syncthreads();
+    const int pick = s_pick != kNoPos ? s_pick : s_last;  // rounding may leave tau at the very end: the last run with weight
+    if (pick >= k0 && pick < k1) {  // the thread that owns the chosen state: the weight in front of it
+        float r2 = front;
+        for (int k = k0; k < pick; ++k) r2 += weight(k);
+        s_base = r2;
+    }
+    __syncthreads();
+    if (tid == 0) { s_pick = kNoPos; s_last = -1; }
+    float base = s_base;
+
+    // the tokens the chosen state stands for
+    const int n_full8 = (a.V >> 3) << 3;
+    int t_lo, t_hi;
+    if (a.tail_state && pick == n_states - 1) {
+        t_lo = n_full8;
+        t_hi = a.V;
+    } else {
+        const long long lim = a.tail_state ? n_full8 : a.V;
+        t_lo = int(min(static_cast<long long>(pick) * a.run_chunks * 256, lim));
+        t_hi = int(min(static_cast<long long>(pick + 1) * a.run_chunks * 256, lim));
+    }
+    constexpr int ES = DT == kBF16 ? 2 : 4;
+    const char* rowp = reinterpret_cast<const char*>(a.logits) + int64_t(row) * a.row_stride * ES;
+    int token = -1;
+    for (int p0 = t_lo; p0 < t_hi; p0 += kSampleThreads * 8) {
+        const int t0 = p0 + tid * 8;
+        float e[8];
+        if (aligned && t0 + 8 <= t_hi) {  // t_lo is a multiple of 8 tokens: 16-byte (bf16) / 32-byte (f32) vectors
+            if (DT == kBF16) {
+                const uint4 v = __ldcg(reinterpret_cast<const uint4*>(rowp + size_t(t0) * 2));
+                e[0] = __uint_as_float(v.x << 16); e[1] = __uint_as_float(v.x & 0xFFFF0000u);
+                e[2] = __uint_as_float(v.y << 16); e[3] = __uint_as_float(v.y & 0xFFFF0000u);
+                e[4] = __uint_as_float(v.z << 16); e[5] = __uint_as_float(v.z & 0xFFFF0000u);
+                e[6] = __uint_as_float(v.w << 16); e[7] = __uint_as_float(v.w & 0xFFFF0000u);
+            } else {
+                const float4 v0 = __ldcg(reinterpret_cast<const float4*>(rowp + size_t(t0) * 4));
+                const float4 v1 = __ldcg(reinterpret_cast<const float4*>(rowp + size_t(t0) * 4 + 16));
+                e[0] = v0.x; e[1] = v0.y; e[2] = v0.z; e[3] = v0.w;
+                e[4] = v1.x; e[5] = v1.y; e[6] = v1.z; e[7] = v1.w;
+            }
+        } else {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) e[q] = t0 + q < t_hi ? ldcg_elem<DT>(rowp, t0 + q) : -INFINITY;
+        }
+        float sum8 = 0.f;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            e[q] = ex2f((e[q] - M) * a.scale);  // a masked logit is -inf: weight 0
+            sum8 += e[q];
+        }
+        float piece;
+        float r3 = base + block_exclusive_scan(sum8, s_warp, piece);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            if (e[q] > 0.f) {
+                atomicMax(&s_last, t0 + q);
+                r3 += e[q];
+                if (r3 > tau) {
+                    atomicMin(&s_pick, t0 + q);
+                    break;
+                }
+            }
+        }
+        __syncthreads();
+        if (s_pick != kNoPos) break;
+        base += piece;
+    }
+    token = s_pick != kNoPos ? s_pick : s_last;  // rounding: the last token with weight in the run
+    if (tid == 0) {
+        float lsev = -INFINITY, lpt = -INFINITY;
+        int repv = -1;
+        if (token >= 0) {
+            const float l = logf(total);
+            lsev = fmaf(M, a.inv_t, l);
+            lpt = (ldcg_elem<DT>(rowp, token) - M) * a.inv_t - l;
+            repv = P.r[P.c32[token]];
+        }
+        a.argmax[row] = token;
+        if (a.rep) a.rep[row] = repv;
+        if (a.lse) a.lse[row] = lsev;
+        if (a.logp_argmax) a.logp_argmax[row] = lpt;
     }
 }
 
