@@ -636,19 +636,22 @@ int cfgzip_load_partition(cfgzip_ctx* ctx, const int32_t* c, int32_t V, const in
     p.KW = ceil_div(K, 32);
     p.VW = ceil_div(V, 32);
     const bool has16 = K <= 65535;  // the value K itself is the padding id
-    // host image of the device block: c32 | r | off | tok | c16 (16-byte aligned pieces)
+    // host image of the device block: c32 | r | off | tok | trep | c16 (16-byte aligned pieces)
     auto align4 = [](size_t n) { return (n + 3) & ~size_t(3); };
     const size_t n_c32 = align4(size_t(V)), n_r = align4(size_t(K)), n_off = align4(size_t(K) + 1), n_tok = align4(size_t(V));
+    const size_t n_trep = align4(size_t(V));
     const size_t n_c16_words = has16 ? size_t(p.VW) * 16 : 0;  // 32*VW uint16 = 16*VW words
-    std::vector<int32_t> img(n_c32 + n_r + n_off + n_tok + n_c16_words, 0);
+    std::vector<int32_t> img(n_c32 + n_r + n_off + n_tok + n_trep + n_c16_words, 0);
     int32_t* h_c32 = img.data();
     int32_t* h_r = h_c32 + n_c32;
     int32_t* h_off = h_r + n_r;
     int32_t* h_tok = h_off + n_off;
-    uint16_t* h_c16 = reinterpret_cast<uint16_t*>(h_tok + n_tok);
+    int32_t* h_trep = h_tok + n_tok;
+    uint16_t* h_c16 = reinterpret_cast<uint16_t*>(h_trep + n_trep);
     std::memcpy(h_c32, c, size_t(V) * 4);
     std::memcpy(h_r, r, size_t(K) * 4);
     build_class_lists_host(c, V, K, h_off, h_tok);
+    for (int32_t i = 0; i < V; ++i) h_trep[i] = r[c[i]];
     if (has16) {
         for (int32_t i = 0; i < V; ++i) h_c16[i] = uint16_t(c[i]);
         for (int32_t i = V; i < 32 * p.VW; ++i) h_c16[i] = uint16_t(K);
@@ -663,7 +666,8 @@ int cfgzip_load_partition(cfgzip_ctx* ctx, const int32_t* c, int32_t V, const in
     p.dev.r = d + n_c32;
     p.dev.off = d + n_c32 + n_r;
     p.dev.tok = d + n_c32 + n_r + n_off;
-    p.dev.c16 = has16 ? reinterpret_cast<const uint16_t*>(d + n_c32 + n_r + n_off + n_tok) : nullptr;
+    p.dev.trep = d + n_c32 + n_r + n_off + n_tok;
+    p.dev.c16 = has16 ? reinterpret_cast<const uint16_t*>(d + n_c32 + n_r + n_off + n_tok + n_trep) : nullptr;
     p.dev.K = K;
     p.dev.KW = p.KW;
     p.dev.V = V;

@@ -23,6 +23,7 @@ struct PartDev {
     const int32_t* r;      // class -> representative token, K entries
     const int32_t* off;    // class -> start in tok, K+1 entries
     const int32_t* tok;    // tokens grouped by class, ascending inside a class
+    const int32_t* trep;   // token -> representative of its class, r[c[t]], V entries (one load instead of two in a chain)
     int32_t K;
     int32_t KW;
     int32_t V;

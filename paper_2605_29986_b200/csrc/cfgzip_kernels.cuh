@@ -86,7 +86,7 @@ __device__ void finalize_row(const StepArgs& a, const PartDev& P, int row, float
                 if (((cm[k >> 5] >> (k & 31)) & 1u) && ldcg_elem<DT>(base, t) == m) tok = t;
             }
         }
-        if (tok >= 0) repv = P.r[P.c32[tok]];
+        if (tok >= 0) repv = P.trep[tok];
         if (m > kRefFloor && s > 0.f) {
             const float l = logf(s);
             lsev = m + l;
@@ -282,13 +282,14 @@ __device__ __forceinline__ void warp_finalize_row(const StepArgs& a, const PartD
     if (pos == kNoPos) {
         cand = first_allowed_share(a, P, row, lane, 32);
     } else {
+        // a position means that m is a finite allowed logit; the row is already masked in memory (disallowed
+        // logits read -inf), so the first token of the octet that holds the value m is the choice. Its
+        // representative is fetched side by side with the logit.
         const int t = 8 * pos + lane;
         if (lane < 8 && t < a.V) {
             const float z = ldcg_elem<DT>(reinterpret_cast<const char*>(a.logits) + int64_t(row) * a.row_stride * (DT == kBF16 ? 2 : 4), t);
-            const int k = P.c32[t];
-            const uint32_t word = a.class_mask[int64_t(row) * a.cm_stride + (k >> 5)];
-            const int repv = P.r[k];
-            if (((word >> (k & 31)) & 1u) && z == m) cand = (static_cast<unsigned long long>(t) << 32) | static_cast<unsigned int>(repv);
+            const int repv = __ldg(P.trep + t);
+            if (z == m) cand = (static_cast<unsigned long long>(t) << 32) | static_cast<unsigned int>(repv);
         }
     }
 #pragma unroll
@@ -1256,7 +1257,7 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample_rows(const __grid_con
             const float l = logf(total);
             lsev = fmaf(M, a.inv_t, l);
             lpt = (ldcg_elem<DT>(rowp, token) - M) * a.inv_t - l;
-            repv = P.r[P.c32[token]];
+            repv = P.trep[token];
         }
         a.argmax[row] = token;
         if (a.rep) a.rep[row] = repv;
@@ -1487,7 +1488,7 @@ __global__ void __launch_bounds__(256) k_map_tokens(const PartDev* parts, int n_
     }
     const int t = tokens[b];
     int rv = -1;
-    if (t >= 0 && t < parts[p].V) rv = parts[p].r[parts[p].c32[t]];
+    if (t >= 0 && t < parts[p].V) rv = parts[p].trep[t];
     else atomicAdd(status + 1, 1);
     reps[b] = rv;
 }
