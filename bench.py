@@ -396,7 +396,7 @@ def run_own(args):
             dist.barrier()
 
     runner = StepRunner(cz, torch, local_rank, args.workload, B=args.batch, mode=args.mode, steps_hint=args.steps,
-                        tune=args.tune)
+                        tune=args.tune, inv_temperature=args.sample_inv_temperature)
     props = torch.cuda.get_device_properties(local_rank)
     sampler = ClockSampler("GPU-" + str(props.uuid))
     seconds, launches = runner.timed(args.steps, args.warmup, barrier, sampler)
@@ -421,8 +421,9 @@ def run_own(args):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": runner.dtype if runner.dtype != "f32" else "f32",
         "data": "synthetic",
         "config": {
-            "workload": "cfg%d %s: V=%d K=%d B=%d %s, fused expand+mask+lse+argmax+rep, %s" % (
-                args.workload, synth.CONFIGS[args.workload]["name"], runner.V, runner.K, runner.B, runner.dtype, args.mode),
+            "workload": "cfg%d %s: V=%d K=%d B=%d %s, fused expand+mask+lse+%s+rep, %s" % (
+                args.workload, synth.CONFIGS[args.workload]["name"], runner.V, runner.K, runner.B, runner.dtype,
+                "argmax" if not args.sample_inv_temperature else "sample(1/T=%g)" % args.sample_inv_temperature, args.mode),
             "rows_per_gpu": runner.B, "global_rows": world * runner.B,
             "l2": "inputs larger than L2: ring of %d working buffers (%.2f GB), refilled with unmasked logits before the "
                   "timed region" % (runner.R, runner.R * runner.B * runner.V * runner.elem / 1e9),
@@ -444,12 +445,13 @@ def run_own(args):
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": traffic, "peak_source": "of " + peak_src, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                      "algorithmic_bytes_per_step": alg, "launches_per_step": launches / max(args.steps, 1),
-                     "kernel": "k_step_dense_pipe (+ k_finalize_rows)" if args.mode != "sparse" else "k_step_sparse"},
+                     "kernel": ("k_step_sparse" if args.mode == "sparse" else
+                                "k_step_dense_pipe (+ %s)" % ("k_sample_rows" if args.sample_inv_temperature else "k_finalize_rows"))},
         "clocks": sampler.summary(),
         "paper_context": "paper reports no timing of this path; its speedups (up to two orders of magnitude in grammar-engine "
                          "latency, up to 7.5x end to end) are for 1x H100 + Xeon Gold 6430 x16 threads, precision unstated",
     }
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.sample_inv_temperature:
         line["cpu_baseline"], line["parity"] = _cpu_baseline(runner, torch)
     runner.close()
     if rank == 0 and world == 1 and not args.no_extras:
@@ -563,6 +565,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=200)
     ap.add_argument("--tune", action="append", default=[], metavar="NAME=VALUE",
                     help="library tuning knob (see cfgzip_set_tuning); may be repeated")
+    ap.add_argument("--sample-inv-temperature", type=float, default=0.0, metavar="1/T",
+                    help="time the sampling step (cfgzip_masked_sample) at this inverse temperature instead of the greedy one")
     ap.add_argument("--no-extras", action="store_true", help="skip the larger-batch sweep")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -435,8 +435,12 @@ int launch_fused(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, in
                 rc = launch(ctx, kern, grid, block, d.smem, st, a);
             }
             // second kernel: one block per row folds the published states and writes the results
-            if (rc == CFGZIP_OK)
-                rc = launch(ctx, k_finalize_rows<DT>, dim3(unsigned(d.n_groups_ub) * kGroupRows), dim3(kFinalizeThreads), 0, st, a);
+            if (rc == CFGZIP_OK) {
+                if (a.slots <= kFinalizeWarpStates)  // few states per row: a warp per row
+                    rc = launch(ctx, k_finalize_rows_warp<DT>, dim3(unsigned(d.n_groups_ub) * (kGroupRows / 8)), dim3(256), 0, st, a);
+                else
+                    rc = launch(ctx, k_finalize_rows<DT>, dim3(unsigned(d.n_groups_ub) * kGroupRows), dim3(kFinalizeThreads), 0, st, a);
+            }
         } else {
             rc = launch(ctx, k_step_generic<DT, true>, dim3(unsigned(a.B)), dim3(256), 0, st, a);
         }

@@ -405,6 +405,43 @@ __global__ void __launch_bounds__(kFinalizeThreads) k_finalize_rows(const __grid
     warp_finalize_row<DT>(a, P, row, m0, s0, p0, lane);
 }
 
+// The same for rows with few published states (at most 4 per lane: large batches, where a group is
+// shared by few blocks): one warp per row, 8 rows per block, no block-level step at all.
+constexpr int kFinalizeWarpStates = 128;
+
+template <int DT>
+__global__ void __launch_bounds__(256) k_finalize_rows_warp(const __grid_constant__ StepArgs a) {
+    pdl_prologue();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int idx = blockIdx.x * 8 + warp;  // (group, row slot)
+    const int g = idx / kGroupRows, j = idx - g * kGroupRows;
+    if (a.n_groups && g >= __ldg(a.n_groups)) return;
+    int row;
+    if (a.group_rows) {
+        row = a.group_rows[g * kGroupRows + j];
+    } else {
+        row = g * kGroupRows + j;
+        if (row >= a.B) row = -1;
+    }
+    if (row < 0) return;
+    const PartDev P = a.group_part ? a.parts[a.group_part[g]] : a.p0;
+    const Partial* src = row_slots(a, g, j);
+    int4 v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const int sp = u * 32 + lane;
+        v[u] = make_int4(__float_as_int(-INFINITY), 0, kNoPos, 0);
+        if (sp < a.slots) v[u] = __ldcg(reinterpret_cast<const int4*>(src + sp));
+    }
+    float m0 = __int_as_float(v[0].x), s0 = __int_as_float(v[0].y), m1 = __int_as_float(v[1].x), s1 = __int_as_float(v[1].y);
+    int p0 = v[0].z, p1 = v[1].z;
+    partial_merge(m0, s0, p0, __int_as_float(v[2].x), __int_as_float(v[2].y), v[2].z);
+    partial_merge(m1, s1, p1, __int_as_float(v[3].x), __int_as_float(v[3].y), v[3].z);
+    partial_merge(m0, s0, p0, m1, s1, p1);
+    partial_warp_allreduce(m0, s0, p0);
+    warp_finalize_row<DT>(a, P, row, m0, s0, p0, lane);
+}
+
 // One whole-vector octet of one row: mask, write back, note the vocab-mask byte, fold into the
 // row state.
 template <int DT>
