@@ -1165,13 +1165,34 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample_rows(const __grid_con
         P = a.parts[part];
     }
     const Partial* src = row_slots(a, g, j);
+    const float u = __ldg(a.u + row);  // needed late: in flight together with the states
     const int n_states = a.slots;
     const int per = (n_states + kSampleThreads - 1) / kSampleThreads;  // consecutive states per thread
     const int k0 = tid * per, k1 = min(k0 + per, n_states);
 
+    // the states of this thread: fetched once, all loads in flight together, kept in registers when there are
+    // at most four of them (otherwise they are fetched again wherever they are needed)
+    constexpr int kKeep = 4;
+    const bool kept = per <= kKeep;
+    float km[kKeep], ks[kKeep];
+#pragma unroll
+    for (int i = 0; i < kKeep; ++i) {
+        km[i] = -INFINITY;
+        ks[i] = 0.f;
+        if (kept && k0 + i < k1) {
+            const int4 raw = __ldcg(reinterpret_cast<const int4*>(src + k0 + i));
+            km[i] = __int_as_float(raw.x);
+            ks[i] = __int_as_float(raw.y);
+        }
+    }
     // the row maximum
     float M = -INFINITY;
-    for (int k = k0; k < k1; ++k) M = fmaxf(M, __ldcg(&src[k].m));
+    if (kept) {
+#pragma unroll
+        for (int i = 0; i < kKeep; ++i) M = fmaxf(M, km[i]);
+    } else {
+        for (int k = k0; k < k1; ++k) M = fmaxf(M, __ldcg(&src[k].m));
+    }
 #pragma unroll
     for (int d = 16; d >= 1; d >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, d));
     if (lane == 0) s_warp[warp] = M;
@@ -1194,18 +1215,23 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample_rows(const __grid_con
     }
 
     // weights of the states relative to M, their exclusive prefix sums in token order, the total
-    float mine = 0.f;
-    for (int k = k0; k < k1; ++k) {
-        const int4 raw = __ldcg(reinterpret_cast<const int4*>(src + k));
-        mine += __int_as_float(raw.y) * ex2f((fmaxf(__int_as_float(raw.x), kRefFloor) - M) * a.scale);
-    }
-    float total;
-    const float front = block_exclusive_scan(mine, s_warp, total);  // weight in front of this thread's states
-    const float tau = __ldg(a.u + row) * total;
+#pragma unroll
+    for (int i = 0; i < kKeep; ++i) ks[i] *= ex2f((fmaxf(km[i], kRefFloor) - M) * a.scale);  // now the weight (0 if unused)
     auto weight = [&](int k) {
+        if (kept) {
+            float w = 0.f;
+#pragma unroll
+            for (int i = 0; i < kKeep; ++i) w = (k - k0 == i) ? ks[i] : w;
+            return w;
+        }
         const int4 raw = __ldcg(reinterpret_cast<const int4*>(src + k));
         return __int_as_float(raw.y) * ex2f((fmaxf(__int_as_float(raw.x), kRefFloor) - M) * a.scale);
     };
+    float mine = 0.f;
+    for (int k = k0; k < k1; ++k) mine += weight(k);
+    float total;
+    const float front = block_exclusive_scan(mine, s_warp, total);  // weight in front of this thread's states
+    const float tau = u * total;
     float run = front;
     for (int k = k0; k < k1; ++k) {
         const float w = weight(k);
@@ -1242,6 +1268,7 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample_rows(const __grid_con
     }
     constexpr int ES = DT == kBF16 ? 2 : 4;
     const char* rowp = reinterpret_cast<const char*>(a.logits) + int64_t(row) * a.row_stride * ES;
+    __shared__ float s_ztok;
     int token = -1;
     for (int p0 = t_lo; p0 < t_hi; p0 += kSampleThreads * 8) {
         const int t0 = p0 + tid * 8;
@@ -1263,37 +1290,47 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample_rows(const __grid_con
 #pragma unroll
             for (int q = 0; q < 8; ++q) e[q] = t0 + q < t_hi ? ldcg_elem<DT>(rowp, t0 + q) : -INFINITY;
         }
-        float sum8 = 0.f;
+        float z8[8], sum8 = 0.f;
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
+            z8[q] = e[q];
             e[q] = ex2f((e[q] - M) * a.scale);  // a masked logit is -inf: weight 0
             sum8 += e[q];
         }
         float piece;
         float r3 = base + block_exclusive_scan(sum8, s_warp, piece);
+        int mine_tok = -1, mine_last = -1;
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
-            if (e[q] > 0.f) {
-                atomicMax(&s_last, t0 + q);
+            if (e[q] > 0.f && mine_tok < 0) {
+                mine_last = t0 + q;
                 r3 += e[q];
-                if (r3 > tau) {
-                    atomicMin(&s_pick, t0 + q);
-                    break;
-                }
+                if (r3 > tau) mine_tok = t0 + q;
             }
         }
+        if (mine_last >= 0) atomicMax(&s_last, mine_last);
+        if (mine_tok >= 0) atomicMin(&s_pick, mine_tok);
         __syncthreads();
-        if (s_pick != kNoPos) break;
+        token = s_pick != kNoPos ? s_pick : -1;
+        const bool last_piece = p0 + kSampleThreads * 8 >= t_hi;
+        if (token < 0 && last_piece) token = s_last;  // rounding: the last token with weight in the run
+        if (token >= t0 && token < t0 + 8) {          // the thread that holds the token hands its logit over
+            float zt = 0.f;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) zt = (token - t0 == q) ? z8[q] : zt;
+            s_ztok = zt;
+        }
+        if (token >= 0) break;
         base += piece;
     }
-    token = s_pick != kNoPos ? s_pick : s_last;  // rounding: the last token with weight in the run
+    __syncthreads();
     if (tid == 0) {
         float lsev = -INFINITY, lpt = -INFINITY;
         int repv = -1;
         if (token >= 0) {
             const float l = logf(total);
             lsev = fmaf(M, a.inv_t, l);
-            lpt = (ldcg_elem<DT>(rowp, token) - M) * a.inv_t - l;
+            lpt = (s_ztok - M) * a.inv_t - l;
             repv = P.trep[token];
         }
         a.argmax[row] = token;
