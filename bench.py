@@ -44,7 +44,7 @@ RING_MAX_BYTES = 24 << 30
 # DRAM traffic of the dominant (streaming) kernel per launch = per step (dram__bytes_read.sum +
 # dram__bytes_write.sum from one ncu capture), keyed by workload; valid only for the kernel sources whose digest is
 # recorded with it. None until a capture of the current sources exists.
-NCU_TRAFFIC = {"cfg2_B32_dense": {"digest": "bf663398c0da422c", "bytes_per_launch": 8538709}}
+NCU_TRAFFIC = {"cfg2_B32_dense": {"digest": "398ff78bcda58931", "bytes_per_launch": 8538965}}
 
 
 def _kernel_digest() -> str:
@@ -505,6 +505,19 @@ def run_own(args):
         s5, _ = r5.timed(2000, 100)
         line["warm_l2_us_per_step"] = s5 / 2000 * 1e6
         r5.close()
+        # the five workloads at their own sizes (cfg2 is the headline above), same protocol, shorter runs
+        five = []
+        for cfg in sorted(synth.CONFIGS):
+            r7 = StepRunner(cz, torch, local_rank, cfg, mode="dense", steps_hint=64, unique=2, tune=args.tune)
+            n = 3 * r7.R
+            s7, l7 = r7.timed(n, r7.R)
+            a7 = r7.alg_bytes() / (s7 / n) / 1e9
+            five.append({"workload": "cfg%d %s: V=%d K=%d B=%d %s, %d partition(s)" % (
+                             cfg, synth.CONFIGS[cfg]["name"], r7.V, r7.K, r7.B, r7.dtype, len(r7.parts)),
+                         "us_per_step": s7 / n * 1e6, "rows_per_s": r7.B * n / s7, "achieved_gbs": a7,
+                         "frac_of_measured": a7 / peak, "launches_per_step": l7 / n, "ring": r7.R})
+            r7.close()
+        line["five_workloads_dense"] = five
         # sparse-mask stress workload (1-5 allowed classes per row): gather path against class-list scatter path
         pair = {}
         for mode in ("dense", "sparse"):

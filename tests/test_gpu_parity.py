@@ -369,3 +369,56 @@ def test_argument_errors_are_reported_before_any_launch():
         cz.cfgzip_free_partition(ctx.h, ctx.ids[0])
         assert fused() == cz.E_RANGE  # freed partition
     assert lib.cfgzip_create(99, ctypes.byref(ctypes.c_void_p())) == cz.E_CUDA
+
+
+# ------------------------------------------------------------------ CUDA graphs
+
+def test_steps_replayed_from_a_cuda_graph_match_the_oracle():
+    # the per-step calls only enqueue work: captured once, replayed on fresh inputs, greedy and sampling
+    w = synth.make_workload(2, B=40, V=20000, K=300)
+    VW = (w.V + 31) // 32
+    with Ctx(w.partitions) as ctx:
+        d_z = torch.empty((w.B, w.V), dtype=torch.int16, device="cuda")
+        d_cm = torch.empty((w.B, (w.K + 31) // 32), dtype=torch.int32, device="cuda")
+        d_u = torch.empty(w.B, dtype=torch.float32, device="cuda")
+        d_vm = torch.zeros((w.B, VW), dtype=torch.int32, device="cuda")
+        outs = [torch.zeros(w.B, dtype=torch.int32, device="cuda") for _ in range(2)]
+        outs += [torch.zeros(w.B, dtype=torch.float32, device="cuda") for _ in range(2)]
+        stream = torch.cuda.Stream()
+        graphs = {}
+        for kind in ("greedy", "sample"):
+            g = torch.cuda.CUDAGraph()
+            stream.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(stream), torch.cuda.graph(g, stream=stream):
+                if kind == "greedy":
+                    cz.cfgzip_masked_logsoftmax_argmax(ctx.h, ctx.ids[0], None, d_cm, d_cm.shape[1], d_z, cz.BF16, w.V, w.B,
+                                                       d_vm, VW, outs[0], outs[1], outs[2], outs[3], None, cz.DENSE, stream)
+                else:
+                    cz.cfgzip_masked_sample(ctx.h, ctx.ids[0], None, d_cm, d_cm.shape[1], d_z, cz.BF16, w.V, w.B, d_vm, VW,
+                                            d_u, 5.0, outs[0], outs[1], outs[2], outs[3], cz.DENSE, stream)
+            graphs[kind] = g
+        for step in (0, 1, 2):
+            cm, z, u = w.class_masks(step), w.logits(step), w.uniforms(step)
+            for kind in ("greedy", "sample"):
+                d_z.copy_(dev(z)); d_cm.copy_(dev(cm)); d_u.copy_(dev(u))
+                torch.cuda.synchronize()
+                graphs[kind].replay()
+                torch.cuda.synchronize()
+                zc = z.copy()
+                if kind == "greedy":
+                    want = oracle.decode_step(w.partitions, None, cm, zc)
+                    assert np.array_equal(outs[0].cpu().numpy(), want["argmax"])
+                    assert np.abs(outs[3].cpu().numpy() - want["lse"]).max() <= LOGP_TOL
+                else:
+                    want = oracle.sample_step(w.partitions, None, cm, zc, 5.0, u.astype(np.float64), want_cdf=True)
+                    got = outs[0].cpu().numpy()
+                    for b in np.flatnonzero(got != want["token"]):  # only within rounding of a CDF boundary
+                        t = int(got[b])
+                        lo = want["cdf"][b, t - 1] if t > 0 else 0.0
+                        assert lo - 2e-5 <= u[b] <= want["cdf"][b, t] + 2e-5
+                    assert (got != want["token"]).sum() <= 1
+                assert np.array_equal(host(d_vm, np.uint32), want["vocab_mask"])
+                assert np.array_equal(host(d_z, np.uint16), zc)
+                part = w.partitions[0]
+                tok = outs[0].cpu().numpy()
+                assert np.array_equal(outs[1].cpu().numpy(), part.r[part.c[tok]])
