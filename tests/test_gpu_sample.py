@@ -204,3 +204,32 @@ def test_sample_full_size_workloads(config, B):
         got = run_sample(ctx, w.row_part, cm, z, w.V, u, 5.0)
         near = check_sample(got, w.partitions, w.row_part, cm, z, w.V, u, 5.0, "cfg%d" % config)
     assert near <= 2
+
+
+def test_sample_huge_vocabulary_many_states_per_row():
+    # a long row shared by every SM: more published states than the sampling kernel keeps in registers
+    V, K, B = 1000003, 500, 2
+    part = synth.zipf_partition(V, K, 1.1, seed=8)
+    cm = synth.class_mask_bernoulli(K, B, 0.2, rng.stream_key(81))
+    z = synth.logits_normal(B, V + 5, 1.5, "f32", (82,))
+    with Ctx([part]) as ctx:
+        plan = cz.cfgzip_plan_query(148, 232448, V, K, B, cz.F32)
+        assert plan["kind"] == 2 and plan["states_per_row"] > 1024
+        for trial in range(3):
+            u = rng.uniform(rng.stream_key(83, trial), B).astype(np.float32)
+            got = run_sample(ctx, None, cm, z, V, u, 3.0, stride=V + 5)
+            check_sample(got, [part], None, cm, z, V, u, 3.0, "trial %d" % trial)
+
+
+def test_sample_unaligned_rows_with_mixed_partitions():
+    V, B, stride = 5003, 21, 5005
+    parts = [synth.zipf_partition(V, K, 1.1, seed=s) for s, K in enumerate((64, 200, 31))]
+    row_part = (rng.u64(rng.stream_key(91), B) % np.uint64(3)).astype(np.int32)
+    cm = synth.class_mask_bernoulli(224, B, 0.3, rng.stream_key(92))
+    cm[:, 0] |= 1
+    z = synth.logits_normal(B, stride, 1.0, "bf16", (93,))
+    u = rng.uniform(rng.stream_key(94), B).astype(np.float32)
+    with Ctx(parts) as ctx:
+        got = run_sample(ctx, row_part, cm, z, V, u, 5.0, stride=stride)
+        check_sample(got, parts, row_part, cm, z, V, u, 5.0)
+        assert cz.cfgzip_poll_status(ctx.h) == (0, 0, 0)
