@@ -77,6 +77,7 @@ struct cfgzip_ctx {
     int32_t pipe_warps = 16;
     int32_t pipe_depth = 2;
     int32_t waves = 1;        // pipelined kernel: blocks launched per resident block slot
+    int32_t stage_alias = 0;  // 1: always lay the class-mask staging area over the rings (default: only where it buys warps)
 };
 
 namespace {
@@ -191,6 +192,8 @@ struct DensePlan {
     int S = 1, per_split = 0, WT = 4, threads = 128, table_words = 0, stage_stride = 0;
     int depth = 0;       // > 0: pipelined kernel with this many stages per warp
     int cm_bulk = 0;     // pipelined kernel: class masks staged by bulk copies
+    int stage_alias = 0; // pipelined kernel: staging area over the start of the rings
+    int hold_warps = 0;
     int ctas_per_sm = 1; // blocks per SM the launch was sized for
     size_t smem = 0;
     int n_groups_ub = 1;
@@ -198,9 +201,11 @@ struct DensePlan {
     bool ok = false;  // false: the dense kernels cannot run this call (generic path instead)
 };
 
-size_t pipe_smem_bytes(int table_words, int n_warps, int depth, int stage_bytes, int stage_stride) {
-    return size_t(table_words) * 4 + kGroupRows * 4 + ((size_t(n_warps) * depth * 12 + 127) & ~size_t(127)) + size_t(n_warps) * depth * stage_bytes +
-           size_t(stage_stride) * kGroupRows * 4;
+// alias: the class-mask staging area shares the space of the rings (it is dead once the table is built)
+size_t pipe_smem_bytes(int table_words, int n_warps, int depth, int stage_bytes, int stage_stride, bool alias = false) {
+    const size_t rings = size_t(n_warps) * depth * stage_bytes, staging = size_t(stage_stride) * kGroupRows * 4;
+    return size_t(table_words) * 4 + kGroupRows * 4 + ((size_t(n_warps) * depth * 12 + 127) & ~size_t(127)) +
+           (alias ? std::max(rings, staging) : rings + staging);
 }
 
 // Launch shape of the register-based dense kernels.
@@ -259,17 +264,24 @@ DensePlan plan_pipe(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, i
     int n_warps = ctx->pipe_warps, depth = ctx->pipe_depth;
     d.cm_bulk = cm_bulk_ok && ps.all_kw_mult4;
     int stride = d.cm_bulk ? ps.maxKW + (ps.maxKW % 8 == 0 ? 4 : 8) : (ps.maxKW | 1);
+    // Where the staging area of the class masks does not fit beside the rings of all warps it is laid over the
+    // first rings (their warps then start copying after the table is built) rather than giving up warps.
+    bool alias = ctx->stage_alias != 0 ||
+                 (pipe_smem_bytes(d.table_words, n_warps, 2, stage_bytes, stride) > cap &&
+                  pipe_smem_bytes(d.table_words, n_warps, 2, stage_bytes, stride, true) <= cap);
     // a staged class-mask fetch is worth giving up warps for (down to 8) when the class table is large
-    while (n_warps > 8 && pipe_smem_bytes(d.table_words, n_warps, 2, stage_bytes, stride) > cap) n_warps -= 4;
-    if (pipe_smem_bytes(d.table_words, n_warps, 2, stage_bytes, stride) > cap) {
+    while (n_warps > 8 && pipe_smem_bytes(d.table_words, n_warps, 2, stage_bytes, stride, alias) > cap) n_warps -= 4;
+    if (pipe_smem_bytes(d.table_words, n_warps, 2, stage_bytes, stride, alias) > cap) {
         n_warps = ctx->pipe_warps;
         stride = 0;
         d.cm_bulk = 0;
+        alias = false;
     }
-    while (depth > 2 && pipe_smem_bytes(d.table_words, n_warps, depth, stage_bytes, stride) > cap) --depth;
-    while (n_warps > 4 && pipe_smem_bytes(d.table_words, n_warps, depth, stage_bytes, stride) > cap) n_warps -= 2;
-    size_t smem = pipe_smem_bytes(d.table_words, n_warps, depth, stage_bytes, stride);
+    while (depth > 2 && pipe_smem_bytes(d.table_words, n_warps, depth, stage_bytes, stride, alias) > cap) --depth;
+    while (n_warps > 4 && pipe_smem_bytes(d.table_words, n_warps, depth, stage_bytes, stride, alias) > cap) n_warps -= 2;
+    size_t smem = pipe_smem_bytes(d.table_words, n_warps, depth, stage_bytes, stride, alias);
     if (smem > cap) return d;
+    if (stride == 0) alias = false;
     d.depth = depth;
     d.stage_stride = stride;
     const int fit = std::max(1, int((cap + 1024) / (smem + 1024)));
@@ -300,7 +312,9 @@ DensePlan plan_pipe(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, i
         per *= 2;
     }
     d.per_split = per;
-    d.smem = pipe_smem_bytes(d.table_words, d.threads / 32, d.depth, stage_bytes, d.stage_stride);
+    d.stage_alias = alias ? 1 : 0;
+    d.hold_warps = alias ? std::min(d.threads / 32, ceil_div(int64_t(d.stage_stride) * kGroupRows * 4, int64_t(d.depth) * stage_bytes)) : 0;
+    d.smem = pipe_smem_bytes(d.table_words, d.threads / 32, d.depth, stage_bytes, d.stage_stride, alias);
     d.ok = true;
     return d;
 }
@@ -336,6 +350,8 @@ void fill_groups(cfgzip_ctx* ctx, StepArgs& a, const DensePlan& d) {
     a.stage_stride = d.stage_stride;
     a.depth = d.depth;
     a.cm_bulk = d.cm_bulk;
+    a.stage_alias = d.stage_alias;
+    a.hold_warps = d.hold_warps;
     a.slots = d.S * d.WT + 1;
     a.p0 = ctx->parts[size_t(a.part0)].dev;
 }
@@ -1009,6 +1025,8 @@ int cfgzip_set_tuning(cfgzip_ctx* ctx, const char* name, int32_t value) {
     } else if (!std::strcmp(name, "waves")) {
         if (value < 1 || value > 16) return CFGZIP_E_ARG;
         ctx->waves = value;
+    } else if (!std::strcmp(name, "stage_alias")) {
+        ctx->stage_alias = value ? 1 : 0;
     } else if (!std::strcmp(name, "pipe_depth")) {
         if (value < 2 || value > 8) return CFGZIP_E_ARG;
         ctx->pipe_depth = value;

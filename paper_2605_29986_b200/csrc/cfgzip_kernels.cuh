@@ -39,6 +39,8 @@ struct StepArgs {
     int32_t stage_stride;       // dense: words per row of the class-mask staging area, 0 = no staging
     int32_t depth;              // pipelined dense kernel: stages per warp
     int32_t cm_bulk;            // pipelined dense kernel: class-mask rows are fetched by bulk copies (16-byte aligned rows)
+    int32_t stage_alias;        // pipelined dense kernel: the class-mask staging area lies over the start of the rings
+    int32_t hold_warps;         // stage_alias: warps whose ring it covers; they start their copies after the table is built
     int32_t run_chunks;         // sampling step: every warp slot of the pipelined kernel takes one contiguous run of this
                                 // many chunks, so that the published states of a row follow the token order
     int32_t tail_state;         // sampling kernel: the last state of a row stands for the octets past the last whole vector
@@ -635,7 +637,10 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
     uint64_t* bars = reinterpret_cast<uint64_t*>(s_row + kGroupRows);  // n_warps * depth
     int* ring_info = reinterpret_cast<int*>(bars + n_warps * a.depth);         // n_warps * depth
     char* ring = reinterpret_cast<char*>(bars) + ((n_warps * a.depth * 12 + 127) & ~127);  // keeps 128-byte alignment
-    uint32_t* stage = reinterpret_cast<uint32_t*>(ring + size_t(n_warps) * a.depth * G::kStageBytes);
+    // The staging area of the class masks is dead once the table is built. Where shared memory is short it
+    // shares the space of the first warps' rings; those warps then start their copies after the table.
+    uint32_t* stage = a.stage_alias ? reinterpret_cast<uint32_t*>(ring)
+                                    : reinterpret_cast<uint32_t*>(ring + size_t(n_warps) * a.depth * G::kStageBytes);
     __shared__ uint64_t cm_bar;
 
     pdl_prologue();
@@ -732,7 +737,7 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
                 bulk_g2s(stage + lane * a.stage_stride, a.class_mask + int64_t(row) * a.cm_stride, uint32_t(P.KW) * 4u, &cm_bar);
         }
     }
-    if (lane == 0)
+    if (lane == 0 && warp >= a.hold_warps)  // hold_warps is 0 unless the staging area lies over the rings
         for (int d = 0; d < depth && !p_end; ++d) issue_next();  // in flight while the table is built
     bool failed = false;
     if (a.cm_bulk) {
@@ -748,6 +753,10 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
     __syncthreads();
     if (__any_sync(0xFFFFFFFFu, failed) && lane == 0) atomicAdd(a.status + 3, 1);  // class masks never arrived
     failed = false;
+    if (lane == 0 && warp < a.hold_warps) {
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the staging area was read and written by plain accesses
+        for (int d = 0; d < depth && !p_end; ++d) issue_next();
+    }
 
     int slot = 0;
     uint32_t phase = 0;
