@@ -76,6 +76,7 @@ struct cfgzip_ctx {
     int32_t tensor_map = 1;   // tiled 2-D copies for row batches that are consecutive rows
     int32_t pipe_warps = 16;
     int32_t pipe_depth = 2;
+    bool pipe_depth_set = false;  // the knob was set: no automatic third stage
     int32_t waves = 1;        // pipelined kernel: blocks launched per resident block slot
     int32_t stage_alias = 0;  // 1: always lay the class-mask staging area over the rings (default: only where it buys warps)
 };
@@ -269,6 +270,17 @@ DensePlan plan_pipe(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, i
     bool alias = ctx->stage_alias != 0 ||
                  (pipe_smem_bytes(d.table_words, n_warps, 2, stage_bytes, stride) > cap &&
                   pipe_smem_bytes(d.table_words, n_warps, 2, stage_bytes, stride, true) <= cap);
+    // Long steps (six or more work items per warp) gain from a third stage where sharing the staging area makes
+    // room for it (measured: B = 256 -4 %, B = 1024 and 2048 -2 %; shorter steps lose to the late start of the
+    // first warps).
+    if (!ctx->pipe_depth_set && depth < 3 && pipe_smem_bytes(d.table_words, n_warps, 3, stage_bytes, stride, true) <= cap) {
+        const int64_t blocks = int64_t(ctx->sm_count) * ctx->waves;
+        const int64_t items = int64_t(ceil_div(B, kGroupRows)) * (((ps.V >> 3) + 31) >> 5) * ceil_div(std::min<int>(B, kGroupRows), kBatchRows);
+        if (items >= 6 * blocks * n_warps) {
+            depth = 3;
+            alias = true;
+        }
+    }
     // a staged class-mask fetch is worth giving up warps for (down to 8) when the class table is large
     while (n_warps > 8 && pipe_smem_bytes(d.table_words, n_warps, 2, stage_bytes, stride, alias) > cap) n_warps -= 4;
     if (pipe_smem_bytes(d.table_words, n_warps, 2, stage_bytes, stride, alias) > cap) {
@@ -1030,6 +1042,7 @@ int cfgzip_set_tuning(cfgzip_ctx* ctx, const char* name, int32_t value) {
     } else if (!std::strcmp(name, "pipe_depth")) {
         if (value < 2 || value > 8) return CFGZIP_E_ARG;
         ctx->pipe_depth = value;
+        ctx->pipe_depth_set = true;
     } else {
         return CFGZIP_E_ARG;
     }
