@@ -179,6 +179,10 @@ int resolve_parts(cfgzip_ctx* ctx, cfgzip_part_id part0, bool mixed, PartSet* ps
     return CFGZIP_OK;
 }
 
+bool aligned32(const void* p, int64_t row_stride_elems, int elem_size) {
+    return (reinterpret_cast<uintptr_t>(p) & 31u) == 0 && ((row_stride_elems * elem_size) & 31) == 0;
+}
+
 bool aligned16(const void* p, int64_t row_stride_elems, int elem_size) {
     return (reinterpret_cast<uintptr_t>(p) & 15u) == 0 && ((row_stride_elems * elem_size) & 15) == 0;
 }
@@ -799,11 +803,11 @@ int cfgzip_mask_logits(cfgzip_ctx* ctx, void* logits, int dtype, int64_t row_str
     if (dtype == CFGZIP_BF16) {
         auto kern = al ? k_mask_logits<kBF16, true> : k_mask_logits<kBF16, false>;
         return launch(ctx, kern, dim3(grid), dim3(256), 0, st, logits, row_stride_elems, int(B), int(V), VW, vocab_mask,
-                      vocab_stride_words);
+                      vocab_stride_words, 0);
     }
     auto kern = al ? k_mask_logits<kF32, true> : k_mask_logits<kF32, false>;
     return launch(ctx, kern, dim3(grid), dim3(256), 0, st, logits, row_stride_elems, int(B), int(V), VW, vocab_mask,
-                  vocab_stride_words);
+                  vocab_stride_words, aligned32(logits, row_stride_elems, 4) ? 1 : 0);
 }
 
 int cfgzip_masked_logsoftmax_argmax(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part,
@@ -849,6 +853,7 @@ int cfgzip_masked_logsoftmax_argmax(cfgzip_ctx* ctx, cfgzip_part_id part0, const
     a.inv_t = 1.f;
     const int es = dtype == CFGZIP_BF16 ? 2 : 4;
     const bool al = aligned16(logits, row_stride_elems, es);
+    a.wide = dtype == CFGZIP_F32 && aligned32(logits, row_stride_elems, 4);
     // measured: early launch of the next kernel helps steps of a few tens of microseconds and costs
     // several percent on long ones
     ctx->pdl_now = int64_t(B) * ps.V * es < (int64_t(48) << 20);
@@ -902,6 +907,7 @@ int cfgzip_masked_sample(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* r
     a.u = u;
     const int es = dtype == CFGZIP_BF16 ? 2 : 4;
     const bool al = aligned16(logits, row_stride_elems, es);
+    a.wide = dtype == CFGZIP_F32 && aligned32(logits, row_stride_elems, 4);
     ctx->pdl_now = int64_t(B) * ps.V * es < (int64_t(48) << 20);
     rc = dtype == CFGZIP_BF16 ? launch_sample<kBF16>(ctx, a, ps, mixed, al, st) : launch_sample<kF32>(ctx, a, ps, mixed, al, st);
     ctx->pdl_now = true;

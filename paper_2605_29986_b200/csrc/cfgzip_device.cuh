@@ -121,6 +121,13 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
 // Streaming 16-byte accesses for the logits (read once, written once).
 __device__ __forceinline__ uint4 ld_stream16(const void* p) { return __ldcs(reinterpret_cast<const uint4*>(p)); }
 __device__ __forceinline__ void st_stream16(void* p, uint4 v) { __stcs(reinterpret_cast<uint4*>(p), v); }
+// One 32-byte store (p 32-byte aligned). Two 16-byte stores per lane would leave every 32-byte sector half
+// written by each of the two instructions of a warp; written whole, a write-only pass runs about twice as fast.
+__device__ __forceinline__ void st_stream32(void* p, uint4 lo, uint4 hi) {
+    asm volatile("st.global.cs.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(lo.x), "r"(lo.y), "r"(lo.z), "r"(lo.w),
+                 "r"(hi.x), "r"(hi.y), "r"(hi.z), "r"(hi.w)
+                 : "memory");
+}
 
 // Logit element access by dtype (scalar, for ragged tails and unaligned buffers).
 template <int DT>
@@ -155,6 +162,8 @@ struct Octet<kBF16> {
         st_stream16(reinterpret_cast<uint16_t*>(row_base) + 8 * int64_t(o), v);
     }
     __device__ __forceinline__ void store_at(void* p) const { st_stream16(p, v); }
+    __device__ __forceinline__ void store(void* row_base, int o, bool) const { store(row_base, o); }
+    __device__ __forceinline__ void store_at(void* p, bool) const { store_at(p); }
     __device__ __forceinline__ void fill_neg_inf() { v = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u); }
     __device__ __forceinline__ void mask(uint32_t byte, float (&f)[8]) {
         const uint32_t xl = nibble_to_byte_msbs(byte & 0xFu), xh = nibble_to_byte_msbs(byte >> 4);
@@ -193,6 +202,13 @@ struct Octet<kF32> {
     __device__ __forceinline__ void store_at(void* p) const {
         st_stream16(p, a);
         st_stream16(reinterpret_cast<char*>(p) + 16, b);
+    }
+    // wide: the octet's address is 32-byte aligned (the caller knows it for the whole buffer)
+    __device__ __forceinline__ void store_at(void* p, bool wide) const {
+        if (wide) st_stream32(p, a, b); else store_at(p);
+    }
+    __device__ __forceinline__ void store(void* row_base, int o, bool wide) const {
+        store_at(reinterpret_cast<float*>(row_base) + 8 * int64_t(o), wide);
     }
     __device__ __forceinline__ void fill_neg_inf() {
         a = make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u);

@@ -39,6 +39,7 @@ struct StepArgs {
     int32_t stage_stride;       // dense: words per row of the class-mask staging area, 0 = no staging
     int32_t depth;              // pipelined dense kernel: stages per warp
     int32_t cm_bulk;            // pipelined dense kernel: class-mask rows are fetched by bulk copies (16-byte aligned rows)
+    int32_t wide;               // every row of the logits starts on a 32-byte boundary: f32 octets go back as one 32-byte store
     int32_t stage_alias;        // pipelined dense kernel: the class-mask staging area lies over the start of the rings
     int32_t hold_warps;         // stage_alias: warps whose ring it covers; they start their copies after the table is built
     int32_t run_chunks;         // sampling step: every warp slot of the pipelined kernel takes one contiguous run of this
@@ -448,10 +449,10 @@ __global__ void __launch_bounds__(256) k_finalize_rows_warp(const __grid_constan
 // row state.
 template <int DT>
 __device__ __forceinline__ void dense_octet_row(Octet<DT>& oc, char* rowp, uint8_t* vmp, int o, uint32_t byte,
-                                                RowAcc& acc) {
+                                                RowAcc& acc, bool wide) {
     float f[8];
     oc.mask(byte, f);
-    oc.store(rowp, o);
+    oc.store(rowp, o, wide);
     if (vmp) vmp[o] = uint8_t(byte);
     acc.add_octet(f, o);
 }
@@ -555,7 +556,7 @@ __global__ void __launch_bounds__(256) k_step_dense(const __grid_constant__ Step
             for (int i = 0; i < kBatchRows; ++i) {
                 if (i < live && active) {
                     const uint32_t byte = ((i < 4 ? lo : hi) >> (8 * (i & 3))) & 0xFFu;
-                    dense_octet_row<DT>(oc[i], rowp[i], vmp[i], o, byte, acc[i]);
+                    dense_octet_row<DT>(oc[i], rowp[i], vmp[i], o, byte, acc[i], a.wide != 0);
                 }
             }
         }
@@ -595,7 +596,8 @@ struct BatchAddr {
 template <int DT, bool FULL, bool CONSEC>
 __device__ __forceinline__ void pipe_consume_item(const char* src, const uint32_t* T, int rb, int live, bool active,
                                                   int o, int lane, const BatchAddr& ba, char* const (&rowp)[kBatchRows],
-                                                  uint8_t* const (&vmp)[kBatchRows], RowAcc (&acc)[kBatchRows], float scale) {
+                                                  uint8_t* const (&vmp)[kBatchRows], RowAcc (&acc)[kBatchRows], float scale,
+                                                  bool wide) {
     using G = PipeGeom<DT>;
     uint4 cv = make_uint4(0, 0, 0, 0);
     if (FULL || active) cv = *reinterpret_cast<const uint4*>(src + kBatchRows * G::kRowBytes + lane * 16);
@@ -610,10 +612,10 @@ __device__ __forceinline__ void pipe_consume_item(const char* src, const uint32_
             float f[8];
             oc.mask(byte, f);
             if (CONSEC) {
-                oc.store_at(ptr_mad(ba.item_base, i, ba.row_bytes));
+                oc.store_at(ptr_mad(ba.item_base, i, ba.row_bytes), wide);
                 if (ba.vm_item) st_global_u8(ptr_mad(reinterpret_cast<char*>(ba.vm_item), i, ba.vm_bytes), byte);
             } else {
-                oc.store(rowp[i], o);
+                oc.store(rowp[i], o, wide);
                 if (vmp[i]) vmp[i][o] = uint8_t(byte);
             }
             acc[i].add_octet(f, o, scale);
@@ -810,9 +812,9 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
         ba.item_base = base0 + size_t(o) * G::kOctetBytes;
         ba.vm_item = vm0 ? vm0 + o : nullptr;
         if (live == kBatchRows && o0 + 32 <= n_full)
-            pipe_consume_item<DT, true, TMAP>(src, T, rb, live, true, o, lane, ba, rowp, vmp, acc, scale);
+            pipe_consume_item<DT, true, TMAP>(src, T, rb, live, true, o, lane, ba, rowp, vmp, acc, scale, a.wide != 0);
         else
-            pipe_consume_item<DT, false, TMAP>(src, T, rb, live, o < n_full, o, lane, ba, rowp, vmp, acc, scale);
+            pipe_consume_item<DT, false, TMAP>(src, T, rb, live, o < n_full, o, lane, ba, rowp, vmp, acc, scale, a.wide != 0);
         ++consumed;
         if (++slot == depth) { slot = 0; phase ^= 1u; }
         __syncwarp();  // every lane has its data out of the slot before it is refilled
@@ -1001,11 +1003,11 @@ __global__ void __launch_bounds__(256) k_step_sparse(const __grid_constant__ Ste
             if (o >= o_vec_end) continue;
             if (byte[u] == 0u) {
                 oc[u].fill_neg_inf();
-                oc[u].store(rowp, o);
+                oc[u].store(rowp, o, a.wide != 0);
             } else {
                 float f[8];
                 oc[u].mask(byte[u], f);
-                if (byte[u] != 0xFFu) oc[u].store(rowp, o);
+                if (byte[u] != 0xFFu) oc[u].store(rowp, o, a.wide != 0);
                 acc.add_octet(f, o);
             }
         }
@@ -1501,7 +1503,7 @@ __global__ void __launch_bounds__(1024) k_plan_rows(const PartDev* parts, int n_
 // ---------------------------------------------------------------------------------------
 template <int DT, bool ALIGNED>
 __global__ void __launch_bounds__(256) k_mask_logits(void* logits, int64_t row_stride, int B, int V, int VW,
-                                                     const uint32_t* vocab_mask, int64_t vm_stride) {
+                                                     const uint32_t* vocab_mask, int64_t vm_stride, int wide) {
     pdl_prologue();
     constexpr int ES = DT == kBF16 ? 2 : 4;
     constexpr int U = 4;
@@ -1533,7 +1535,7 @@ __global__ void __launch_bounds__(256) k_mask_logits(void* logits, int64_t row_s
             float f[8];
             if (ALIGNED && o < n_full) {
                 if (byte[u] == 0u) oc[u].fill_neg_inf(); else oc[u].mask(byte[u], f);
-                oc[u].store(rowp, o);
+                oc[u].store(rowp, o, wide != 0);
             } else {
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
