@@ -896,7 +896,7 @@ __global__ void __launch_bounds__(256) k_expand_dense(const __grid_constant__ St
 // streamed: octets with no allowed token are overwritten with -inf without being read.
 // FUSED = false stops after writing the vocab mask.
 // ---------------------------------------------------------------------------------------
-constexpr int kBigClass = 4096;  // classes at least this large are scattered by the whole block
+constexpr int kBigClass = 256;   // classes at least this large are scattered by the whole block
 constexpr int kBigListCap = 64;
 
 __device__ __forceinline__ int lower_bound_tok(const int32_t* tok, int lo, int hi, int t) {
@@ -952,9 +952,13 @@ __global__ void __launch_bounds__(256) k_step_sparse(const __grid_constant__ Ste
                     continue;
                 }
             }
-            for (int i = lo + lane; i < hi; i += 32) {
-                const int t = __ldg(P.tok + i);
-                atomicOr(bits + ((t >> 5) - w_begin), 1u << (t & 31));
+            for (int i = lo + lane; i < hi; i += 4 * 32) {  // four member ids in flight per lane
+                int t[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) t[q] = i + 32 * q < hi ? __ldg(P.tok + i + 32 * q) : -1;
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    if (t[q] >= 0) atomicOr(bits + ((t[q] >> 5) - w_begin), 1u << (t[q] & 31));
             }
         }
     }
@@ -967,9 +971,13 @@ __global__ void __launch_bounds__(256) k_step_sparse(const __grid_constant__ Ste
             lo = lower_bound_tok(P.tok, lo, hi, t0);
             hi = lower_bound_tok(P.tok, lo, hi, t1);
         }
-        for (int i = lo + tid; i < hi; i += blockDim.x) {
-            const int t = __ldg(P.tok + i);
-            atomicOr(bits + ((t >> 5) - w_begin), 1u << (t & 31));
+        for (int i = lo + tid; i < hi; i += 4 * blockDim.x) {
+            int t[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) t[q] = i + int(blockDim.x) * q < hi ? __ldg(P.tok + i + blockDim.x * q) : -1;
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                if (t[q] >= 0) atomicOr(bits + ((t[q] >> 5) - w_begin), 1u << (t[q] & 31));
         }
     }
     __syncthreads();
