@@ -44,7 +44,7 @@ RING_MAX_BYTES = 24 << 30
 # DRAM traffic of the dominant (streaming) kernel per launch = per step (dram__bytes_read.sum +
 # dram__bytes_write.sum from one ncu capture), keyed by workload; valid only for the kernel sources whose digest is
 # recorded with it. None until a capture of the current sources exists.
-NCU_TRAFFIC = {"cfg2_B32_dense": {"digest": "398ff78bcda58931", "bytes_per_launch": 8538965}}
+NCU_TRAFFIC = {"cfg2_B32_dense": {"digest": "c459a6edd57fc699", "bytes_per_launch": 8539051}}
 
 
 def _kernel_digest() -> str:
@@ -324,6 +324,12 @@ class StepRunner:
         return int(self.B * (self.V * self.elem + 4 * self.VW + 4 * self.KW + 16) + allowed_tokens * (4 + self.elem))
 
 
+def _extra_steps(runner: StepRunner, passes: int = 3, min_steps: int = 300) -> int:
+    """Steps of a secondary measurement: whole passes over the ring, at least `min_steps` steps, so that the timed
+    region lasts tens of milliseconds (a few milliseconds right after host-side set-up measured up to 10 % slow)."""
+    return runner.R * max(passes, -(-min_steps // runner.R))
+
+
 def _e2e(runner: StepRunner, torch, n_steps: int):
     """Rows/s through cfgzip_decode_step_host: pinned host inputs in, results out, every step."""
     cz = runner.cz
@@ -473,7 +479,7 @@ def run_own(args):
         for B in (128, 256, 1024):
             r2 = StepRunner(cz, torch, local_rank, args.workload, B=B, mode=args.mode, steps_hint=8, unique=2,
                             tune=args.tune)
-            n = 3 * r2.R
+            n = _extra_steps(r2)
             s2, l2 = r2.timed(n, r2.R)
             a2 = r2.alg_bytes() / (s2 / n) / 1e9
             extras.append({"B": B, "us_per_step": s2 / n * 1e6, "rows_per_s": B * n / s2, "achieved_gbs": a2,
@@ -484,7 +490,7 @@ def run_own(args):
         # the vocab mask is written and read back, so it moves more bytes for less work
         r3 = StepRunner(cz, torch, local_rank, args.workload, B=args.batch, mode=args.mode, steps_hint=256, unique=2,
                         tune=args.tune, unfused=True)
-        n = 2 * r3.R
+        n = _extra_steps(r3, 2)
         s3, l3 = r3.timed(n, r3.R)
         line["unfused_expand_then_mask"] = {"us_per_step": s3 / n * 1e6, "launches_per_step": l3 / n}
         r3.close()
@@ -493,7 +499,7 @@ def run_own(args):
         for B in (args.batch or synth.CONFIGS[args.workload]["B"], 1024):
             r6 = StepRunner(cz, torch, local_rank, args.workload, B=B, mode=args.mode, steps_hint=64, unique=2,
                             tune=args.tune, inv_temperature=5.0)
-            n = 3 * r6.R
+            n = _extra_steps(r6)
             s6, l6 = r6.timed(n, r6.R)
             samp.append({"B": B, "us_per_step": s6 / n * 1e6, "launches_per_step": l6 / n,
                          "frac_of_measured": r6.alg_bytes() / (s6 / n) / 1e9 / peak})
@@ -509,7 +515,7 @@ def run_own(args):
         five = []
         for cfg in sorted(synth.CONFIGS):
             r7 = StepRunner(cz, torch, local_rank, cfg, mode="dense", steps_hint=64, unique=2, tune=args.tune)
-            n = 3 * r7.R
+            n = _extra_steps(r7)
             s7, l7 = r7.timed(n, r7.R)
             a7 = r7.alg_bytes() / (s7 / n) / 1e9
             five.append({"workload": "cfg%d %s: V=%d K=%d B=%d %s, %d partition(s)" % (
@@ -522,7 +528,7 @@ def run_own(args):
         pair = {}
         for mode in ("dense", "sparse"):
             r4 = StepRunner(cz, torch, local_rank, 5, mode=mode, steps_hint=4, unique=1, tune=args.tune)
-            n = 4 * r4.R
+            n = _extra_steps(r4, 4)
             s4, _ = r4.timed(n, r4.R)
             pair[mode + "_us_per_step"] = s4 / n * 1e6
             pair[mode + "_algorithmic_bytes"] = r4.alg_bytes()
