@@ -189,6 +189,11 @@ class StepRunner:
         self.row_part_host = None if self.w.row_part is None else \
             (np.arange(self.B) % len(self.parts)).astype(np.int32)
         self.row_part = None if self.row_part_host is None else torch.from_numpy(self.row_part_host).cuda()
+        self.row_part_arg = self.row_part
+        if self.row_part is not None:
+            # the rows keep their grammars over the steps: group them by partition once, outside the steps
+            cz.cfgzip_plan_rows(self.ctx, self.parts[0], self.row_part, self.B)
+            self.row_part_arg = cz.ROWS_AS_PLANNED
         self.work = torch.empty((self.R, self.B, self.V), dtype=tdt, device="cuda")
         self.vm = torch.empty((self.R, self.B, self.VW), dtype=torch.int32, device="cuda")
         self.am = torch.empty((self.R, self.B), dtype=torch.int32, device="cuda")
@@ -226,12 +231,12 @@ class StepRunner:
             return
         if self.u is not None:
             cz.cfgzip_masked_sample(
-                self.ctx, self.parts[0], self.row_part, self.cm[j], self.KW, self.work[j],
+                self.ctx, self.parts[0], self.row_part_arg, self.cm[j], self.KW, self.work[j],
                 cz.BF16 if self.dtype == "bf16" else cz.F32, self.V, self.B, self.vm[j], self.VW, self.u[j],
                 self.inv_temperature, self.am[j], self.rep[j], self.lpa[j], self.lse[j], self.mode, stream)
             return
         cz.cfgzip_masked_logsoftmax_argmax(
-            self.ctx, self.parts[0], self.row_part, self.cm[j], self.KW, self.work[j],
+            self.ctx, self.parts[0], self.row_part_arg, self.cm[j], self.KW, self.work[j],
             cz.BF16 if self.dtype == "bf16" else cz.F32, self.V, self.B, self.vm[j], self.VW, self.am[j], self.rep[j],
             self.lpa[j], self.lse[j], None, self.mode, stream)
 
@@ -451,6 +456,8 @@ def run_own(args):
                       "%.0f kernels per step (streaming pass + per-row finalize)" % (
                 min(runner.R, args.steps), launches / max(args.steps, 1)),
             "parallelism": "rows sharded over %d GPU(s), no collective on the path" % world,
+            "row_grouping": ("rows grouped by partition once before the steps (cfgzip_plan_rows), reused by every step"
+                             if runner.row_part is not None else "one partition: rows grouped implicitly"),
         },
         "us_per_step": seconds / args.steps * 1e6,
         "us_per_step_over_ring_passes": (

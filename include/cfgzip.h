@@ -102,6 +102,21 @@ int cfgzip_free_partition(cfgzip_ctx* ctx, cfgzip_part_id id);
  */
 
 /*
+ * Batches whose rows keep their partitions over many decode steps (one grammar per request: Section 4 runs
+ * one CFG per schema on the JSON task) need not be regrouped at every step. cfgzip_plan_rows groups the rows
+ * of `row_part` (dev int32 [B]) by partition once, on `stream`; afterwards a per-step call on the same context
+ * may pass CFGZIP_ROWS_AS_PLANNED in place of row_part (with the same B, and a part0 of the same V) and skips its
+ * grouping launch. The caller keeps `row_part` alive and unchanged meanwhile. The kept grouping does not survive
+ * a per-step call that passes an explicit row_part (assume it gone after any such call), another
+ * cfgzip_plan_rows, cfgzip_reserve_rows, or loading or freeing a partition; CFGZIP_ROWS_AS_PLANNED without a
+ * valid kept grouping gives CFGZIP_E_ARG. B above the reserved
+ * rows gives CFGZIP_E_NOMEM (see cfgzip_reserve_rows).
+ */
+#define CFGZIP_ROWS_AS_PLANNED ((const int32_t*)(uintptr_t)1)
+int cfgzip_plan_rows(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part /*dev [B]*/, int32_t B,
+                     void* stream);
+
+/*
  * Expand class masks to vocab masks: vocab bit (b, i) = class bit (b, c[i])
  * (Section 3.1, "Inference": the mask entry applied to token i is m_{c_i}; Figure 1b).
  *   class_mask : dev uint32 [B, class_stride_words], class_stride_words >= KW

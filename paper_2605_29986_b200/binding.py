@@ -33,6 +33,7 @@ _SIGNATURES = {
                                                _vp, _vp, _vp, _int, _vp]),
     "cfgzip_masked_sample": (_int, [_vp, _i32, _vp, _vp, _i64, _vp, _int, _i64, _i32, _vp, _i64, _vp, ctypes.c_float, _vp,
                                     _vp, _vp, _vp, _int, _vp]),
+    "cfgzip_plan_rows": (_int, [_vp, _i32, _vp, _i32, _vp]),
     "cfgzip_map_tokens": (_int, [_vp, _i32, _vp, _vp, _vp, _i32, _vp]),
     "cfgzip_decode_step_host": (_int, [_vp, _i32, _vp, _vp, _i64, _vp, _int, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _int,
                                        _vp]),
@@ -165,6 +166,13 @@ def cfgzip_masked_sample(ctx: int, part0: int, row_part, class_mask, class_strid
         ctx, part0, _ptr(row_part), _ptr(class_mask), class_stride_words, _ptr(logits), dtype, row_stride_elems, B,
         _ptr(vocab_mask), vocab_stride_words, _ptr(u), inv_temperature, _ptr(token), _ptr(rep), _ptr(logp_token),
         _ptr(lse), mode, _stream(stream)), "cfgzip_masked_sample")
+
+
+ROWS_AS_PLANNED = 1  # pass as row_part after cfgzip_plan_rows: the kept grouping of that call is reused
+
+
+def cfgzip_plan_rows(ctx: int, part0: int, row_part, B: int, stream=None) -> None:
+    _check(load_library().cfgzip_plan_rows(ctx, part0, _ptr(row_part), B, _stream(stream)), "cfgzip_plan_rows")
 
 
 def cfgzip_map_tokens(ctx: int, part0: int, row_part, tokens, reps, B: int, stream=None) -> None:

@@ -62,6 +62,11 @@ struct cfgzip_ctx {
     int32_t* st_small = nullptr;  // row_part, argmax, rep, lse, logp_argmax: 5 arrays of st_rows
     int32_t st_rows = 0;
     int64_t launches = 0;
+    // row plan kept by cfgzip_plan_rows (valid until anything overwrites the plan buffers or the partitions change)
+    bool plan_valid = false;
+    bool plan_in_use = false;  // set for the duration of a call that passed CFGZIP_ROWS_AS_PLANNED
+    const int32_t* plan_row_part = nullptr;
+    int32_t plan_B = 0, plan_V = 0;
     // tuning
     int32_t ctas_per_sm = 4;
     int32_t token_warps = 0;
@@ -335,6 +340,26 @@ DensePlan plan_pipe(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, i
     return d;
 }
 
+// A call may pass CFGZIP_ROWS_AS_PLANNED for its row -> partition vector: it then means the vector given to the
+// last cfgzip_plan_rows, whose grouping is still in the plan buffers.
+int resolve_row_part(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t** row_part, int32_t B, bool* planned) {
+    *planned = false;
+    if (*row_part != CFGZIP_ROWS_AS_PLANNED) return CFGZIP_OK;
+    if (!ctx) return CFGZIP_E_ARG;
+    if (!ctx->plan_valid || ctx->plan_B != B || part0 < 0 || size_t(part0) >= ctx->parts.size() ||
+        !ctx->parts[size_t(part0)].live || ctx->parts[size_t(part0)].V != ctx->plan_V)
+        return CFGZIP_E_ARG;
+    *row_part = ctx->plan_row_part;
+    *planned = true;
+    return CFGZIP_OK;
+}
+
+struct PlanUse {  // marks the kept plan as in use for the lifetime of a call
+    cfgzip_ctx* ctx;
+    PlanUse(cfgzip_ctx* c, bool planned) : ctx(c) { if (ctx) ctx->plan_in_use = planned; }
+    ~PlanUse() { if (ctx) ctx->plan_in_use = false; }
+};
+
 int check_step_args(cfgzip_ctx* ctx, const uint32_t* class_mask, int64_t cm_stride, int32_t B, int mode) {
     if (!ctx || B < 0) return CFGZIP_E_ARG;
     if (mode != CFGZIP_AUTO && mode != CFGZIP_DENSE && mode != CFGZIP_SPARSE) return CFGZIP_E_ARG;
@@ -344,6 +369,8 @@ int check_step_args(cfgzip_ctx* ctx, const uint32_t* class_mask, int64_t cm_stri
 
 int run_plan_kernel(cfgzip_ctx* ctx, const int32_t* row_part, int32_t B, int32_t V, const DensePlan& d,
                     cudaStream_t st) {
+    if (ctx->plan_in_use) return CFGZIP_OK;  // the call runs on the grouping cfgzip_plan_rows left in the buffers
+    ctx->plan_valid = false;                 // this launch overwrites them
     return launch(ctx, k_plan_rows, dim3(1), dim3(1024), 0, st, (const PartDev*)ctx->d_parts, int(ctx->parts.size()),
                   row_part, int(B), int(V), d.n_groups_ub, ctx->d_group_part, ctx->d_group_rows, ctx->d_n_groups,
                   ctx->d_status);
@@ -479,9 +506,8 @@ int launch_fused(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, in
     }
     if (rc != CFGZIP_OK) return rc;
     if (logp_full) {
-        const int64_t total = int64_t(a.B) * a.V;
-        const unsigned grid = unsigned(std::min<int64_t>((total + 255) / 256, int64_t(ctx->sm_count) * 16));
-        rc = launch(ctx, k_logp_full<DT>, dim3(grid), dim3(256), 0, st, (const void*)a.logits, a.row_stride, int(a.B),
+        const dim3 grid(unsigned(std::min(ceil_div(a.V, 256 * 4), 64)), unsigned(std::min<int32_t>(a.B, 65535)));
+        rc = launch(ctx, k_logp_full<DT>, grid, dim3(256), 0, st, (const void*)a.logits, a.row_stride, int(a.B),
                     int(a.V), (const float*)a.lse, logp_full);
     }
     return rc;
@@ -569,6 +595,7 @@ int cfgzip_reserve_rows(cfgzip_ctx* ctx, int32_t max_rows) {
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return CFGZIP_E_CUDA;
     cudaDeviceSynchronize();
+    ctx->plan_valid = false;
     cudaFree(ctx->d_tickets);
     cudaFree(ctx->d_group_part);
     cudaFree(ctx->d_group_rows);
@@ -718,6 +745,7 @@ int cfgzip_load_partition(cfgzip_ctx* ctx, const int32_t* c, int32_t V, const in
         return CFGZIP_E_CUDA;
     }
     ctx->parts[slot] = p;
+    ctx->plan_valid = false;
     *out_id = cfgzip_part_id(slot);
     return CFGZIP_OK;
 }
@@ -728,6 +756,7 @@ int cfgzip_free_partition(cfgzip_ctx* ctx, cfgzip_part_id id) {
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return CFGZIP_E_CUDA;
     cudaDeviceSynchronize();
+    ctx->plan_valid = false;
     Part& p = ctx->parts[size_t(id)];
     cudaFree(p.block);
     p = Part();
@@ -741,6 +770,9 @@ int cfgzip_expand_mask(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row
                        int mode, void* stream) {
     int rc = check_step_args(ctx, class_mask, class_stride_words, B, mode);
     if (rc != CFGZIP_OK) return rc;
+    bool planned;
+    if ((rc = resolve_row_part(ctx, part0, &row_part, B, &planned)) != CFGZIP_OK) return rc;
+    PlanUse plan_use(ctx, planned);
     PartSet ps;
     const bool mixed = row_part != nullptr;
     if ((rc = resolve_parts(ctx, part0, mixed, &ps)) != CFGZIP_OK) return rc;
@@ -818,6 +850,9 @@ int cfgzip_masked_logsoftmax_argmax(cfgzip_ctx* ctx, cfgzip_part_id part0, const
     int rc = check_step_args(ctx, class_mask, class_stride_words, B, mode);
     if (rc != CFGZIP_OK) return rc;
     if (dtype != CFGZIP_F32 && dtype != CFGZIP_BF16) return CFGZIP_E_ARG;
+    bool planned;
+    if ((rc = resolve_row_part(ctx, part0, &row_part, B, &planned)) != CFGZIP_OK) return rc;
+    PlanUse plan_use(ctx, planned);
     PartSet ps;
     const bool mixed = row_part != nullptr;
     if ((rc = resolve_parts(ctx, part0, mixed, &ps)) != CFGZIP_OK) return rc;
@@ -872,6 +907,9 @@ int cfgzip_masked_sample(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* r
     if (dtype != CFGZIP_F32 && dtype != CFGZIP_BF16) return CFGZIP_E_ARG;
     if (mode == CFGZIP_SPARSE) return CFGZIP_E_ARG;  // the class-list kernel does not leave its states in token order
     if (!(inv_temperature > 0.f) || !(inv_temperature <= 1e6f)) return CFGZIP_E_ARG;
+    bool planned;
+    if ((rc = resolve_row_part(ctx, part0, &row_part, B, &planned)) != CFGZIP_OK) return rc;
+    PlanUse plan_use(ctx, planned);
     PartSet ps;
     const bool mixed = row_part != nullptr;
     if ((rc = resolve_parts(ctx, part0, mixed, &ps)) != CFGZIP_OK) return rc;
@@ -914,11 +952,34 @@ int cfgzip_masked_sample(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* r
     return rc;
 }
 
+int cfgzip_plan_rows(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part, int32_t B, void* stream) {
+    if (!ctx || !row_part || row_part == CFGZIP_ROWS_AS_PLANNED || B <= 0) return CFGZIP_E_ARG;
+    PartSet ps;
+    int rc = resolve_parts(ctx, part0, true, &ps);
+    if (rc != CFGZIP_OK) return rc;
+    if (B > ctx->reserved_rows) return CFGZIP_E_NOMEM;
+    DensePlan d;
+    d.n_groups_ub = ceil_div(B, kGroupRows) + ps.n_live_same_v;
+    if (d.n_groups_ub > ctx->max_groups) return CFGZIP_E_NOMEM;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return CFGZIP_E_CUDA;
+    ctx->plan_in_use = false;
+    if ((rc = run_plan_kernel(ctx, row_part, B, ps.V, d, static_cast<cudaStream_t>(stream))) != CFGZIP_OK) return rc;
+    ctx->plan_valid = true;
+    ctx->plan_row_part = row_part;
+    ctx->plan_B = B;
+    ctx->plan_V = ps.V;
+    return CFGZIP_OK;
+}
+
 int cfgzip_map_tokens(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part, const int32_t* tokens,
                       int32_t* reps, int32_t B, void* stream) {
     if (!ctx || B < 0) return CFGZIP_E_ARG;
+    bool planned;
+    int rc = resolve_row_part(ctx, part0, &row_part, B, &planned);
+    if (rc != CFGZIP_OK) return rc;
     PartSet ps;
-    int rc = resolve_parts(ctx, part0, row_part != nullptr, &ps);
+    rc = resolve_parts(ctx, part0, row_part != nullptr, &ps);
     if (rc != CFGZIP_OK) return rc;
     if (B == 0) return CFGZIP_OK;
     if (!tokens || !reps) return CFGZIP_E_ARG;

@@ -1558,12 +1558,13 @@ template <int DT>
 __global__ void __launch_bounds__(256) k_logp_full(const void* logits, int64_t row_stride, int B, int V, const float* lse,
                                                    float* out) {
     pdl_prologue();
-    const int64_t total = int64_t(B) * V;
-    for (int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += int64_t(gridDim.x) * blockDim.x) {
-        const int row = int(i / V), t = int(i - int64_t(row) * V);
+    // grid: x strides over the tokens of a row, y over the rows
+    for (int row = blockIdx.y; row < B; row += gridDim.y) {
         const float l = lse[row];
-        const float z = load_elem<DT>(logits, int64_t(row) * row_stride + t);
-        out[i] = (l == -INFINITY || z == -INFINITY) ? -INFINITY : z - l;
+        for (int t = blockIdx.x * blockDim.x + threadIdx.x; t < V; t += gridDim.x * blockDim.x) {
+            const float z = load_elem<DT>(logits, int64_t(row) * row_stride + t);
+            out[int64_t(row) * V + t] = (l == -INFINITY || z == -INFINITY) ? -INFINITY : z - l;
+        }
     }
 }
 

@@ -422,3 +422,45 @@ def test_steps_replayed_from_a_cuda_graph_match_the_oracle():
                 part = w.partitions[0]
                 tok = outs[0].cpu().numpy()
                 assert np.array_equal(outs[1].cpu().numpy(), part.r[part.c[tok]])
+
+
+# ------------------------------------------------------------------ kept row grouping
+
+def test_kept_row_grouping_gives_the_same_steps_and_is_dropped_when_it_must():
+    w = synth.make_workload(4, B=70, V=30000, K=700)
+    VW = (w.V + 31) // 32
+    lib = cz.load_library()
+    with Ctx(w.partitions) as ctx:
+        d_rp = dev(w.row_part)
+        d_tok = torch.zeros(w.B, dtype=torch.int32, device="cuda")
+        # nothing planned yet: the sentinel is an argument error
+        assert lib.cfgzip_map_tokens(ctx.h, ctx.ids[0], cz.ROWS_AS_PLANNED, d_tok.data_ptr(), d_tok.data_ptr(), w.B, None) == cz.E_ARG
+        cz.cfgzip_plan_rows(ctx.h, ctx.ids[0], d_rp, w.B)
+        for step in range(3):
+            cm, z = w.class_masks(step), w.logits(step)
+            want = oracle_step(w.partitions, w.row_part, cm, z, w.V)
+            d_z, d_cm = dev(z), dev(cm)
+            d_vm = torch.zeros((w.B, VW), dtype=torch.int32, device="cuda")
+            d_am = torch.zeros(w.B, dtype=torch.int32, device="cuda")
+            d_rep = torch.zeros_like(d_am)
+            d_lse = torch.zeros(w.B, dtype=torch.float32, device="cuda")
+            d_lpa = torch.zeros_like(d_lse)
+            before = cz.cfgzip_launch_count(ctx.h)
+            cz.cfgzip_masked_logsoftmax_argmax(ctx.h, ctx.ids[0], cz.ROWS_AS_PLANNED, d_cm, cm.shape[1], d_z, cz.BF16, w.V, w.B,
+                                               d_vm, VW, d_am, d_rep, d_lpa, d_lse, None, cz.DENSE)
+            assert cz.cfgzip_launch_count(ctx.h) - before == 2  # no grouping launch
+            torch.cuda.synchronize()
+            got = dict(logits=host(d_z, z.dtype), vocab_mask=host(d_vm, np.uint32), argmax=d_am.cpu().numpy(),
+                       rep=d_rep.cpu().numpy(), lse=d_lse.cpu().numpy(), logp_argmax=d_lpa.cpu().numpy())
+            compare_step(got, want, w.V, "kept grouping, step %d" % step)
+            d_map = torch.zeros_like(d_am)
+            cz.cfgzip_map_tokens(ctx.h, ctx.ids[0], cz.ROWS_AS_PLANNED, d_am, d_map, w.B)
+            torch.cuda.synchronize()
+            assert np.array_equal(d_map.cpu().numpy(), want["rep"])
+        # another batch size, or a call that regroups with an explicit vector, ends the kept grouping
+        assert lib.cfgzip_map_tokens(ctx.h, ctx.ids[0], cz.ROWS_AS_PLANNED, d_tok.data_ptr(), d_tok.data_ptr(), w.B - 1, None) == cz.E_ARG
+        got = run_fused(ctx, w.row_part, w.class_masks(5), w.logits(5), w.V)
+        compare_step(got, oracle_step(w.partitions, w.row_part, w.class_masks(5), w.logits(5), w.V), w.V, "explicit")
+        assert lib.cfgzip_map_tokens(ctx.h, ctx.ids[0], cz.ROWS_AS_PLANNED, d_tok.data_ptr(), d_tok.data_ptr(), w.B, None) == cz.E_ARG
+        assert lib.cfgzip_plan_rows(ctx.h, ctx.ids[0], None, w.B, None) == cz.E_ARG
+        assert cz.cfgzip_poll_status(ctx.h) == (0, 0, 0)
