@@ -73,3 +73,49 @@ def test_full_size_workload(config):
         sub = {k: (v[rows] if v is not None else None) for k, v in got.items()}
         want = oracle_step(w.partitions, None if row_part is None else row_part[rows], cm[rows], z[rows], V)
         compare_step(sub, want, V, "config %d step %d" % (config, step))
+
+
+@pytest.mark.parametrize("B", [256, 1024])
+def test_llama_size_large_batches_three_stage_launch(B):
+    # from 256 rows on the bf16 step runs three stages per warp with the class-mask staging area laid over the
+    # first rings: the launch shape the bench's larger batches use
+    plan = cz.cfgzip_plan_query(148, 232448, 128256, 2048, B, cz.BF16)
+    assert plan["kind"] == 2 and plan["depth"] == 3
+    wu = synth.make_workload(2, B=64)
+    wf = synth.make_workload(2, B=B)
+    z = np.tile(wu.logits(3), (B // 64, 1))
+    cm = wf.class_masks(3)
+    with Ctx(wf.partitions) as ctx:
+        got = run_fused(ctx, None, cm, z, wf.V, mode=cz.DENSE)
+        assert cz.cfgzip_poll_status(ctx.h) == (0, 0, 0)
+    _properties(wf, None, cm, got, wf.V)
+    rows = np.unique(np.linspace(0, B - 1, 96).astype(np.int64))
+    sub = {k: (v[rows] if v is not None else None) for k, v in got.items()}
+    compare_step(sub, oracle_step(wf.partitions, None, cm[rows], z[rows], wf.V), wf.V, "B=%d" % B)
+
+
+def test_heavy_tail_workload_with_kept_row_grouping():
+    # the bench groups the rows of the mixed batch once (cfgzip_plan_rows) and reuses the grouping at every step
+    w, row_part, cm, z = _inputs(4, 2)
+    V, B = w.V, cm.shape[0]
+    VW = (V + 31) // 32
+    from _gpu_util import dev, host
+    with Ctx(w.partitions) as ctx:
+        d_rp = dev(row_part)
+        cz.cfgzip_plan_rows(ctx.h, ctx.ids[0], d_rp, B)
+        d_z, d_cm = dev(z), dev(cm)
+        d_vm = torch.zeros((B, VW), dtype=torch.int32, device="cuda")
+        d_am = torch.zeros(B, dtype=torch.int32, device="cuda")
+        d_rep = torch.zeros_like(d_am)
+        d_lse = torch.zeros(B, dtype=torch.float32, device="cuda")
+        d_lpa = torch.zeros_like(d_lse)
+        cz.cfgzip_masked_logsoftmax_argmax(ctx.h, ctx.ids[0], cz.ROWS_AS_PLANNED, d_cm, cm.shape[1], d_z, cz.BF16, V, B, d_vm,
+                                           VW, d_am, d_rep, d_lpa, d_lse, None, cz.DENSE)
+        torch.cuda.synchronize()
+        assert cz.cfgzip_poll_status(ctx.h) == (0, 0, 0)
+        got = dict(logits=host(d_z, z.dtype), vocab_mask=host(d_vm, np.uint32), argmax=d_am.cpu().numpy(),
+                   rep=d_rep.cpu().numpy(), lse=d_lse.cpu().numpy(), logp_argmax=d_lpa.cpu().numpy(), logp_full=None)
+    _properties(w, row_part, cm, got, V)
+    rows = np.unique(np.linspace(0, B - 1, 48).astype(np.int64))
+    sub = {k: (v[rows] if v is not None else None) for k, v in got.items()}
+    compare_step(sub, oracle_step(w.partitions, row_part[rows], cm[rows], z[rows], V), V, "kept grouping")
