@@ -276,7 +276,12 @@ int cfgzip_launch_count(cfgzip_ctx* ctx, int64_t* out);
  *                  tensor map (default), 0 = one bulk copy per row
  *   "pipe_warps"   warps per thread block of the pipelined kernel (1..16)
  *   "waves"        thread blocks launched per resident block slot of the pipelined kernel (1..16)
- *   "pipe_depth"   stages per warp of the pipelined kernel (2..8; lowered to fit shared memory)
+ *   "pipe_depth"   stages per warp of the pipelined kernel (2..8; lowered to fit shared memory); unset, long
+ *                  steps take a third stage where it fits
+ *   "stage_alias"  1 = always lay the class-mask staging area over the first warps' rings (default 0: only where
+ *                  that keeps warps or buys the third stage)
+ *   "spread"       1 = launches sized for one block per SM ask for more than half of an SM's shared memory, so
+ *                  that the blocks of a small batch cannot share an SM (default), 0 = only what the block needs
  * Unknown names give CFGZIP_E_ARG.
  */
 int cfgzip_set_tuning(cfgzip_ctx* ctx, const char* name, int32_t value);
