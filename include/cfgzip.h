@@ -280,8 +280,9 @@ int cfgzip_launch_count(cfgzip_ctx* ctx, int64_t* out);
  *                  steps take a third stage where it fits
  *   "stage_alias"  1 = always lay the class-mask staging area over the first warps' rings (default 0: only where
  *                  that keeps warps or buys the third stage)
- *   "spread"       1 = launches sized for one block per SM ask for more than half of an SM's shared memory, so
- *                  that the blocks of a small batch cannot share an SM (default), 0 = only what the block needs
+ *   "spread"       1 = launches of at most one block per SM (the streaming kernel of a small batch, the per-row
+ *                  kernels of 32 to 148 rows) ask for more than half of an SM's shared memory, so that two of
+ *                  their blocks never share an SM (default), 0 = only what the block needs
  * Unknown names give CFGZIP_E_ARG.
  */
 int cfgzip_set_tuning(cfgzip_ctx* ctx, const char* name, int32_t value);
