@@ -403,8 +403,19 @@ __global__ void __launch_bounds__(kFinalizeThreads) k_finalize_rows(const __grid
     if (lane == 0) s_red[warp] = Partial{m0, s0, p0, 0};
     __syncthreads();
     if (warp != 0) return;
+    // the eight warp states: one per lane, three butterfly steps, the result handed to every lane
+    const Partial mine = lane < kFinalizeThreads / 32 ? s_red[lane] : partial_empty();
+    m0 = mine.m; s0 = mine.s; p0 = mine.pos;
 #pragma unroll
-    for (int w = 1; w < kFinalizeThreads / 32; ++w) partial_merge(m0, s0, p0, s_red[w].m, s_red[w].s, s_red[w].pos);
+    for (int d = kFinalizeThreads / 64; d >= 1; d >>= 1) {
+        const float m2 = __shfl_xor_sync(0xFFFFFFFFu, m0, d);
+        const float s2 = __shfl_xor_sync(0xFFFFFFFFu, s0, d);
+        const int p2 = __shfl_xor_sync(0xFFFFFFFFu, p0, d);
+        partial_merge(m0, s0, p0, m2, s2, p2);
+    }
+    m0 = __shfl_sync(0xFFFFFFFFu, m0, 0);
+    s0 = __shfl_sync(0xFFFFFFFFu, s0, 0);
+    p0 = __shfl_sync(0xFFFFFFFFu, p0, 0);
     warp_finalize_row<DT>(a, P, row, m0, s0, p0, lane);
 }
 
@@ -650,6 +661,20 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = blockIdx.x / a.S, split = blockIdx.x - g * a.S;
     if (a.n_groups && g >= __ldg(a.n_groups)) return;
+    // Without a row plan the rows of the group are g*32 .. g*32+31 and its partition is part0: the class masks,
+    // whose arrival everything else waits for, are asked for before anything else is set up.
+    const bool early_cm = a.cm_bulk && !a.group_rows;
+    if (early_cm && warp == 0) {
+        if (lane == 0) {
+            mbar_init(&cm_bar, 1);
+            mbar_init_fence();
+            mbar_expect_tx(&cm_bar, uint32_t(min(kGroupRows, a.B - g * kGroupRows)) * uint32_t(a.p0.KW) * 4u);
+        }
+        __syncwarp();
+        const int row = g * kGroupRows + lane;
+        if (row < a.B)
+            bulk_g2s(stage + lane * a.stage_stride, a.class_mask + int64_t(row) * a.cm_stride, uint32_t(a.p0.KW) * 4u, &cm_bar);
+    }
     const int part = group_rows_setup(a, g, s_row, tid);
     __syncthreads();
     const PartDev P = a.group_part ? a.parts[part] : a.p0;
@@ -725,10 +750,10 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
 
     if (lane == 0) {
         for (int d = 0; d < depth; ++d) mbar_init(bar + d, 1);
-        if (warp == 0) mbar_init(&cm_bar, 1);
+        if (warp == 0 && !early_cm) mbar_init(&cm_bar, 1);
         mbar_init_fence();
     }
-    if (a.cm_bulk) {
+    if (a.cm_bulk && !early_cm) {
         __syncthreads();  // the class-mask barrier is initialised for everybody
         if (warp == 0) {
             // one bulk copy per row of the group, issued side by side by the lanes of one warp
