@@ -54,6 +54,11 @@ struct StepArgs {
     int32_t* status;            // [0] empty rows, [1] bad tokens, [2] bad rows, [3] copies that never arrived
 };
 
+// The two halves separately, for a kernel that sets itself up (nothing read from memory) while the kernel in
+// front of it is still running and only then waits for it.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ void pdl_prologue() {
     // Let the next kernel of the stream start its launch early, then wait until everything
     // launched before this kernel has completed. Both are no-ops without the launch attribute.
@@ -656,24 +661,22 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
                                     : reinterpret_cast<uint32_t*>(ring + size_t(n_warps) * a.depth * G::kStageBytes);
     __shared__ uint64_t cm_bar;
 
-    pdl_prologue();
+    // Without a row plan nothing of the set-up reads memory (the rows of the group are g*32 .. g*32+31, its
+    // partition is part0): it runs while the kernel in front is still finishing, and the wait for that kernel
+    // comes just before the first copies. With a row plan the wait comes first, as the plan is read at once.
+    pdl_launch_dependents();
+    const bool implicit = !a.group_rows;
+    if (!implicit) pdl_wait();
     const float scale = TEMPERED ? a.scale : kLog2e;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = blockIdx.x / a.S, split = blockIdx.x - g * a.S;
     if (a.n_groups && g >= __ldg(a.n_groups)) return;
-    // Without a row plan the rows of the group are g*32 .. g*32+31 and its partition is part0: the class masks,
-    // whose arrival everything else waits for, are asked for before anything else is set up.
-    const bool early_cm = a.cm_bulk && !a.group_rows;
-    if (early_cm && warp == 0) {
-        if (lane == 0) {
-            mbar_init(&cm_bar, 1);
-            mbar_init_fence();
-            mbar_expect_tx(&cm_bar, uint32_t(min(kGroupRows, a.B - g * kGroupRows)) * uint32_t(a.p0.KW) * 4u);
-        }
-        __syncwarp();
-        const int row = g * kGroupRows + lane;
-        if (row < a.B)
-            bulk_g2s(stage + lane * a.stage_stride, a.class_mask + int64_t(row) * a.cm_stride, uint32_t(a.p0.KW) * 4u, &cm_bar);
+    const bool early_cm = a.cm_bulk && implicit;
+    if (early_cm && tid == 0) {
+        mbar_init(&cm_bar, 1);
+        mbar_init_fence();
+        mbar_expect_tx(&cm_bar, uint32_t(min(kGroupRows, a.B - g * kGroupRows)) * uint32_t(a.p0.KW) * 4u);
+        if (TMAP) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");
     }
     const int part = group_rows_setup(a, g, s_row, tid);
     __syncthreads();
@@ -752,6 +755,15 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
         for (int d = 0; d < depth; ++d) mbar_init(bar + d, 1);
         if (warp == 0 && !early_cm) mbar_init(&cm_bar, 1);
         mbar_init_fence();
+    }
+    if (implicit) pdl_wait();
+    if (early_cm) {
+        // the class masks first (everything waits for them): the rows dealt over the warps, so that no warp
+        // issues more than a few copies; the barrier was set up by thread 0 before the block met above
+        const int r = warp + n_warps * lane;
+        if (r < kGroupRows && g * kGroupRows + r < a.B)
+            bulk_g2s(stage + r * a.stage_stride, a.class_mask + int64_t(g * kGroupRows + r) * a.cm_stride, uint32_t(a.p0.KW) * 4u,
+                     &cm_bar);
     }
     if (a.cm_bulk && !early_cm) {
         __syncthreads();  // the class-mask barrier is initialised for everybody
