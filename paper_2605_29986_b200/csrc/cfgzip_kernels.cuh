@@ -371,7 +371,6 @@ constexpr int kFinalizeThreads = 256;
 
 template <int DT>
 __global__ void __launch_bounds__(kFinalizeThreads) k_finalize_rows(const __grid_constant__ StepArgs a) {
-    __shared__ Partial s_red[kFinalizeThreads / 32];
     pdl_prologue();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = blockIdx.x / kGroupRows, j = blockIdx.x - g * kGroupRows;
@@ -386,42 +385,71 @@ __global__ void __launch_bounds__(kFinalizeThreads) k_finalize_rows(const __grid
     if (row < 0) return;
     const PartDev P = a.group_part ? a.parts[a.group_part[g]] : a.p0;
     const Partial* src = row_slots(a, g, j);
-    // each thread fetches up to four states in one batch (all loads in flight together), folds them
-    // as two independent chains; then a shuffle tree and a fold over the warps
-    float m0 = -INFINITY, s0 = 0.f, m1 = -INFINITY, s1 = 0.f;
-    int p0 = kNoPos, p1 = kNoPos;
-    for (int base = 0; base < a.slots; base += 4 * kFinalizeThreads) {
-        int4 v[4];
+    // Two passes over the states, which stay in registers (up to four per thread, all loads in flight together):
+    // first the row maximum (shuffles and max only), then every state's sum brought to that maximum with one
+    // exponential per state, summed, and the lowest position among the states that hold the maximum. No
+    // exponential sits inside a reduction chain, and the three reductions run side by side.
+    constexpr int kWarps = kFinalizeThreads / 32;
+    __shared__ float s_max[kWarps], s_sum[kWarps];
+    __shared__ int s_pos[kWarps];
+    auto fetch = [&](int base, int4 (&v)[4]) {
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const int sp = base + u * kFinalizeThreads + tid;
             v[u] = make_int4(__float_as_int(-INFINITY), 0, kNoPos, 0);
             if (sp < a.slots) v[u] = __ldcg(reinterpret_cast<const int4*>(src + sp));
         }
-        partial_merge(m0, s0, p0, __int_as_float(v[0].x), __int_as_float(v[0].y), v[0].z);
-        partial_merge(m1, s1, p1, __int_as_float(v[1].x), __int_as_float(v[1].y), v[1].z);
-        partial_merge(m0, s0, p0, __int_as_float(v[2].x), __int_as_float(v[2].y), v[2].z);
-        partial_merge(m1, s1, p1, __int_as_float(v[3].x), __int_as_float(v[3].y), v[3].z);
+    };
+    int4 v0[4];
+    fetch(0, v0);
+    float M = fmaxf(fmaxf(__int_as_float(v0[0].x), __int_as_float(v0[1].x)), fmaxf(__int_as_float(v0[2].x), __int_as_float(v0[3].x)));
+    for (int base = 4 * kFinalizeThreads; base < a.slots; base += 4 * kFinalizeThreads) {  // more than 1024 states: rare
+        int4 w[4];
+        fetch(base, w);
+        M = fmaxf(M, fmaxf(fmaxf(__int_as_float(w[0].x), __int_as_float(w[1].x)), fmaxf(__int_as_float(w[2].x), __int_as_float(w[3].x))));
     }
-    partial_merge(m0, s0, p0, m1, s1, p1);
-    partial_warp_allreduce(m0, s0, p0);
-    if (lane == 0) s_red[warp] = Partial{m0, s0, p0, 0};
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, d));
+    if (lane == 0) s_max[warp] = M;
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) M = fmaxf(M, s_max[w]);
+    const float Mf = fmaxf(M, kRefFloor);
+    float sum = 0.f;
+    int pos = kNoPos;
+    auto gather = [&](const int4 (&v)[4]) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const float m = __int_as_float(v[u].x);
+            sum = fmaf(__int_as_float(v[u].y), ex2f((fmaxf(m, kRefFloor) - Mf) * kLog2e), sum);
+            pos = (m == M) ? min(pos, v[u].z) : pos;
+        }
+    };
+    gather(v0);
+    for (int base = 4 * kFinalizeThreads; base < a.slots; base += 4 * kFinalizeThreads) {
+        int4 w[4];
+        fetch(base, w);
+        gather(w);
+    }
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, d);
+        pos = min(pos, __shfl_xor_sync(0xFFFFFFFFu, pos, d));
+    }
+    if (lane == 0) {
+        s_sum[warp] = sum;
+        s_pos[warp] = pos;
+    }
     __syncthreads();
     if (warp != 0) return;
-    // the eight warp states: one per lane, three butterfly steps, the result handed to every lane
-    const Partial mine = lane < kFinalizeThreads / 32 ? s_red[lane] : partial_empty();
-    m0 = mine.m; s0 = mine.s; p0 = mine.pos;
+    sum = 0.f;
+    pos = kNoPos;
 #pragma unroll
-    for (int d = kFinalizeThreads / 64; d >= 1; d >>= 1) {
-        const float m2 = __shfl_xor_sync(0xFFFFFFFFu, m0, d);
-        const float s2 = __shfl_xor_sync(0xFFFFFFFFu, s0, d);
-        const int p2 = __shfl_xor_sync(0xFFFFFFFFu, p0, d);
-        partial_merge(m0, s0, p0, m2, s2, p2);
+    for (int w = 0; w < kWarps; ++w) {  // every lane of warp 0 takes the same eight values in the same order
+        sum += s_sum[w];
+        pos = min(pos, s_pos[w]);
     }
-    m0 = __shfl_sync(0xFFFFFFFFu, m0, 0);
-    s0 = __shfl_sync(0xFFFFFFFFu, s0, 0);
-    p0 = __shfl_sync(0xFFFFFFFFu, p0, 0);
-    warp_finalize_row<DT>(a, P, row, m0, s0, p0, lane);
+    warp_finalize_row<DT>(a, P, row, M, sum, pos, lane);
 }
 
 // The same for rows with few published states (at most 4 per lane: large batches, where a group is
