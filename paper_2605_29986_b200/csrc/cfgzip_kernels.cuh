@@ -501,39 +501,52 @@ __device__ __forceinline__ void dense_octet_row(Octet<DT>& oc, char* rowp, uint8
     acc.add_octet(f, o);
 }
 
+// Order-preserving map between floats and signed integers (for the integer warp reductions).
+__device__ __forceinline__ int float_order_key(float x) {
+    const int i = __float_as_int(x);
+    return i >= 0 ? i : i ^ 0x7FFFFFFF;
+}
+__device__ __forceinline__ float float_from_order_key(int k) { return __int_as_float(k >= 0 ? k : k ^ 0x7FFFFFFF); }
+
 // Reduce the 8 row states of a warp over its 32 lanes and publish them in the warp's slot of each row.
-// Recursive halving: lanes first trade half of their rows with the lane 16 away and fold the
-// half they keep, then 2 of 4 with the lane 8 away, then 1 of 2; two butterfly steps finish
-// the single row left (nine folds instead of forty).
 __device__ __forceinline__ void warp_rows_publish(const StepArgs& a, RowAcc (&acc)[kBatchRows], int live, int g, int slot,
                                                   int rb, int lane, float scale = kLog2e) {
-    Partial p[kBatchRows];
+    // Two passes, no exponential inside a reduction chain: the maximum of every row over the lanes (one integer
+    // warp reduction each), every lane's sum brought to it with one exponential, the lowest position among the
+    // lanes that hold the maximum (one more integer reduction), and the eight sums reduced by recursive halving
+    // (lanes trade half of their rows with the lane 16 away, then 2 of 4 with the lane 8 away, then 1 of 2; two
+    // butterfly steps finish the single row left).
+    float M[kBatchRows], w[kBatchRows];
+    int pos[kBatchRows];
 #pragma unroll
-    for (int i = 0; i < kBatchRows; ++i) p[i] = acc[i].to_partial(scale);
+    for (int i = 0; i < kBatchRows; ++i) M[i] = float_from_order_key(__reduce_max_sync(0xFFFFFFFFu, float_order_key(acc[i].m)));
+#pragma unroll
+    for (int i = 0; i < kBatchRows; ++i) {
+        w[i] = M[i] > kRefFloor ? acc[i].s * ex2f(-fmaf(M[i], scale, acc[i].nrl)) : 0.f;
+        pos[i] = __reduce_min_sync(0xFFFFFFFFu, acc[i].m == M[i] ? acc[i].pos : kNoPos);
+    }
 #pragma unroll
     for (int half = 4; half >= 1; half >>= 1) {
         const int d = 4 * half;  // 16, 8, 4
         const bool up = lane & d;
 #pragma unroll
         for (int k = 0; k < half; ++k) {
-            const Partial keep = up ? p[k + half] : p[k];
-            const Partial send = up ? p[k] : p[k + half];
-            const float m2 = __shfl_xor_sync(0xFFFFFFFFu, send.m, d);
-            const float s2 = __shfl_xor_sync(0xFFFFFFFFu, send.s, d);
-            const int p2 = __shfl_xor_sync(0xFFFFFFFFu, send.pos, d);
-            p[k] = keep;
-            partial_merge(p[k].m, p[k].s, p[k].pos, m2, s2, p2, scale);
+            const float keep = up ? w[k + half] : w[k];
+            const float send = up ? w[k] : w[k + half];
+            w[k] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, d);
         }
     }
-#pragma unroll
-    for (int d = 2; d >= 1; d >>= 1) {
-        const float m2 = __shfl_xor_sync(0xFFFFFFFFu, p[0].m, d);
-        const float s2 = __shfl_xor_sync(0xFFFFFFFFu, p[0].s, d);
-        const int p2 = __shfl_xor_sync(0xFFFFFFFFu, p[0].pos, d);
-        partial_merge(p[0].m, p[0].s, p[0].pos, m2, s2, p2, scale);
-    }
+    w[0] += __shfl_xor_sync(0xFFFFFFFFu, w[0], 2);
+    w[0] += __shfl_xor_sync(0xFFFFFFFFu, w[0], 1);
     const int i = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);  // the row this lane ended with
-    if ((lane & 3) == 0 && i < live) row_slots(a, g, rb * kBatchRows + i)[slot] = p[0];
+    float Mi = M[0];
+    int pi = pos[0];
+#pragma unroll
+    for (int k = 1; k < kBatchRows; ++k) {
+        Mi = i == k ? M[k] : Mi;
+        pi = i == k ? pos[k] : pi;
+    }
+    if ((lane & 3) == 0 && i < live) row_slots(a, g, rb * kBatchRows + i)[slot] = Partial{Mi, w[0], pi, 0};
 }
 
 // ---------------------------------------------------------------------------------------
