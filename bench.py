@@ -172,6 +172,9 @@ class StepRunner:
         if ring_override:
             self.R = ring_override  # a short ring stays in L2: only for the figure labelled warm
         self.U = min(self.R, unique)
+        # steps per CUDA graph: one pass over the ring; a short (L2-resident) ring is cycled 500 times per graph so
+        # that the replay cost of a graph stays negligible there too
+        self.G = self.R if not ring_override else 500 * self.R
         tile = -(-self.B // self.w.B)
         tdt = torch.int16 if self.dtype == "bf16" else torch.float32
         self.host_logits = []
@@ -251,26 +254,26 @@ class StepRunner:
             with torch.cuda.stream(self.stream):
                 with torch.cuda.graph(g, stream=self.stream):
                     for j in range(n):
-                        self.call(j, self.stream)
+                        self.call(j % self.R, self.stream)
             self.launches[n] = self.cz.cfgzip_launch_count(self.ctx) - before
             self.graphs[n] = g
         return self.graphs[n]
 
     def prepare(self, n_steps: int):
-        full, rem = divmod(n_steps, self.R)
+        full, rem = divmod(n_steps, self.G)
         if full:
-            self.graph(self.R)
+            self.graph(self.G)
         if rem:
             self.graph(rem)
 
     def run(self, n_steps: int) -> int:
         """Enqueue n_steps steps (ring order, wrapping) on self.stream; returns kernels launched."""
-        full, rem = divmod(n_steps, self.R)
+        full, rem = divmod(n_steps, self.G)
         launched = 0
         with self.torch.cuda.stream(self.stream):
             for _ in range(full):
-                self.graph(self.R).replay()
-                launched += self.launches[self.R]
+                self.graph(self.G).replay()
+                launched += self.launches[self.G]
                 if self.pass_events is not None:  # one event per pass over the ring, inside the timed region
                     ev = self.torch.cuda.Event(enable_timing=True)
                     ev.record(self.stream)
@@ -288,8 +291,8 @@ class StepRunner:
         self.run(max(warmup, 3))
         # every CUDA graph the timed region replays has run once before it (the first replay of a graph
         # also uploads it): these are extra untimed steps on top of the warm-up
-        full, rem = divmod(n_steps, self.R)
-        self.run((self.R if full else 0) + rem)
+        full, rem = divmod(n_steps, self.G)
+        self.run((self.G if full else 0) + rem)
         self.stream.synchronize()
         self.restore()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -305,7 +308,7 @@ class StepRunner:
         self.stream.synchronize()
         torch.cuda.synchronize()
         marks, self.pass_events = [e0] + self.pass_events, None
-        self.pass_us_per_step = [a.elapsed_time(b) * 1e3 / self.R for a, b in zip(marks, marks[1:])]
+        self.pass_us_per_step = [a.elapsed_time(b) * 1e3 / self.G for a, b in zip(marks, marks[1:])]
         if sampler:
             sampler.stop()
         if barrier:
