@@ -268,7 +268,7 @@ int cfgzip_launch_count(cfgzip_ctx* ctx, int64_t* out);
  *   "ctas_per_sm"  target resident thread blocks per SM for the fused kernel (1..16)
  *   "token_warps"  0 = automatic, else warps side by side along the vocabulary (1..16)
  *   "row_warps"    0 = automatic, else 1, 2 or 4 row batches handled by separate warps
- *   "pdl"          1 = programmatic dependent launch where it pays (steps under 48 MB of logits;
+ *   "pdl"          1 = programmatic dependent launch where it pays (steps under 192 MB of logits;
  *                  default), 0 = never, 2 = always
  *   "pipeline"     1 = aligned logits stream through per-warp rings of bulk asynchronous copies
  *                  in shared memory (default), 0 = plain 16-byte loads into registers
