@@ -280,13 +280,13 @@ DensePlan plan_pipe(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, i
     bool alias = ctx->stage_alias != 0 ||
                  (pipe_smem_bytes(d.table_words, n_warps, 2, stage_bytes, stride) > cap &&
                   pipe_smem_bytes(d.table_words, n_warps, 2, stage_bytes, stride, true) <= cap);
-    // Long steps (six or more work items per warp) gain from a third stage where sharing the staging area makes
-    // room for it (measured: B = 256 -4 %, B = 1024 and 2048 -2 %; shorter steps lose to the late start of the
-    // first warps).
+    // Long steps (twenty or more work items per warp) gain from a third stage where sharing the staging area makes
+    // room for it (measured at V = 128256, bf16: B = 1024 -0.7 %, B = 2048 -1.4 %; B = 256 .. 512 lose 1 to 2 % to
+    // the late start of the first warps).
     if (!ctx->pipe_depth_set && depth < 3 && pipe_smem_bytes(d.table_words, n_warps, 3, stage_bytes, stride, true) <= cap) {
         const int64_t blocks = int64_t(ctx->sm_count) * ctx->waves;
         const int64_t items = int64_t(ceil_div(B, kGroupRows)) * (((ps.V >> 3) + 31) >> 5) * ceil_div(std::min<int>(B, kGroupRows), kBatchRows);
-        if (items >= 6 * blocks * n_warps) {
+        if (items >= 20 * blocks * n_warps) {
             depth = 3;
             alias = true;
         }
