@@ -61,6 +61,7 @@ struct cfgzip_ctx {
     size_t st_vm_bytes = 0;
     int32_t* st_small = nullptr;  // row_part, argmax, rep, lse, logp_argmax: 5 arrays of st_rows
     int32_t st_rows = 0;
+    int32_t* st_small_host = nullptr;  // pinned mirror of the four result arrays: they come back in one copy
     int64_t launches = 0;
     // row plan kept by cfgzip_plan_rows (valid until anything overwrites the plan buffers or the partitions change)
     bool plan_valid = false;
@@ -698,6 +699,7 @@ int cfgzip_destroy(cfgzip_ctx* ctx) {
     cudaFree(ctx->st_cm);
     cudaFree(ctx->st_vm);
     cudaFree(ctx->st_small);
+    if (ctx->st_small_host) cudaFreeHost(ctx->st_small_host);
     cudaGetLastError();
     delete ctx;
     return CFGZIP_OK;
@@ -1043,6 +1045,12 @@ int cfgzip_decode_step_host(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t
                 return rc;
             }
             ctx->st_rows = B;
+            if (ctx->st_small_host) cudaFreeHost(ctx->st_small_host);
+            ctx->st_small_host = nullptr;
+            if (cudaHostAlloc(reinterpret_cast<void**>(&ctx->st_small_host), size_t(B) * 16, cudaHostAllocDefault) != cudaSuccess) {
+                cudaGetLastError();
+                ctx->st_small_host = nullptr;  // the four results then come back one by one
+            }
         }
     }
     int32_t* d_rp = ctx->st_small;
@@ -1067,13 +1075,29 @@ int cfgzip_decode_step_host(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t
     };
     back(masked_logits, ctx->st_logits, logit_bytes);
     back(vocab_mask_host, ctx->st_vm, vm_bytes);
-    back(argmax, d_am, size_t(B) * 4);
-    back(rep, d_rep, size_t(B) * 4);
-    back(lse, d_lse, size_t(B) * 4);
-    back(logp_argmax, d_lpa, size_t(B) * 4);
+    // the four small result arrays sit side by side on the device: one copy into a pinned mirror, handed out
+    // after the stream has drained (four separate small copies cost more than the kernels of a short step)
+    const bool one_copy = ctx->st_small_host != nullptr && (argmax || rep || lse || logp_argmax);
+    const size_t span = (size_t(ctx->st_rows) * 3 + size_t(B)) * 4;  // argmax .. logp_argmax, st_rows apart
+    if (one_copy) {
+        back(ctx->st_small_host, d_am, span);
+    } else {
+        back(argmax, d_am, size_t(B) * 4);
+        back(rep, d_rep, size_t(B) * 4);
+        back(lse, d_lse, size_t(B) * 4);
+        back(logp_argmax, d_lpa, size_t(B) * 4);
+    }
     if (!ok || cudaStreamSynchronize(st) != cudaSuccess) {
         cudaGetLastError();
         return CFGZIP_E_CUDA;
+    }
+    if (one_copy) {
+        const int32_t* h = ctx->st_small_host;
+        const size_t n = size_t(B) * 4, step = size_t(ctx->st_rows);
+        if (argmax) std::memcpy(argmax, h, n);
+        if (rep) std::memcpy(rep, h + step, n);
+        if (lse) std::memcpy(lse, h + 2 * step, n);
+        if (logp_argmax) std::memcpy(logp_argmax, h + 3 * step, n);
     }
     return CFGZIP_OK;
 }
