@@ -1222,8 +1222,7 @@ __device__ __forceinline__ float block_exclusive_scan(float v, float* s_warp, fl
         const float up = __shfl_up_sync(0xFFFFFFFFu, inc, d);
         if (lane >= d) inc += up;
     }
-    __syncthreads();  // s_warp may still be read from an earlier call
-    if (lane == 31) s_warp[warp] = inc;
+    if (lane == 31) s_warp[warp] = inc;  // the caller gives every call an array no thread may still be reading
     __syncthreads();
     float before = 0.f, all = 0.f;
 #pragma unroll
@@ -1238,8 +1237,9 @@ __device__ __forceinline__ float block_exclusive_scan(float v, float* s_warp, fl
 
 template <int DT>
 __global__ void __launch_bounds__(kSampleThreads) k_sample_rows(const __grid_constant__ StepArgs a, int aligned) {
-    __shared__ float s_warp[kSampleThreads / 32];
+    __shared__ float s_warp[kSampleThreads / 32], s_scan_states[kSampleThreads / 32], s_scan_tokens[kSampleThreads / 32];
     __shared__ int s_pick, s_last;
+    __shared__ int s_pick_state, s_last_state;
     __shared__ float s_base;
     pdl_prologue();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -1293,7 +1293,12 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample_rows(const __grid_con
 #pragma unroll
     for (int d = 16; d >= 1; d >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, d));
     if (lane == 0) s_warp[warp] = M;
-    if (tid == 0) { s_pick = kNoPos; s_last = -1; }
+    if (tid == 0) {
+        s_pick = kNoPos;
+        s_last = -1;
+        s_pick_state = kNoPos;
+        s_last_state = -1;
+    }
     __syncthreads();
 #pragma unroll
     for (int w = 0; w < kSampleThreads / 32; ++w) M = fmaxf(M, s_warp[w]);
@@ -1327,29 +1332,29 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample_rows(const __grid_con
     float mine = 0.f;
     for (int k = k0; k < k1; ++k) mine += weight(k);
     float total;
-    const float front = block_exclusive_scan(mine, s_warp, total);  // weight in front of this thread's states
+    const float front = block_exclusive_scan(mine, s_scan_states, total);  // weight in front of this thread's states
     const float tau = u * total;
     float run = front;
     for (int k = k0; k < k1; ++k) {
         const float w = weight(k);
         if (w > 0.f) {
-            atomicMax(&s_last, k);
+            atomicMax(&s_last_state, k);
             if (run + w > tau) {
-                atomicMin(&s_pick, k);
+                atomicMin(&s_pick_state, k);
                 break;
             }
         }
         run += w;
     }
     __syncthreads();
-    const int pick = s_pick != kNoPos ? s_pick : s_last;  // rounding may leave tau at the very end: the last run with weight
+    // rounding may leave tau at the very end: then the last run with weight
+    const int pick = s_pick_state != kNoPos ? s_pick_state : s_last_state;
     if (pick >= k0 && pick < k1) {  // the thread that owns the chosen state: the weight in front of it
         float r2 = front;
         for (int k = k0; k < pick; ++k) r2 += weight(k);
         s_base = r2;
     }
     __syncthreads();
-    if (tid == 0) { s_pick = kNoPos; s_last = -1; }
     float base = s_base;
 
     // the tokens the chosen state stands for
@@ -1365,11 +1370,7 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample_rows(const __grid_con
     }
     constexpr int ES = DT == kBF16 ? 2 : 4;
     const char* rowp = reinterpret_cast<const char*>(a.logits) + int64_t(row) * a.row_stride * ES;
-    __shared__ float s_ztok;
-    int token = -1;
-    for (int p0 = t_lo; p0 < t_hi; p0 += kSampleThreads * 8) {
-        const int t0 = p0 + tid * 8;
-        float e[8];
+    auto load8 = [&](int t0, float (&e)[8]) {
         if (aligned && t0 + 8 <= t_hi) {  // t_lo is a multiple of 8 tokens: 16-byte (bf16) / 32-byte (f32) vectors
             if (DT == kBF16) {
                 const uint4 v = __ldcg(reinterpret_cast<const uint4*>(rowp + size_t(t0) * 2));
@@ -1387,6 +1388,29 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample_rows(const __grid_con
 #pragma unroll
             for (int q = 0; q < 8; ++q) e[q] = t0 + q < t_hi ? ldcg_elem<DT>(rowp, t0 + q) : -INFINITY;
         }
+    };
+    auto write_token = [&](int token, float zt, int repv) {
+        const float l = logf(total);
+        a.argmax[row] = token;
+        if (a.rep) a.rep[row] = repv;
+        if (a.lse) a.lse[row] = fmaf(M, a.inv_t, l);
+        if (a.logp_argmax) a.logp_argmax[row] = (zt - M) * a.inv_t - l;
+    };
+    auto write_empty = [&]() {  // no token of the run carried weight: report the row as empty
+        a.argmax[row] = -1;
+        if (a.rep) a.rep[row] = -1;
+        if (a.lse) a.lse[row] = -INFINITY;
+        if (a.logp_argmax) a.logp_argmax[row] = -INFINITY;
+    };
+    if (pick < 0) {  // no state carried weight
+        if (tid == 0) write_empty();
+        return;
+    }
+    int token = -1;
+    for (int p0 = t_lo; p0 < t_hi; p0 += kSampleThreads * 8) {
+        const int t0 = p0 + tid * 8;
+        float e[8];
+        load8(t0, e);
         float z8[8], sum8 = 0.f;
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
@@ -1395,7 +1419,7 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample_rows(const __grid_con
             sum8 += e[q];
         }
         float piece;
-        float r3 = base + block_exclusive_scan(sum8, s_warp, piece);
+        float r3 = base + block_exclusive_scan(sum8, s_scan_tokens, piece);
         int mine_tok = -1, mine_last = -1;
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
@@ -1407,34 +1431,22 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample_rows(const __grid_con
         }
         if (mine_last >= 0) atomicMax(&s_last, mine_last);
         if (mine_tok >= 0) atomicMin(&s_pick, mine_tok);
+        int my_rep = mine_tok >= 0 ? __ldg(P.trep + mine_tok) : -1;  // in flight across the barrier
         __syncthreads();
         token = s_pick != kNoPos ? s_pick : -1;
         const bool last_piece = p0 + kSampleThreads * 8 >= t_hi;
         if (token < 0 && last_piece) token = s_last;  // rounding: the last token with weight in the run
-        if (token >= t0 && token < t0 + 8) {          // the thread that holds the token hands its logit over
+        if (token >= t0 && token < t0 + 8) {          // the thread that holds the token writes the row's results
             float zt = 0.f;
 #pragma unroll
             for (int q = 0; q < 8; ++q) zt = (token - t0 == q) ? z8[q] : zt;
-            s_ztok = zt;
+            if (token != mine_tok) my_rep = __ldg(P.trep + token);
+            write_token(token, zt, my_rep);
         }
         if (token >= 0) break;
         base += piece;
     }
-    __syncthreads();
-    if (tid == 0) {
-        float lsev = -INFINITY, lpt = -INFINITY;
-        int repv = -1;
-        if (token >= 0) {
-            const float l = logf(total);
-            lsev = fmaf(M, a.inv_t, l);
-            lpt = (s_ztok - M) * a.inv_t - l;
-            repv = P.trep[token];
-        }
-        a.argmax[row] = token;
-        if (a.rep) a.rep[row] = repv;
-        if (a.lse) a.lse[row] = lsev;
-        if (a.logp_argmax) a.logp_argmax[row] = lpt;
-    }
+    if (token < 0 && tid == 0) write_empty();
 }
 
 // ---------------------------------------------------------------------------------------
