@@ -233,3 +233,22 @@ def test_sample_unaligned_rows_with_mixed_partitions():
         got = run_sample(ctx, row_part, cm, z, V, u, 5.0, stride=stride)
         check_sample(got, parts, row_part, cm, z, V, u, 5.0)
         assert cz.cfgzip_poll_status(ctx.h) == (0, 0, 0)
+
+
+@pytest.mark.parametrize("inv_t", [0.25, 1.0])
+def test_sample_uniforms_at_both_ends_of_the_range_many_rows(inv_t):
+    # u = 0 draws the first allowed token with weight; u just under 1 lands in the last run, where the summation
+    # order of the prefix decides whether the threshold is crossed at all (if not: the last token with weight).
+    # Flat distributions (high temperature) keep weight on the tail, so both cases occur across 96 rows.
+    w = synth.make_workload(2, B=96)
+    cm, z = w.class_masks(11), w.logits(11)
+    u = np.where(np.arange(96) % 3 == 0, np.float32(0.0), np.float32(1.0) - np.float32(2.0 ** -24)).astype(np.float32)
+    with Ctx(w.partitions) as ctx:
+        got = run_sample(ctx, None, cm, z, w.V, u, inv_t)
+        assert cz.cfgzip_poll_status(ctx.h)[1:] == (0, 0)
+    check_sample(got, w.partitions, None, cm, z, w.V, u, inv_t, "1/T=%g" % inv_t)
+    allowed = synth.unpack_bits(got["vocab_mask"], w.V)
+    for b in range(96):
+        assert allowed[b, got["token"][b]]
+        if u[b] == 0.0:
+            assert got["token"][b] == np.flatnonzero(allowed[b])[0]   # every allowed logit is finite: weight > 0
