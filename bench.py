@@ -13,7 +13,12 @@ Prints ONE JSON line (rank 0). ``value`` is rows/s over all GPUs with inputs res
 HBM; ``e2e`` is the same metric through the host-buffer entry point with the copies inside
 the timed region; ``roofline`` relates the fused kernel to the measured HBM copy rate;
 ``cpu_baseline`` is the CPU oracle timed on this machine's host cores (a reported baseline,
-not a target). ``--impl reference`` times only that oracle.
+not a target); ``parity`` compares GPU results with that oracle. ``--impl reference`` times
+only the oracle. With ``--gpus N`` > 1 and no launcher in the environment the script starts
+N ranks of itself (one per GPU).
+
+The timed region always consists of whole passes over the ring of working buffers and lasts
+at least 20 ms: ``steps`` echoes the request, ``timed_steps`` is what was timed.
 """
 from __future__ import annotations
 
@@ -32,6 +37,7 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 import synth  # noqa: E402
+from paper_2605_29986_b200 import rows as ranks  # noqa: E402  (host-only helpers: no CUDA needed to import)
 
 METRIC = "masked_rows_per_s"
 UNIT = "rows/s"
@@ -40,11 +46,13 @@ FALLBACK_HBM_GBS = 6650.0
 RING_BYTES = 1 << 30          # working buffers cover at least this much, several times the 126 MB L2
 RING_MAX_STEPS = 1000
 RING_MAX_BYTES = 24 << 30
+MIN_TIMED_SECONDS = 0.02      # shorter regions read slow: the replay cost of a graph sits inside them
+LOG_TOL = 1e-4                # absolute, fp32-accumulated log quantities against the fp64 oracle
 
 # DRAM traffic of the dominant (streaming) kernel per launch = per step (dram__bytes_read.sum +
-# dram__bytes_write.sum from one ncu capture), keyed by workload; valid only for the kernel sources whose digest is
-# recorded with it. None until a capture of the current sources exists.
-NCU_TRAFFIC = {"cfg2_B32_dense": {"digest": "59571828e471fddd", "bytes_per_launch": 8539051}}
+# dram__bytes_write.sum from one ncu capture, see profiles/), keyed by workload; valid only for the kernel
+# sources whose digest is recorded with it. A workload without a capture of the current sources reports null.
+NCU_TRAFFIC = {}
 
 
 def _kernel_digest() -> str:
@@ -54,11 +62,6 @@ def _kernel_digest() -> str:
         if name.endswith(".cuh"):  # the kernels; the launch shape of the headline workload is pinned by tests/test_planner.py
             h.update(open(os.path.join(csrc, name), "rb").read())
     return h.hexdigest()[:16]
-
-
-def _dist_env():
-    return (int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")),
-            int(os.environ.get("WORLD_SIZE", "1")))
 
 
 def _host_threads() -> int:
@@ -81,6 +84,71 @@ def algorithmic_bytes(B: int, V: int, K: int, elem: int, n_partitions: int = 1, 
     class masks, write four 4-byte results per row, read the token->class vector once per partition."""
     VW, KW = (V + 31) // 32, (K + 31) // 32
     return B * (2 * V * elem + 4 * VW + 4 * KW + 16) + n_partitions * V * class_id_bytes
+
+
+# ----------------------------------------------------------------------------- step and slot bookkeeping
+
+def ring_steps(step_bytes: int, steps_hint: int) -> int:
+    """Working buffers in the ring: at least RING_BYTES of logits (several times L2), at least min(steps_hint,
+    RING_MAX_STEPS) buffers, never more than RING_MAX_BYTES."""
+    ring = max(4, -(-RING_BYTES // step_bytes))
+    ring = max(ring, min(steps_hint, RING_MAX_STEPS))
+    return int(max(1, min(ring, RING_MAX_BYTES // step_bytes)))
+
+
+def timed_steps_for(requested: int, steps_per_pass: int, pass_seconds: float, min_seconds: float = MIN_TIMED_SECONDS) -> int:
+    """Steps the timed region runs: whole passes over the ring, at least the requested steps, at least min_seconds."""
+    passes = max(1, -(-requested // steps_per_pass))
+    if pass_seconds > 0:
+        passes = max(passes, int(np.ceil(min_seconds / pass_seconds)))
+    return passes * steps_per_pass
+
+
+def spread(n: int, k: int) -> list:
+    """k indices spread evenly over range(n) (all of them when k >= n), ascending and distinct."""
+    if k >= n:
+        return list(range(n))
+    return sorted(set(int(x) for x in np.linspace(0, n - 1, k)))
+
+
+def check_slots(runner, slots, row_ids=None, threads: int = 1, budget_s: float = 30.0, full_logits: int = 2) -> dict:
+    """Parity of ring slots against the CPU oracle. `runner.execute_slots(slots, rows)` runs exactly these steps
+    once more (untimed, on freshly refilled buffers) and returns the outputs of the chosen rows, so no slot is
+    compared that was not executed. Rows `row_ids` (all when None) of each slot are compared: vocab mask, argmax
+    and representative bit for bit, lse and logp_argmax within LOG_TOL, and the masked logits bit for bit on the
+    first `full_logits` slots. Stops early when the oracle has used `budget_s` seconds."""
+    import oracle
+    slots = list(slots)
+    rows_sel = np.arange(runner.B) if row_ids is None else np.asarray(sorted(row_ids), dtype=np.int64)
+    got = runner.execute_slots(slots, rows_sel, full_logits)
+    rp = None if runner.row_part_host is None else runner.row_part_host[rows_sel]
+    checked, mismatches, max_err, spent = 0, 0, 0.0, 0.0
+    for n, j in enumerate(slots):
+        z = np.ascontiguousarray(runner.host_logits_of(j)[rows_sel]).copy()
+        t0 = time.perf_counter()
+        want = oracle.decode_step(runner.partitions, rp, np.ascontiguousarray(runner.host_cm[j][rows_sel]), z,
+                                  threads=threads)
+        spent += time.perf_counter() - t0
+        ok = np.array_equal(got["argmax"][n], want["argmax"]) and np.array_equal(got["rep"][n], want["rep"])
+        ok = ok and np.array_equal(got["vocab_mask"][n], want["vocab_mask"])
+        if n < full_logits:
+            ok = ok and np.array_equal(got["logits"][n].view(np.uint8), z.view(np.uint8))
+        for key in ("lse", "logp_argmax"):
+            g = got[key][n].astype(np.float64)
+            fin = np.isfinite(want[key])
+            ok = ok and np.array_equal(np.isfinite(g), fin)
+            if fin.any():
+                err = float(np.abs(g[fin] - want[key][fin]).max())
+                max_err = max(max_err, err)
+                ok = ok and err <= LOG_TOL
+        checked += 1
+        mismatches += 0 if ok else 1
+        if spent > budget_s:
+            break
+    return {"steps_checked": checked, "of_ring_steps": runner.R, "rows_per_step": int(len(rows_sel)), "of_rows": runner.B,
+            "mismatching_steps": mismatches, "max_abs_err_log": max_err, "tolerance_log": LOG_TOL,
+            "what": "steps re-run untimed on refilled buffers, compared with the CPU oracle: vocab mask, argmax, rep bit-exact "
+                    "(masked logits too on the first %d), lse and logp_argmax within the tolerance" % full_logits}
 
 
 # ----------------------------------------------------------------------------- clocks
@@ -145,198 +213,210 @@ class ClockSampler(threading.Thread):
 # ----------------------------------------------------------------------------- workload on the device
 
 class StepRunner:
-    """A ring of resident working buffers for one workload and CUDA graphs that run steps over it."""
+    """A ring of resident working buffers for one workload and a CUDA graph that runs one pass of steps over it."""
 
     def __init__(self, cz, torch, device: int, config: int, B: int = None, mode: str = "dense", steps_hint: int = 1000,
-                 unique: int = 8, tune=(), unfused: bool = False, ring: int = 0, inv_temperature: float = 0.0):
+                 unique: int = 8, tune=(), kind: str = "fused", ring: int = 0, inv_temperature: float = 0.0):
         self.cz, self.torch = cz, torch
-        self.unfused = unfused  # separate expand + mask calls instead of the fused step (no reductions)
+        # kind: "fused" the whole step; "unfused" separate expand + mask calls (no reductions); "floor" the in-place
+        # read-modify-write kernel over the same buffers (what a pass over these bytes costs at least)
+        self.kind = kind
         self.inv_temperature = inv_temperature  # > 0: the sampling step (cfgzip_masked_sample) instead of the greedy one
         spec = synth.CONFIGS[config]
-        self.w = synth.make_workload(config, B=min(B or spec["B"], 64))  # unique rows; tiled up to B below
         self.B = B or spec["B"]
+        wl = synth.make_workload(config, B=min(self.B, 64))  # unique logits rows; tiled up to B below
+        # every row has its own class mask (and partition) at every batch size; only the logits rows repeat
+        self.w = wl if self.B <= 64 else synth.make_workload(config, B=self.B)
+        self.partitions = self.w.partitions
         self.V, self.K, self.dtype = self.w.V, self.w.K, self.w.dtype
         self.elem = 2 if self.dtype == "bf16" else 4
         self.VW, self.KW = (self.V + 31) // 32, (self.K + 31) // 32
+        self.mode_name = mode
         self.mode = {"dense": cz.DENSE, "sparse": cz.SPARSE, "auto": cz.AUTO}[mode]
         self.ctx = cz.cfgzip_create(device)
         for item in tune:
             name, value = item.split("=")
             cz.cfgzip_set_tuning(self.ctx, name, int(value))
-        self.parts = [cz.cfgzip_load_partition(self.ctx, p.c, p.V, p.r, p.K) for p in self.w.partitions]
-        ring_override = ring
+        self.parts = [cz.cfgzip_load_partition(self.ctx, p.c, p.V, p.r, p.K) for p in self.partitions]
         step_bytes = self.B * self.V * self.elem
-        ring = max(4, -(-RING_BYTES // step_bytes))
-        ring = max(ring, min(steps_hint, RING_MAX_STEPS))
-        self.R = int(max(1, min(ring, RING_MAX_BYTES // step_bytes)))
-        if ring_override:
-            self.R = ring_override  # a short ring stays in L2: only for the figure labelled warm
+        self.R = ring if ring else ring_steps(step_bytes, steps_hint)  # a short ring stays in L2: only for the figure labelled warm
         self.U = min(self.R, unique)
         # steps per CUDA graph: one pass over the ring; a short (L2-resident) ring is cycled 500 times per graph so
         # that the replay cost of a graph stays negligible there too
-        self.G = self.R if not ring_override else 500 * self.R
-        tile = -(-self.B // self.w.B)
+        self.G = self.R if not ring else 500 * self.R
+        tile = -(-self.B // wl.B)
         tdt = torch.int16 if self.dtype == "bf16" else torch.float32
         self.host_logits = []
         self.pristine = []
         for u in range(self.U):
-            z = self.w.logits(u)
-            z = np.tile(z, (tile, 1))[: self.B]
+            z = np.tile(wl.logits(u), (tile, 1))[: self.B]
             self.host_logits.append(z)
             self.pristine.append(torch.from_numpy(z.view(np.int16) if self.dtype == "bf16" else z).cuda())
-        cms = []
-        for j in range(self.R):
-            cm = self.w.class_masks(j)
-            cms.append(np.tile(cm, (tile, 1))[: self.B])
-        self.host_cm = np.stack(cms)
+        self.host_cm = np.stack([self.w.class_masks(j) for j in range(self.R)])
         self.cm = torch.from_numpy(self.host_cm.view(np.int32)).cuda()
-        self.row_part_host = None if self.w.row_part is None else \
-            (np.arange(self.B) % len(self.parts)).astype(np.int32)
+        self.row_part_host = None if self.w.row_part is None else np.ascontiguousarray(self.w.row_part, dtype=np.int32)
         self.row_part = None if self.row_part_host is None else torch.from_numpy(self.row_part_host).cuda()
         self.row_part_arg = self.row_part
-        if self.row_part is not None:
+        if self.row_part is not None and kind == "fused":
             # the rows keep their grammars over the steps: group them by partition once, outside the steps
             cz.cfgzip_plan_rows(self.ctx, self.parts[0], self.row_part, self.B)
             self.row_part_arg = cz.ROWS_AS_PLANNED
         self.work = torch.empty((self.R, self.B, self.V), dtype=tdt, device="cuda")
-        self.vm = torch.empty((self.R, self.B, self.VW), dtype=torch.int32, device="cuda")
-        self.am = torch.empty((self.R, self.B), dtype=torch.int32, device="cuda")
-        self.rep = torch.empty_like(self.am)
-        self.lse = torch.empty((self.R, self.B), dtype=torch.float32, device="cuda")
-        self.lpa = torch.empty_like(self.lse)
+        self.vm = torch.zeros((self.R, self.B, self.VW), dtype=torch.int32, device="cuda")
+        self.am = torch.full((self.R, self.B), -9, dtype=torch.int32, device="cuda")
+        self.rep = torch.full_like(self.am, -9)
+        self.lse = torch.full((self.R, self.B), float("nan"), dtype=torch.float32, device="cuda")
+        self.lpa = torch.full_like(self.lse, float("nan"))
         self.u = None
         if inv_temperature > 0:
-            us = np.stack([np.tile(self.w.uniforms(j), tile)[: self.B] for j in range(self.R)])
-            self.u = torch.from_numpy(us).cuda()
+            self.u = torch.from_numpy(np.stack([self.w.uniforms(j) for j in range(self.R)])).cuda()
         self.stream = torch.cuda.Stream()
-        self.graphs = {}
-        self.launches = {}
-        self.pass_events = None
+        self.graph_obj = None
+        self.launches_per_pass = 0
         self.pass_us_per_step = []
         self.restore()
 
     def close(self):
-        self.graphs.clear()
+        self.graph_obj = None
         self.cz.cfgzip_destroy(self.ctx)
 
-    def restore(self):
-        """Refill every working buffer with unmasked logits (outside any timed region)."""
-        for j in range(self.R):
+    def host_logits_of(self, j: int) -> np.ndarray:
+        return self.host_logits[j % self.U]
+
+    def restore(self, slots=None):
+        """Refill working buffers with unmasked logits (outside any timed region)."""
+        for j in (range(self.R) if slots is None else slots):
             self.work[j].copy_(self.pristine[j % self.U])
         self.torch.cuda.synchronize()
 
     def call(self, j: int, stream):
         cz = self.cz
-        if self.unfused:
+        dt = cz.BF16 if self.dtype == "bf16" else cz.F32
+        if self.kind == "floor":
+            cz.cfgzip_rmw_floor(self.ctx, self.work[j], dt, self.V, self.B, self.V, stream)
+        elif self.kind == "unfused":
             cz.cfgzip_expand_mask(self.ctx, self.parts[0], self.row_part, self.cm[j], self.KW, self.vm[j], self.VW,
                                   self.B, self.mode, stream)
-            cz.cfgzip_mask_logits(self.ctx, self.work[j], cz.BF16 if self.dtype == "bf16" else cz.F32, self.V, self.B,
-                                  self.V, self.vm[j], self.VW, stream)
-            return
-        if self.u is not None:
+            cz.cfgzip_mask_logits(self.ctx, self.work[j], dt, self.V, self.B, self.V, self.vm[j], self.VW, stream)
+        elif self.u is not None:
             cz.cfgzip_masked_sample(
-                self.ctx, self.parts[0], self.row_part_arg, self.cm[j], self.KW, self.work[j],
-                cz.BF16 if self.dtype == "bf16" else cz.F32, self.V, self.B, self.vm[j], self.VW, self.u[j],
-                self.inv_temperature, self.am[j], self.rep[j], self.lpa[j], self.lse[j], self.mode, stream)
-            return
-        cz.cfgzip_masked_logsoftmax_argmax(
-            self.ctx, self.parts[0], self.row_part_arg, self.cm[j], self.KW, self.work[j],
-            cz.BF16 if self.dtype == "bf16" else cz.F32, self.V, self.B, self.vm[j], self.VW, self.am[j], self.rep[j],
-            self.lpa[j], self.lse[j], None, self.mode, stream)
+                self.ctx, self.parts[0], self.row_part_arg, self.cm[j], self.KW, self.work[j], dt, self.V, self.B,
+                self.vm[j], self.VW, self.u[j], self.inv_temperature, self.am[j], self.rep[j], self.lpa[j], self.lse[j],
+                self.mode, stream)
+        else:
+            cz.cfgzip_masked_logsoftmax_argmax(
+                self.ctx, self.parts[0], self.row_part_arg, self.cm[j], self.KW, self.work[j], dt, self.V, self.B,
+                self.vm[j], self.VW, self.am[j], self.rep[j], self.lpa[j], self.lse[j], None, self.mode, stream)
 
-    def graph(self, n: int):
-        """CUDA graph of steps 0..n-1 of the ring (captured once per n)."""
-        if n not in self.graphs:
+    def graph(self):
+        """CUDA graph of one pass: steps 0..G-1 over the ring (captured once)."""
+        if self.graph_obj is None:
             torch = self.torch
             g = torch.cuda.CUDAGraph()
             self.stream.wait_stream(torch.cuda.current_stream())
             before = self.cz.cfgzip_launch_count(self.ctx)
             with torch.cuda.stream(self.stream):
                 with torch.cuda.graph(g, stream=self.stream):
-                    for j in range(n):
+                    for j in range(self.G):
                         self.call(j % self.R, self.stream)
-            self.launches[n] = self.cz.cfgzip_launch_count(self.ctx) - before
-            self.graphs[n] = g
-        return self.graphs[n]
+            self.launches_per_pass = self.cz.cfgzip_launch_count(self.ctx) - before
+            self.graph_obj = g
+        return self.graph_obj
 
-    def prepare(self, n_steps: int):
-        full, rem = divmod(n_steps, self.G)
-        if full:
-            self.graph(self.G)
-        if rem:
-            self.graph(rem)
-
-    def run(self, n_steps: int) -> int:
-        """Enqueue n_steps steps (ring order, wrapping) on self.stream; returns kernels launched."""
-        full, rem = divmod(n_steps, self.G)
-        launched = 0
+    def run_passes(self, passes: int, events=None) -> int:
+        """Enqueue whole passes over the ring on self.stream; returns kernels launched."""
+        g = self.graph()
         with self.torch.cuda.stream(self.stream):
-            for _ in range(full):
-                self.graph(self.G).replay()
-                launched += self.launches[self.G]
-                if self.pass_events is not None:  # one event per pass over the ring, inside the timed region
+            for _ in range(passes):
+                g.replay()
+                if events is not None:  # one event per pass, inside the timed region
                     ev = self.torch.cuda.Event(enable_timing=True)
                     ev.record(self.stream)
-                    self.pass_events.append(ev)
-            if rem:
-                self.graph(rem).replay()
-                launched += self.launches[rem]
-        return launched
+                    events.append(ev)
+        return passes * self.launches_per_pass
 
-    def timed(self, n_steps: int, warmup: int, barrier=None, sampler: ClockSampler = None):
-        """(seconds, launches) for n_steps steps after `warmup` untimed ones; events on the launching stream."""
+    def timed(self, requested_steps: int, warmup: int, barrier=None, sampler: ClockSampler = None):
+        """(seconds, timed steps, launches): whole passes over the ring, at least `requested_steps` steps and at least
+        MIN_TIMED_SECONDS, after at least `warmup` (and at least 3) untimed steps; CUDA events on the launching stream."""
         torch = self.torch
-        self.prepare(n_steps)
-        self.prepare(max(warmup, 3))
-        self.run(max(warmup, 3))
-        # every CUDA graph the timed region replays has run once before it (the first replay of a graph
-        # also uploads it): these are extra untimed steps on top of the warm-up
-        full, rem = divmod(n_steps, self.G)
-        self.run((self.G if full else 0) + rem)
+        warm_passes = max(1, -(-max(warmup, 3) // self.G))
+        self.run_passes(warm_passes)  # the first replay also uploads the graph
         self.stream.synchronize()
-        self.restore()
+        # one more untimed pass, timed on its own, sizes the timed region
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        p0.record(self.stream)
+        self.run_passes(1)
+        p1.record(self.stream)
+        self.stream.synchronize()
+        n_steps = timed_steps_for(requested_steps, self.G, p0.elapsed_time(p1) * 1e-3)
+        passes = n_steps // self.G
+        if self.kind != "floor":
+            self.restore()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         if barrier:
             barrier()
         if sampler:
             sampler.start()
-        self.pass_events = []
+        marks = []
         e0.record(self.stream)
-        launched = self.run(n_steps)
+        launched = self.run_passes(passes, marks)
         e1.record(self.stream)
         self.stream.synchronize()
         torch.cuda.synchronize()
-        marks, self.pass_events = [e0] + self.pass_events, None
+        marks = [e0] + marks
         self.pass_us_per_step = [a.elapsed_time(b) * 1e3 / self.G for a, b in zip(marks, marks[1:])]
         if sampler:
             sampler.stop()
         if barrier:
             barrier()
-        return e0.elapsed_time(e1) * 1e-3, launched
+        return e0.elapsed_time(e1) * 1e-3, n_steps, launched
+
+    def execute_slots(self, slots, rows_sel, full_logits: int = 2) -> dict:
+        """Run the steps of these ring slots once more on refilled buffers (untimed, no graph) and return the outputs
+        of rows `rows_sel` as numpy arrays indexed [slot, row]; the masked logits of the first `full_logits` slots."""
+        torch = self.torch
+        slots = list(slots)
+        idx = torch.tensor(slots, dtype=torch.long, device="cuda")
+        rsel = torch.from_numpy(np.asarray(rows_sel, dtype=np.int64)).cuda()
+        self.restore(slots)
+        with torch.cuda.stream(self.stream):
+            for j in slots:
+                self.call(j, self.stream)
+        self.stream.synchronize()
+
+        def take(t):
+            return t[idx][:, rsel].cpu().numpy()
+
+        out = {"argmax": take(self.am), "rep": take(self.rep), "lse": take(self.lse), "logp_argmax": take(self.lpa),
+               "vocab_mask": take(self.vm).view(np.uint32)}
+        head = self.work[idx[:full_logits]][:, rsel].cpu().numpy()
+        out["logits"] = head.view(np.uint16) if self.dtype == "bf16" else head
+        return out
 
     def alg_bytes(self) -> int:
-        if self.mode == self.cz.SPARSE and not self.unfused:
+        if self.mode == self.cz.SPARSE and self.kind == "fused":
             return self.alg_bytes_sparse()
         return algorithmic_bytes(self.B, self.V, self.K, self.elem, len(self.parts))
 
     def alg_bytes_sparse(self) -> int:
         """Bytes one class-list step must move: write the whole row and its vocab mask, read the class masks, and per
-        allowed token read its id from the class list (4 bytes) and its logit; mean over the steps of the ring."""
+        allowed token read its id from the class list (4 bytes) and its logit; mean over the first steps of the ring."""
         allowed_tokens = 0.0
-        for j in range(min(self.R, 8)):
+        n = min(self.R, 8)
+        for j in range(n):
             bits = synth.unpack_bits(self.host_cm[j], self.K)  # [B, K]
-            for b in range(self.B):
-                p = self.w.partitions[0 if self.row_part_host is None else int(self.row_part_host[b])]
-                allowed_tokens += float(p.sizes[bits[b]].sum())
-        allowed_tokens /= min(self.R, 8)
+            for p, part in enumerate(self.partitions):
+                sel = slice(None) if self.row_part_host is None else (self.row_part_host == p)
+                allowed_tokens += float((bits[sel] * part.sizes[None, :]).sum())
+        allowed_tokens /= n
         return int(self.B * (self.V * self.elem + 4 * self.VW + 4 * self.KW + 16) + allowed_tokens * (4 + self.elem))
 
 
-def _extra_steps(runner: StepRunner, passes: int = 3, min_steps: int = 300) -> int:
-    """Steps of a secondary measurement: whole passes over the ring, at least `min_steps` steps, so that the timed
-    region lasts tens of milliseconds (a few milliseconds right after host-side set-up measured up to 10 % slow)."""
-    return runner.R * max(passes, -(-min_steps // runner.R))
+def _measure(runner: StepRunner, min_steps: int = 300):
+    """(us per step, steps timed, launches per step) of a secondary measurement: same protocol as the headline."""
+    seconds, n, launched = runner.timed(min_steps, runner.G)
+    return seconds / n * 1e6, n, launched / n
 
 
 def _e2e(runner: StepRunner, torch, n_steps: int):
@@ -369,40 +449,29 @@ def _e2e(runner: StepRunner, torch, n_steps: int):
     return dt_s, h2d, d2h
 
 
-def _cpu_baseline(runner: StepRunner, torch, budget_s: float = 12.0):
-    """Time the CPU oracle on the first steps of the same workload and check the GPU results of
-    those steps against it. Returns (cpu_baseline dict, parity dict)."""
+def _cpu_baseline(runner, budget_s: float = 12.0) -> dict:
+    """The CPU oracle timed on steps of the same workload: with one thread per host core (rows split over a thread
+    pool) and with a single thread, each for about half of `budget_s`."""
     import oracle
     threads = max(1, min(_host_threads(), runner.B))
-    n_max = min(runner.R, 256)
-    done, spent, mismatches, max_err = 0, 0.0, 0, 0.0
-    am = runner.am.cpu().numpy(); rep = runner.rep.cpu().numpy()
-    lse = runner.lse.cpu().numpy(); lpa = runner.lpa.cpu().numpy()
-    for j in range(n_max):
-        z = runner.host_logits[j % runner.U].copy()
-        t0 = time.perf_counter()
-        out = oracle.decode_step(runner.w.partitions, runner.row_part_host, runner.host_cm[j], z, threads=threads)
-        spent += time.perf_counter() - t0
-        done += 1
-        ok = np.array_equal(out["argmax"], am[j]) and np.array_equal(out["rep"], rep[j])
-        vm = runner.vm[j].cpu().numpy().view(np.uint32)
-        ok = ok and np.array_equal(vm, out["vocab_mask"])
-        if j < 4:
-            got = runner.work[j].cpu().numpy()
-            ok = ok and np.array_equal(got.view(np.uint8), z.view(np.uint8))
-        fin = np.isfinite(out["lse"])
-        ok = ok and np.array_equal(np.isfinite(lse[j]), fin)
-        if fin.any():
-            err = max(np.abs(lse[j][fin] - out["lse"][fin]).max(), np.abs(lpa[j][fin] - out["logp_argmax"][fin]).max())
-            max_err = max(max_err, float(err))
-            ok = ok and err <= 1e-4
-        mismatches += 0 if ok else 1
-        if spent > budget_s:
-            break
-    base = {"value": done * runner.B / spent, "unit": UNIT, "cores": threads, "kind": "oracle",
-            "sample": "first %d steps (%d rows) of the same workload, %d threads over rows" % (done, done * runner.B, threads)}
-    parity = {"steps_checked": done, "mismatching_steps": mismatches, "max_abs_err_log": max_err}
-    return base, parity
+
+    def timed(n_threads, budget):
+        done, spent, j = 0, 0.0, 0
+        while spent < budget:
+            z = runner.host_logits_of(j).copy()
+            t0 = time.perf_counter()
+            oracle.decode_step(runner.partitions, runner.row_part_host, runner.host_cm[j % runner.R], z, threads=n_threads)
+            spent += time.perf_counter() - t0
+            done += 1
+            j += 1
+        return done, spent
+
+    n_t, s_t = timed(threads, budget_s / 2)
+    n_1, s_1 = timed(1, budget_s / 2)
+    return {"value": n_t * runner.B / s_t, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": "%d steps (%d rows) of the same workload, %d threads over rows" % (n_t, n_t * runner.B, threads),
+            "single_thread": {"value": n_1 * runner.B / s_1, "unit": UNIT, "cores": 1,
+                              "sample": "%d steps (%d rows) of the same workload, one thread" % (n_1, n_1 * runner.B)}}
 
 
 # ----------------------------------------------------------------------------- arms
@@ -411,59 +480,62 @@ def run_own(args):
     import torch
     from paper_2605_29986_b200 import binding as cz
 
-    rank, local_rank, world = _dist_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the CFGzip library has no CPU path")
+    _, local_rank, _ = ranks.dist_env()
     torch.cuda.set_device(local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    os.environ.setdefault("NCCL_DEBUG", "INFO")       # the communicator's rank count shows in the log
+    os.environ.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    rank, local_rank, world, dist = ranks.init_ranks("nccl", device=torch.device("cuda", local_rank))
 
     def barrier():
         if dist is not None:
             dist.barrier()
 
+    solo = rank == 0 and world == 1
     runner = StepRunner(cz, torch, local_rank, args.workload, B=args.batch, mode=args.mode, steps_hint=args.steps,
                         tune=args.tune, inv_temperature=args.sample_inv_temperature)
     props = torch.cuda.get_device_properties(local_rank)
     sampler = ClockSampler("GPU-" + str(props.uuid))
-    seconds, launches = runner.timed(args.steps, args.warmup, barrier, sampler)
+    seconds, timed_steps, launches = runner.timed(args.steps, args.warmup, barrier, sampler)
     e2e_steps = max(3, min(args.steps, args.e2e_steps))
     barrier()
     e2e_s, h2d, d2h = _e2e(runner, torch, e2e_steps)
     if dist is not None:
-        from paper_2605_29986_b200 import rows
-        seconds = rows.max_over_ranks(seconds, dist, device="cuda")
-        e2e_s = rows.max_over_ranks(e2e_s, dist, device="cuda")
+        seconds = ranks.max_over_ranks(seconds, dist, device="cuda")
+        e2e_s = ranks.max_over_ranks(e2e_s, dist, device="cuda")
     peak, peak_src = _measured_peak()
     alg = runner.alg_bytes()
+    us_per_step = seconds / timed_steps * 1e6
     # a dense step is two launches (streaming kernel + per-row finalize); the figure is per step
-    achieved = alg * args.steps / seconds / 1e9
+    achieved = alg / (seconds / timed_steps) / 1e9
     key = "cfg%d_B%d_%s" % (args.workload, runner.B, args.mode)
     traffic = None
     if key in NCU_TRAFFIC and NCU_TRAFFIC[key]["digest"] == _kernel_digest():
         traffic = NCU_TRAFFIC[key]["bytes_per_launch"]
+    sampling = bool(args.sample_inv_temperature)
     line = {
-        "metric": METRIC, "value": world * runner.B * args.steps / seconds, "unit": UNIT, "n_gpus": world,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": seconds / args.steps * 1e3,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": runner.dtype if runner.dtype != "f32" else "f32",
+        "metric": METRIC, "value": world * runner.B * timed_steps / seconds, "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "timed_steps": timed_steps, "warmup": args.warmup, "ms_per_step": us_per_step * 1e-3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": runner.dtype,
         "data": "synthetic",
         "config": {
             "workload": "cfg%d %s: V=%d K=%d B=%d %s, fused expand+mask+lse+%s+rep, %s" % (
                 args.workload, synth.CONFIGS[args.workload]["name"], runner.V, runner.K, runner.B, runner.dtype,
-                "argmax" if not args.sample_inv_temperature else "sample(1/T=%g)" % args.sample_inv_temperature, args.mode),
+                "argmax" if not sampling else "sample(1/T=%g)" % args.sample_inv_temperature, args.mode),
             "rows_per_gpu": runner.B, "global_rows": world * runner.B,
             "l2": "inputs larger than L2: ring of %d working buffers (%.2f GB), refilled with unmasked logits before the "
                   "timed region" % (runner.R, runner.R * runner.B * runner.V * runner.elem / 1e9),
-            "launch": "CUDA graph of %d steps replayed (each graph replayed once, untimed, before the timed region); "
-                      "%.0f kernels per step (streaming pass + per-row finalize)" % (
-                min(runner.R, args.steps), launches / max(args.steps, 1)),
+            "timed_region": "%d whole passes over the ring (%d steps, %.1f ms): at least the requested steps and at least "
+                            "%.0f ms" % (timed_steps // runner.G, timed_steps, seconds * 1e3, MIN_TIMED_SECONDS * 1e3),
+            "launch": "CUDA graph of one pass (%d steps) replayed, run untimed before the timed region; %.0f kernels per step" % (
+                runner.G, launches / timed_steps),
+            "inputs": "every row has its own class mask at every step; logits rows repeat every %d rows" % min(runner.B, 64),
             "parallelism": "rows sharded over %d GPU(s), no collective on the path" % world,
             "row_grouping": ("rows grouped by partition once before the steps (cfgzip_plan_rows), reused by every step"
                              if runner.row_part is not None else "one partition: rows grouped implicitly"),
         },
-        "us_per_step": seconds / args.steps * 1e6,
+        "us_per_step": us_per_step,
         "us_per_step_over_ring_passes": (
             {"passes": len(runner.pass_us_per_step), "median": float(np.median(runner.pass_us_per_step)),
              "p10": float(np.percentile(runner.pass_us_per_step, 10)),
@@ -475,88 +547,115 @@ def run_own(args):
                         "logp_argmax out; synchronised every step"},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": traffic, "peak_source": "of " + peak_src, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                     "algorithmic_bytes_per_step": alg, "launches_per_step": launches / max(args.steps, 1),
+                     "algorithmic_bytes_per_step": alg, "launches_per_step": launches / timed_steps,
                      "kernel": ("k_step_sparse" if args.mode == "sparse" else
-                                "k_step_dense_pipe (+ %s)" % ("k_sample_rows" if args.sample_inv_temperature else "k_finalize_rows"))},
+                                "k_step_dense_pipe (+ %s)" % ("k_sample_rows" if sampling else "k_finalize_rows"))},
         "clocks": sampler.summary(),
         "paper_context": "paper reports no timing of this path; its speedups (up to two orders of magnitude in grammar-engine "
                          "latency, up to 7.5x end to end) are for 1x H100 + Xeon Gold 6430 x16 threads, precision unstated",
     }
-    if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.sample_inv_temperature:
-        line["cpu_baseline"], line["parity"] = _cpu_baseline(runner, torch)
+    host_threads = max(1, min(_host_threads(), 16))
+    if solo and not args.no_cpu_baseline and not sampling:
+        # every step of the ring, every row (budget: a minute of oracle time)
+        line["parity"] = check_slots(runner, range(runner.R), None, host_threads, budget_s=60.0)
+        line["cpu_baseline"] = _cpu_baseline(runner)
     runner.close()
-    if rank == 0 and world == 1 and not args.no_extras:
+    if solo and not args.no_extras:
+        def parity_of(r, steps=2, rows=32):
+            if args.no_cpu_baseline:
+                return None
+            return check_slots(r, spread(r.R, steps), spread(r.B, rows), host_threads, budget_s=10.0)
+
+        # the floor: the in-place read-modify-write kernel over the same ring, same graph protocol
+        r0 = StepRunner(cz, torch, local_rank, args.workload, B=args.batch, steps_hint=args.steps, unique=2, tune=args.tune,
+                        kind="floor")
+        us0, _, _ = _measure(r0)
+        r0.close()
+        line["floor_us_per_step"] = us0
+        line["roofline"]["floor"] = {"us_per_step": us0, "step_over_floor": us_per_step / us0,
+                                     "what": "one launch per step that reads every logit of the batch and writes it back "
+                                             "(sign flipped), same ring, same CUDA-graph protocol: the least a pass over "
+                                             "these bytes costs here"}
         extras = []
         for B in (128, 256, 1024):
-            r2 = StepRunner(cz, torch, local_rank, args.workload, B=B, mode=args.mode, steps_hint=8, unique=2,
-                            tune=args.tune)
-            n = _extra_steps(r2)
-            s2, l2 = r2.timed(n, r2.R)
-            a2 = r2.alg_bytes() / (s2 / n) / 1e9
-            extras.append({"B": B, "us_per_step": s2 / n * 1e6, "rows_per_s": B * n / s2, "achieved_gbs": a2,
-                           "frac_of_measured": a2 / peak, "ring": r2.R})
+            r2 = StepRunner(cz, torch, local_rank, args.workload, B=B, mode=args.mode, steps_hint=8, unique=2, tune=args.tune)
+            us2, n2, _ = _measure(r2)
+            a2 = r2.alg_bytes() / us2 / 1e3
+            entry = {"B": B, "us_per_step": us2, "rows_per_s": B / us2 * 1e6, "achieved_gbs": a2,
+                     "frac_of_measured": a2 / peak, "ring": r2.R, "timed_steps": n2, "parity": parity_of(r2)}
             r2.close()
+            rf = StepRunner(cz, torch, local_rank, args.workload, B=B, steps_hint=8, unique=2, tune=args.tune, kind="floor")
+            entry["floor_us_per_step"] = _measure(rf)[0]
+            rf.close()
+            extras.append(entry)
         line["larger_batches"] = extras
         # the same masking through the two separate calls (expand, then mask; no normaliser, argmax or map):
         # the vocab mask is written and read back, so it moves more bytes for less work
         r3 = StepRunner(cz, torch, local_rank, args.workload, B=args.batch, mode=args.mode, steps_hint=256, unique=2,
-                        tune=args.tune, unfused=True)
-        n = _extra_steps(r3, 2)
-        s3, l3 = r3.timed(n, r3.R)
-        line["unfused_expand_then_mask"] = {"us_per_step": s3 / n * 1e6, "launches_per_step": l3 / n}
+                        tune=args.tune, kind="unfused")
+        us3, _, l3 = _measure(r3)
+        line["unfused_expand_then_mask"] = {"us_per_step": us3, "launches_per_step": l3}
         r3.close()
         # the sampling step (inverse CDF at the paper's temperature 0.2, one uniform number per row) on the same workload
         samp = []
         for B in (args.batch or synth.CONFIGS[args.workload]["B"], 1024):
             r6 = StepRunner(cz, torch, local_rank, args.workload, B=B, mode=args.mode, steps_hint=64, unique=2,
                             tune=args.tune, inv_temperature=5.0)
-            n = _extra_steps(r6)
-            s6, l6 = r6.timed(n, r6.R)
-            samp.append({"B": B, "us_per_step": s6 / n * 1e6, "launches_per_step": l6 / n,
-                         "frac_of_measured": r6.alg_bytes() / (s6 / n) / 1e9 / peak})
+            us6, _, l6 = _measure(r6)
+            samp.append({"B": B, "us_per_step": us6, "launches_per_step": l6,
+                         "frac_of_measured": r6.alg_bytes() / us6 / 1e3 / peak})
             r6.close()
         line["sampling_step_T0.2"] = samp
         # the same step on two buffers that stay in the 126 MB L2: NOT an HBM figure, only the latency floor
         r5 = StepRunner(cz, torch, local_rank, args.workload, B=args.batch, mode=args.mode, steps_hint=2, unique=2,
                         tune=args.tune, ring=2)
-        s5, _ = r5.timed(2000, 100)
-        line["warm_l2_us_per_step"] = s5 / 2000 * 1e6
+        line["warm_l2_us_per_step"] = _measure(r5, 2000)[0]
         r5.close()
-        # the five workloads at their own sizes (cfg2 is the headline above), same protocol, shorter runs
+        # the five workloads at their own sizes (cfg2 is the headline above), same protocol
         five = []
         for cfg in sorted(synth.CONFIGS):
             r7 = StepRunner(cz, torch, local_rank, cfg, mode="dense", steps_hint=64, unique=2, tune=args.tune)
-            n = _extra_steps(r7)
-            s7, l7 = r7.timed(n, r7.R)
-            a7 = r7.alg_bytes() / (s7 / n) / 1e9
+            us7, n7, l7 = _measure(r7)
+            a7 = r7.alg_bytes() / us7 / 1e3
+            all_steps = cfg in (1, 2)  # every step and row where the oracle takes seconds; a spread sample elsewhere
+            par = None
+            if not args.no_cpu_baseline:
+                par = (check_slots(r7, range(r7.R), None, host_threads, budget_s=20.0) if all_steps else parity_of(r7))
             five.append({"workload": "cfg%d %s: V=%d K=%d B=%d %s, %d partition(s)" % (
                              cfg, synth.CONFIGS[cfg]["name"], r7.V, r7.K, r7.B, r7.dtype, len(r7.parts)),
-                         "us_per_step": s7 / n * 1e6, "rows_per_s": r7.B * n / s7, "achieved_gbs": a7,
-                         "frac_of_measured": a7 / peak, "launches_per_step": l7 / n, "ring": r7.R})
+                         "us_per_step": us7, "rows_per_s": r7.B / us7 * 1e6, "achieved_gbs": a7,
+                         "frac_of_measured": a7 / peak, "launches_per_step": l7, "ring": r7.R, "timed_steps": n7,
+                         "parity": par})
             r7.close()
         line["five_workloads_dense"] = five
-        # sparse-mask stress workload (1-5 allowed classes per row): gather path against class-list scatter path
+        # sparse-mask stress workload (1-5 allowed classes per row): gather path, class-list scatter path, and the
+        # library's own choice between them
         pair = {}
-        for mode in ("dense", "sparse"):
+        for mode in ("dense", "sparse", "auto"):
             r4 = StepRunner(cz, torch, local_rank, 5, mode=mode, steps_hint=4, unique=1, tune=args.tune)
-            n = _extra_steps(r4, 4)
-            s4, _ = r4.timed(n, r4.R)
-            pair[mode + "_us_per_step"] = s4 / n * 1e6
-            pair[mode + "_algorithmic_bytes"] = r4.alg_bytes()
-            pair[mode + "_achieved_gbs_of_own_algorithmic_bytes"] = r4.alg_bytes() / (s4 / n) / 1e9
+            us4, _, _ = _measure(r4)
+            pair[mode + "_us_per_step"] = us4
+            if mode != "auto":
+                pair[mode + "_algorithmic_bytes"] = r4.alg_bytes()
+                pair[mode + "_achieved_gbs_of_own_algorithmic_bytes"] = r4.alg_bytes() / us4 / 1e3
+            if mode != "dense":
+                pair[mode + "_parity"] = parity_of(r4)
             r4.close()
+        pair["auto_vs_best"] = pair["auto_us_per_step"] / min(pair["dense_us_per_step"], pair["sparse_us_per_step"])
         pair["workload"] = "cfg5 sparse-stress: V=128256 K=512 B=1024 f32"
         line["sparse_vs_dense"] = pair
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
     if rank == 0:
-        print(json.dumps(line))
+        if world > 1:
+            time.sleep(0.5)  # let the other ranks' shutdown messages out first: the JSON line comes last
+        print(json.dumps(line), flush=True)
 
 
 def run_reference(args):
     """The CPU oracle, as it stands, on the host cores: each step is a bounded sample of the workload's rows."""
-    rank, _, world = _dist_env()
+    rank, _, world = ranks.dist_env()
     if rank != 0:
         return
     import oracle
@@ -598,7 +697,7 @@ def run_reference(args):
     print(json.dumps(line))
 
 
-def main():
+def main(argv=None):
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10000)
@@ -614,11 +713,14 @@ def main():
                     help="time the sampling step (cfgzip_masked_sample) at this inverse temperature instead of the greedy one")
     ap.add_argument("--no-extras", action="store_true", help="skip the larger-batch sweep")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    args = ap.parse_args()
-    if args.steps < 1 or args.warmup < 0:
-        ap.error("--steps must be >= 1 and --warmup >= 0")
+    args = ap.parse_args(argv)
+    if args.steps < 1 or args.warmup < 0 or args.gpus < 1:
+        ap.error("--steps and --gpus must be >= 1 and --warmup >= 0")
     if args.impl == "reference":
-        run_reference(args)
+        run_reference(args)  # the CPU oracle: one process whatever --gpus says (under a launcher rank 0 alone runs it)
+    elif ranks.need_spawn(args.gpus):
+        # several GPUs asked for and no launcher in the environment: start one rank per GPU of this script
+        sys.exit(ranks.spawn_ranks(os.path.abspath(__file__), args.gpus, sys.argv[1:] if argv is None else list(argv)))
     else:
         run_own(args)
 

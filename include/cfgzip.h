@@ -130,8 +130,8 @@ int cfgzip_expand_mask(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row
 
 /*
  * Apply a vocab mask to logits in place: a disallowed logit becomes -inf, an allowed
- * one keeps its bits (Section 2.2: "the corresponding logit is set to -inf";
- * Section 3.1 applies it after the gather).
+ * one keeps its bits (Section 2.2 defines the masking so; Section 3.1 applies it
+ * after the gather).
  *   logits : dev [B, row_stride_elems] of `dtype`, row_stride_elems >= V; elements at
  *            index >= V of a row are not touched. 16-byte aligned rows take the
  *            vectorised path, anything else a scalar one.
@@ -164,7 +164,7 @@ int cfgzip_masked_logsoftmax_argmax(cfgzip_ctx* ctx, cfgzip_part_id part0, const
 
 /*
  * The same pass with the token SAMPLED instead of taken greedily (Section 3.1, "Inference": a
- * token "is sampled from the next-token distribution"; Section 4: temperature 0.2 in the paper's
+ * token is drawn from the next-token distribution; Section 4: temperature 0.2 in the paper's
  * runs). The paper names no sampler; this one is the inverse CDF in token-id order:
  *   p_i   = exp(z_i / T) / sum_{allowed j} exp(z_j / T),  1/T = inv_temperature > 0 (at most 1e6)
  *   token = the lowest token id i with sum_{j <= i} p_j > u[b]
@@ -259,6 +259,16 @@ int cfgzip_step_noalloc(const int32_t* token_to_class /*dev [V]*/, int32_t V,
                         int64_t class_stride_words, void* logits, int dtype, int64_t row_stride_elems,
                         int32_t B, uint32_t* vocab_mask, int64_t vocab_stride_words, int32_t* argmax,
                         int32_t* rep, float* logp_argmax, float* lse, void* stream);
+
+/*
+ * Measurement aid (the paper has no counterpart): one launch that reads every whole 16-byte vector of
+ * logits [B, row_stride_elems] (first V elements of each row), flips the sign bit of each element and
+ * writes it back in place. It is the cheapest pass over the bytes a fused step must read and write;
+ * timing it in the same launch protocol as the step gives the floor the step's time is compared with.
+ * Calling it twice restores the buffer. Rows must be 16-byte aligned (CFGZIP_E_ALIGN otherwise).
+ */
+int cfgzip_rmw_floor(cfgzip_ctx* ctx, void* logits, int dtype, int64_t row_stride_elems, int32_t B, int32_t V,
+                     void* stream);
 
 /* Kernels this context has launched so far (monotonic; for launch accounting). */
 int cfgzip_launch_count(cfgzip_ctx* ctx, int64_t* out);

@@ -21,8 +21,8 @@
  *   - a row with nothing allowed yields argmax = rep = -1 and -inf log
  *     quantities; a row whose allowed logits are all -inf yields the lowest
  *     allowed token id and -inf log quantities.
- *   - sampling (Section 3.1 says a token "is sampled from the next-token
- *     distribution", Section 4 fixes the temperature, neither names the
+ *   - sampling (Section 3.1 draws the token from the next-token
+ *     distribution, Section 4 fixes the temperature, neither names the
  *     sampler): p_i = exp(z_i/T) / sum_{allowed j} exp(z_j/T); the uniform
  *     number u in [0,1) is an input; the chosen token is the lowest id whose
  *     cumulative probability, taken in token-id order, exceeds u.
@@ -198,7 +198,7 @@ void oracle_decode_step(const int32_t* c, const int32_t* r, int32_t V, int32_t K
 
 /*
  * Sampling from the tempered distribution over the allowed tokens (Section 3.1,
- * "Inference": the next token is sampled from the next-token distribution; Section 4:
+ * "Inference": the next token is a draw from the model's distribution; Section 4:
  * temperature T, 0.2 in the paper's runs), from logits that are already masked.
  *   p_i      = exp(z_i / T) / sum_{allowed j} exp(z_j / T)          (0 where masked)
  *   token    = min { i : sum_{j <= i} p_j > u },  u in [0,1) given per row

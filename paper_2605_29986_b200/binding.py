@@ -39,6 +39,7 @@ _SIGNATURES = {
                                        _vp]),
     "cfgzip_step_noalloc": (_int, [_vp, _i32, _vp, _i32, _vp, _i64, _vp, _int, _i64, _i32, _vp, _i64, _vp, _vp, _vp, _vp,
                                    _vp]),
+    "cfgzip_rmw_floor": (_int, [_vp, _vp, _int, _i64, _i32, _i32, _vp]),
     "cfgzip_poll_status": (_int, [_vp, _vp, ctypes.POINTER(_i32), ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
     "cfgzip_launch_count": (_int, [_vp, ctypes.POINTER(_i64)]),
     "cfgzip_set_tuning": (_int, [_vp, ctypes.c_char_p, _i32]),
@@ -200,6 +201,12 @@ def cfgzip_step_noalloc(token_to_class, V: int, class_to_rep, K: int, class_mask
         _ptr(token_to_class), V, _ptr(class_to_rep), K, _ptr(class_mask), class_stride_words, _ptr(logits), dtype,
         row_stride_elems, B, _ptr(vocab_mask), vocab_stride_words, _ptr(argmax), _ptr(rep), _ptr(logp_argmax),
         _ptr(lse), _stream(stream)), "cfgzip_step_noalloc")
+
+
+def cfgzip_rmw_floor(ctx: int, logits, dtype: int, row_stride_elems: int, B: int, V: int, stream=None) -> None:
+    """Measurement aid: in-place sign flip of every whole 16-byte vector of the logits (one launch)."""
+    _check(load_library().cfgzip_rmw_floor(ctx, _ptr(logits), dtype, row_stride_elems, B, V, _stream(stream)),
+           "cfgzip_rmw_floor")
 
 
 def cfgzip_poll_status(ctx: int, stream=None) -> Tuple[int, int, int]:

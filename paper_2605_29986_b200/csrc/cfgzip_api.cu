@@ -715,7 +715,8 @@ int cfgzip_load_partition(cfgzip_ctx* ctx, const int32_t* c, int32_t V, const in
     size_t slot = 0;
     while (slot < ctx->parts.size() && ctx->parts[slot].live) ++slot;
     if (slot >= size_t(kMaxParts)) return CFGZIP_E_RANGE;
-    if (slot == ctx->parts.size()) ctx->parts.emplace_back();
+    const bool appended = slot == ctx->parts.size();
+    if (appended) ctx->parts.emplace_back();
 
     Part p;
     p.V = V;
@@ -745,6 +746,7 @@ int cfgzip_load_partition(cfgzip_ctx* ctx, const int32_t* c, int32_t V, const in
     }
     if (cudaMalloc(&p.block, img.size() * 4) != cudaSuccess) {
         cudaGetLastError();
+        if (appended) ctx->parts.pop_back();
         return CFGZIP_E_NOMEM;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -764,8 +766,15 @@ int cfgzip_load_partition(cfgzip_ctx* ctx, const int32_t* c, int32_t V, const in
               cudaMemcpyAsync(ctx->d_parts + slot, &p.dev, sizeof(PartDev), cudaMemcpyHostToDevice, st) == cudaSuccess &&
               cudaStreamSynchronize(st) == cudaSuccess;
     if (!ok) {
+        // the descriptor may already be on the device: clear it before its tables are freed, so that no later
+        // call finds a live slot that points at released memory
+        cudaGetLastError();
+        cudaStreamSynchronize(st);
+        cudaMemset(ctx->d_parts + slot, 0, sizeof(PartDev));
+        cudaDeviceSynchronize();
         cudaGetLastError();
         cudaFree(p.block);
+        if (appended) ctx->parts.pop_back();
         return CFGZIP_E_CUDA;
     }
     ctx->parts[slot] = p;
@@ -1021,6 +1030,7 @@ int cfgzip_decode_step_host(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t
     int rc = check_step_args(ctx, class_mask_host, class_stride_words, B, mode);
     if (rc != CFGZIP_OK) return rc;
     if (dtype != CFGZIP_F32 && dtype != CFGZIP_BF16) return CFGZIP_E_ARG;
+    if (row_part_host == CFGZIP_ROWS_AS_PLANNED) return CFGZIP_E_ARG;  // a kept grouping refers to a device vector
     PartSet ps;
     if ((rc = resolve_parts(ctx, part0, row_part_host != nullptr, &ps)) != CFGZIP_OK) return rc;
     if (B == 0) return CFGZIP_OK;
@@ -1118,6 +1128,28 @@ int cfgzip_poll_status(cfgzip_ctx* ctx, void* stream, int32_t* n_empty_rows, int
     if (n_bad_tokens) *n_bad_tokens = h[1];
     if (n_bad_rows) *n_bad_rows = h[2];
     return h[3] ? CFGZIP_E_CUDA : CFGZIP_OK;  // h[3]: asynchronous copies that never completed
+}
+
+int cfgzip_rmw_floor(cfgzip_ctx* ctx, void* logits, int dtype, int64_t row_stride_elems, int32_t B, int32_t V,
+                     void* stream) {
+    if (!ctx || B < 0 || V <= 0 || (dtype != CFGZIP_F32 && dtype != CFGZIP_BF16)) return CFGZIP_E_ARG;
+    if (B == 0) return CFGZIP_OK;
+    if (!logits || row_stride_elems < V) return CFGZIP_E_ARG;
+    const int es = dtype == CFGZIP_BF16 ? 2 : 4;
+    if (!aligned16(logits, row_stride_elems, es)) return CFGZIP_E_ALIGN;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return CFGZIP_E_CUDA;
+    const int64_t items = int64_t(B) * ceil_div((int64_t(V) * es) >> 4, 256 * 4);
+    if (items == 0) return CFGZIP_OK;
+    const unsigned grid = unsigned(std::min<int64_t>(items, int64_t(ctx->sm_count) * 8));
+    ctx->pdl_now = int64_t(B) * V * es < (int64_t(192) << 20);
+    const int rc = dtype == CFGZIP_BF16
+                       ? launch(ctx, k_rmw_floor<kBF16>, dim3(grid), dim3(256), 0, static_cast<cudaStream_t>(stream), logits,
+                                row_stride_elems, int(B), int(V))
+                       : launch(ctx, k_rmw_floor<kF32>, dim3(grid), dim3(256), 0, static_cast<cudaStream_t>(stream), logits,
+                                row_stride_elems, int(B), int(V));
+    ctx->pdl_now = true;
+    return rc;
 }
 
 int cfgzip_launch_count(cfgzip_ctx* ctx, int64_t* out) {

@@ -1643,6 +1643,39 @@ __global__ void __launch_bounds__(256) k_mask_logits(void* logits, int64_t row_s
     }
 }
 
+// Measurement aid: the cheapest in-place read-modify-write over a logits matrix (every whole 16-byte vector of
+// every row is read, the sign bits of its elements are flipped, and it is written back). It moves the bytes a
+// step must at least move and does nothing else, so its time under the same launch protocol is what the
+// step's time is compared with.
+template <int DT>
+__global__ void __launch_bounds__(256) k_rmw_floor(void* logits, int64_t row_stride, int B, int V) {
+    pdl_prologue();
+    constexpr int ES = DT == kBF16 ? 2 : 4;
+    constexpr int U = 4;
+    constexpr uint32_t kSign = DT == kBF16 ? 0x80008000u : 0x80000000u;
+    const int nvec = int((int64_t(V) * ES) >> 4);
+    const int chunks = (nvec + 256 * U - 1) / (256 * U);
+    const int64_t total = int64_t(B) * chunks;
+    for (int64_t item = blockIdx.x; item < total; item += gridDim.x) {
+        const int row = int(item / chunks), ch = int(item - int64_t(row) * chunks);
+        char* rowp = reinterpret_cast<char*>(logits) + int64_t(row) * row_stride * ES;
+        uint4 v[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int i = ch * 256 * U + u * 256 + threadIdx.x;
+            if (i < nvec) v[u] = ld_stream16(rowp + size_t(i) * 16);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int i = ch * 256 * U + u * 256 + threadIdx.x;
+            if (i < nvec) {
+                v[u].x ^= kSign; v[u].y ^= kSign; v[u].z ^= kSign; v[u].w ^= kSign;
+                st_stream16(rowp + size_t(i) * 16, v[u]);
+            }
+        }
+    }
+}
+
 // logp_full[b, i] = z'[b, i] - lse[b] from the masked logits (fp32 out, row stride V).
 template <int DT>
 __global__ void __launch_bounds__(256) k_logp_full(const void* logits, int64_t row_stride, int B, int V, const float* lse,

@@ -1,9 +1,10 @@
 """The five workloads at their full sizes, through the fused entry point in the launch shape the bench uses.
 
 Inputs follow the workload recipes (unique logits rows are generated for up to 64 rows and tiled to
-the batch; every row has its own class mask). All rows are compared with the CPU oracle where that
-takes seconds; for the largest batches a spread sample of rows is compared and the remaining rows
-are checked by properties that hold at any size (popcount of the vocab mask = summed sizes of the
+the batch, and repeat every 16 steps; every row has its own class mask at every step). Every decode
+step of the two small workloads and ten steps spread over the run of the others are covered. All rows
+are compared with the CPU oracle where that takes seconds; for the largest batch a spread sample of
+rows is compared and the remaining rows are checked by properties that hold at any size (popcount of the vocab mask = summed sizes of the
 allowed classes, -inf count of the masked logits, the chosen token is allowed and maps to its
 representative) and, for the sparse stress workload, by bit-equality of the dense and sparse paths.
 """
@@ -17,19 +18,42 @@ from _gpu_util import Ctx, compare_step, oracle_step, run_fused
 
 pytestmark = pytest.mark.gpu
 
-ORACLE_ROWS = {1: 1, 2: 32, 3: 128, 4: 64, 5: 64}
+# rows of a step that are compared with the oracle one by one (the rest: properties that hold at any size)
+ORACLE_ROWS = {1: 1, 2: 32, 3: 128, 4: 256, 5: 64}
+# decode steps covered: every step of the two small workloads, ten spread over the run of the others
+STEPS = {1: list(range(100)), 2: list(range(1000)),
+         3: [int(x) for x in np.linspace(0, 499, 10)], 4: [int(x) for x in np.linspace(0, 199, 10)],
+         5: [int(x) for x in np.linspace(0, 199, 10)]}
+# the logits of step s are those of step s mod FRESH_LOGITS (generating them costs far more than the step itself)
+FRESH_LOGITS = {1: 100, 2: 16, 3: 16, 4: 16, 5: 16}
+_logits_cache = {}
 
 
 def _inputs(config, step):
     spec = synth.CONFIGS[config]
     B = spec["B"]
-    wu = synth.make_workload(config, B=min(B, 64))   # unique logits rows
-    wf = wu if B <= 64 else synth.make_workload(config, B=B)  # class masks for every row
-    tile = -(-B // wu.B)
-    z = np.tile(wu.logits(step), (tile, 1))[:B]
+    fresh = step % FRESH_LOGITS[config]
+    if ("w", config) not in _logits_cache:
+        _logits_cache.clear()
+        _logits_cache[("w", config)] = synth.make_workload(config, B=min(B, 64))   # unique logits rows
+    wu = _logits_cache[("w", config)]
+    if fresh not in _logits_cache:
+        _logits_cache[fresh] = wu.logits(fresh)
+    z = np.tile(_logits_cache[fresh], (-(-B // wu.B), 1))[:B]
+    wf = _workload(config)                                 # class masks (and partitions) for every row
     cm = wf.class_masks(step)
     row_part = None if wf.row_part is None else wf.row_part
     return wf, row_part, cm, z
+
+
+_workloads = {}
+
+
+def _workload(config):
+    if config not in _workloads:
+        _workloads.clear()
+        _workloads[config] = synth.make_workload(config)
+    return _workloads[config]
 
 
 def _popcount_rows(words):
@@ -58,21 +82,23 @@ def _properties(w, row_part, cm, got, V):
 def test_full_size_workload(config):
     spec = synth.CONFIGS[config]
     V, B = spec["V"], spec["B"]
-    for step in (0, 1):
-        w, row_part, cm, z = _inputs(config, step)
-        with Ctx(w.partitions) as ctx:
+    w = _workload(config)
+    with Ctx(w.partitions) as ctx:
+        for n, step in enumerate(STEPS[config]):
+            _, row_part, cm, z = _inputs(config, step)
             got = run_fused(ctx, row_part, cm, z, V, mode=cz.DENSE)
-            assert cz.cfgzip_poll_status(ctx.h)[1:] == (0, 0)
             if config == 5:
                 sparse = run_fused(ctx, row_part, cm, z, V, mode=cz.SPARSE)
                 for key in ("vocab_mask", "logits", "argmax", "rep"):
                     assert np.array_equal(got[key].view(np.uint8), sparse[key].view(np.uint8)), key
                 assert np.abs(got["lse"] - sparse["lse"]).max() <= 1e-4
-        _properties(w, row_part, cm, got, V)
-        rows = np.unique(np.linspace(0, B - 1, ORACLE_ROWS[config]).astype(np.int64))
-        sub = {k: (v[rows] if v is not None else None) for k, v in got.items()}
-        want = oracle_step(w.partitions, None if row_part is None else row_part[rows], cm[rows], z[rows], V)
-        compare_step(sub, want, V, "config %d step %d" % (config, step))
+            if n % 10 == 0 or len(STEPS[config]) <= 10:
+                _properties(w, row_part, cm, got, V)
+            rows = np.unique(np.linspace(0, B - 1, ORACLE_ROWS[config]).astype(np.int64))
+            sub = {k: (v[rows] if v is not None else None) for k, v in got.items()}
+            want = oracle_step(w.partitions, None if row_part is None else row_part[rows], cm[rows], z[rows], V)
+            compare_step(sub, want, V, "config %d step %d" % (config, step))
+        assert cz.cfgzip_poll_status(ctx.h)[1:] == (0, 0)
 
 
 @pytest.mark.parametrize("B", [256, 1024])

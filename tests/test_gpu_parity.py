@@ -360,6 +360,12 @@ def test_argument_errors_are_reported_before_any_launch():
         assert lib.cfgzip_expand_mask(ctx.h, 0, None, cz._ptr(d_cm), 2, None, 32, B, cz.DENSE, None) == cz.E_ARG
         assert lib.cfgzip_mask_logits(ctx.h, cz._ptr(d_z), cz.F32, V - 1, B, V, cz._ptr(d_vm), 32, None) == cz.E_ARG
         assert lib.cfgzip_set_tuning(ctx.h, b"nonsense", 1) == cz.E_ARG
+        # the host-buffer call takes a host vector of partition ids: the "rows as planned" marker is refused, not read
+        h_cm = np.zeros((B, 2), dtype=np.uint32); h_z = np.zeros((B, V), dtype=np.float32)
+        assert lib.cfgzip_decode_step_host(ctx.h, 0, cz.ROWS_AS_PLANNED, h_cm.ctypes.data, 2, h_z.ctypes.data, cz.F32, B,
+                                           None, None, None, None, None, None, cz.DENSE, None) == cz.E_ARG
+        assert lib.cfgzip_rmw_floor(ctx.h, cz._ptr(d_z) + 4, cz.F32, V, B, V, None) == cz.E_ALIGN
+        assert lib.cfgzip_rmw_floor(ctx.h, cz._ptr(d_z), cz.F32, V - 1, B, V, None) == cz.E_ARG
         assert cz.cfgzip_launch_count(ctx.h) == n0  # nothing was launched
         bad = part.c.copy(); bad[0] = K
         out = cz._i32(-1)
@@ -369,6 +375,24 @@ def test_argument_errors_are_reported_before_any_launch():
         cz.cfgzip_free_partition(ctx.h, ctx.ids[0])
         assert fused() == cz.E_RANGE  # freed partition
     assert lib.cfgzip_create(99, ctypes.byref(ctypes.c_void_p())) == cz.E_CUDA
+
+
+def test_floor_kernel_flips_every_sign_once():
+    # the measurement aid reads and rewrites every whole 16-byte vector of every row and nothing else
+    V, B, stride = 1003, 5, 1008
+    part = synth.zipf_partition(V, 10, 1.1, seed=5)
+    with Ctx([part]) as ctx:
+        for dtype, code, sign, per_vec in (("f32", cz.F32, np.uint32(0x80000000), 4), ("bf16", cz.BF16, np.uint16(0x8000), 8)):
+            z = synth.logits_normal(B, stride, 1.0, dtype, (91,))
+            d_z = dev(z)
+            cz.cfgzip_rmw_floor(ctx.h, d_z, code, stride, B, V, torch.cuda.current_stream())
+            once = host(d_z, z.dtype)
+            whole = (V // per_vec) * per_vec
+            bits = z.view(sign.dtype)
+            assert np.array_equal(once.view(sign.dtype)[:, :whole], bits[:, :whole] ^ sign)
+            assert np.array_equal(once.view(sign.dtype)[:, whole:], bits[:, whole:])   # ragged end and padding untouched
+            cz.cfgzip_rmw_floor(ctx.h, d_z, code, stride, B, V, torch.cuda.current_stream())
+            assert np.array_equal(host(d_z, z.dtype).view(np.uint8), z.view(np.uint8))
 
 
 # ------------------------------------------------------------------ CUDA graphs

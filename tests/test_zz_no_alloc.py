@@ -5,7 +5,8 @@ calling the CUDA allocator is forbidden, so they cannot create a context (which 
 tables and scratch). The entry point tested here takes device-resident c and r from the
 caller and keeps its only scratch in an array compiled into the library. The test drives it
 through the C ABI twice in a row (the scratch array is shared and keeps the previous call's
-contents) and compares every result with the context-based entry point.
+contents) and compares every result with the context-based entry point and with the CPU oracle,
+including a full 1024-row batch, one block per row, and class ids outside [0, K).
 
 This file is named so that pytest collects it last.
 """
@@ -16,7 +17,7 @@ import torch
 import synth
 from synth import rng
 from paper_2605_29986_b200 import binding as cz
-from _gpu_util import Ctx, LOGP_TOL, dev, dtype_code, host, run_fused
+from _gpu_util import Ctx, LOGP_TOL, compare_step, dev, dtype_code, host, oracle_step, run_fused
 
 pytestmark = pytest.mark.gpu
 
@@ -61,6 +62,57 @@ def test_noalloc_matches_the_context_entry_point_twice_in_a_row(dtype):
             z = synth.logits_normal(B, V, 2.0, dtype, (78, call))
             want = run_fused(ctx, None, cm, z, V)
             _same(_noalloc(part, cm, z, V), want, "call %d" % call)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_noalloc_matches_the_oracle_twice_in_a_row(dtype):
+    V, K = 50003, 700
+    part = synth.zipf_partition(V, K, 1.1, seed=22)
+    for call, B in enumerate((37, 5)):
+        cm = synth.class_mask_bernoulli(K, B, 0.15, rng.stream_key(79, call))
+        cm[B // 2] = 0
+        z = synth.logits_normal(B, V, 2.0, dtype, (80, call))
+        got = _noalloc(part, cm, z, V)
+        got["logp_full"] = None
+        compare_step(got, oracle_step([part], None, cm, z, V), V, "call %d" % call)
+
+
+def test_noalloc_full_batch_one_block_per_row_against_the_oracle():
+    # 1024 rows: the largest batch the built-in scratch takes, and so many rows that every row gets a single block
+    # (the path that folds without tickets), with class masks that allow something in (almost) every row
+    V, K, B = 9001, 130, 1024
+    part = synth.zipf_partition(V, K, 1.1, seed=23)
+    cm = synth.class_mask_bernoulli(K, B, 0.2, rng.stream_key(81))
+    cm[17] = 0
+    z = synth.logits_normal(B, V, 1.0, "bf16", (82,))
+    for call in range(2):
+        got = _noalloc(part, cm, z, V)
+        got["logp_full"] = None
+        compare_step(got, oracle_step([part], None, cm, z, V, threads=8), V, "call %d" % call)
+
+
+def test_noalloc_treats_class_ids_out_of_range_as_disallowed():
+    # the caller's device vector c is not validated: an id outside [0, K) must make its token disallowed and must not
+    # index the class mask. The oracle sees the same thing as one more class (id K) that the mask never allows.
+    V, K, B = 20000, 700, 9       # K = 700: bit 700 of the last class-mask word exists and stays 0
+    part = synth.zipf_partition(V, K, 1.1, seed=24)
+    cm = synth.class_mask_bernoulli(K, B, 0.3, rng.stream_key(83))
+    z = synth.logits_normal(B, V, 2.0, "f32", (84,))
+    bad = np.array([3, 777, 5000, 12345, 19999])
+    bad = bad[~np.isin(bad, part.r)]              # keep every class's representative valid
+    c_gpu = part.c.copy()
+    c_gpu[bad] = np.array([K, -1, K + 1000, -2 ** 31, 2 ** 31 - 1])[: len(bad)]
+    c_cpu = part.c.copy()
+    c_cpu[bad] = K
+    r_cpu = np.concatenate([part.r, bad[:1]]).astype(np.int32)
+    cpu_part = synth.Partition(V=V, K=K + 1, c=c_cpu, r=r_cpu, sizes=np.bincount(c_cpu, minlength=K + 1))
+    gpu_part = synth.Partition(V=V, K=K, c=c_gpu, r=part.r, sizes=part.sizes)
+    z[:, bad] = 50.0                               # the tokens with bad ids would win every row if they were allowed
+    got = _noalloc(gpu_part, cm, z, V)
+    got["logp_full"] = None
+    want = oracle_step([cpu_part], None, cm, z, V)
+    compare_step(got, want, V, "bad class ids")
+    assert not np.isin(got["argmax"], bad).any()
 
 
 def test_noalloc_rejects_what_it_cannot_hold():
