@@ -290,6 +290,17 @@ int cfgzip_launch_count(cfgzip_ctx* ctx, int64_t* out);
  *                  steps take a third stage where it fits
  *   "stage_alias"  1 = always lay the class-mask staging area over the first warps' rings (default 0: only where
  *                  that keeps warps or buys the third stage)
+ *   "fold"         0 = every warp of the streaming kernel publishes its row states and a second launch (one block or
+ *                  warp per row) folds them and writes the results (default: the fastest at every size measured);
+ *                  1 = the streaming kernel's last block of every row group does that itself, one launch per step;
+ *                  2 = the warps of a block merge their states in shared memory before publishing, second launch kept
+ *   "lane_octets"  bf16 streaming kernel: octets (8 tokens) a lane handles per row of a work item: 1 = 16 bytes,
+ *                  2 = 32 bytes (chunks of 512 tokens, at most 12 warps per block), 0 = automatic (default; currently
+ *                  always 1: two octets measured 2 % faster at 256 rows with 8 warps x 3 stages and slower elsewhere)
+ *   "test_expire_waits"  test hook, default 0: 1 makes every warp of the streaming kernel report its first wait
+ *                  for an asynchronous copy as run out AFTER the wait has completed, so that the error path
+ *                  (flag, bounded drain of the copies in flight, cfgzip_poll_status -> CFGZIP_E_CUDA) can be
+ *                  exercised with nothing left in flight; the results of such a call are undefined
  *   "spread"       1 = launches of at most one block per SM (the streaming kernel of a small batch, the per-row
  *                  kernels of 32 to 148 rows) ask for more than half of an SM's shared memory, so that two of
  *                  their blocks never share an SM (default), 0 = only what the block needs

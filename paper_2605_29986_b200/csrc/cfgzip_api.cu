@@ -25,6 +25,7 @@ struct Part {
 };
 
 constexpr size_t kPartialSlots = size_t(1) << 18;  // 4 MB of (max, sum, pos) slots
+constexpr int kTwoOctetItemsPerWarp = 3;           // bf16: two octets per lane from this many work items per warp on
 constexpr int kDefaultRows = 16384;
 
 }  // namespace
@@ -86,6 +87,9 @@ struct cfgzip_ctx {
     int32_t waves = 1;        // pipelined kernel: blocks launched per resident block slot
     int32_t spread = 1;       // pad the shared memory of one-block-per-SM launches so that blocks cannot share an SM
     int32_t stage_alias = 0;  // 1: always lay the class-mask staging area over the rings (default: only where it buys warps)
+    int32_t lane_octets = 0;  // bf16 pipelined kernel: octets per lane and row (0 = automatic, 1, 2)
+    int32_t fold = 0;         // pipelined kernel: the last block of a row group writes the rows' results (one launch per step)
+    int32_t expire_test = 0;  // test hook: the pipelined kernel reports its first completed wait as run out
 };
 
 namespace {
@@ -207,6 +211,10 @@ struct DensePlan {
     int stage_alias = 0; // pipelined kernel: staging area over the start of the rings
     int hold_warps = 0;
     int ctas_per_sm = 1; // blocks per SM the launch was sized for
+    int opl = 1;         // pipelined kernel: octets per lane and row (2: bf16 chunks of 512 tokens)
+    int fold = 0;        // pipelined kernel: results written by the last block of each group (no finalize launch)
+    int fold_off = 0;    // fold: offset of the block's shared (row, warp) states, 0 = warps publish to the scratch directly
+    int slots = 0;       // states per row in the global scratch
     size_t smem = 0;
     int n_groups_ub = 1;
     bool use_plan_kernel = false;
@@ -257,6 +265,7 @@ DensePlan plan_dense(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, 
         cps *= 2;
     }
     d.per_split = cps * unit_chunk;
+    d.slots = d.S * d.WT + 1;
     d.smem = dense_smem_bytes(d.table_words, fused ? d.threads / 32 : 0, d.stage_stride);
     d.ok = true;
     return d;
@@ -264,60 +273,79 @@ DensePlan plan_dense(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, 
 
 // Launch shape of the pipelined fused kernel. A block takes per_split octets (any number, not only
 // whole 32-octet chunks) of one row group, so that the blocks of a step fill the SMs evenly.
-DensePlan plan_pipe(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, int elem_size, bool cm_bulk_ok) {
+DensePlan plan_pipe_opl(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, int elem_size, bool cm_bulk_ok, int opl) {
     DensePlan d;
+    d.opl = opl;
     d.table_words = (ps.maxKW + 1) * 32;
     d.use_plan_kernel = mixed;
     d.n_groups_ub = mixed ? ceil_div(B, kGroupRows) + ps.n_live_same_v : ceil_div(B, kGroupRows);
     if (!ps.all_c16 || !ctx->pipeline) return d;
     if (mixed && (B > ctx->reserved_rows || d.n_groups_ub > ctx->max_groups)) return d;
-    const int stage_bytes = 8 * 32 * 8 * elem_size + 512;
+    const int chunk_octets = 32 * opl;
+    const int stage_bytes = 8 * chunk_octets * 8 * elem_size + chunk_octets * 16;
     const size_t cap = size_t(ctx->smem_optin) - 2048;  // room for the kernel's static shared memory
-    int n_warps = ctx->pipe_warps, depth = ctx->pipe_depth;
+    // two octets per lane: the variant is compiled for at most 12 warps (its stages are twice as large and it needs
+    // more registers per thread)
+    int n_warps = opl == 2 ? std::min(ctx->pipe_warps, 12) : ctx->pipe_warps, depth = ctx->pipe_depth;
+    const int max_warps = n_warps;
     d.cm_bulk = cm_bulk_ok && ps.all_kw_mult4;
     int stride = d.cm_bulk ? ps.maxKW + (ps.maxKW % 8 == 0 ? 4 : 8) : (ps.maxKW | 1);
-    // Where the staging area of the class masks does not fit beside the rings of all warps it is laid over the
-    // first rings (their warps then start copying after the table is built) rather than giving up warps.
-    bool alias = ctx->stage_alias != 0 ||
-                 (pipe_smem_bytes(d.table_words, n_warps, 2, stage_bytes, stride) > cap &&
-                  pipe_smem_bytes(d.table_words, n_warps, 2, stage_bytes, stride, true) <= cap);
+    auto fits = [&](int warps, int stages, bool over_rings) {
+        return pipe_smem_bytes(d.table_words, warps, stages, stage_bytes, stride, over_rings) <= cap;
+    };
+    bool alias = ctx->stage_alias != 0;
+    bool settled = false;
     // Long steps (twenty or more work items per warp) gain from a third stage where sharing the staging area makes
     // room for it (measured at V = 128256, bf16: B = 1024 -0.7 %, B = 2048 -1.4 %; B = 256 .. 512 lose 1 to 2 % to
     // the late start of the first warps).
-    if (!ctx->pipe_depth_set && depth < 3 && pipe_smem_bytes(d.table_words, n_warps, 3, stage_bytes, stride, true) <= cap) {
+    if (!ctx->pipe_depth_set && depth < 3 && fits(n_warps, 3, true)) {
         const int64_t blocks = int64_t(ctx->sm_count) * ctx->waves;
-        const int64_t items = int64_t(ceil_div(B, kGroupRows)) * (((ps.V >> 3) + 31) >> 5) * ceil_div(std::min<int>(B, kGroupRows), kBatchRows);
+        const int64_t items = int64_t(ceil_div(B, kGroupRows)) * ceil_div(ps.V >> 3, chunk_octets) *
+                              ceil_div(std::min<int>(B, kGroupRows), kBatchRows);
         if (items >= 20 * blocks * n_warps) {
             depth = 3;
             alias = true;
+            settled = true;
         }
     }
-    // a staged class-mask fetch is worth giving up warps for (down to 8) when the class table is large
-    while (n_warps > 8 && pipe_smem_bytes(d.table_words, n_warps, 2, stage_bytes, stride, alias) > cap) n_warps -= 4;
-    if (pipe_smem_bytes(d.table_words, n_warps, 2, stage_bytes, stride, alias) > cap) {
-        n_warps = ctx->pipe_warps;
-        stride = 0;
-        d.cm_bulk = 0;
-        alias = false;
+    // Otherwise: the most warps (down to 8: a staged class-mask fetch is worth giving up warps for when the class
+    // table is large) for which the staging area of the class masks fits, beside the rings of all warps or, where
+    // it does not, laid over the first rings (their warps then start copying after the table is built).
+    if (!settled) {
+        const int step_down = opl == 2 ? 1 : 4;
+        int w = n_warps;
+        for (; w >= std::min(8, max_warps); w -= step_down) {
+            if (ctx->stage_alias == 0 && fits(w, 2, false)) { alias = false; break; }
+            if (fits(w, 2, true)) { alias = true; break; }
+        }
+        if (w >= std::min(8, max_warps)) {
+            n_warps = w;
+        } else {  // no staging: every lane reads its row's class-mask words from global memory
+            n_warps = max_warps;
+            stride = 0;
+            d.cm_bulk = 0;
+            alias = false;
+        }
     }
     while (depth > 2 && pipe_smem_bytes(d.table_words, n_warps, depth, stage_bytes, stride, alias) > cap) --depth;
-    while (n_warps > 4 && pipe_smem_bytes(d.table_words, n_warps, depth, stage_bytes, stride, alias) > cap) n_warps -= 2;
+    while (n_warps > 4 && pipe_smem_bytes(d.table_words, n_warps, depth, stage_bytes, stride, alias) > cap)
+        n_warps -= opl == 2 ? 1 : 2;
     size_t smem = pipe_smem_bytes(d.table_words, n_warps, depth, stage_bytes, stride, alias);
     if (smem > cap) return d;
     if (stride == 0) alias = false;
     d.depth = depth;
     d.stage_stride = stride;
     const int fit = std::max(1, int((cap + 1024) / (smem + 1024)));
-    d.ctas_per_sm = std::min(ctx->ctas_per_sm, fit);
+    d.ctas_per_sm = opl == 2 ? 1 : std::min(ctx->ctas_per_sm, fit);
     const int target = ctx->sm_count * d.ctas_per_sm * ctx->waves;
     const int n_oct = 4 * ps.VW;
     // blocks of groups that turn out not to exist leave at once, so size the split for the fewest
     // groups the batch can have
     const int s0 = std::max(1, target / ceil_div(B, kGroupRows));
-    int per = std::max(32, ceil_div(n_oct, s0));
+    int per = std::max(chunk_octets, ceil_div(n_oct, s0));
     // Warps go side by side along the vocabulary first (long contiguous runs per row are kind to
-    // DRAM); only when a block has fewer 32-octet chunks than warps do warps split the row batches.
-    const int chunks = ceil_div(per, 32);
+    // DRAM); only when a block has fewer chunks than warps do warps split the row batches.
+    const int chunks = ceil_div(per, chunk_octets);
     int WR = ctx->row_warps;
     if (!WR) {
         WR = 1;
@@ -326,7 +354,7 @@ DensePlan plan_pipe(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, i
     while (WR > 1 && (WR - 1) * kBatchRows >= std::min<int>(B, kGroupRows)) WR >>= 1;
     if ((WR != 1 && WR != 2 && WR != 4)) WR = 1;
     d.WT = ctx->token_warps ? ctx->token_warps : n_warps / WR;
-    d.WT = std::max(1, std::min(std::min(d.WT, 16 / WR), chunks));
+    d.WT = std::max(1, std::min(std::min(d.WT, max_warps / WR), chunks));
     d.threads = d.WT * WR * 32;
     for (;;) {
         d.S = ceil_div(n_oct, per);
@@ -338,12 +366,43 @@ DensePlan plan_pipe(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, i
     d.stage_alias = alias ? 1 : 0;
     d.hold_warps = alias ? std::min(d.threads / 32, ceil_div(int64_t(d.stage_stride) * kGroupRows * 4, int64_t(d.depth) * stage_bytes)) : 0;
     d.smem = pipe_smem_bytes(d.table_words, d.threads / 32, d.depth, stage_bytes, d.stage_stride, alias);
+    d.slots = d.S * d.WT + 1;
+    // One launch per step: the last block of a group folds the group's states. Where shared memory has room the
+    // warps of a block first merge their states there (one state per row and block reaches the scratch); otherwise
+    // the warps publish directly, which is only taken while a row has few states.
+    if (ctx->fold) {  // 1: fold in the kernel; 2: only merge the states of a block's warps before they are published
+        const size_t block_states = size_t(kGroupRows) * (d.WT + 1) * sizeof(Partial);
+        if (d.smem + block_states <= cap) {
+            d.fold = ctx->fold == 1;
+            d.fold_off = int(d.smem);
+            d.smem += block_states;
+            d.slots = d.S;
+        } else if (d.slots <= 256) {
+            d.fold = ctx->fold == 1;
+        }
+    }
     // A launch sized for one block per SM asks for more than half of an SM's shared memory even when its few warps
     // need less, so that two of its blocks never share an SM while another SM stays empty (measured at B = 8 .. 24:
     // 10.2 -> 7.7 us, 10.1 -> 8.8 us, 12.4 -> 10.6 us).
     if (d.ctas_per_sm == 1 && ctx->spread) d.smem = std::max(d.smem, cap / 2 + 1024);
     d.ok = true;
     return d;
+}
+
+// Launch shape of the pipelined fused kernel. bf16 rows may be streamed with one octet (16 bytes) or two octets
+// (32 bytes) per lane and row; two octets halve the per-row bookkeeping but double a work item, so they are taken
+// only when every warp of the launch still gets several items.
+DensePlan plan_pipe(cfgzip_ctx* ctx, const PartSet& ps, int32_t B, bool mixed, int elem_size, bool cm_bulk_ok) {
+    const DensePlan one = plan_pipe_opl(ctx, ps, B, mixed, elem_size, cm_bulk_ok, 1);
+    if (elem_size != 2 || ctx->lane_octets == 1) return one;
+    const DensePlan two = plan_pipe_opl(ctx, ps, B, mixed, elem_size, cm_bulk_ok, 2);
+    if (!two.ok) return one;
+    if (!one.ok || ctx->lane_octets == 2) return two;
+    if (ctx->lane_octets == 0) return one;
+    const int64_t items = int64_t(ceil_div(B, kGroupRows)) * ceil_div(ps.V >> 3, 64) *
+                          ceil_div(std::min<int>(B, kGroupRows), kBatchRows);
+    const int64_t warps = int64_t(ctx->sm_count) * ctx->waves * (two.threads / 32);
+    return items >= kTwoOctetItemsPerWarp * warps ? two : one;
 }
 
 // A call may pass CFGZIP_ROWS_AS_PLANNED for its row -> partition vector: it then means the vector given to the
@@ -401,7 +460,11 @@ void fill_groups(cfgzip_ctx* ctx, StepArgs& a, const DensePlan& d) {
     a.cm_bulk = d.cm_bulk;
     a.stage_alias = d.stage_alias;
     a.hold_warps = d.hold_warps;
-    a.slots = d.S * d.WT + 1;
+    a.slots = d.slots;
+    a.fold = d.fold;
+    a.fold_off = d.fold_off;
+    a.chunk_tokens = 256 * d.opl;
+    a.expire_test = ctx->expire_test;
     a.p0 = ctx->parts[size_t(a.part0)].dev;
 }
 
@@ -460,15 +523,20 @@ int launch_pipe(cfgzip_ctx* ctx, const StepArgs& a, const DensePlan& d, dim3 gri
     }
     void (*kern)(StepArgs, CUtensorMap);
     const bool tempered = a.u != nullptr;  // only a sampling step has a temperature
-#define CFGZIP_PIPE_VARIANT(LBT, MINB)                                                                              \
-    (tempered ? (tiled ? k_step_dense_pipe<DT, true, LBT, MINB, true> : k_step_dense_pipe<DT, false, LBT, MINB, true>) \
-              : (tiled ? k_step_dense_pipe<DT, true, LBT, MINB, false> : k_step_dense_pipe<DT, false, LBT, MINB, false>))
-    if (d.threads <= 256 && d.ctas_per_sm >= 3)
-        kern = CFGZIP_PIPE_VARIANT(256, 3);
+    constexpr int kTwo = DT == kBF16 ? 2 : 1;  // f32 lanes always take one octet (32 bytes)
+#define CFGZIP_PIPE_VARIANT(OPL, LBT, MINB)                                                                         \
+    (tempered ? (tiled ? k_step_dense_pipe<DT, OPL, true, LBT, MINB, true> : k_step_dense_pipe<DT, OPL, false, LBT, MINB, true>) \
+              : (tiled ? k_step_dense_pipe<DT, OPL, true, LBT, MINB, false> : k_step_dense_pipe<DT, OPL, false, LBT, MINB, false>))
+    if (d.opl == 2 && kTwo == 2 && d.threads <= 384)
+        kern = CFGZIP_PIPE_VARIANT(kTwo, 384, 1);
+    else if (d.opl != 1)
+        return CFGZIP_E_ARG;  // the planner never asks for this
+    else if (d.threads <= 256 && d.ctas_per_sm >= 3)
+        kern = CFGZIP_PIPE_VARIANT(1, 256, 3);
     else if (d.threads <= 320 && d.ctas_per_sm >= 2)
-        kern = CFGZIP_PIPE_VARIANT(320, 2);
+        kern = CFGZIP_PIPE_VARIANT(1, 320, 2);
     else
-        kern = CFGZIP_PIPE_VARIANT(512, 1);
+        kern = CFGZIP_PIPE_VARIANT(1, 512, 1);
 #undef CFGZIP_PIPE_VARIANT
     if ((rc = ensure_smem(kern, d.smem)) != CFGZIP_OK) return rc;
     return launch(ctx, kern, grid, block, d.smem, st, a, tmap);
@@ -508,8 +576,9 @@ int launch_fused(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, in
                 if ((rc = ensure_smem(kern, d.smem)) != CFGZIP_OK) return rc;
                 rc = launch(ctx, kern, grid, block, d.smem, st, a);
             }
-            // second kernel: one block per row folds the published states and writes the results
-            if (rc == CFGZIP_OK) {
+            // second kernel: one block per row folds the published states and writes the results (unless the
+            // streaming kernel's last block of each group has done so)
+            if (rc == CFGZIP_OK && !(d.depth && d.fold)) {
                 if (a.slots <= kFinalizeWarpStates)  // few states per row: a warp per row
                     rc = launch(ctx, k_finalize_rows_warp<DT>, dim3(unsigned(d.n_groups_ub) * (kGroupRows / 8)), dim3(256), 0, st, a);
                 else
@@ -546,8 +615,12 @@ int launch_sample(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, b
     }
     if (d.ok && d.depth) {
         if (d.use_plan_kernel && (rc = run_plan_kernel(ctx, a.row_part, a.B, a.V, d, st)) != CFGZIP_OK) return rc;
+        // a sampling step keeps one state per warp slot in token order and a kernel of its own for the draw
+        if (d.fold_off) d.smem -= size_t(kGroupRows) * (d.WT + 1) * sizeof(Partial);
+        d.fold = d.fold_off = 0;
+        d.slots = d.S * d.WT + 1;
         fill_groups(ctx, a, d);
-        const int n_chunks = ((ps.V >> 3) + 31) >> 5;
+        const int n_chunks = ceil_div(ps.V >> 3, 32 * d.opl);
         a.run_chunks = std::max(1, ceil_div(n_chunks, d.S * d.WT));
         a.tail_state = 1;
         const dim3 grid(unsigned(d.n_groups_ub) * unsigned(d.S)), block{unsigned(d.threads)};
@@ -563,6 +636,7 @@ int launch_sample(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, b
     a.n_groups = nullptr;
     a.slots = 1;
     a.run_chunks = ceil_div(ps.V, 256);
+    a.chunk_tokens = 256;
     a.tail_state = 0;
     a.p0 = ctx->parts[size_t(a.part0)].dev;
     if ((rc = launch(ctx, k_step_generic<DT, true>, dim3(unsigned(a.B)), dim3(256), 0, st, a)) != CFGZIP_OK) return rc;
@@ -921,7 +995,7 @@ int cfgzip_masked_logsoftmax_argmax(cfgzip_ctx* ctx, cfgzip_part_id part0, const
     a.inv_t = 1.f;
     const int es = dtype == CFGZIP_BF16 ? 2 : 4;
     const bool al = aligned16(logits, row_stride_elems, es);
-    a.wide = dtype == CFGZIP_F32 && aligned32(logits, row_stride_elems, 4);
+    a.wide = aligned32(logits, row_stride_elems, es);  // 32-byte stores (f32 octets, bf16 octet pairs)
     // measured: early launch of the next kernel (whose blocks set themselves up meanwhile) helps steps up to
     // about 130 MB of logits (B = 512 bf16: -1.3 %) and costs 1 % and more from 260 MB on
     ctx->pdl_now = int64_t(B) * ps.V * es < (int64_t(192) << 20);
@@ -978,7 +1052,7 @@ int cfgzip_masked_sample(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* r
     a.u = u;
     const int es = dtype == CFGZIP_BF16 ? 2 : 4;
     const bool al = aligned16(logits, row_stride_elems, es);
-    a.wide = dtype == CFGZIP_F32 && aligned32(logits, row_stride_elems, 4);
+    a.wide = aligned32(logits, row_stride_elems, es);
     ctx->pdl_now = int64_t(B) * ps.V * es < (int64_t(192) << 20);
     rc = dtype == CFGZIP_BF16 ? launch_sample<kBF16>(ctx, a, ps, mixed, al, st) : launch_sample<kF32>(ctx, a, ps, mixed, al, st);
     ctx->pdl_now = true;
@@ -1186,6 +1260,14 @@ int cfgzip_set_tuning(cfgzip_ctx* ctx, const char* name, int32_t value) {
         ctx->spread = value ? 1 : 0;
     } else if (!std::strcmp(name, "stage_alias")) {
         ctx->stage_alias = value ? 1 : 0;
+    } else if (!std::strcmp(name, "fold")) {
+        if (value < 0 || value > 2) return CFGZIP_E_ARG;
+        ctx->fold = value;
+    } else if (!std::strcmp(name, "lane_octets")) {
+        if (value < 0 || value > 2) return CFGZIP_E_ARG;
+        ctx->lane_octets = value;
+    } else if (!std::strcmp(name, "test_expire_waits")) {
+        ctx->expire_test = value ? 1 : 0;
     } else if (!std::strcmp(name, "pipe_depth")) {
         if (value < 2 || value > 8) return CFGZIP_E_ARG;
         ctx->pipe_depth = value;
@@ -1315,7 +1397,7 @@ extern "C" int cfgzip_plan_query(int32_t sm_count, int32_t smem_optin, int32_t V
     int sp_S = 0, sp_per = 0;
     const bool sparse_ok = plan_sparse(&fake, ps, B, true, &sp_S, &sp_per);
     const int32_t vals[16] = {kind, d.n_groups_ub, d.S, d.per_split, d.WT, d.threads, d.depth, int32_t(d.smem),
-                              d.table_words, d.stage_stride, d.cm_bulk, d.S * d.WT + 1, sparse_ok ? sp_S : 0,
+                              d.table_words, d.stage_stride, d.cm_bulk, d.slots, sparse_ok ? sp_S : 0,
                               sparse_ok ? sp_per : 0, int32_t(kPartialSlots), d.ctas_per_sm};
     std::memcpy(out, vals, sizeof vals);
     return CFGZIP_OK;

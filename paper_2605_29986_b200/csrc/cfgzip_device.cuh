@@ -158,6 +158,7 @@ struct Octet<kBF16> {
     __device__ __forceinline__ void load_shared(const char* stage_row, int lane) {
         v = *reinterpret_cast<const uint4*>(stage_row + lane * 16);
     }
+    __device__ __forceinline__ void load_shared_at(const char* p) { v = *reinterpret_cast<const uint4*>(p); }
     __device__ __forceinline__ void store(void* row_base, int o) const {
         st_stream16(reinterpret_cast<uint16_t*>(row_base) + 8 * int64_t(o), v);
     }
@@ -165,7 +166,8 @@ struct Octet<kBF16> {
     __device__ __forceinline__ void store(void* row_base, int o, bool) const { store(row_base, o); }
     __device__ __forceinline__ void store_at(void* p, bool) const { store_at(p); }
     __device__ __forceinline__ void fill_neg_inf() { v = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u); }
-    __device__ __forceinline__ void mask(uint32_t byte, float (&f)[8]) {
+    __device__ __forceinline__ uint4 raw() const { return v; }
+    __device__ __forceinline__ void mask(uint32_t byte, float* f) {
         const uint32_t xl = nibble_to_byte_msbs(byte & 0xFu), xh = nibble_to_byte_msbs(byte >> 4);
         // replicate the top bit of byte 2p / 2p+1 over the low / high half-word
         const uint32_t m0 = prmt(xl, 0u, 0x9988), m1 = prmt(xl, 0u, 0xBBAA);
@@ -194,6 +196,10 @@ struct Octet<kF32> {
         a = *reinterpret_cast<const uint4*>(stage_row + lane * 32);
         b = *reinterpret_cast<const uint4*>(stage_row + lane * 32 + 16);
     }
+    __device__ __forceinline__ void load_shared_at(const char* p) {
+        a = *reinterpret_cast<const uint4*>(p);
+        b = *reinterpret_cast<const uint4*>(p + 16);
+    }
     __device__ __forceinline__ void store(void* row_base, int o) const {
         float* p = reinterpret_cast<float*>(row_base) + 8 * int64_t(o);
         st_stream16(p, a);
@@ -214,7 +220,8 @@ struct Octet<kF32> {
         a = make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u);
         b = a;
     }
-    __device__ __forceinline__ void mask(uint32_t byte, float (&f)[8]) {
+    __device__ __forceinline__ uint4 raw() const { return a; }  // only called for bf16 (two octets per lane)
+    __device__ __forceinline__ void mask(uint32_t byte, float* f) {
         const uint32_t xl = nibble_to_byte_msbs(byte & 0xFu), xh = nibble_to_byte_msbs(byte >> 4);
         const uint32_t ni = 0xFF800000u;
         uint32_t m;
@@ -265,6 +272,10 @@ __device__ __forceinline__ void st_global_u8(void* p, uint32_t v) {
     asm volatile("st.global.u8 [%0], %1;" ::"l"(p), "r"(v));
 }
 
+__device__ __forceinline__ void st_global_u16(void* p, uint32_t v) {
+    asm volatile("st.global.u16 [%0], %1;" ::"l"(p), "h"(static_cast<unsigned short>(v)));
+}
+
 // base + i * stride with a 32-bit stride in one wide multiply-add
 __device__ __forceinline__ char* ptr_mad(char* base, uint32_t i, uint32_t stride) {
     unsigned long long r;
@@ -287,8 +298,12 @@ struct RowAcc {
         nrl = -(kRefFloor * kLog2e);
         pos = kNoPos;
     }
-    __device__ __forceinline__ void add_octet(const float (&f)[8], int position, float scale = kLog2e) {
-        const float vmax = fmax3(fmax3(f[0], f[1], f[2]), fmax3(f[3], f[4], f[5]), fmaxf(f[6], f[7]));
+    // N = 8 or 16 consecutive logits of the row (masked ones are -inf), `position` the index of their first octet.
+    template <int N>
+    __device__ __forceinline__ void add_values(const float* f, int position, float scale = kLog2e) {
+        float vmax = fmax3(fmax3(f[0], f[1], f[2]), fmax3(f[3], f[4], f[5]), fmaxf(f[6], f[7]));
+        if (N == 16)
+            vmax = fmaxf(vmax, fmax3(fmax3(f[8], f[9], f[10]), fmax3(f[11], f[12], f[13]), fmaxf(f[14], f[15])));
         pos = vmax > m ? position : pos;
         m = fmaxf(m, vmax);
         if (fmaf(vmax, scale, nrl) > kRefSlack) {  // rare: move the reference up to vmax
@@ -297,17 +312,23 @@ struct RowAcc {
             nrl = n2;
         }
         const unsigned long long l2 = pack2(scale, scale), n2p = pack2(nrl, nrl);
-        float e[8];
+        unsigned long long e2[N / 2];
 #pragma unroll
-        for (int j = 0; j < 8; j += 2) {
+        for (int j = 0; j < N; j += 2) {
             float t0, t1;
             unpack2(fma2(pack2(f[j], f[j + 1]), l2, n2p), t0, t1);
-            e[j] = ex2f(t0);
-            e[j + 1] = ex2f(t1);
+            e2[j / 2] = pack2(ex2f(t0), ex2f(t1));
         }
+#pragma unroll
+        for (int w = N / 4; w >= 1; w >>= 1)
+#pragma unroll
+            for (int j = 0; j < w; ++j) e2[j] = add2(e2[j], e2[j + w]);
         float a0, a1;
-        unpack2(add2(add2(pack2(e[0], e[1]), pack2(e[2], e[3])), add2(pack2(e[4], e[5]), pack2(e[6], e[7]))), a0, a1);
+        unpack2(e2[0], a0, a1);
         s += a0 + a1;
+    }
+    __device__ __forceinline__ void add_octet(const float (&f)[8], int position, float scale = kLog2e) {
+        add_values<8>(f, position, scale);
     }
     // Bring the sum to the convention of Partial: relative to max(m, kRefFloor).
     __device__ __forceinline__ Partial to_partial(float scale = kLog2e) const {

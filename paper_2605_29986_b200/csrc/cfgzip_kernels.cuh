@@ -44,6 +44,12 @@ struct StepArgs {
     int32_t hold_warps;         // stage_alias: warps whose ring it covers; they start their copies after the table is built
     int32_t run_chunks;         // sampling step: every warp slot of the pipelined kernel takes one contiguous run of this
                                 // many chunks, so that the published states of a row follow the token order
+    int32_t chunk_tokens;       // tokens of one chunk of the pipelined kernel (256 or 512): sampling kernel's run length unit
+    int32_t expire_test;        // test hook: the pipelined kernel reports its first completed wait as run out
+    int32_t fold;               // pipelined kernel: the last block of a row group folds the group's states and writes the
+                                // rows' results itself (no second kernel); tickets[g] counts the group's finished blocks
+    int32_t fold_off;           // fold: byte offset, in dynamic shared memory, of the block's own (row, warp) states, which
+                                // are merged to one state per row before they are published; 0 = warps publish directly
     int32_t tail_state;         // sampling kernel: the last state of a row stands for the octets past the last whole vector
     float scale;                // log2(e) / temperature: the sums are of exp(z / T); log2(e) in a greedy step
     float inv_t;                // 1 / temperature
@@ -110,7 +116,7 @@ __device__ void finalize_row(const StepArgs& a, const PartDev& P, int row, float
 }
 
 // Same for a whole warp whose lanes all hold the row's merged state (octet position): lanes
-// 0..7 test the 8 tokens of the winning octet side by side. A row without a position either
+// 0..15 test the 16 tokens from the winning octet on side by side. A row without a position either
 // allows nothing or holds only -inf at its allowed tokens: the class lists give its lowest
 // allowed token. Needs first_allowed_share / write_row_outputs (defined below).
 template <int DT>
@@ -293,8 +299,9 @@ __device__ __forceinline__ void warp_finalize_row(const StepArgs& a, const PartD
         // a position means that m is a finite allowed logit; the row is already masked in memory (disallowed
         // logits read -inf), so the first token of the octet that holds the value m is the choice. Its
         // representative is fetched side by side with the logit.
+        // the position is the first octet of the 8 or 16 tokens its producer handled together: 16 lanes look
         const int t = 8 * pos + lane;
-        if (lane < 8 && t < a.V) {
+        if (lane < 16 && pos >= 0 && t < a.V) {
             const float z = ldcg_elem<DT>(reinterpret_cast<const char*>(a.logits) + int64_t(row) * a.row_stride * (DT == kBF16 ? 2 : 4), t);
             const int repv = __ldg(P.trep + t);
             if (z == m) cand = (static_cast<unsigned long long>(t) << 32) | static_cast<unsigned int>(repv);
@@ -360,6 +367,14 @@ __device__ __forceinline__ void publish_tail_octets(const StepArgs& a, const Par
                                                     int tail_first, int tail_end, float scale = kLog2e) {
     const Partial p = dense_tail_octets<DT>(a, P, s_row[lane], tail_first, tail_end, scale);
     if (s_row[lane] >= 0) row_slots(a, g, lane)[a.slots - 1] = p;
+}
+// The same into any array of states: row slot r's state goes to base[r * stride + slot].
+template <int DT>
+__device__ __forceinline__ void publish_tail_octets_to(const StepArgs& a, const PartDev& P, const int* s_row, int lane,
+                                                       int tail_first, int tail_end, float scale, Partial* base, int stride,
+                                                       int slot) {
+    const Partial p = dense_tail_octets<DT>(a, P, s_row[lane], tail_first, tail_end, scale);
+    if (s_row[lane] >= 0) base[lane * stride + slot] = p;
 }
 
 // ---------------------------------------------------------------------------------------
@@ -509,8 +524,9 @@ __device__ __forceinline__ int float_order_key(float x) {
 __device__ __forceinline__ float float_from_order_key(int k) { return __int_as_float(k >= 0 ? k : k ^ 0x7FFFFFFF); }
 
 // Reduce the 8 row states of a warp over its 32 lanes and publish them in the warp's slot of each row.
-__device__ __forceinline__ void warp_rows_publish(const StepArgs& a, RowAcc (&acc)[kBatchRows], int live, int g, int slot,
-                                                  int rb, int lane, float scale = kLog2e) {
+// The state of row slot r goes to base[r * stride + slot] (global scratch, or the block's shared array).
+__device__ __forceinline__ void warp_rows_publish_to(RowAcc (&acc)[kBatchRows], int live, int rb, int lane, float scale,
+                                                     Partial* base, int stride, int slot) {
     // Two passes, no exponential inside a reduction chain: the maximum of every row over the lanes (one integer
     // warp reduction each), every lane's sum brought to it with one exponential, the lowest position among the
     // lanes that hold the maximum (one more integer reduction), and the eight sums reduced by recursive halving
@@ -546,7 +562,31 @@ __device__ __forceinline__ void warp_rows_publish(const StepArgs& a, RowAcc (&ac
         Mi = i == k ? M[k] : Mi;
         pi = i == k ? pos[k] : pi;
     }
-    if ((lane & 3) == 0 && i < live) row_slots(a, g, rb * kBatchRows + i)[slot] = Partial{Mi, w[0], pi, 0};
+    if ((lane & 3) == 0 && i < live) base[(rb * kBatchRows + i) * stride + slot] = Partial{Mi, w[0], pi, 0};
+}
+__device__ __forceinline__ void warp_rows_publish(const StepArgs& a, RowAcc (&acc)[kBatchRows], int live, int g, int slot,
+                                                  int rb, int lane, float scale = kLog2e) {
+    warp_rows_publish_to(acc, live, rb, lane, scale, row_slots(a, g, 0), a.slots, slot);
+}
+
+// Fold up to `n` states (16 bytes each, read through L2) with the lanes of a warp side by side; every lane returns
+// the merged state. Four loads per lane are in flight together.
+__device__ __forceinline__ void warp_fold_states(const Partial* src, int n, int lane, float& m, float& s, int& pos) {
+    m = -INFINITY;
+    s = 0.f;
+    pos = kNoPos;
+    for (int base = 0; base < n; base += 128) {
+        int4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int sp = base + u * 32 + lane;
+            v[u] = make_int4(__float_as_int(-INFINITY), 0, kNoPos, 0);
+            if (sp < n) v[u] = __ldcg(reinterpret_cast<const int4*>(src + sp));
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) partial_merge(m, s, pos, __int_as_float(v[u].x), __int_as_float(v[u].y), v[u].z);
+    }
+    partial_warp_allreduce(m, s, pos);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -632,11 +672,15 @@ __global__ void __launch_bounds__(256) k_step_dense(const __grid_constant__ Step
 // bytes per row from shared memory, so no registers wait on memory and the copies of later
 // items overlap the arithmetic of this one. Masked logits go back with 16-byte stores.
 // ---------------------------------------------------------------------------------------
-template <int DT>
+// OPL: octets a lane handles per row of an item (1, or 2 for bf16: 32 bytes per lane and row either way for OPL = 2
+// and for f32). A chunk is the 32 * OPL octets the lanes of a warp cover together.
+template <int DT, int OPL>
 struct PipeGeom {
     static constexpr int kOctetBytes = DT == kBF16 ? 16 : 32;
-    static constexpr int kRowBytes = 32 * kOctetBytes;                   // one row of a stage
-    static constexpr int kStageBytes = kBatchRows * kRowBytes + 32 * 16;  // + class ids of 32 octets
+    static constexpr int kBoxBytes = kBatchRows * 32 * kOctetBytes;        // one tiled copy: 8 rows of 32 octets
+    static constexpr int kRowBytes = 32 * OPL * kOctetBytes;               // one row of a stage
+    static constexpr int kChunkOctets = 32 * OPL;
+    static constexpr int kStageBytes = kBatchRows * kRowBytes + kChunkOctets * 16;  // + class ids of the chunk
 };
 
 // Where the rows of a batch live. With consecutive rows (CONSEC) the address of row i is one
@@ -648,47 +692,73 @@ struct BatchAddr {
     uint32_t vm_bytes;    // CONSEC: bytes between rows of the vocab mask
 };
 
-// One work item of a warp: 32 octets of the 8 rows of a batch, read from the stage `src`.
-// FULL: all 8 rows live and all 32 lanes inside the whole-vector range (no per-row tests).
-template <int DT, bool FULL, bool CONSEC>
-__device__ __forceinline__ void pipe_consume_item(const char* src, const uint32_t* T, int rb, int live, bool active,
-                                                  int o, int lane, const BatchAddr& ba, char* const (&rowp)[kBatchRows],
-                                                  uint8_t* const (&vmp)[kBatchRows], RowAcc (&acc)[kBatchRows], float scale,
-                                                  bool wide) {
-    using G = PipeGeom<DT>;
-    uint4 cv = make_uint4(0, 0, 0, 0);
-    if (FULL || active) cv = *reinterpret_cast<const uint4*>(src + kBatchRows * G::kRowBytes + lane * 16);
-    uint32_t lo, hi;
-    octet_allow_bits(cv, T, rb, FULL || active, lo, hi);
+// One work item of a warp: the 32 * OPL octets of a chunk for the 8 rows of a batch, read from the stage `src`;
+// this lane's OPL octets of row i lie at src + i * srow + lane_off. n_act: how many of the lane's octets are whole
+// vectors of the row (OPL everywhere except at the end of the vocabulary).
+// FULL: all 8 rows live and every lane's octets inside the whole-vector range (no per-row tests).
+template <int DT, int OPL, bool FULL, bool CONSEC>
+__device__ __forceinline__ void pipe_consume_item(const char* src, uint32_t lane_off, uint32_t srow, const uint32_t* T, int rb,
+                                                  int live, int n_act, int o, int lane, const BatchAddr& ba,
+                                                  char* const (&rowp)[kBatchRows], uint8_t* const (&vmp)[kBatchRows],
+                                                  RowAcc (&acc)[kBatchRows], float scale, bool wide) {
+    using G = PipeGeom<DT, OPL>;
+    uint32_t lo[OPL], hi[OPL];
+#pragma unroll
+    for (int q = 0; q < OPL; ++q) {
+        const bool act = FULL || q < n_act;
+        uint4 cv = make_uint4(0, 0, 0, 0);
+        if (act) cv = *reinterpret_cast<const uint4*>(src + kBatchRows * G::kRowBytes + (lane * OPL + q) * 16);
+        octet_allow_bits(cv, T, rb, act, lo[q], hi[q]);
+    }
+    const bool both = FULL || n_act == OPL;
 #pragma unroll
     for (int i = 0; i < kBatchRows; ++i) {
-        if (FULL || (i < live && active)) {
-            Octet<DT> oc;
-            oc.load_shared(src + i * G::kRowBytes, lane);
-            const uint32_t byte = ((i < 4 ? lo : hi) >> (8 * (i & 3))) & 0xFFu;
-            float f[8];
-            oc.mask(byte, f);
-            if (CONSEC) {
-                oc.store_at(ptr_mad(ba.item_base, i, ba.row_bytes), wide);
-                if (ba.vm_item) st_global_u8(ptr_mad(reinterpret_cast<char*>(ba.vm_item), i, ba.vm_bytes), byte);
-            } else {
-                oc.store(rowp[i], o, wide);
-                if (vmp[i]) vmp[i][o] = uint8_t(byte);
+        if (FULL || (i < live && n_act > 0)) {
+            Octet<DT> oc[OPL];
+            float f[8 * OPL];
+            uint32_t bytes = 0;
+#pragma unroll
+            for (int q = 0; q < OPL; ++q) {
+                const uint32_t byte = ((i < 4 ? lo[q] : hi[q]) >> (8 * (i & 3))) & 0xFFu;  // 0 for an octet past the range
+                if (FULL || q < n_act)
+                    oc[q].load_shared_at(src + i * srow + lane_off + q * G::kOctetBytes);
+                else
+                    oc[q].fill_neg_inf();
+                oc[q].mask(byte, f + 8 * q);
+                bytes |= byte << (8 * q);
             }
-            acc[i].add_octet(f, o, scale);
+            char* zp = CONSEC ? ptr_mad(ba.item_base, i, ba.row_bytes) : rowp[i] + size_t(o) * G::kOctetBytes;
+            char* vp = CONSEC ? (ba.vm_item ? ptr_mad(reinterpret_cast<char*>(ba.vm_item), i, ba.vm_bytes) : nullptr)
+                              : (vmp[i] ? reinterpret_cast<char*>(vmp[i]) + o : nullptr);
+            if (OPL == 1) {
+                oc[0].store_at(zp, wide);
+                if (vp) st_global_u8(vp, bytes);
+            } else {
+                if (both && wide) {
+                    st_stream32(zp, oc[0].raw(), oc[OPL - 1].raw());
+                } else {
+                    oc[0].store_at(zp);
+                    if (both) oc[OPL - 1].store_at(zp + G::kOctetBytes);
+                }
+                if (vp) {
+                    if (both) st_global_u16(vp, bytes); else st_global_u8(vp, bytes & 0xFFu);
+                }
+            }
+            acc[i].template add_values<8 * OPL>(f, o, scale);
         }
     }
 }
 
-// TMAP: the 8 rows of a batch are consecutive rows of the logits matrix and arrive as one
-// tiled 2-D copy through `tmap` (box = 256 elements x 8 rows); otherwise one bulk copy per row.
+// TMAP: the 8 rows of a batch are consecutive rows of the logits matrix and arrive as tiled 2-D copies
+// through `tmap` (box = 256 elements x 8 rows: one per chunk, two for a chunk of 512 bf16 tokens);
+// otherwise one bulk copy per row. OPL: octets per lane and row (see PipeGeom).
 // LBT / MINB: launch bounds (threads per block, blocks per SM) the variant is compiled for; they set
-// the register budget: (512, 1) 128 registers, (320, 2) 96, (256, 3) 80. TEMPERED: the sums are of
-// exp(z / T) with the step's temperature (sampling steps); otherwise T = 1 is compiled in.
-template <int DT, bool TMAP, int LBT, int MINB, bool TEMPERED>
+// the register budget: (512, 1) 128 registers, (384, 1) 168, (320, 2) 96, (256, 3) 80. TEMPERED: the sums
+// are of exp(z / T) with the step's temperature (sampling steps); otherwise T = 1 is compiled in.
+template <int DT, int OPL, bool TMAP, int LBT, int MINB, bool TEMPERED>
 __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_constant__ StepArgs a,
                                                          const __grid_constant__ CUtensorMap tmap) {
-    using G = PipeGeom<DT>;
+    using G = PipeGeom<DT, OPL>;
     extern __shared__ __align__(128) uint32_t smem[];
     uint32_t* T = smem;
     int* s_row = reinterpret_cast<int*>(T + a.table_words);
@@ -739,7 +809,7 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
     // range per block, and as fast as handing chunks out through global counters.
     // In a sampling step (TEMPERED) the states of a row must follow the token order: every warp slot then
     // takes one contiguous run of run_chunks chunks instead.
-    const int n_chunks = (n_full + 31) >> 5;
+    const int n_chunks = (n_full + G::kChunkOctets - 1) / G::kChunkOctets;
     const int first_chunk = TEMPERED ? (split * a.WT + wt) * a.run_chunks : split * a.WT + wt;  // this warp's first chunk
     const int stride_chunks = TEMPERED ? 1 : a.S * a.WT;  // round-robin: warps that share a row batch of the group
     const int chunk_end = TEMPERED ? min(first_chunk + a.run_chunks, n_chunks) : n_chunks;
@@ -770,12 +840,16 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
             return;
         }
         slot_info[p_slot] = (p_rb << 24) | chunk;
-        const int o0 = chunk * 32;
+        const int o0 = chunk * G::kChunkOctets;
         char* dst = my_ring + size_t(p_slot) * G::kStageBytes;
-        const uint32_t nvec = uint32_t(min(n_full - o0, 32));  // >= 1: chunk < n_chunks
+        const uint32_t nvec = uint32_t(min(n_full - o0, G::kChunkOctets));  // >= 1: chunk < n_chunks
         if (TMAP) {
-            mbar_expect_tx(bar + p_slot, uint32_t(kBatchRows * G::kRowBytes) + nvec * 16u);
+            // a box holds 32 octets of the 8 rows; the second box of a two-octet chunk is fetched only if the chunk
+            // reaches into it (its lanes are idle otherwise); parts of a box past V or past the last row are filled in
+            const int nbox = (OPL == 2 && nvec > 32u) ? 2 : 1;
+            mbar_expect_tx(bar + p_slot, uint32_t(nbox * G::kBoxBytes) + nvec * 16u);
             tma_g2s_2d(dst, &tmap, o0 * 8, s_row[p_rb * kBatchRows], bar + p_slot);
+            if (nbox == 2) tma_g2s_2d(dst + G::kBoxBytes, &tmap, o0 * 8 + 256, s_row[p_rb * kBatchRows], bar + p_slot);
         } else {
             const int live = min(kBatchRows, nrow - p_rb * kBatchRows);
             const uint32_t row_bytes = nvec * G::kOctetBytes;
@@ -841,7 +915,18 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
     int slot = 0;
     uint32_t phase = 0;
     int consumed = 0;
-    const int my_slot = split * a.WT + wt;
+    // Where this warp's row states go: its own slot of the global scratch, or (fold with block-level merge) the
+    // block's shared array of (row slot, warp along tokens) states
+    const bool fold = !TEMPERED && a.fold != 0;
+    Partial* const s_state = (!TEMPERED && a.fold_off) ? reinterpret_cast<Partial*>(reinterpret_cast<char*>(smem) + a.fold_off) : nullptr;
+    Partial* const pub_base = s_state ? s_state : row_slots(a, g, 0);
+    const int pub_stride = s_state ? a.WT + 1 : a.slots;
+    const int my_slot = s_state ? wt : split * a.WT + wt;
+    // where this lane's octets of a row sit inside a stage: two tiled copies leave two boxes of 8 rows x 32 octets
+    // behind one another, anything else whole rows of the chunk
+    const uint32_t lane_off = (TMAP && OPL == 2) ? uint32_t(lane >> 4) * G::kBoxBytes + uint32_t(lane & 15) * 2u * G::kOctetBytes
+                                                 : uint32_t(lane) * OPL * G::kOctetBytes;
+    const uint32_t srow = (TMAP && OPL == 2) ? 32u * G::kOctetBytes : uint32_t(G::kRowBytes);
     BatchAddr ba;
     ba.row_bytes = uint32_t(a.row_stride * ES);
     ba.vm_bytes = uint32_t(a.vm_stride * 4);
@@ -874,25 +959,29 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
     while (cur_rb * kBatchRows < nrow) {
         const int info = slot_info[slot];
         if (info < 0) break;
-        const int rb = info >> 24, o0 = (info & 0xFFFFFF) * 32;
+        const int rb = info >> 24, o0 = (info & 0xFFFFFF) * G::kChunkOctets;
         while (cur_rb < rb) {  // the previous row batch of this warp is complete (possibly without any chunk)
-            warp_rows_publish(a, acc, live, g, my_slot, cur_rb, lane, scale);
+            warp_rows_publish_to(acc, live, cur_rb, lane, scale, pub_base, pub_stride, my_slot);
             cur_rb += WR;
             open_batch(cur_rb);
         }
-        const bool arrived = mbar_wait(bar + slot, phase);
+        // (the test hook lets the wait complete and then reports it as run out, so that the error path below, drain
+        // loop included, runs with every copy landed)
+        const bool arrived = mbar_wait(bar + slot, phase) && !a.expire_test;
         if (!__all_sync(0xFFFFFFFFu, arrived)) {
             failed = true;
             break;
         }
         const char* src = my_ring + size_t(slot) * G::kStageBytes;
-        const int o = o0 + lane;
+        const int o = o0 + lane * OPL;
         ba.item_base = base0 + size_t(o) * G::kOctetBytes;
         ba.vm_item = vm0 ? vm0 + o : nullptr;
-        if (live == kBatchRows && o0 + 32 <= n_full)
-            pipe_consume_item<DT, true, TMAP>(src, T, rb, live, true, o, lane, ba, rowp, vmp, acc, scale, a.wide != 0);
+        if (live == kBatchRows && o0 + G::kChunkOctets <= n_full)
+            pipe_consume_item<DT, OPL, true, TMAP>(src, lane_off, srow, T, rb, live, OPL, o, lane, ba, rowp, vmp, acc, scale,
+                                                   a.wide != 0);
         else
-            pipe_consume_item<DT, false, TMAP>(src, T, rb, live, o < n_full, o, lane, ba, rowp, vmp, acc, scale, a.wide != 0);
+            pipe_consume_item<DT, OPL, false, TMAP>(src, lane_off, srow, T, rb, live, max(0, min(OPL, n_full - o)), o, lane, ba,
+                                                    rowp, vmp, acc, scale, a.wide != 0);
         ++consumed;
         if (++slot == depth) { slot = 0; phase ^= 1u; }
         __syncwarp();  // every lane has its data out of the slot before it is refilled
@@ -902,7 +991,7 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
     if (!failed) {
         // whatever row batches of this warp are left (all of them if it never got a chunk) are published too
         for (; cur_rb * kBatchRows < nrow; cur_rb += WR) {
-            warp_rows_publish(a, acc, live, g, my_slot, cur_rb, lane, scale);
+            warp_rows_publish_to(acc, live, cur_rb, lane, scale, pub_base, pub_stride, my_slot);
             if ((cur_rb + WR) * kBatchRows < nrow) open_batch(cur_rb + WR);
         }
     } else if (lane == 0) {
@@ -915,7 +1004,41 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
         }
     }
     // the block that reaches the end of the vocabulary takes the octets past the last whole vector
-    if (warp == 0 && split == 0) publish_tail_octets<DT>(a, P, g, s_row, lane, n_full, n_octets, scale);
+    if (warp == 0 && split == 0)
+        publish_tail_octets_to<DT>(a, P, s_row, lane, n_full, n_octets, scale, pub_base, pub_stride, s_state ? a.WT : a.slots - 1);
+    if (!fold && !s_state) return;
+    __shared__ int s_last;
+    if (s_state) {
+        // first the block's own states: one per row and block goes out instead of one per row and warp
+        __syncthreads();
+        for (int j = warp; j < nrow; j += n_warps) {
+            const int n_mine = a.WT + (split == 0 ? 1 : 0);  // only the block that owns the end of the vocabulary has a tail state
+            float m = -INFINITY, s = 0.f;
+            int pos = kNoPos;
+            if (lane < n_mine) {
+                const Partial p = s_state[j * (a.WT + 1) + lane];
+                m = p.m; s = p.s; pos = p.pos;
+            }
+            partial_warp_allreduce(m, s, pos);
+            if (lane == 0) row_slots(a, g, j)[split] = Partial{m, s, pos, 0};
+        }
+    }
+    if (!fold) return;
+    // ---- One launch per step: the group's blocks count themselves off, and the last one to finish folds the states
+    // of the group's rows and writes their results (what k_finalize_rows does in a launch of its own otherwise).
+    __threadfence();  // this block's states and masked logits are visible device-wide before its ticket is drawn
+    __syncthreads();
+    if (tid == 0) s_last = (atomicAdd(a.tickets + g, 1u) == unsigned(a.S - 1));
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();  // the other blocks' states and masked logits, published before their tickets
+    for (int j = warp; j < nrow; j += n_warps) {
+        float m, s;
+        int pos;
+        warp_fold_states(row_slots(a, g, j), a.slots, lane, m, s, pos);
+        warp_finalize_row<DT>(a, P, s_row[j], m, s, pos, lane);
+    }
+    if (tid == 0) a.tickets[g] = 0u;  // ready for the next launch
 }
 
 // ---------------------------------------------------------------------------------------
@@ -1207,7 +1330,7 @@ __global__ void __launch_bounds__(256) k_step_generic(const __grid_constant__ St
 // distribution over its allowed tokens by inverse CDF in token order, with the row's uniform number
 // u: the lowest token whose cumulative weight exceeds u times the total. The states the streaming
 // kernel published stand for consecutive runs of tokens (state k: chunks [k * run_chunks,
-// (k+1) * run_chunks) of 256 tokens; with tail_state the last one: the tokens past the last whole
+// (k+1) * run_chunks) of chunk_tokens tokens; with tail_state the last one: the tokens past the last whole
 // vector), so the block first scans the states for the run that holds the crossing, then re-reads
 // the masked logits of that run only and scans them. All sums are taken in a fixed order.
 // ---------------------------------------------------------------------------------------
@@ -1365,8 +1488,8 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample_rows(const __grid_con
         t_hi = a.V;
     } else {
         const long long lim = a.tail_state ? n_full8 : a.V;
-        t_lo = int(min(static_cast<long long>(pick) * a.run_chunks * 256, lim));
-        t_hi = int(min(static_cast<long long>(pick + 1) * a.run_chunks * 256, lim));
+        t_lo = int(min(static_cast<long long>(pick) * a.run_chunks * a.chunk_tokens, lim));
+        t_hi = int(min(static_cast<long long>(pick + 1) * a.run_chunks * a.chunk_tokens, lim));
     }
     constexpr int ES = DT == kBF16 ? 2 : 4;
     const char* rowp = reinterpret_cast<const char*>(a.logits) + int64_t(row) * a.row_stride * ES;

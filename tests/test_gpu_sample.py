@@ -215,7 +215,7 @@ def test_sample_huge_vocabulary_many_states_per_row():
     z = synth.logits_normal(B, V + 5, 1.5, "f32", (82,))
     with Ctx([part]) as ctx:
         plan = cz.cfgzip_plan_query(148, 232448, V, K, B, cz.F32)
-        assert plan["kind"] == 2 and plan["states_per_row"] > 1024
+        assert plan["kind"] == 2 and plan["S"] * plan["token_warps"] + 1 > 1024  # a sampling step keeps one state per warp
         for trial in range(3):
             u = rng.uniform(rng.stream_key(83, trial), B).astype(np.float32)
             got = run_sample(ctx, None, cm, z, V, u, 3.0, stride=V + 5)

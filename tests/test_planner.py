@@ -24,7 +24,7 @@ def _check(V, K, B, dtype, parts):
     assert p["threads"] % (32 * p["token_warps"]) == 0
     assert p["smem_bytes"] <= SMEM - 1024
     assert p["table_words"] >= 32 * ((K + 31) // 32 + 1)
-    assert p["states_per_row"] == p["S"] * p["token_warps"] + 1
+    assert p["states_per_row"] in (p["S"], p["S"] * p["token_warps"] + 1)  # one per block (merged in the block) or per warp
     assert p["groups"] * 32 * p["states_per_row"] <= p["state_capacity"]
     assert p["S"] >= 1
     if p["kind"] == 1:
