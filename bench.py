@@ -640,8 +640,14 @@ def run_own(args):
                 pair[mode + "_achieved_gbs_of_own_algorithmic_bytes"] = r4.alg_bytes() / us4 / 1e3
             if mode != "dense":
                 pair[mode + "_parity"] = parity_of(r4)
+            if mode == "auto":
+                chosen = cz.cfgzip_choose_mode(r4.ctx, r4.parts[0], r4.row_part_host, r4.host_cm[0], r4.KW, r4.B, cz.F32)
+                pair["host_side_choice"] = {cz.DENSE: "dense", cz.SPARSE: "sparse"}[chosen]
             r4.close()
         pair["auto_vs_best"] = pair["auto_us_per_step"] / min(pair["dense_us_per_step"], pair["sparse_us_per_step"])
+        pair["auto_what"] = ("CFGZIP_AUTO on device-resident masks: the class-list kernel runs first and decides per batch of 8 "
+                             "rows, the gather kernel takes the rest (one extra launch); with the masks still on the host "
+                             "cfgzip_choose_mode picks the mode without any launch")
         pair["workload"] = "cfg5 sparse-stress: V=128256 K=512 B=1024 f32"
         line["sparse_vs_dense"] = pair
     if dist is not None:

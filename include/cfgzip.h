@@ -122,7 +122,8 @@ int cfgzip_plan_rows(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_p
  *   class_mask : dev uint32 [B, class_stride_words], class_stride_words >= KW
  *   vocab_mask : dev uint32 [B, vocab_stride_words], vocab_stride_words >= VW (written)
  *   mode       : CFGZIP_DENSE gathers through c; CFGZIP_SPARSE clears the row and
- *                scatters the members of each allowed class; CFGZIP_AUTO = dense.
+ *                scatters the members of each allowed class; CFGZIP_AUTO = dense here (the
+ *                fused step below is where the automatic mode chooses).
  */
 int cfgzip_expand_mask(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part,
                        const uint32_t* class_mask, int64_t class_stride_words, uint32_t* vocab_mask,
@@ -150,6 +151,16 @@ int cfgzip_mask_logits(cfgzip_ctx* ctx, void* logits, int dtype, int64_t row_str
  *   logp_argmax : nullable dev float [B]; z_argmax - lse
  *   logp_full   : nullable dev float [B, V] (row stride V); z_i - lse, -inf where masked
  *   vocab_mask  : nullable; as in cfgzip_expand_mask
+ *   mode        : CFGZIP_DENSE streams every row through the gather; CFGZIP_SPARSE builds each row's vocab
+ *                 mask from the class->token lists of its allowed classes and never reads a logit that
+ *                 is not allowed; CFGZIP_AUTO decides on the GPU, for the 8 rows of a row batch at a
+ *                 time (the rows the gather kernel streams together): the class-list kernel runs first,
+ *                 adds up the sizes of the classes the batch's rows allow and finishes the batches that
+ *                 allow under 4 % (f32) or 1 % (bf16) of their tokens, the measured break-even; the
+ *                 gather kernel behind it streams the other batches. The extra launch costs about
+ *                 10 us, so steps of less than 384 MB of logits are dense outright. Callers whose
+ *                 class masks are still on the host can choose for free: see cfgzip_choose_mode. The
+ *                 results do not depend on the mode.
  * A row with no allowed token, or whose allowed logits are all -inf, gets lse =
  * logp_argmax = -inf (the latter still returns the lowest allowed id). +inf and NaN
  * logits are outside the contract for the reductions (the masking itself still copies
@@ -197,6 +208,18 @@ int cfgzip_map_tokens(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_
                       void* stream);
 
 /*
+ * Host-only choice between CFGZIP_DENSE and CFGZIP_SPARSE for a batch whose class masks are still in host memory,
+ * which is where the grammar engine leaves them (Section 3.1, "Inference": the engine produces the mask over the
+ * classes; Section 4 runs it on the CPU). Adds up the sizes of the classes every row allows and returns
+ * CFGZIP_SPARSE when under 4 % (f32) or 1 % (bf16) of the batch's tokens are allowed (the measured break-even of the
+ * two kernels; tuning knob "auto_sparse_permille"), else CFGZIP_DENSE; a negative status on bad arguments. Touches
+ * no GPU and launches nothing. row_part_host: NULL or host int32 [B].
+ */
+int cfgzip_choose_mode(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part_host,
+                       const uint32_t* class_mask_host /*host [B, class_stride_words]*/, int64_t class_stride_words,
+                       int32_t B, int dtype);
+
+/*
  * The same step for callers whose data lives on the host: copies the class masks and
  * logits (pinned or pageable host memory) to staging buffers owned by the context,
  * runs cfgzip_masked_logsoftmax_argmax, copies the requested results back and waits
@@ -205,6 +228,7 @@ int cfgzip_map_tokens(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_
  *   masked_logits   : nullable host [B, V]; receives the masked logits
  *   vocab_mask_host : nullable host uint32 [B, VW]
  *   argmax/rep/lse/logp_argmax : nullable host [B]
+ *   mode            : CFGZIP_AUTO chooses with cfgzip_choose_mode from the host masks (no extra launch)
  */
 int cfgzip_decode_step_host(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part_host,
                             const uint32_t* class_mask_host, int64_t class_stride_words,
@@ -290,6 +314,10 @@ int cfgzip_launch_count(cfgzip_ctx* ctx, int64_t* out);
  *                  steps take a third stage where it fits
  *   "stage_alias"  1 = always lay the class-mask staging area over the first warps' rings (default 0: only where
  *                  that keeps warps or buys the third stage)
+ *   "auto_sparse_permille"  CFGZIP_AUTO: a row batch stays with the class-list kernel when under this many
+ *                  thousandths of its tokens are allowed (0..1000; 0 = always dense; -1 = by element type, the default: 40 for
+ *                  f32, 10 for bf16)
+ *   "auto_min_mbytes"  CFGZIP_AUTO: steps with fewer megabytes of logits are dense without looking (default 384)
  *   "fold"         0 = every warp of the streaming kernel publishes its row states and a second launch (one block or
  *                  warp per row) folds them and writes the results (default: the fastest at every size measured);
  *                  1 = the streaming kernel's last block of every row group does that itself, one launch per step;

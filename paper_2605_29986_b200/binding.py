@@ -35,6 +35,7 @@ _SIGNATURES = {
                                     _vp, _vp, _vp, _int, _vp]),
     "cfgzip_plan_rows": (_int, [_vp, _i32, _vp, _i32, _vp]),
     "cfgzip_map_tokens": (_int, [_vp, _i32, _vp, _vp, _vp, _i32, _vp]),
+    "cfgzip_choose_mode": (_int, [_vp, _i32, _vp, _vp, _i64, _i32, _int]),
     "cfgzip_decode_step_host": (_int, [_vp, _i32, _vp, _vp, _i64, _vp, _int, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _int,
                                        _vp]),
     "cfgzip_step_noalloc": (_int, [_vp, _i32, _vp, _i32, _vp, _i64, _vp, _int, _i64, _i32, _vp, _i64, _vp, _vp, _vp, _vp,
@@ -179,6 +180,16 @@ def cfgzip_plan_rows(ctx: int, part0: int, row_part, B: int, stream=None) -> Non
 def cfgzip_map_tokens(ctx: int, part0: int, row_part, tokens, reps, B: int, stream=None) -> None:
     _check(load_library().cfgzip_map_tokens(ctx, part0, _ptr(row_part), _ptr(tokens), _ptr(reps), B, _stream(stream)),
            "cfgzip_map_tokens")
+
+
+def cfgzip_choose_mode(ctx: int, part0: int, row_part_host, class_mask_host, class_stride_words: int, B: int,
+                       dtype: int) -> int:
+    """DENSE or SPARSE for a batch whose class masks are in host memory (host-only, nothing is launched)."""
+    mode = load_library().cfgzip_choose_mode(ctx, part0, _ptr(row_part_host), _ptr(class_mask_host), class_stride_words,
+                                             B, dtype)
+    if mode < 0:
+        raise CfgzipError(mode, "cfgzip_choose_mode")
+    return mode
 
 
 def cfgzip_decode_step_host(ctx: int, part0: int, row_part_host, class_mask_host, class_stride_words: int,

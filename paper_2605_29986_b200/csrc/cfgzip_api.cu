@@ -22,6 +22,7 @@ struct Part {
     int32_t V = 0, K = 0, KW = 0, VW = 0;
     void* block = nullptr;  // one device allocation holding every table of the partition
     PartDev dev{};
+    std::vector<int32_t> sizes;  // host copy of the class sizes (cfgzip_choose_mode)
 };
 
 constexpr size_t kPartialSlots = size_t(1) << 18;  // 4 MB of (max, sum, pos) slots
@@ -51,6 +52,7 @@ struct cfgzip_ctx {
     int32_t* d_group_part = nullptr;
     int32_t* d_group_rows = nullptr;
     int32_t* d_n_groups = nullptr;
+    int32_t* d_row_mode = nullptr;      // automatic mode: which rows the class-list kernel has finished
     int32_t reserved_rows = 0;
     int32_t max_groups = 0;
     // staging for cfgzip_decode_step_host
@@ -88,6 +90,9 @@ struct cfgzip_ctx {
     int32_t spread = 1;       // pad the shared memory of one-block-per-SM launches so that blocks cannot share an SM
     int32_t stage_alias = 0;  // 1: always lay the class-mask staging area over the rings (default: only where it buys warps)
     int32_t lane_octets = 0;  // bf16 pipelined kernel: octets per lane and row (0 = automatic, 1, 2)
+    int32_t auto_permille = -1;  // automatic mode: groups that allow under this many thousandths of their tokens go to the
+                                 // class lists; -1 = by element type (measured break-even: f32 40, bf16 10)
+    int64_t auto_min_bytes = int64_t(384) << 20;  // automatic mode: steps with fewer bytes of logits are dense outright
     int32_t fold = 0;         // pipelined kernel: the last block of a row group writes the rows' results (one launch per step)
     int32_t expire_test = 0;  // test hook: the pipelined kernel reports its first completed wait as run out
 };
@@ -567,7 +572,34 @@ int launch_fused(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, in
         if (!d.ok) d = plan_dense(ctx, ps, a.B, mixed, 4 * ps.VW, 32, true);
         if (d.ok) {
             if (d.use_plan_kernel && (rc = run_plan_kernel(ctx, a.row_part, a.B, a.V, d, st)) != CFGZIP_OK) return rc;
+            // Automatic mode on a long step: the class-list kernel runs first, keeps the row batches (the 8 rows the
+            // gather kernel streams together) that allow few tokens (it never reads a logit that is not allowed) and
+            // marks the others for the gather kernel behind it.
+            // Short steps are dense outright (the extra launch would cost more than the class lists can save).
+            int sp_S = 0, sp_per = 0;
+            const int permille = ctx->auto_permille >= 0 ? ctx->auto_permille : (DT == kBF16 ? 10 : 40);
+            const bool choose = mode == CFGZIP_AUTO && d.depth > 0 && permille > 0 && ctx->d_row_mode != nullptr &&
+                                a.B <= ctx->reserved_rows && int64_t(a.B) * a.V * (DT == kBF16 ? 2 : 4) >= ctx->auto_min_bytes &&
+                                plan_sparse(ctx, ps, a.B, true, &sp_S, &sp_per);
+            if (choose) {
+                if (d.fold_off) d.smem -= size_t(kGroupRows) * (d.WT + 1) * sizeof(Partial);
+                d.fold = d.fold_off = 0;                // the tickets belong to the class-list kernel here
+                d.slots = d.S * d.WT + 1;
+            }
             fill_groups(ctx, a, d);
+            if (choose) {
+                a.row_mode = ctx->d_row_mode;
+                a.auto_permille = permille;
+                StepArgs b = a;  // one row per S blocks
+                b.S = sp_S;
+                b.per_split = sp_per;
+                const size_t smem = size_t(sp_per) * 4;
+                auto kern = k_step_sparse<DT, true>;
+                if ((rc = ensure_smem(kern, smem)) != CFGZIP_OK) return rc;
+                if ((rc = launch(ctx, kern, dim3(unsigned(d.n_groups_ub) * kGroupRows * unsigned(sp_S)), dim3(256), smem, st, b)) !=
+                    CFGZIP_OK)
+                    return rc;
+            }
             const dim3 grid(unsigned(d.n_groups_ub) * unsigned(d.S)), block{unsigned(d.threads)};
             if (d.depth) {
                 rc = launch_pipe<DT>(ctx, a, d, grid, block, st);
@@ -696,14 +728,16 @@ int cfgzip_reserve_rows(cfgzip_ctx* ctx, int32_t max_rows) {
     cudaFree(ctx->d_tickets);
     cudaFree(ctx->d_group_part);
     cudaFree(ctx->d_group_rows);
+    cudaFree(ctx->d_row_mode);
     ctx->d_tickets = nullptr;
-    ctx->d_group_part = ctx->d_group_rows = nullptr;
+    ctx->d_group_part = ctx->d_group_rows = ctx->d_row_mode = nullptr;
     ctx->reserved_rows = 0;
     const int32_t groups = ceil_div(max_rows, kGroupRows) + kMaxParts;
     const size_t tickets = size_t(std::max(max_rows, groups));
     if (cudaMalloc(&ctx->d_tickets, tickets * sizeof(unsigned int)) != cudaSuccess ||
         cudaMalloc(&ctx->d_group_part, size_t(groups) * sizeof(int32_t)) != cudaSuccess ||
-        cudaMalloc(&ctx->d_group_rows, size_t(groups) * kGroupRows * sizeof(int32_t)) != cudaSuccess) {
+        cudaMalloc(&ctx->d_group_rows, size_t(groups) * kGroupRows * sizeof(int32_t)) != cudaSuccess ||
+        cudaMalloc(&ctx->d_row_mode, size_t(max_rows) * sizeof(int32_t)) != cudaSuccess) {
         cudaGetLastError();
         return CFGZIP_E_NOMEM;
     }
@@ -768,6 +802,7 @@ int cfgzip_destroy(cfgzip_ctx* ctx) {
     cudaFree(ctx->d_status);
     cudaFree(ctx->d_group_part);
     cudaFree(ctx->d_group_rows);
+    cudaFree(ctx->d_row_mode);
     cudaFree(ctx->d_n_groups);
     cudaFree(ctx->st_logits);
     cudaFree(ctx->st_cm);
@@ -813,6 +848,8 @@ int cfgzip_load_partition(cfgzip_ctx* ctx, const int32_t* c, int32_t V, const in
     std::memcpy(h_c32, c, size_t(V) * 4);
     std::memcpy(h_r, r, size_t(K) * 4);
     build_class_lists_host(c, V, K, h_off, h_tok);
+    p.sizes.resize(size_t(K));
+    for (int32_t k = 0; k < K; ++k) p.sizes[size_t(k)] = h_off[k + 1] - h_off[k];
     for (int32_t i = 0; i < V; ++i) h_trep[i] = r[c[i]];
     if (has16) {
         for (int32_t i = 0; i < V; ++i) h_c16[i] = uint16_t(c[i]);
@@ -1097,6 +1134,35 @@ int cfgzip_map_tokens(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_
                   int(ps.V), ctx->d_status);
 }
 
+int cfgzip_choose_mode(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part_host,
+                       const uint32_t* class_mask_host, int64_t class_stride_words, int32_t B, int dtype) {
+    if (!ctx || B < 0 || (dtype != CFGZIP_F32 && dtype != CFGZIP_BF16)) return CFGZIP_E_ARG;
+    if (row_part_host == CFGZIP_ROWS_AS_PLANNED) return CFGZIP_E_ARG;
+    PartSet ps;
+    int rc = resolve_parts(ctx, part0, row_part_host != nullptr, &ps);
+    if (rc != CFGZIP_OK) return rc;
+    if (B == 0) return CFGZIP_DENSE;
+    if (!class_mask_host || class_stride_words < ps.maxKW) return CFGZIP_E_ARG;
+    unsigned long long allowed = 0, rows = 0;
+    for (int32_t b = 0; b < B; ++b) {
+        const int32_t id = row_part_host ? row_part_host[b] : part0;
+        if (id < 0 || size_t(id) >= ctx->parts.size() || !ctx->parts[size_t(id)].live || ctx->parts[size_t(id)].V != ps.V) continue;
+        const Part& p = ctx->parts[size_t(id)];
+        const uint32_t* m = class_mask_host + int64_t(b) * class_stride_words;
+        for (int32_t kw = 0; kw < p.KW; ++kw) {
+            uint32_t word = m[kw];
+            if (kw == p.KW - 1 && (p.K & 31)) word &= (1u << (p.K & 31)) - 1u;
+            while (word) {
+                allowed += unsigned(p.sizes[size_t(kw) * 32 + size_t(__builtin_ctz(word))]);
+                word &= word - 1u;
+            }
+        }
+        ++rows;
+    }
+    const int permille = ctx->auto_permille >= 0 ? ctx->auto_permille : (dtype == CFGZIP_BF16 ? 10 : 40);
+    return allowed * 1000ull < static_cast<unsigned long long>(permille) * rows * unsigned(ps.V) ? CFGZIP_SPARSE : CFGZIP_DENSE;
+}
+
 int cfgzip_decode_step_host(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part_host,
                             const uint32_t* class_mask_host, int64_t class_stride_words, const void* logits_host,
                             int dtype, int32_t B, void* masked_logits, uint32_t* vocab_mask_host, int32_t* argmax,
@@ -1149,6 +1215,10 @@ int cfgzip_decode_step_host(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t
     if (!ok) {
         cudaGetLastError();
         return CFGZIP_E_CUDA;
+    }
+    if (mode == CFGZIP_AUTO) {  // the class masks are in host memory: the choice costs no launch
+        const int chosen = cfgzip_choose_mode(ctx, part0, row_part_host, class_mask_host, class_stride_words, B, dtype);
+        if (chosen > 0) mode = chosen;
     }
     rc = cfgzip_masked_logsoftmax_argmax(ctx, part0, row_part_host ? d_rp : nullptr, ctx->st_cm, class_stride_words,
                                          ctx->st_logits, dtype, ps.V, B, vocab_mask_host ? ctx->st_vm : nullptr, ps.VW,
@@ -1260,6 +1330,12 @@ int cfgzip_set_tuning(cfgzip_ctx* ctx, const char* name, int32_t value) {
         ctx->spread = value ? 1 : 0;
     } else if (!std::strcmp(name, "stage_alias")) {
         ctx->stage_alias = value ? 1 : 0;
+    } else if (!std::strcmp(name, "auto_sparse_permille")) {
+        if (value < -1 || value > 1000) return CFGZIP_E_ARG;
+        ctx->auto_permille = value;
+    } else if (!std::strcmp(name, "auto_min_mbytes")) {
+        if (value < 0) return CFGZIP_E_ARG;
+        ctx->auto_min_bytes = int64_t(value) << 20;
     } else if (!std::strcmp(name, "fold")) {
         if (value < 0 || value > 2) return CFGZIP_E_ARG;
         ctx->fold = value;

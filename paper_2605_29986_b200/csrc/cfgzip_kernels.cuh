@@ -50,6 +50,9 @@ struct StepArgs {
                                 // rows' results itself (no second kernel); tickets[g] counts the group's finished blocks
     int32_t fold_off;           // fold: byte offset, in dynamic shared memory, of the block's own (row, warp) states, which
                                 // are merged to one state per row before they are published; 0 = warps publish directly
+    int32_t* row_mode;          // automatic mode: dev [B], written by the class-list kernel, which runs first (1 = the row
+                                // allowed so few tokens that that kernel finished it), read by the kernels after it; else null
+    int32_t auto_permille;      // automatic mode: a row stays with the class lists when under this many thousandths of its tokens are allowed
     int32_t tail_state;         // sampling kernel: the last state of a row stands for the octets past the last whole vector
     float scale;                // log2(e) / temperature: the sums are of exp(z / T); log2(e) in a greedy step
     float inv_t;                // 1 / temperature
@@ -398,6 +401,7 @@ __global__ void __launch_bounds__(kFinalizeThreads) k_finalize_rows(const __grid
         if (row >= a.B) row = -1;
     }
     if (row < 0) return;
+    if (a.row_mode && a.row_mode[row]) return;  // automatic mode: the class-list kernel has finished this row
     const PartDev P = a.group_part ? a.parts[a.group_part[g]] : a.p0;
     const Partial* src = row_slots(a, g, j);
     // Two passes over the states, which stay in registers (up to four per thread, all loads in flight together):
@@ -486,6 +490,7 @@ __global__ void __launch_bounds__(256) k_finalize_rows_warp(const __grid_constan
         if (row >= a.B) row = -1;
     }
     if (row < 0) return;
+    if (a.row_mode && a.row_mode[row]) return;  // automatic mode: the class-list kernel has finished this row
     const PartDev P = a.group_part ? a.parts[a.group_part[g]] : a.p0;
     const Partial* src = row_slots(a, g, j);
     int4 v[4];
@@ -815,12 +820,24 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
     const int chunk_end = TEMPERED ? min(first_chunk + a.run_chunks, n_chunks) : n_chunks;
     int* const slot_info = ring_info + warp * depth; // (rb << 24) | chunk of the item in each slot, -1 = no more items
 
+    // automatic mode: bit r = row slot r was finished by the class-list kernel (set after the wait below)
+    uint32_t rows_done = 0u;
+    auto batch_done = [&](int rb) {
+        const int n = min(kBatchRows, nrow - rb * kBatchRows);
+        const uint32_t all = n >= 8 ? 0xFFu : (1u << n) - 1u;
+        return ((rows_done >> (rb * kBatchRows)) & 0xFFu) == all;
+    };
     // producer cursor (meaningful in lane 0)
     int p_rb = wr, p_slot = 0, p_issued = 0, p_chunk = 0;
     bool p_first = true, p_done = wr * kBatchRows >= nrow, p_end = false;
     auto issue_next = [&]() {
         int chunk = -1;
         while (!p_done) {
+            if (p_first && rows_done && batch_done(p_rb)) {  // nothing left to do for this row batch
+                p_rb += WR;
+                p_done = p_rb * kBatchRows >= nrow;
+                continue;
+            }
             if (p_first) {
                 chunk = first_chunk;
                 p_first = false;
@@ -872,6 +889,12 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
         mbar_init_fence();
     }
     if (implicit) pdl_wait();
+    // automatic mode: row batches that allow few tokens were finished by the class-list kernel in front and get no
+    // work items here (that kernel decides for the 8 row slots of a batch together).
+    if (a.row_mode) {
+        rows_done = __ballot_sync(0xFFFFFFFFu, s_row[lane] >= 0 && a.row_mode[s_row[lane]] != 0);
+        if (rows_done == __ballot_sync(0xFFFFFFFFu, s_row[lane] >= 0)) return;  // the whole group is done
+    }
     if (early_cm) {
         // the class masks first (everything waits for them): the rows dealt over the warps, so that no warp
         // issues more than a few copies; the barrier was set up by thread 0 before the block met above
@@ -1119,20 +1142,67 @@ __global__ void __launch_bounds__(256) k_step_sparse(const __grid_constant__ Ste
 
     pdl_prologue();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, n_warps = blockDim.x >> 5;
-    const int row = blockIdx.x / a.S, split = blockIdx.x - row * a.S;
+    int row = blockIdx.x / a.S;
+    const int split = blockIdx.x - row * a.S;
+    __shared__ int s_batch[kBatchRows];
+    if (a.row_mode) {
+        // Automatic mode: the grid covers the (group, row slot) pairs of the gather kernel, and the choice is made
+        // for the 8 row slots that kernel streams together (its row batch), so that no row is done twice.
+        const int g = row / kGroupRows, j = row - g * kGroupRows;
+        if (a.n_groups && g >= __ldg(a.n_groups)) return;
+        if (tid < kBatchRows) {
+            const int slot = g * kGroupRows + (j & ~(kBatchRows - 1)) + tid;
+            int r = a.group_rows ? a.group_rows[slot] : slot;
+            if (r >= a.B) r = -1;
+            s_batch[tid] = r;
+        }
+        __syncthreads();
+        row = s_batch[j & (kBatchRows - 1)];
+        if (row < 0) return;
+    }
     const int part = a.row_part ? a.row_part[row] : a.part0;
     if (part < 0 || part >= a.n_parts || !a.parts[part].live || a.parts[part].V != a.V) {
-        if (tid == 0 && split == 0) atomicAdd(a.status + 2, 1);
+        if (tid == 0 && split == 0) atomicAdd(a.status + 2, 1);  // (never in automatic mode: only grouped rows come here)
         return;
     }
     const PartDev P = a.parts[part];
     const int w_begin = split * a.per_split, w_end = min(w_begin + a.per_split, a.VW);
     const int t0 = w_begin * 32, t1 = min(w_end * 32, a.V);
+    const uint32_t* cm = a.class_mask + int64_t(row) * a.cm_stride;
+    if (a.row_mode) {
+        // This kernel runs first and keeps the row batches that allow few tokens (it never reads a logit that is not
+        // allowed); the others it leaves, marked, to the gather kernel launched behind it. The tokens a row allows
+        // are the summed sizes of its allowed classes; the rows of a batch share their partition.
+        __shared__ unsigned long long s_allowed;
+        if (tid == 0) s_allowed = 0ull;
+        __syncthreads();
+        unsigned long long mine = 0ull;
+        int n_live = 0;
+#pragma unroll
+        for (int q = 0; q < kBatchRows; ++q) n_live += s_batch[q] >= 0;
+        // a thread per class: how many of the batch's rows allow it (their mask words are the same address for the 32
+        // lanes of a warp), times its size; the cost does not depend on how many classes are allowed
+        for (int k = tid; k < P.K; k += blockDim.x) {
+            int cnt = 0;
+#pragma unroll
+            for (int q = 0; q < kBatchRows; ++q) {
+                const int r = s_batch[q];
+                if (r >= 0) cnt += (__ldg(a.class_mask + int64_t(r) * a.cm_stride + (k >> 5)) >> (k & 31)) & 1u;
+            }
+            if (cnt) mine += static_cast<unsigned long long>(cnt) * static_cast<unsigned>(__ldg(P.off + k + 1) - __ldg(P.off + k));
+        }
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, d);
+        if (lane == 0 && mine) atomicAdd(&s_allowed, mine);
+        __syncthreads();
+        const bool keep = s_allowed * 1000ull < static_cast<unsigned long long>(a.auto_permille) * unsigned(n_live) * unsigned(a.V);
+        if (tid == 0 && split == 0) a.row_mode[row] = keep ? 1 : 0;
+        if (!keep) return;
+    }
     for (int i = tid; i < a.per_split; i += blockDim.x) bits[i] = 0u;
     if (tid == 0) s_nbig = 0;
     __syncthreads();
 
-    const uint32_t* cm = a.class_mask + int64_t(row) * a.cm_stride;
     for (int kw = warp; kw < P.KW; kw += n_warps) {
         uint32_t word = __ldg(cm + kw);
         if (kw == P.KW - 1 && (P.K & 31)) word &= (1u << (P.K & 31)) - 1u;
