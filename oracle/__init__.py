@@ -39,7 +39,7 @@ def _load():
         _lib = ctypes.CDLL(build())
         for name in ("oracle_expand_mask", "oracle_build_csr", "oracle_expand_mask_csr", "oracle_mask_logits",
                      "oracle_logsoftmax_argmax", "oracle_map_tokens", "oracle_decode_step", "oracle_sample",
-                     "oracle_sample_step"):
+                     "oracle_sample_step", "oracle_multi_mask_step"):
             getattr(_lib, name).restype = None
     return _lib
 
@@ -235,3 +235,26 @@ def sample_step(partitions: Sequence, row_part, class_mask, logits: np.ndarray, 
         with ThreadPoolExecutor(max_workers=threads) as ex:
             list(ex.map(run, chunks))
     return dict(vocab_mask=vm, token=tok, rep=rp, lse=lse, logp_token=lpt, cdf=cdf)
+
+
+def multi_mask_step(partition, class_masks, masks_per_row: int, logits: np.ndarray):
+    """Several class masks per logits row: ``class_masks`` is uint32 [B * masks_per_row, >=ceil(K/32)], entry
+    (b, j) at row b * masks_per_row + j; ``logits`` [B, V] is left unchanged. Returns dict(vocab_mask, argmax, rep,
+    lse, logp_argmax), every array with B * masks_per_row entries in the same order."""
+    assert logits.flags.c_contiguous and logits.ndim == 2
+    class_masks = _u32(class_masks)
+    B, V = logits.shape[0], len(partition.c)
+    n = B * masks_per_row
+    assert class_masks.shape[0] == n
+    c, r = _i32(partition.c), _i32(partition.r)
+    vm = np.empty((n, (V + 31) // 32), dtype=np.uint32)
+    am = np.empty(n, dtype=np.int32)
+    rp = np.empty(n, dtype=np.int32)
+    lse = np.empty(n, dtype=np.float64)
+    lpa = np.empty(n, dtype=np.float64)
+    _load().oracle_multi_mask_step(
+        _p(c), _p(r), ctypes.c_int32(V), ctypes.c_int32(int(partition.K)), _p(class_masks),
+        ctypes.c_int64(class_masks.shape[1]), ctypes.c_int32(masks_per_row), _p(logits), ctypes.c_int(_dtype_code(logits)),
+        ctypes.c_int64(logits.shape[1]), ctypes.c_int32(B), _p(vm), ctypes.c_int64(vm.shape[1]), _p(am), _p(rp), _p(lse),
+        _p(lpa))
+    return dict(vocab_mask=vm, argmax=am, rep=rp, lse=lse, logp_argmax=lpa)

@@ -28,8 +28,8 @@
  *     cumulative probability, taken in token-id order, exceeds u.
  *
  * Parity pins: every function here is pinned by tests/test_oracle_pins.py
- * (closed forms, invariants, a library log-softmax, brute force); nothing in
- * this file is "parity unpinned".
+ * (closed forms, invariants, a library log-softmax, brute force, hand-worked
+ * examples); nothing in this file is "parity unpinned".
  */
 #include <math.h>
 #include <stdint.h>
@@ -258,4 +258,29 @@ void oracle_sample_step(const int32_t* c, const int32_t* r, int32_t V, int32_t K
     oracle_sample(logits, dtype, row_stride_elems, B, V, vocab_mask, vocab_stride_words, inv_temperature, u, token, lse,
                   logp_token, cdf);
     oracle_map_tokens(c, r, V, K, token, rep, B);
+}
+
+/*
+ * Several class masks against one logits row (tree or speculative decoding: one next-token
+ * distribution, several grammar states). Not in the paper as such: it is the decode step of
+ * Section 3.1 ("Inference") taken once per mask on a private copy of the row, so the caller's
+ * logits stay as they are. Entry (b, j) of every output sits at index b * masks_per_row + j;
+ * class_masks and vocab_masks hold one row per (b, j) in that order.
+ */
+void oracle_multi_mask_step(const int32_t* c, const int32_t* r, int32_t V, int32_t K, const uint32_t* class_masks,
+                            int64_t class_stride_words, int32_t masks_per_row, const void* logits, int dtype,
+                            int64_t row_stride_elems, int32_t B, uint32_t* vocab_masks, int64_t vocab_stride_words,
+                            int32_t* argmax, int32_t* rep, double* lse, double* logp_argmax) {
+    size_t elem = dtype == ORACLE_BF16 ? 2 : 4;
+    void* row = malloc((size_t)V * elem);
+    for (int32_t b = 0; b < B; ++b) {
+        for (int32_t j = 0; j < masks_per_row; ++j) {
+            int64_t e = (int64_t)b * masks_per_row + j;
+            memcpy(row, (const char*)logits + (size_t)b * (size_t)row_stride_elems * elem, (size_t)V * elem);
+            oracle_decode_step(c, r, V, K, class_masks + e * class_stride_words, class_stride_words, row, dtype, V, 1,
+                               vocab_masks + e * vocab_stride_words, vocab_stride_words, argmax + e, rep + e, lse + e,
+                               logp_argmax + e, NULL);
+        }
+    }
+    free(row);
 }

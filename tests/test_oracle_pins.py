@@ -488,3 +488,66 @@ def test_sample_step_is_the_composition_of_its_steps():
         assert oracle.map_tokens(p.c, p.r, tok)[0] == out["rep"][b]
         t = int(tok[0])
         assert (int(vm[0, t // 32]) >> (t % 32)) & 1 == 1
+
+
+# ------------------------------------------------------------------ several masks per logits row
+
+def test_multi_mask_hand_worked_example():
+    # six tokens in three classes (0, 1, 2, 0, 1, 2), logits 1..6; mask {0} allows tokens 0 and 3, mask {1, 2} the rest
+    part = synth.Partition(V=6, K=3, c=np.array([0, 1, 2, 0, 1, 2], dtype=np.int32), r=np.array([0, 1, 2], dtype=np.int32),
+                           sizes=np.array([2, 2, 2]))
+    z = np.array([[1.0, 2.0, 3.0, 4.0, 5.0, 6.0]], dtype=np.float32)
+    cms = np.array([[0b001], [0b110]], dtype=np.uint32)
+    out = oracle.multi_mask_step(part, cms, 2, z)
+    assert out["argmax"].tolist() == [3, 5] and out["rep"].tolist() == [0, 2]
+    assert out["vocab_mask"][:, 0].tolist() == [0b001001, 0b110110]
+    assert abs(out["lse"][0] - math.log(math.exp(1.0) + math.exp(4.0))) < 1e-12
+    assert abs(out["lse"][1] - math.log(math.exp(2.0) + math.exp(3.0) + math.exp(5.0) + math.exp(6.0))) < 1e-12
+    assert abs(out["logp_argmax"][0] - (4.0 - out["lse"][0])) < 1e-12
+    assert z.tolist() == [[1.0, 2.0, 3.0, 4.0, 5.0, 6.0]]  # the logits are left alone
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_multi_mask_is_one_step_per_mask_and_order_free(dtype):
+    V, K, B, M = 3001, 77, 5, 4
+    part = synth.zipf_partition(V, K, 1.1, seed=3)
+    z = synth.logits_normal(B, V, 2.0, dtype, (21,))
+    cms = synth.class_mask_bernoulli(K, B * M, 0.3, rng.stream_key(22))
+    cms[6] = 0                                     # one (row, mask) with nothing allowed
+    z0 = z.copy()
+    out = oracle.multi_mask_step(part, cms, M, z)
+    assert np.array_equal(z.view(np.uint8), z0.view(np.uint8))
+    # one mask per row is the plain step
+    one = oracle.multi_mask_step(part, cms[::M], 1, z)
+    plain = oracle.decode_step([part], None, cms[::M], z.copy())
+    for key in ("vocab_mask", "argmax", "rep", "lse", "logp_argmax"):
+        assert np.array_equal(one[key], plain[key]), key
+        assert np.array_equal(out[key][::M], plain[key]), key
+    # the masks of a row do not see one another: reversing their order reverses the results
+    rev = cms.reshape(B, M, -1)[:, ::-1].reshape(B * M, -1)
+    out_rev = oracle.multi_mask_step(part, rev, M, z)
+    for key in ("vocab_mask", "argmax", "rep", "lse", "logp_argmax"):
+        got = out_rev[key].reshape((B, M) + out_rev[key].shape[1:])[:, ::-1].reshape(out[key].shape)
+        assert np.array_equal(got, out[key]), key
+    assert out["argmax"][6] == -1 and out["rep"][6] == -1 and np.isneginf(out["lse"][6])
+
+
+def test_multi_mask_disjoint_masks_add_up():
+    # masks A and B allow disjoint class sets, C = A | B: the allowed tokens split, so the normalisers add and the
+    # greedy choice under C is the better of the two choices (the lower token id on a tie)
+    V, K, B = 4000, 64, 6
+    part = synth.zipf_partition(V, K, 1.1, seed=4)
+    z = synth.logits_normal(B, V, 2.0, "bf16", (23,))      # bf16: ties at the maximum do occur
+    a = synth.class_mask_bernoulli(K, B, 0.4, rng.stream_key(24))
+    b = synth.class_mask_bernoulli(K, B, 0.4, rng.stream_key(25)) & ~a
+    cms = np.stack([a, b, a | b], axis=1).reshape(B * 3, -1)
+    out = oracle.multi_mask_step(part, cms, 3, z)
+    zf = rng.bf16_bits_to_f32(z.reshape(-1)).reshape(z.shape).astype(np.float64)
+    for row in range(B):
+        ia, ib, ic = 3 * row, 3 * row + 1, 3 * row + 2
+        assert np.array_equal(out["vocab_mask"][ic], out["vocab_mask"][ia] | out["vocab_mask"][ib])
+        assert not np.any(out["vocab_mask"][ia] & out["vocab_mask"][ib])
+        assert abs(math.exp(out["lse"][ic]) - math.exp(out["lse"][ia]) - math.exp(out["lse"][ib])) <= 1e-9 * math.exp(out["lse"][ic])
+        ta, tb = int(out["argmax"][ia]), int(out["argmax"][ib])
+        best = max((zf[row, ta], -ta), (zf[row, tb], -tb))
+        assert out["argmax"][ic] == -best[1]
