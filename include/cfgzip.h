@@ -199,6 +199,25 @@ int cfgzip_masked_sample(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* r
                          int32_t* rep, float* logp_token, float* lse, int mode, void* stream);
 
 /*
+ * Several class masks against ONE logits row (tree or speculative decoding: the same next-token distribution is
+ * needed under the grammar states of several candidate continuations). The masking of Section 3.1 ("Inference":
+ * mask entry m_{c_i} per token i) is applied once per mask, the logits themselves are read once and NOT modified.
+ * Row (b, j) below stands for logits row b under its j-th mask, stored at index b * masks_per_row + j:
+ *   class_masks : dev uint32 [B * masks_per_row, class_stride_words]
+ *   logits      : dev [B, row_stride_elems] of `dtype`, rows 16-byte aligned (CFGZIP_E_ALIGN otherwise); read only
+ *   vocab_masks : nullable dev uint32 [B * masks_per_row, vocab_stride_words]
+ *   argmax, rep, logp_argmax, lse : dev [B * masks_per_row] (rep, logp_argmax, lse nullable), each as in
+ *                 cfgzip_masked_logsoftmax_argmax for the row masked by that one mask
+ * One partition (part0) for the whole call. B * masks_per_row above the reserved rows gives CFGZIP_E_NOMEM;
+ * partitions with more than 65535 classes give CFGZIP_E_RANGE.
+ */
+int cfgzip_multi_mask_logsoftmax_argmax(cfgzip_ctx* ctx, cfgzip_part_id part0, const uint32_t* class_masks,
+                                        int64_t class_stride_words, int32_t masks_per_row, const void* logits,
+                                        int dtype, int64_t row_stride_elems, int32_t B, uint32_t* vocab_masks,
+                                        int64_t vocab_stride_words, int32_t* argmax, int32_t* rep,
+                                        float* logp_argmax, float* lse, void* stream);
+
+/*
  * Token -> representative of its class, reps[b] = r[c[tokens[b]]] (Section 3.1,
  * "Inference": the engine is fed r_{c_i} instead of t^(i); Figure 1a). A token id
  * outside [0, V) gives -1 and counts as a bad token.

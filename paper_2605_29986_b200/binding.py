@@ -33,6 +33,8 @@ _SIGNATURES = {
                                                _vp, _vp, _vp, _int, _vp]),
     "cfgzip_masked_sample": (_int, [_vp, _i32, _vp, _vp, _i64, _vp, _int, _i64, _i32, _vp, _i64, _vp, ctypes.c_float, _vp,
                                     _vp, _vp, _vp, _int, _vp]),
+    "cfgzip_multi_mask_logsoftmax_argmax": (_int, [_vp, _i32, _vp, _i64, _i32, _vp, _int, _i64, _i32, _vp, _i64, _vp, _vp, _vp,
+                                                   _vp, _vp]),
     "cfgzip_plan_rows": (_int, [_vp, _i32, _vp, _i32, _vp]),
     "cfgzip_map_tokens": (_int, [_vp, _i32, _vp, _vp, _vp, _i32, _vp]),
     "cfgzip_choose_mode": (_int, [_vp, _i32, _vp, _vp, _i64, _i32, _int]),
@@ -168,6 +170,16 @@ def cfgzip_masked_sample(ctx: int, part0: int, row_part, class_mask, class_strid
         ctx, part0, _ptr(row_part), _ptr(class_mask), class_stride_words, _ptr(logits), dtype, row_stride_elems, B,
         _ptr(vocab_mask), vocab_stride_words, _ptr(u), inv_temperature, _ptr(token), _ptr(rep), _ptr(logp_token),
         _ptr(lse), mode, _stream(stream)), "cfgzip_masked_sample")
+
+
+def cfgzip_multi_mask_logsoftmax_argmax(ctx: int, part0: int, class_masks, class_stride_words: int, masks_per_row: int,
+                                        logits, dtype: int, row_stride_elems: int, B: int, vocab_masks,
+                                        vocab_stride_words: int, argmax, rep=None, logp_argmax=None, lse=None,
+                                        stream=None) -> None:
+    _check(load_library().cfgzip_multi_mask_logsoftmax_argmax(
+        ctx, part0, _ptr(class_masks), class_stride_words, masks_per_row, _ptr(logits), dtype, row_stride_elems, B,
+        _ptr(vocab_masks), vocab_stride_words, _ptr(argmax), _ptr(rep), _ptr(logp_argmax), _ptr(lse), _stream(stream)),
+        "cfgzip_multi_mask_logsoftmax_argmax")
 
 
 ROWS_AS_PLANNED = 1  # pass as row_part after cfgzip_plan_rows: the kept grouping of that call is reused

@@ -1096,6 +1096,63 @@ int cfgzip_masked_sample(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* r
     return rc;
 }
 
+int cfgzip_multi_mask_logsoftmax_argmax(cfgzip_ctx* ctx, cfgzip_part_id part0, const uint32_t* class_masks,
+                                        int64_t class_stride_words, int32_t masks_per_row, const void* logits, int dtype,
+                                        int64_t row_stride_elems, int32_t B, uint32_t* vocab_masks,
+                                        int64_t vocab_stride_words, int32_t* argmax, int32_t* rep, float* logp_argmax,
+                                        float* lse, void* stream) {
+    if (!ctx || B < 0 || masks_per_row < 1 || (dtype != CFGZIP_F32 && dtype != CFGZIP_BF16)) return CFGZIP_E_ARG;
+    PartSet ps;
+    int rc = resolve_parts(ctx, part0, false, &ps);
+    if (rc != CFGZIP_OK) return rc;
+    if (B == 0) return CFGZIP_OK;
+    if (int64_t(B) * masks_per_row > ctx->reserved_rows) return CFGZIP_E_NOMEM;
+    if (!class_masks || !logits || !argmax || class_stride_words < ps.maxKW || row_stride_elems < ps.V) return CFGZIP_E_ARG;
+    if (vocab_masks && vocab_stride_words < ps.VW) return CFGZIP_E_ARG;
+    const int es = dtype == CFGZIP_BF16 ? 2 : 4;
+    if (!aligned16(logits, row_stride_elems, es)) return CFGZIP_E_ALIGN;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return CFGZIP_E_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int32_t rows = B * masks_per_row;  // one "row" of masks, vocab masks and results per (logits row, mask)
+    StepArgs a{};
+    a.parts = ctx->d_parts;
+    a.part0 = part0;
+    a.n_parts = int32_t(ctx->parts.size());
+    a.class_mask = class_masks;
+    a.cm_stride = class_stride_words;
+    a.logits = const_cast<void*>(logits);  // never written: masks_per_row > 0 switches the write-back off
+    a.row_stride = row_stride_elems;
+    a.vocab_mask = vocab_masks;
+    a.vm_stride = vocab_stride_words;
+    a.argmax = argmax;
+    a.rep = rep;
+    a.logp_argmax = logp_argmax;
+    a.lse = lse;
+    a.B = rows;
+    a.V = ps.V;
+    a.VW = ps.VW;
+    a.partials = ctx->d_partials;
+    a.tickets = ctx->d_tickets;
+    a.status = ctx->d_status;
+    a.scale = kLog2e;
+    a.inv_t = 1.f;
+    a.masks_per_row = masks_per_row;
+    const DensePlan d = plan_dense(ctx, ps, rows, false, 4 * ps.VW, 32, true);
+    if (!d.ok) return CFGZIP_E_RANGE;  // more than 65535 classes, or a class table beyond shared memory
+    fill_groups(ctx, a, d);
+    ctx->pdl_now = int64_t(B) * ps.V * es < (int64_t(192) << 20);
+    auto kern = dtype == CFGZIP_BF16 ? k_step_dense<kBF16> : k_step_dense<kF32>;
+    if ((rc = ensure_smem(kern, d.smem)) == CFGZIP_OK)
+        rc = launch(ctx, kern, dim3(unsigned(d.n_groups_ub) * unsigned(d.S)), dim3(unsigned(d.threads)), d.smem, st, a);
+    if (rc == CFGZIP_OK) {
+        auto fin = dtype == CFGZIP_BF16 ? k_finalize_rows<kBF16> : k_finalize_rows<kF32>;
+        rc = launch(ctx, fin, dim3(unsigned(d.n_groups_ub) * kGroupRows), dim3(kFinalizeThreads), 0, st, a);
+    }
+    ctx->pdl_now = true;
+    return rc;
+}
+
 int cfgzip_plan_rows(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part, int32_t B, void* stream) {
     if (!ctx || !row_part || row_part == CFGZIP_ROWS_AS_PLANNED || B <= 0) return CFGZIP_E_ARG;
     PartSet ps;

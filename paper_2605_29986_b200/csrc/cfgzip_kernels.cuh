@@ -53,6 +53,8 @@ struct StepArgs {
     int32_t* row_mode;          // automatic mode: dev [B], written by the class-list kernel, which runs first (1 = the row
                                 // allowed so few tokens that that kernel finished it), read by the kernels after it; else null
     int32_t auto_permille;      // automatic mode: a row stays with the class lists when under this many thousandths of its tokens are allowed
+    int32_t masks_per_row;      // > 0: several class masks per logits row (register dense kernel only): row r of the masks,
+                                // vocab masks and results belongs to logits row r / masks_per_row, and the logits are not modified
     int32_t tail_state;         // sampling kernel: the last state of a row stands for the octets past the last whole vector
     float scale;                // log2(e) / temperature: the sums are of exp(z / T); log2(e) in a greedy step
     float inv_t;                // 1 / temperature
@@ -62,6 +64,9 @@ struct StepArgs {
     unsigned int* tickets;
     int32_t* status;            // [0] empty rows, [1] bad tokens, [2] bad rows, [3] copies that never arrived
 };
+
+// The logits row behind row r of the masks and results (they differ when a logits row has several masks).
+__device__ __forceinline__ int64_t logits_row(const StepArgs& a, int r) { return a.masks_per_row > 0 ? r / a.masks_per_row : r; }
 
 // The two halves separately, for a kernel that sets itself up (nothing read from memory) while the kernel in
 // front of it is still running and only then waits for it.
@@ -305,9 +310,14 @@ __device__ __forceinline__ void warp_finalize_row(const StepArgs& a, const PartD
         // the position is the first octet of the 8 or 16 tokens its producer handled together: 16 lanes look
         const int t = 8 * pos + lane;
         if (lane < 16 && pos >= 0 && t < a.V) {
-            const float z = ldcg_elem<DT>(reinterpret_cast<const char*>(a.logits) + int64_t(row) * a.row_stride * (DT == kBF16 ? 2 : 4), t);
+            const float z = ldcg_elem<DT>(reinterpret_cast<const char*>(a.logits) + logits_row(a, row) * a.row_stride * (DT == kBF16 ? 2 : 4), t);
             const int repv = __ldg(P.trep + t);
-            if (z == m) cand = (static_cast<unsigned long long>(t) << 32) | static_cast<unsigned int>(repv);
+            bool ok = z == m;
+            if (a.masks_per_row > 0) {  // the logits were left as they are: ask this row's class mask
+                const int k = __ldg(P.c32 + t);
+                ok = ok && ((__ldg(a.class_mask + int64_t(row) * a.cm_stride + (k >> 5)) >> (k & 31)) & 1u);
+            }
+            if (ok) cand = (static_cast<unsigned long long>(t) << 32) | static_cast<unsigned int>(repv);
         }
     }
 #pragma unroll
@@ -330,7 +340,7 @@ __device__ __forceinline__ Partial dense_tail_octets(const StepArgs& a, const Pa
     int pos = kNoPos;
     if (row < 0) return Partial{m, s, pos, 0};
     const uint32_t* cm = a.class_mask + int64_t(row) * a.cm_stride;
-    char* rowp = reinterpret_cast<char*>(a.logits) + int64_t(row) * a.row_stride * ES;
+    char* rowp = reinterpret_cast<char*>(a.logits) + logits_row(a, row) * a.row_stride * ES;
     uint8_t* vmp = a.vocab_mask ? reinterpret_cast<uint8_t*>(a.vocab_mask) + int64_t(row) * a.vm_stride * 4 : nullptr;
     for (int o = o_first; o < o_end; ++o) {
         uint32_t byte = 0;
@@ -346,7 +356,7 @@ __device__ __forceinline__ Partial dense_tail_octets(const StepArgs& a, const Pa
                 m = fmaxf(m, z);
                 const float ref = fmaxf(m, kRefFloor);
                 s = fmaf(s, ex2f((ref_old - ref) * scale), ex2f((z - ref) * scale));
-            } else {
+            } else if (a.masks_per_row == 0) {
                 store_neg_inf<DT>(rowp, t);
             }
         }
@@ -513,10 +523,10 @@ __global__ void __launch_bounds__(256) k_finalize_rows_warp(const __grid_constan
 // row state.
 template <int DT>
 __device__ __forceinline__ void dense_octet_row(Octet<DT>& oc, char* rowp, uint8_t* vmp, int o, uint32_t byte,
-                                                RowAcc& acc, bool wide) {
+                                                RowAcc& acc, bool wide, bool write_back = true) {
     float f[8];
     oc.mask(byte, f);
-    oc.store(rowp, o, wide);
+    if (write_back) oc.store(rowp, o, wide);
     if (vmp) vmp[o] = uint8_t(byte);
     acc.add_octet(f, o);
 }
@@ -638,7 +648,7 @@ __global__ void __launch_bounds__(256) k_step_dense(const __grid_constant__ Step
         for (int i = 0; i < kBatchRows; ++i) {
             acc[i].init();
             const int row = s_row[min(rb * kBatchRows + i, kGroupRows - 1)];
-            rowp[i] = reinterpret_cast<char*>(a.logits) + int64_t(max(row, 0)) * a.row_stride * ES;
+            rowp[i] = reinterpret_cast<char*>(a.logits) + logits_row(a, max(row, 0)) * a.row_stride * ES;
             vmp[i] = vm8 ? vm8 + int64_t(max(row, 0)) * a.vm_stride * 4 : nullptr;
         }
         const int live = min(kBatchRows, nrow - rb * kBatchRows);
@@ -658,7 +668,7 @@ __global__ void __launch_bounds__(256) k_step_dense(const __grid_constant__ Step
             for (int i = 0; i < kBatchRows; ++i) {
                 if (i < live && active) {
                     const uint32_t byte = ((i < 4 ? lo : hi) >> (8 * (i & 3))) & 0xFFu;
-                    dense_octet_row<DT>(oc[i], rowp[i], vmp[i], o, byte, acc[i], a.wide != 0);
+                    dense_octet_row<DT>(oc[i], rowp[i], vmp[i], o, byte, acc[i], a.wide != 0, a.masks_per_row == 0);
                 }
             }
         }
