@@ -4,6 +4,7 @@ This package holds input recipes only; it imports neither the CPU oracle nor
 the CUDA library, and contains none of the masking path's arithmetic.
 """
 from . import rng  # noqa: F401
+from . import grammars  # noqa: F401
 from .workloads import (  # noqa: F401
     CONFIGS,
     Partition,
