@@ -313,6 +313,60 @@ int cfgzip_step_noalloc(const int32_t* token_to_class /*dev [V]*/, int32_t V,
 int cfgzip_rmw_floor(cfgzip_ctx* ctx, void* logits, int dtype, int64_t row_stride_elems, int32_t B, int32_t V,
                      void* stream);
 
+/*
+ * ---- Offline step (Section 3.1 "Pre-Computation", Section 3.2, Appendix C): from a grammar and a vocabulary to
+ * the vectors c and r that cfgzip_load_partition takes. Done once per tokenizer / grammar pair.
+ *
+ * A grammar in Greibach normal form (Section 2.1): production i is  prod_head[i] -> prod_terminal[i] beta_i  with
+ * beta_i = prod_rhs[prod_rhs_off[i] .. prod_rhs_off[i+1]) a possibly empty sequence of non-terminals 0 ..
+ * n_nonterminals-1 (host arrays, copied). The production S -> epsilon, if the grammar has one, is left out: it
+ * consumes no character and plays no part below. cfgzip_grammar_create also computes the stack-adjacency relation
+ * of Appendix C (graph over the non-terminals, breadth-first search from the non-terminal in front of each
+ * non-terminal Z of a right-hand side to the non-terminals that have a production pushing nothing).
+ * CFGZIP_E_RANGE: a symbol outside [0, n_nonterminals).
+ */
+typedef struct cfgzip_grammar cfgzip_grammar;
+int cfgzip_grammar_create(int32_t n_nonterminals, int32_t start, const int32_t* prod_head, const uint8_t* prod_terminal,
+                          const int32_t* prod_rhs_off /*host [n_prod + 1]*/, const int32_t* prod_rhs, int32_t n_prod,
+                          cfgzip_grammar** out);
+int cfgzip_grammar_destroy(cfgzip_grammar* g);
+/* adjacency[y * n_nonterminals + z] = 1 when z may be popped right after y was popped by a production that pushes
+ * nothing (Appendix C); host uint8 [n_nonterminals^2]. */
+int cfgzip_grammar_adjacency(const cfgzip_grammar* g, uint8_t* adjacency);
+
+/*
+ * Displacement of every token (Algorithm 1 with the stack backtrack restricted by the adjacency relation: the
+ * symbol guessed for the input stack must be adjacent to the symbol popped last; no restriction for the first
+ * symbol), written as one signature row per token: row[0] = n, then n integers: the (input stack, output stack)
+ * pairs in lexicographic order, each as  len(sigma_i), sigma_i.., len(sigma_o), sigma_o..  (stacks top first), then
+ * zeros up to row_words. Two tokens have equal displacement exactly when their rows are equal.
+ *   token_bytes / token_off : host; token i is bytes [token_off[i], token_off[i+1])
+ *   signatures              : host int32 [V, row_words] (written)
+ *   signature_words         : nullable host int32 [V]; the n of each token (-1: more than max_pairs pairs)
+ * Returns CFGZIP_E_RANGE when some token needs more than row_words - 1 integers or more than max_pairs pairs (the
+ * rows of the other tokens are still written; the offending rows are zero). Host only, touches no GPU.
+ */
+int cfgzip_displacement_signatures(const cfgzip_grammar* g, const uint8_t* token_bytes, const int64_t* token_off,
+                                   int32_t V, int32_t row_words, int32_t* signatures, int32_t* signature_words,
+                                   int64_t max_pairs);
+
+/*
+ * Grouping on the GPU (Section 3.1, "Pre-Computation": tokens with equal displacement form a class, the byte-wise
+ * shortest member represents it, c maps tokens to classes and r classes to representatives). Rows are compared
+ * word for word (a hash only picks where to look first), so the grouping is exact.
+ *   signatures     : dev int32 [V, row_words]          token_len : dev int32 [V], byte length of each token
+ *   token_to_class : dev int32 [V] (written): classes numbered in the order of their lowest token id
+ *   class_to_rep   : dev int32 [V] (first *n_classes entries written): shortest member, lowest id among the shortest
+ *   n_classes      : dev int32 [1]
+ *   class_off / class_tok : both NULL, or dev int32 [V + 1] / [V]: the class -> token lists in ascending token id
+ *                    (entries of class_off past n_classes read V)
+ * Runs on the current device; allocates its scratch (about 50 bytes per token), synchronises `stream` before it
+ * returns and frees the scratch: an offline call, not a per-step one. No context is needed.
+ */
+int cfgzip_group_tokens(const int32_t* signatures, int32_t row_words, const int32_t* token_len, int32_t V,
+                        int32_t* token_to_class, int32_t* class_to_rep, int32_t* n_classes, int32_t* class_off,
+                        int32_t* class_tok, void* stream);
+
 /* Kernels this context has launched so far (monotonic; for launch accounting). */
 int cfgzip_launch_count(cfgzip_ctx* ctx, int64_t* out);
 

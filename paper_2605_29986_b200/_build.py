@@ -37,7 +37,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         raise RuntimeError("nvcc not found: the CFGzip CUDA library cannot be built")
     tmp = LIB_PATH + ".%d.tmp" % os.getpid()
     cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + [
-        "-I", _INCLUDE, "-I", _CSRC, "-o", tmp, os.path.join(_CSRC, "cfgzip_api.cu")]
+        "-I", _INCLUDE, "-I", _CSRC, "-o", tmp, os.path.join(_CSRC, "cfgzip_api.cu"),
+        os.path.join(_CSRC, "cfgzip_offline.cu")]
     subprocess.check_call(cmd)
     os.replace(tmp, LIB_PATH)
     return LIB_PATH

@@ -43,6 +43,11 @@ _SIGNATURES = {
     "cfgzip_step_noalloc": (_int, [_vp, _i32, _vp, _i32, _vp, _i64, _vp, _int, _i64, _i32, _vp, _i64, _vp, _vp, _vp, _vp,
                                    _vp]),
     "cfgzip_rmw_floor": (_int, [_vp, _vp, _int, _i64, _i32, _i32, _vp]),
+    "cfgzip_grammar_create": (_int, [_i32, _i32, _vp, _vp, _vp, _vp, _i32, ctypes.POINTER(_vp)]),
+    "cfgzip_grammar_destroy": (_int, [_vp]),
+    "cfgzip_grammar_adjacency": (_int, [_vp, _vp]),
+    "cfgzip_displacement_signatures": (_int, [_vp, _vp, _vp, _i32, _i32, _vp, _vp, _i64]),
+    "cfgzip_group_tokens": (_int, [_vp, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "cfgzip_poll_status": (_int, [_vp, _vp, ctypes.POINTER(_i32), ctypes.POINTER(_i32), ctypes.POINTER(_i32)]),
     "cfgzip_launch_count": (_int, [_vp, ctypes.POINTER(_i64)]),
     "cfgzip_set_tuning": (_int, [_vp, ctypes.c_char_p, _i32]),
@@ -230,6 +235,39 @@ def cfgzip_rmw_floor(ctx: int, logits, dtype: int, row_stride_elems: int, B: int
     """Measurement aid: in-place sign flip of every whole 16-byte vector of the logits (one launch)."""
     _check(load_library().cfgzip_rmw_floor(ctx, _ptr(logits), dtype, row_stride_elems, B, V, _stream(stream)),
            "cfgzip_rmw_floor")
+
+
+def cfgzip_grammar_create(n_nonterminals: int, start: int, prod_head, prod_terminal, prod_rhs_off, prod_rhs) -> int:
+    """Grammar handle from host arrays (int32 heads, uint8 terminals, int32 offsets [n_prod + 1], int32 symbols)."""
+    out = _vp()
+    _check(load_library().cfgzip_grammar_create(n_nonterminals, start, _ptr(prod_head), _ptr(prod_terminal), _ptr(prod_rhs_off),
+                                                _ptr(prod_rhs), len(prod_head), ctypes.byref(out)), "cfgzip_grammar_create")
+    return out.value
+
+
+def cfgzip_grammar_destroy(g: int) -> None:
+    _check(load_library().cfgzip_grammar_destroy(g), "cfgzip_grammar_destroy")
+
+
+def cfgzip_grammar_adjacency(g: int, adjacency) -> None:
+    _check(load_library().cfgzip_grammar_adjacency(g, _ptr(adjacency)), "cfgzip_grammar_adjacency")
+
+
+def cfgzip_displacement_signatures(g: int, token_bytes, token_off, V: int, row_words: int, signatures, signature_words=None,
+                                   max_pairs: int = 1 << 20) -> int:
+    """Returns the status (OK, or E_RANGE when some row did not fit); raises on argument errors."""
+    rc = load_library().cfgzip_displacement_signatures(g, _ptr(token_bytes), _ptr(token_off), V, row_words, _ptr(signatures),
+                                                       _ptr(signature_words), max_pairs)
+    if rc not in (OK, E_RANGE):
+        raise CfgzipError(rc, "cfgzip_displacement_signatures")
+    return rc
+
+
+def cfgzip_group_tokens(signatures, row_words: int, token_len, V: int, token_to_class, class_to_rep, n_classes, class_off=None,
+                        class_tok=None, stream=None) -> None:
+    _check(load_library().cfgzip_group_tokens(_ptr(signatures), row_words, _ptr(token_len), V, _ptr(token_to_class),
+                                              _ptr(class_to_rep), _ptr(n_classes), _ptr(class_off), _ptr(class_tok),
+                                              _stream(stream)), "cfgzip_group_tokens")
 
 
 def cfgzip_poll_status(ctx: int, stream=None) -> Tuple[int, int, int]:
