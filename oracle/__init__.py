@@ -39,7 +39,7 @@ def _load():
         _lib = ctypes.CDLL(build())
         for name in ("oracle_expand_mask", "oracle_build_csr", "oracle_expand_mask_csr", "oracle_mask_logits",
                      "oracle_logsoftmax_argmax", "oracle_map_tokens", "oracle_decode_step", "oracle_sample",
-                     "oracle_sample_step", "oracle_multi_mask_step"):
+                     "oracle_sample_step", "oracle_multi_mask_step", "oracle_sample_filtered"):
             getattr(_lib, name).restype = None
     return _lib
 
@@ -258,3 +258,44 @@ def multi_mask_step(partition, class_masks, masks_per_row: int, logits: np.ndarr
         ctypes.c_int64(logits.shape[1]), ctypes.c_int32(B), _p(vm), ctypes.c_int64(vm.shape[1]), _p(am), _p(rp), _p(lse),
         _p(lpa))
     return dict(vocab_mask=vm, argmax=am, rep=rp, lse=lse, logp_argmax=lpa)
+
+
+def sample_filtered(logits: np.ndarray, V: int, vocab_mask, inv_temperature: float, top_k: int, top_p: float, u,
+                    want_kept: bool = False):
+    """Top-k / top-p sampling from masked logits: dict(token, lse, logp_token, n_kept, p_margin, kept or None)."""
+    assert logits.flags.c_contiguous and logits.ndim == 2
+    vocab_mask = _u32(vocab_mask)
+    B = logits.shape[0]
+    u = np.ascontiguousarray(u, dtype=np.float64)
+    assert u.shape == (B,)
+    token = np.empty(B, dtype=np.int32)
+    lse = np.empty(B, dtype=np.float64)
+    lpt = np.empty(B, dtype=np.float64)
+    n_kept = np.empty(B, dtype=np.int32)
+    margin = np.empty(B, dtype=np.float64)
+    kept = np.empty((B, V), dtype=np.uint8) if want_kept else None
+    _load().oracle_sample_filtered(
+        _p(logits), ctypes.c_int(_dtype_code(logits)), ctypes.c_int64(logits.shape[1]), ctypes.c_int32(B), ctypes.c_int32(V),
+        _p(vocab_mask), ctypes.c_int64(vocab_mask.shape[1]), ctypes.c_double(inv_temperature), ctypes.c_int32(top_k),
+        ctypes.c_double(top_p), _p(u), _p(token), _p(lse), _p(lpt), _p(n_kept), _p(margin), _p(kept))
+    return dict(token=token, lse=lse, logp_token=lpt, n_kept=n_kept, p_margin=margin, kept=kept)
+
+
+def sample_filtered_step(partitions: Sequence, row_part, class_mask, logits: np.ndarray, inv_temperature: float, top_k: int,
+                         top_p: float, u, want_kept: bool = False):
+    """One whole filtered sampling step: expand, mask (in place on ``logits``), sample among the top-k / top-p tokens,
+    map the token to its representative. Returns dict(vocab_mask, token, rep, lse, logp_token, n_kept, p_margin, kept)."""
+    class_mask = _u32(class_mask)
+    B = logits.shape[0]
+    V = len(partitions[0].c)
+    part_of = np.zeros(B, dtype=np.int64) if row_part is None else np.asarray(row_part, dtype=np.int64)
+    vm = np.empty((B, (V + 31) // 32), dtype=np.uint32)
+    for b in range(B):
+        p = partitions[int(part_of[b])]
+        vm[b] = expand_mask(p.c, int(p.K), class_mask[b:b + 1])[0]
+    mask_logits(logits, V, vm)
+    out = sample_filtered(logits, V, vm, inv_temperature, top_k, top_p, u, want_kept)
+    out["vocab_mask"] = vm
+    out["rep"] = np.array([-1 if t < 0 else int(partitions[int(part_of[b])].r[partitions[int(part_of[b])].c[t]])
+                           for b, t in enumerate(out["token"])], dtype=np.int32)
+    return out

@@ -284,3 +284,98 @@ void oracle_multi_mask_step(const int32_t* c, const int32_t* r, int32_t V, int32
     }
     free(row);
 }
+
+/*
+ * Sampling restricted to the most probable tokens (top-k, top-p) of the tempered distribution over the allowed
+ * tokens. The paper only says that the token is sampled (Section 3.1, "Inference") at a temperature (Section 4);
+ * the two filters are the customary ones, read as follows on logits that are already masked:
+ *   order    : the allowed tokens by value, largest first, equal values by token id, lowest first;
+ *   top_k    : > 0 keeps the first min(top_k, allowed) tokens of that order, 0 keeps all;
+ *   top_p    : < 1 then keeps the shortest beginning of what top_k kept whose weight sum_{kept} exp((z_i - M) / T)
+ *              reaches top_p times the weight of all that top_k kept (at least one token); >= 1 keeps all;
+ *   sampling : among the kept tokens F as in oracle_sample, inverse CDF in token-id order with u:
+ *              p_i = exp(z_i / T) / sum_{F} exp(z_j / T), token = min { i in F : sum_{j in F, j <= i} p_j > u };
+ *   lse      = log sum_{F} exp(z_i / T),   logp_tok = z_token / T - lse.
+ * n_kept receives |F|; kept (nullable, [B, V] bytes) the membership of F; p_margin (nullable) how far, as a
+ * fraction of the weight top_k kept, the top_p target lies from the nearer of the two cumulative weights around
+ * the cut (+inf when top_p keeps all): a test can tell from it whether rounding may move the cut.
+ * Degenerate rows as in oracle_sample (nothing allowed: -1; allowed logits all -inf: the lowest allowed id).
+ */
+typedef struct { float z; int32_t id; } oracle_entry;
+
+static int oracle_entry_before(const void* a, const void* b) {
+    const oracle_entry* x = (const oracle_entry*)a;
+    const oracle_entry* y = (const oracle_entry*)b;
+    if (x->z > y->z) return -1;
+    if (x->z < y->z) return 1;
+    return (x->id > y->id) - (x->id < y->id);
+}
+
+void oracle_sample_filtered(const void* logits, int dtype, int64_t row_stride_elems, int32_t B, int32_t V,
+                            const uint32_t* vocab_mask, int64_t vocab_stride_words, double inv_temperature,
+                            int32_t top_k, double top_p, const double* u, int32_t* token, double* lse,
+                            double* logp_token, int32_t* n_kept, double* p_margin, uint8_t* kept) {
+    oracle_entry* order = (oracle_entry*)malloc((size_t)(V > 0 ? V : 1) * sizeof(oracle_entry));
+    uint8_t* in_f = (uint8_t*)malloc((size_t)(V > 0 ? V : 1));
+    for (int32_t b = 0; b < B; ++b) {
+        const uint32_t* v = vocab_mask + (int64_t)b * vocab_stride_words;
+        int64_t base = (int64_t)b * row_stride_elems;
+        int32_t n = 0;
+        for (int32_t i = 0; i < V; ++i) {
+            in_f[i] = 0;
+            if (get_bit(v, i)) {
+                order[n].z = load_logit(logits, dtype, base + i);
+                order[n].id = i;
+                ++n;
+            }
+        }
+        qsort(order, (size_t)n, sizeof(oracle_entry), oracle_entry_before);
+        double M = n > 0 ? (double)order[0].z : -INFINITY;
+        int finite = n > 0 && M > -INFINITY;
+        int32_t keep = n;
+        if (top_k > 0 && top_k < keep) keep = top_k;
+        double margin = INFINITY;
+        if (finite && top_p < 1.0) {
+            double Sk = 0.0;
+            for (int32_t j = 0; j < keep; ++j) Sk += exp(((double)order[j].z - M) * inv_temperature);
+            double target = top_p * Sk, run = 0.0;
+            int32_t cut = keep;
+            for (int32_t j = 0; j < keep; ++j) {
+                double before = run;
+                run += exp(((double)order[j].z - M) * inv_temperature);
+                if (run >= target) {
+                    cut = j + 1;
+                    margin = fmin(run - target, target - before) / Sk;
+                    break;
+                }
+            }
+            keep = cut;
+        }
+        for (int32_t j = 0; j < keep; ++j) in_f[order[j].id] = 1;
+        double S = 0.0;
+        if (finite)
+            for (int32_t i = 0; i < V; ++i)
+                if (in_f[i]) S += exp(((double)load_logit(logits, dtype, base + i) - M) * inv_temperature);
+        int32_t pick = -1, last_pos = -1, first = n > 0 ? V : -1;
+        for (int32_t j = 0; j < n; ++j)
+            if (order[j].id < first) first = order[j].id;
+        if (!finite) pick = first;
+        double run = 0.0;
+        for (int32_t i = 0; i < V && finite; ++i) {
+            if (!in_f[i]) continue;
+            double w = exp(((double)load_logit(logits, dtype, base + i) - M) * inv_temperature);
+            run += w;
+            if (w > 0.0) last_pos = i;
+            if (pick < 0 && run > u[b] * S) pick = i;
+        }
+        if (finite && pick < 0) pick = last_pos;
+        token[b] = pick;
+        lse[b] = finite ? M * inv_temperature + log(S) : -INFINITY;
+        logp_token[b] = finite ? ((double)load_logit(logits, dtype, base + pick) - M) * inv_temperature - log(S) : -INFINITY;
+        if (n_kept) n_kept[b] = keep;
+        if (p_margin) p_margin[b] = margin;
+        if (kept) memcpy(kept + (size_t)b * (size_t)V, in_f, (size_t)V);
+    }
+    free(order);
+    free(in_f);
+}

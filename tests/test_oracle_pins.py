@@ -551,3 +551,93 @@ def test_multi_mask_disjoint_masks_add_up():
         ta, tb = int(out["argmax"][ia]), int(out["argmax"][ib])
         best = max((zf[row, ta], -ta), (zf[row, tb], -tb))
         assert out["argmax"][ic] == -best[1]
+
+
+# ------------------------------------------------------------------ top-k / top-p sampling
+
+def _weights_row(ws):
+    """One row whose tempered weights at T = 1 are ws (logits log w), all allowed."""
+    z = np.log(np.asarray(ws, dtype=np.float64)).astype(np.float32)[None, :]
+    return z, _full_mask(len(ws))
+
+
+def test_filtered_sampling_hand_worked():
+    # weights 1 : 2 : 3 : 4 on tokens 0..3
+    z, vm = _weights_row([1, 2, 3, 4])
+    def run(k, p, u):
+        return oracle.sample_filtered(z.copy(), 4, vm, 1.0, k, p, [u], want_kept=True)
+    o = run(2, 1.0, 0.4)                                  # top-2 keeps tokens 3 and 2 (weights 4 and 3): CDF 3/7, 1
+    assert o["kept"][0].tolist() == [0, 0, 1, 1] and o["n_kept"][0] == 2 and o["token"][0] == 2
+    assert abs(o["lse"][0] - math.log(7.0)) < 1e-6 and abs(o["logp_token"][0] - math.log(3.0 / 7.0)) < 1e-6
+    assert run(2, 1.0, 0.5)["token"][0] == 3
+    o = run(0, 0.5, 0.0)                                  # top-p 0.5 of 10: 4 < 5 <= 4 + 3 keeps tokens 3 and 2
+    assert o["kept"][0].tolist() == [0, 0, 1, 1] and abs(o["p_margin"][0] - 0.1) < 1e-6
+    assert run(0, 0.39, 0.0)["kept"][0].tolist() == [0, 0, 0, 1]     # 3.9 <= 4: the top token alone
+    assert run(0, 0.71, 0.0)["kept"][0].tolist() == [0, 1, 1, 1]     # 7 < 7.1 <= 9
+    o = run(3, 0.5, 0.99)                                 # top-3 first (weights 4, 3, 2 = 9), then half of 9: 4 < 4.5 <= 7
+    assert o["kept"][0].tolist() == [0, 0, 1, 1] and o["token"][0] == 3
+
+
+def test_filtered_sampling_ties_keep_the_lowest_ids():
+    z, vm = _weights_row([5, 2, 5, 5, 1, 5])             # four equal maxima at tokens 0, 2, 3, 5
+    o = oracle.sample_filtered(z.copy(), 6, vm, 1.0, 2, 1.0, [0.0], want_kept=True)
+    assert o["kept"][0].tolist() == [1, 0, 1, 0, 0, 0]
+    o = oracle.sample_filtered(z.copy(), 6, vm, 1.0, 0, 0.6, [0.0], want_kept=True)     # 0.6 * 23 = 13.8: three maxima
+    assert o["kept"][0].tolist() == [1, 0, 1, 1, 0, 0]
+
+
+def test_filtered_sampling_reduces_to_the_plain_cases():
+    V = 700
+    z = rng.normal_f32(rng.stream_key(9, 1), 6 * V, 2.0).reshape(6, V)
+    bits = rng.uniform(rng.stream_key(9, 2), 6 * V).reshape(6, V) < 0.4
+    vm = synth.pack_bits(bits)
+    oracle.mask_logits(z, V, vm)
+    u = rng.uniform(rng.stream_key(9, 3), 6)
+    plain = oracle.sample(z.copy(), V, vm, 5.0, u)
+    allowed = bits.sum(axis=1)
+    for k, p in ((0, 1.0), (int(allowed.max()), 1.0), (V + 5, 1.5)):                      # no filter at all
+        o = oracle.sample_filtered(z.copy(), V, vm, 5.0, k, p, u)
+        assert np.array_equal(o["token"], plain[0]) and np.allclose(o["lse"], plain[1], atol=1e-12)
+        assert np.allclose(o["logp_token"], plain[2], atol=1e-12) and np.all(o["n_kept"] == allowed)
+    am, _, _, _ = oracle.logsoftmax_argmax(z.copy(), V, vm)
+    for uu in (0.0, 0.5, 0.999999):                                                        # top-1 is the greedy choice
+        o = oracle.sample_filtered(z.copy(), V, vm, 5.0, 1, 1.0, [uu] * 6)
+        assert np.array_equal(o["token"], am) and np.allclose(o["logp_token"], 0.0, atol=1e-12)
+        o = oracle.sample_filtered(z.copy(), V, vm, 5.0, 0, 1e-9, [uu] * 6)                # a tiny top-p too
+        assert np.array_equal(o["token"], am)
+
+
+def test_filtered_sampling_keeps_a_top_set_of_the_right_size_and_weight():
+    V, B = 3000, 8
+    z = rng.normal_f32(rng.stream_key(9, 4), B * V, 2.0).reshape(B, V)
+    bits = rng.uniform(rng.stream_key(9, 5), B * V).reshape(B, V) < 0.5
+    vm = synth.pack_bits(bits)
+    oracle.mask_logits(z, V, vm)
+    u = rng.uniform(rng.stream_key(9, 6), B)
+    for k, p, inv_t in ((50, 1.0, 1.0), (0, 0.9, 1.0), (200, 0.5, 2.0), (7, 0.999, 5.0)):
+        o = oracle.sample_filtered(z.copy(), V, vm, inv_t, k, p, u, want_kept=True)
+        for b in range(B):
+            kept = o["kept"][b].astype(bool)
+            assert not np.any(kept & ~bits[b]) and kept[o["token"][b]]
+            assert z[b][kept].min() >= z[b][bits[b] & ~kept].max()           # nothing dropped beats anything kept
+            w = np.exp((z[b].astype(np.float64) - z[b][bits[b]].max()) * inv_t)
+            if p >= 1.0:
+                assert kept.sum() == min(k, bits[b].sum())
+            else:
+                top = np.sort(w[bits[b]])[::-1][: (k or V)]
+                target = p * top.sum()
+                assert w[kept].sum() >= target * (1 - 1e-12)                  # reaches the target ...
+                assert w[kept].sum() - w[kept].min() < target * (1 + 1e-12)  # ... and would not without its last token
+            assert abs(o["lse"][b] - (float(z[b][bits[b]].max()) * inv_t + math.log(w[kept].sum()))) < 1e-9
+
+
+def test_filtered_sampling_degenerate_rows():
+    V = 40
+    z = np.zeros((2, V), dtype=np.float32)
+    bits = np.zeros((2, V), dtype=bool)
+    bits[1, [7, 30]] = True
+    z[1, [7, 30]] = -np.inf
+    vm = synth.pack_bits(bits)
+    oracle.mask_logits(z, V, vm)
+    o = oracle.sample_filtered(z, V, vm, 1.0, 3, 0.5, [0.3, 0.3])
+    assert o["token"].tolist() == [-1, 7] and np.isneginf(o["lse"]).all() and np.isneginf(o["logp_token"]).all()
