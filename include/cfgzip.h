@@ -199,6 +199,26 @@ int cfgzip_masked_sample(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* r
                          int32_t* rep, float* logp_token, float* lse, int mode, void* stream);
 
 /*
+ * cfgzip_masked_sample with the draw restricted to the most probable allowed tokens (the paper names no sampler,
+ * Section 3.1 / Section 4; these are the two customary filters, applied to the masked, tempered distribution):
+ *   order : the allowed tokens by logit, largest first; equal logits by token id, lowest first
+ *   top_k : > 0 keeps the first min(top_k, allowed) tokens of that order; 0 keeps all
+ *   top_p : in (0, 1) then keeps the shortest beginning of what top_k kept whose weight, sum of exp(z_i / T),
+ *           reaches top_p times the weight of all that top_k kept (at least one token); >= 1 keeps all
+ * The token is drawn among the kept tokens by inverse CDF in token-id order with u[b]; lse and logp_token are those
+ * of the distribution renormalised over the kept tokens. top_k = 0 and top_p >= 1 give cfgzip_masked_sample.
+ * Weights are summed as 40-bit fixed-point integers, so the result is deterministic; where top_p times the weight
+ * lies within rounding (about 1e-6 of the weight) of a cumulative weight of the order, the kept set may end one
+ * token earlier or later than in exact arithmetic. top_k < 0 or top_p <= 0 give CFGZIP_E_ARG.
+ */
+int cfgzip_masked_sample_filtered(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part,
+                                  const uint32_t* class_mask, int64_t class_stride_words, void* logits, int dtype,
+                                  int64_t row_stride_elems, int32_t B, uint32_t* vocab_mask,
+                                  int64_t vocab_stride_words, const float* u, float inv_temperature, int32_t top_k,
+                                  float top_p, int32_t* token, int32_t* rep, float* logp_token, float* lse, int mode,
+                                  void* stream);
+
+/*
  * Several class masks against ONE logits row (tree or speculative decoding: the same next-token distribution is
  * needed under the grammar states of several candidate continuations). The masking of Section 3.1 ("Inference":
  * mask entry m_{c_i} per token i) is applied once per mask, the logits themselves are read once and NOT modified.

@@ -298,7 +298,8 @@ void oracle_multi_mask_step(const int32_t* c, const int32_t* r, int32_t V, int32
  *   lse      = log sum_{F} exp(z_i / T),   logp_tok = z_token / T - lse.
  * n_kept receives |F|; kept (nullable, [B, V] bytes) the membership of F; p_margin (nullable) how far, as a
  * fraction of the weight top_k kept, the top_p target lies from the nearer of the two cumulative weights around
- * the cut (+inf when top_p keeps all): a test can tell from it whether rounding may move the cut.
+ * the cut, leaving out a side on which the cut cannot move (+inf when top_p keeps all): a test can tell from it
+ * whether rounding may move the cut.
  * Degenerate rows as in oracle_sample (nothing allowed: -1; allowed logits all -inf: the lowest allowed id).
  */
 typedef struct { float z; int32_t id; } oracle_entry;
@@ -345,7 +346,10 @@ void oracle_sample_filtered(const void* logits, int dtype, int64_t row_stride_el
                 run += exp(((double)order[j].z - M) * inv_temperature);
                 if (run >= target) {
                     cut = j + 1;
-                    margin = fmin(run - target, target - before) / Sk;
+                    /* the cut cannot move before the first token nor behind the last one top_k kept */
+                    margin = INFINITY;
+                    if (j > 0) margin = fmin(margin, (target - before) / Sk);
+                    if (j + 1 < keep) margin = fmin(margin, (run - target) / Sk);
                     break;
                 }
             }

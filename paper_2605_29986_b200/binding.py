@@ -33,6 +33,8 @@ _SIGNATURES = {
                                                _vp, _vp, _vp, _int, _vp]),
     "cfgzip_masked_sample": (_int, [_vp, _i32, _vp, _vp, _i64, _vp, _int, _i64, _i32, _vp, _i64, _vp, ctypes.c_float, _vp,
                                     _vp, _vp, _vp, _int, _vp]),
+    "cfgzip_masked_sample_filtered": (_int, [_vp, _i32, _vp, _vp, _i64, _vp, _int, _i64, _i32, _vp, _i64, _vp, ctypes.c_float,
+                                             _i32, ctypes.c_float, _vp, _vp, _vp, _vp, _int, _vp]),
     "cfgzip_multi_mask_logsoftmax_argmax": (_int, [_vp, _i32, _vp, _i64, _i32, _vp, _int, _i64, _i32, _vp, _i64, _vp, _vp, _vp,
                                                    _vp, _vp]),
     "cfgzip_plan_rows": (_int, [_vp, _i32, _vp, _i32, _vp]),
@@ -175,6 +177,16 @@ def cfgzip_masked_sample(ctx: int, part0: int, row_part, class_mask, class_strid
         ctx, part0, _ptr(row_part), _ptr(class_mask), class_stride_words, _ptr(logits), dtype, row_stride_elems, B,
         _ptr(vocab_mask), vocab_stride_words, _ptr(u), inv_temperature, _ptr(token), _ptr(rep), _ptr(logp_token),
         _ptr(lse), mode, _stream(stream)), "cfgzip_masked_sample")
+
+
+def cfgzip_masked_sample_filtered(ctx: int, part0: int, row_part, class_mask, class_stride_words: int, logits, dtype: int,
+                                  row_stride_elems: int, B: int, vocab_mask, vocab_stride_words: int, u,
+                                  inv_temperature: float, top_k: int, top_p: float, token, rep=None, logp_token=None,
+                                  lse=None, mode: int = AUTO, stream=None) -> None:
+    _check(load_library().cfgzip_masked_sample_filtered(
+        ctx, part0, _ptr(row_part), _ptr(class_mask), class_stride_words, _ptr(logits), dtype, row_stride_elems, B,
+        _ptr(vocab_mask), vocab_stride_words, _ptr(u), inv_temperature, top_k, top_p, _ptr(token), _ptr(rep),
+        _ptr(logp_token), _ptr(lse), mode, _stream(stream)), "cfgzip_masked_sample_filtered")
 
 
 def cfgzip_multi_mask_logsoftmax_argmax(ctx: int, part0: int, class_masks, class_stride_words: int, masks_per_row: int,

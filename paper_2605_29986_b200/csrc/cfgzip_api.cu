@@ -638,7 +638,9 @@ int launch_fused(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, in
 // (one block per row) draws the token. Rows off the 16-byte grid, and shapes the pipelined kernel does not
 // take, go through the per-row kernel, whose single state per row stands for the whole row.
 template <int DT>
-int launch_sample(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, bool aligned, cudaStream_t st) {
+int launch_sample(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, bool aligned, int top_k, float top_p,
+                  cudaStream_t st) {
+    const bool filtered = top_k > 0 || top_p < 1.f;  // the draw is restricted to the most probable tokens
     int rc;
     DensePlan d;
     if (aligned) {
@@ -658,6 +660,8 @@ int launch_sample(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, b
         const dim3 grid(unsigned(d.n_groups_ub) * unsigned(d.S)), block{unsigned(d.threads)};
         if ((rc = launch_pipe<DT>(ctx, a, d, grid, block, st)) != CFGZIP_OK) return rc;
         const unsigned rows_grid = unsigned(d.n_groups_ub) * kGroupRows;
+        if (filtered)
+            return launch(ctx, k_sample_filtered<DT>, dim3(rows_grid), dim3(kFiltThreads), 0, st, a, 1, top_k, top_p);
         const size_t pad = row_blocks_pad(ctx, rows_grid, a.B);
         if (pad && (rc = ensure_smem(k_sample_rows<DT>, pad)) != CFGZIP_OK) return rc;
         return launch(ctx, k_sample_rows<DT>, dim3(rows_grid), dim3(kSampleThreads), pad, st, a, 1);
@@ -672,6 +676,9 @@ int launch_sample(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, b
     a.tail_state = 0;
     a.p0 = ctx->parts[size_t(a.part0)].dev;
     if ((rc = launch(ctx, k_step_generic<DT, true>, dim3(unsigned(a.B)), dim3(256), 0, st, a)) != CFGZIP_OK) return rc;
+    if (filtered)
+        return launch(ctx, k_sample_filtered<DT>, dim3(unsigned(ceil_div(a.B, kGroupRows)) * kGroupRows), dim3(kFiltThreads), 0,
+                      st, a, aligned ? 1 : 0, top_k, top_p);
     return launch(ctx, k_sample_rows<DT>, dim3(unsigned(ceil_div(a.B, kGroupRows)) * kGroupRows), dim3(kSampleThreads), 0, st,
                   a, aligned ? 1 : 0);
 }
@@ -1046,6 +1053,17 @@ int cfgzip_masked_sample(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* r
                          int64_t class_stride_words, void* logits, int dtype, int64_t row_stride_elems, int32_t B,
                          uint32_t* vocab_mask, int64_t vocab_stride_words, const float* u, float inv_temperature,
                          int32_t* token, int32_t* rep, float* logp_token, float* lse, int mode, void* stream) {
+    return cfgzip_masked_sample_filtered(ctx, part0, row_part, class_mask, class_stride_words, logits, dtype, row_stride_elems,
+                                         B, vocab_mask, vocab_stride_words, u, inv_temperature, 0, 1.f, token, rep, logp_token,
+                                         lse, mode, stream);
+}
+
+int cfgzip_masked_sample_filtered(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part,
+                                  const uint32_t* class_mask, int64_t class_stride_words, void* logits, int dtype,
+                                  int64_t row_stride_elems, int32_t B, uint32_t* vocab_mask, int64_t vocab_stride_words,
+                                  const float* u, float inv_temperature, int32_t top_k, float top_p, int32_t* token,
+                                  int32_t* rep, float* logp_token, float* lse, int mode, void* stream) {
+    if (top_k < 0 || !(top_p > 0.f)) return CFGZIP_E_ARG;
     int rc = check_step_args(ctx, class_mask, class_stride_words, B, mode);
     if (rc != CFGZIP_OK) return rc;
     if (dtype != CFGZIP_F32 && dtype != CFGZIP_BF16) return CFGZIP_E_ARG;
@@ -1091,7 +1109,8 @@ int cfgzip_masked_sample(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* r
     const bool al = aligned16(logits, row_stride_elems, es);
     a.wide = aligned32(logits, row_stride_elems, es);
     ctx->pdl_now = int64_t(B) * ps.V * es < (int64_t(192) << 20);
-    rc = dtype == CFGZIP_BF16 ? launch_sample<kBF16>(ctx, a, ps, mixed, al, st) : launch_sample<kF32>(ctx, a, ps, mixed, al, st);
+    rc = dtype == CFGZIP_BF16 ? launch_sample<kBF16>(ctx, a, ps, mixed, al, top_k, top_p, st)
+                              : launch_sample<kF32>(ctx, a, ps, mixed, al, top_k, top_p, st);
     ctx->pdl_now = true;
     return rc;
 }

@@ -1653,6 +1653,339 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample_rows(const __grid_con
 }
 
 // ---------------------------------------------------------------------------------------
+// Second kernel of a sampling step with top-k / top-p: one block per row keeps, of the row's allowed tokens in the
+// order (value, largest first; equal values by token id, lowest first), the first top_k (0 = all) and of those the
+// shortest beginning whose weight reaches top_p times the weight of what top_k kept (>= 1: all), then draws among
+// the kept tokens by inverse CDF in token order with the row's uniform number.
+// The kept set is { key > tau } plus the first m tokens, in token order, with key == tau, where key is an
+// order-preserving integer image of the logit; tau is found by bisection on the key with counts and weights of
+// { key >= mid } as the test. Weights are 40-bit fixed-point integers (exp((z - M) / T) * 2^40), so every sum is
+// exact whatever the order of the addends: the result is deterministic. The tokens whose weight is at least 2^-24
+// are first collected in shared memory (up to kFiltList of them): when the searched threshold lies among them,
+// which is the rule at the temperatures used for constrained decoding, the bisection never goes back to the row.
+// ---------------------------------------------------------------------------------------
+constexpr int kFiltThreads = 256;
+constexpr int kFiltList = 2048;
+constexpr float kFixOne = 1099511627776.f;  // 2^40
+
+__device__ __forceinline__ uint32_t logit_key(float z) {
+    z = z == 0.f ? 0.f : z;  // -0.0 and +0.0 are the same value
+    const uint32_t b = __float_as_uint(z);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float key_logit(uint32_t k) {
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
+}
+__device__ __forceinline__ unsigned long long fixed_weight(float z, float M, float scale) {
+    return __float2ull_rz(ex2f((z - M) * scale) * kFixOne);
+}
+
+struct CountMass {
+    unsigned int n;
+    unsigned long long w;
+};
+
+// Sum of one (count, weight) pair per thread over the block; everybody gets the total. s_n / s_w: one entry per warp.
+__device__ __forceinline__ CountMass block_sum(CountMass v, unsigned int* s_n, unsigned long long* s_w) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) {
+        v.n += __shfl_xor_sync(0xFFFFFFFFu, v.n, d);
+        v.w += __shfl_xor_sync(0xFFFFFFFFu, v.w, d);
+    }
+    __syncthreads();  // the arrays may still be read from the call before
+    if (lane == 0) {
+        s_n[warp] = v.n;
+        s_w[warp] = v.w;
+    }
+    __syncthreads();
+    CountMass t{0u, 0ull};
+#pragma unroll
+    for (int w = 0; w < kFiltThreads / 32; ++w) {
+        t.n += s_n[w];
+        t.w += s_w[w];
+    }
+    return t;
+}
+
+// Exclusive prefix sum of one 64-bit value per thread in thread order; total to everybody.
+__device__ __forceinline__ unsigned long long block_exclusive_scan_u64(unsigned long long v, unsigned long long* s_w,
+                                                                       unsigned long long& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned long long inc = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const unsigned long long up = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+        if (lane >= d) inc += up;
+    }
+    __syncthreads();
+    if (lane == 31) s_w[warp] = inc;
+    __syncthreads();
+    unsigned long long before = 0ull, all = 0ull;
+#pragma unroll
+    for (int w = 0; w < kFiltThreads / 32; ++w) {
+        const unsigned long long t = s_w[w];
+        if (w < warp) before += t;
+        all += t;
+    }
+    total = all;
+    return before + inc - v;
+}
+
+// Visit every token of a row, the block's threads side by side (8 consecutive tokens per thread and round).
+template <int DT, typename F>
+__device__ __forceinline__ void row_visit(const char* rowp, int V, bool aligned, F&& f) {
+    for (int t0 = threadIdx.x * 8; t0 < V; t0 += kFiltThreads * 8) {
+        float e[8];
+        if (aligned && t0 + 8 <= V) {
+            if (DT == kBF16) {
+                const uint4 v = __ldcg(reinterpret_cast<const uint4*>(rowp + size_t(t0) * 2));
+                e[0] = __uint_as_float(v.x << 16); e[1] = __uint_as_float(v.x & 0xFFFF0000u);
+                e[2] = __uint_as_float(v.y << 16); e[3] = __uint_as_float(v.y & 0xFFFF0000u);
+                e[4] = __uint_as_float(v.z << 16); e[5] = __uint_as_float(v.z & 0xFFFF0000u);
+                e[6] = __uint_as_float(v.w << 16); e[7] = __uint_as_float(v.w & 0xFFFF0000u);
+            } else {
+                const float4 v0 = __ldcg(reinterpret_cast<const float4*>(rowp + size_t(t0) * 4));
+                const float4 v1 = __ldcg(reinterpret_cast<const float4*>(rowp + size_t(t0) * 4 + 16));
+                e[0] = v0.x; e[1] = v0.y; e[2] = v0.z; e[3] = v0.w;
+                e[4] = v1.x; e[5] = v1.y; e[6] = v1.z; e[7] = v1.w;
+            }
+        } else {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) e[q] = t0 + q < V ? ldcg_elem<DT>(rowp, t0 + q) : -INFINITY;
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+            if (e[q] > kRefFloor) f(t0 + q, e[q]);  // masked logits are -inf
+    }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_constant__ StepArgs a, int aligned, int top_k,
+                                                                  float top_p) {
+    __shared__ uint32_t l_key[kFiltList];
+    __shared__ unsigned long long l_w[kFiltList];
+    __shared__ unsigned int s_n[kFiltThreads / 32];
+    __shared__ unsigned long long s_w[kFiltThreads / 32];
+    __shared__ float s_max[kFiltThreads / 32];
+    __shared__ unsigned int s_list_n;
+    pdl_prologue();
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int g = blockIdx.x / kGroupRows, j = blockIdx.x - g * kGroupRows;
+    if (a.n_groups && g >= __ldg(a.n_groups)) return;
+    int row;
+    if (a.group_rows) {
+        row = a.group_rows[g * kGroupRows + j];
+    } else {
+        row = g * kGroupRows + j;
+        if (row >= a.B) row = -1;
+    }
+    if (row < 0) return;
+    PartDev P = a.p0;
+    if (a.group_part) {
+        P = a.parts[a.group_part[g]];
+    } else if (a.row_part) {
+        const int part = a.row_part[row];
+        if (part < 0 || part >= a.n_parts || !a.parts[part].live || a.parts[part].V != a.V) return;  // counted by the step kernel
+        P = a.parts[part];
+    }
+    // the row maximum from the states the streaming kernel published
+    const Partial* src = row_slots(a, g, j);
+    float M = -INFINITY;
+    for (int k = tid; k < a.slots; k += kFiltThreads) M = fmaxf(M, __ldcg(&src[k].m));
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, d));
+    if (lane == 0) s_max[warp] = M;
+    if (tid == 0) s_list_n = 0u;
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < kFiltThreads / 32; ++w) M = fmaxf(M, s_max[w]);
+    if (!(M > kRefFloor)) {
+        // nothing allowed, or only -inf allowed: the lowest allowed token (if any) and -inf logs
+        if (warp == 0) {
+            unsigned long long cand = first_allowed_share(a, P, row, lane, 32);
+#pragma unroll
+            for (int d = 16; d >= 1; d >>= 1) {
+                const unsigned long long other = __shfl_xor_sync(0xFFFFFFFFu, cand, d);
+                cand = other < cand ? other : cand;
+            }
+            if (lane == 0) write_row_outputs(a, row, -INFINITY, 0.f, cand);
+        }
+        return;
+    }
+    constexpr int ES = DT == kBF16 ? 2 : 4;
+    const char* rowp = reinterpret_cast<const char*>(a.logits) + int64_t(row) * a.row_stride * ES;
+    const float scale = a.scale;
+    const uint32_t key_max = logit_key(M);
+    // candidates of weight >= 2^-24 go to the list; counts and weights of the whole row on the way
+    const uint32_t key_list = logit_key(M - 24.f / scale);
+    CountMass mine{0u, 0ull};
+    row_visit<DT>(rowp, a.V, aligned != 0, [&](int, float z) {
+        const unsigned long long w = fixed_weight(z, M, scale);
+        mine.n += 1u;
+        mine.w += w;
+        const uint32_t key = logit_key(z);
+        if (key >= key_list) {
+            const unsigned int at = atomicAdd(&s_list_n, 1u);
+            if (at < kFiltList) {
+                l_key[at] = key;
+                l_w[at] = w;
+            }
+        }
+    });
+    const CountMass all = block_sum(mine, s_n, s_w);
+    const unsigned int n_list = s_list_n;
+    const bool list_whole = n_list <= kFiltList;
+
+    // (count, weight) of the tokens with key >= lo: from the list when it is known to hold them all, else from the row
+    auto above = [&](uint32_t lo, bool from_list) {
+        CountMass v{0u, 0ull};
+        if (from_list) {
+            for (unsigned int i = tid; i < n_list; i += kFiltThreads)
+                if (l_key[i] >= lo) {
+                    v.n += 1u;
+                    v.w += l_w[i];
+                }
+        } else {
+            row_visit<DT>(rowp, a.V, aligned != 0, [&](int, float z) {
+                if (logit_key(z) >= lo) {
+                    v.n += 1u;
+                    v.w += fixed_weight(z, M, scale);
+                }
+            });
+        }
+        return block_sum(v, s_n, s_w);
+    };
+    // kept so far: { key > tau } and the first m tokens with key == tau; S their weight
+    uint32_t tau = 0u;
+    unsigned int m = 0xFFFFFFFFu;
+    unsigned long long S = all.w;
+    if (top_k > 0 && unsigned(top_k) < all.n) {
+        const bool use_list = list_whole && n_list >= unsigned(top_k);
+        uint32_t lo = use_list ? key_list : 0u, hi = key_max;  // count(>= lo) >= top_k holds
+        while (lo < hi) {
+            const uint32_t mid = lo + (hi - lo + 1u) / 2u;
+            if (above(mid, use_list).n >= unsigned(top_k)) lo = mid; else hi = mid - 1u;
+        }
+        tau = lo;
+        const CountMass gt = tau == key_max ? CountMass{0u, 0ull} : above(tau + 1u, use_list);
+        m = unsigned(top_k) - gt.n;
+        S = gt.w + static_cast<unsigned long long>(m) * fixed_weight(key_logit(tau), M, scale);
+    }
+    if (top_p < 1.f) {
+        // the target: top_p times the weight kept so far, rounded up; at least one unit so that one token is kept
+        unsigned long long target = static_cast<unsigned long long>(ceil(static_cast<double>(S) * static_cast<double>(top_p)));
+        target = target < 1ull ? 1ull : (target > S ? S : target);
+        // the list serves when it holds everything above tau, or when its weight alone reaches the target
+        bool use_list = list_whole && tau >= key_list;
+        if (!use_list && list_whole) use_list = above(key_list, true).w >= target;
+        const CountMass gt_tau = tau >= key_max ? CountMass{0u, 0ull} : above(tau + 1u, use_list);
+        if (gt_tau.w >= target) {
+            uint32_t lo = tau + 1u, hi = key_max;  // weight(>= lo) >= target holds
+            while (lo < hi) {
+                const uint32_t mid = lo + (hi - lo + 1u) / 2u;
+                if (above(mid, use_list).w >= target) lo = mid; else hi = mid - 1u;
+            }
+            const CountMass ge = above(lo, use_list);
+            const CountMass gt = lo == key_max ? CountMass{0u, 0ull} : above(lo + 1u, use_list);
+            const unsigned long long w_tie = fixed_weight(key_logit(lo), M, scale);
+            unsigned int need = ge.n - gt.n;  // all the ties unless fewer reach the target
+            if (w_tie > 0ull) {
+                const unsigned long long q = (target - gt.w + w_tie - 1ull) / w_tie;
+                if (q < need) need = unsigned(q);
+            }
+            tau = lo;
+            m = need < 1u ? 1u : need;
+            S = gt.w + static_cast<unsigned long long>(m) * w_tie;
+        } else {
+            // the target is reached among the ties at tau itself
+            const unsigned long long w_tie = fixed_weight(key_logit(tau), M, scale);
+            if (w_tie > 0ull) {
+                const unsigned long long q = (target - gt_tau.w + w_tie - 1ull) / w_tie;
+                if (q < m) m = unsigned(q < 1ull ? 1ull : q);
+            }
+            S = gt_tau.w + static_cast<unsigned long long>(m) * w_tie;
+        }
+    }
+
+    // Draw in token order. Every thread owns one contiguous segment of the row: first the ties per segment (their
+    // rank decides which of them are kept), then the kept weight per segment, then the one thread whose segment
+    // holds the crossing walks it once more.
+    const int seg = ((a.V + kFiltThreads - 1) / kFiltThreads + 7) & ~7;
+    const int t_lo = min(tid * seg, a.V), t_hi = min(t_lo + seg, a.V);
+    auto seg_visit = [&](auto&& f) {
+        for (int t0 = t_lo; t0 < t_hi; t0 += 8) {
+            float e[8];
+            if (aligned && t0 + 8 <= t_hi) {
+                if (DT == kBF16) {
+                    const uint4 v = __ldcg(reinterpret_cast<const uint4*>(rowp + size_t(t0) * 2));
+                    e[0] = __uint_as_float(v.x << 16); e[1] = __uint_as_float(v.x & 0xFFFF0000u);
+                    e[2] = __uint_as_float(v.y << 16); e[3] = __uint_as_float(v.y & 0xFFFF0000u);
+                    e[4] = __uint_as_float(v.z << 16); e[5] = __uint_as_float(v.z & 0xFFFF0000u);
+                    e[6] = __uint_as_float(v.w << 16); e[7] = __uint_as_float(v.w & 0xFFFF0000u);
+                } else {
+                    const float4 v0 = __ldcg(reinterpret_cast<const float4*>(rowp + size_t(t0) * 4));
+                    const float4 v1 = __ldcg(reinterpret_cast<const float4*>(rowp + size_t(t0) * 4 + 16));
+                    e[0] = v0.x; e[1] = v0.y; e[2] = v0.z; e[3] = v0.w;
+                    e[4] = v1.x; e[5] = v1.y; e[6] = v1.z; e[7] = v1.w;
+                }
+            } else {
+#pragma unroll
+                for (int q = 0; q < 8; ++q) e[q] = t0 + q < t_hi ? ldcg_elem<DT>(rowp, t0 + q) : -INFINITY;
+            }
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                if (e[q] > kRefFloor) f(t0 + q, e[q]);
+        }
+    };
+    unsigned long long my_ties = 0ull;
+    seg_visit([&](int, float z) { my_ties += logit_key(z) == tau ? 1ull : 0ull; });
+    unsigned long long total_ties;
+    const unsigned long long tie_base = block_exclusive_scan_u64(my_ties, s_w, total_ties);
+    unsigned long long my_w = 0ull, ties_seen = tie_base;
+    seg_visit([&](int, float z) {
+        const uint32_t key = logit_key(z);
+        if (key > tau || (key == tau && ties_seen++ < m)) my_w += fixed_weight(z, M, scale);
+    });
+    unsigned long long S_drawn;
+    const unsigned long long w_base = block_exclusive_scan_u64(my_w, s_w, S_drawn);
+    // u * S rounded down: the first token whose cumulative weight exceeds it is drawn
+    const float u = __ldg(a.u + row);
+    unsigned long long thr = static_cast<unsigned long long>(static_cast<double>(u) * static_cast<double>(S_drawn));
+    if (S_drawn > 0ull && thr >= S_drawn) thr = S_drawn - 1ull;
+    if (S_drawn == 0ull) {  // cannot happen while the row maximum is kept; reported as an empty row
+        if (tid == 0) {
+            a.argmax[row] = -1;
+            if (a.rep) a.rep[row] = -1;
+            if (a.lse) a.lse[row] = -INFINITY;
+            if (a.logp_argmax) a.logp_argmax[row] = -INFINITY;
+        }
+        return;
+    }
+    if (my_w > 0ull && w_base <= thr && thr < w_base + my_w) {
+        unsigned long long cum = w_base;
+        int token = -1;
+        float zt = 0.f;
+        ties_seen = tie_base;
+        seg_visit([&](int t, float z) {
+            const uint32_t key = logit_key(z);
+            if (key > tau || (key == tau && ties_seen++ < m)) {
+                cum += fixed_weight(z, M, scale);
+                if (token < 0 && cum > thr) {
+                    token = t;
+                    zt = z;
+                }
+            }
+        });
+        const float l = logf(static_cast<float>(S_drawn) * (1.f / kFixOne));
+        a.argmax[row] = token;
+        if (a.rep) a.rep[row] = token >= 0 ? __ldg(P.trep + token) : -1;
+        if (a.lse) a.lse[row] = fmaf(M, a.inv_t, l);
+        if (a.logp_argmax) a.logp_argmax[row] = (zt - M) * a.inv_t - l;
+    }
+}
+
+// ---------------------------------------------------------------------------------------
 // Row-split step on caller-provided tables: the per-row kernel above, with each row shared by
 // S blocks that meet through a scratch area of (max, sum-exp, token) states and one ticket
 // per row, exactly as the sparse kernel's blocks do. It touches no context: token->class and
