@@ -216,12 +216,14 @@ class StepRunner:
     """A ring of resident working buffers for one workload and a CUDA graph that runs one pass of steps over it."""
 
     def __init__(self, cz, torch, device: int, config: int, B: int = None, mode: str = "dense", steps_hint: int = 1000,
-                 unique: int = 8, tune=(), kind: str = "fused", ring: int = 0, inv_temperature: float = 0.0):
+                 unique: int = 8, tune=(), kind: str = "fused", ring: int = 0, inv_temperature: float = 0.0, top_k: int = 0,
+                 top_p: float = 1.0):
         self.cz, self.torch = cz, torch
         # kind: "fused" the whole step; "unfused" separate expand + mask calls (no reductions); "floor" the in-place
         # read-modify-write kernel over the same buffers (what a pass over these bytes costs at least)
         self.kind = kind
         self.inv_temperature = inv_temperature  # > 0: the sampling step (cfgzip_masked_sample) instead of the greedy one
+        self.top_k, self.top_p = top_k, top_p   # sampling step: restricted to the most probable tokens when set
         spec = synth.CONFIGS[config]
         self.B = B or spec["B"]
         wl = synth.make_workload(config, B=min(self.B, 64))  # unique logits rows; tiled up to B below
@@ -299,10 +301,10 @@ class StepRunner:
                                   self.B, self.mode, stream)
             cz.cfgzip_mask_logits(self.ctx, self.work[j], dt, self.V, self.B, self.V, self.vm[j], self.VW, stream)
         elif self.u is not None:
-            cz.cfgzip_masked_sample(
+            cz.cfgzip_masked_sample_filtered(
                 self.ctx, self.parts[0], self.row_part_arg, self.cm[j], self.KW, self.work[j], dt, self.V, self.B,
-                self.vm[j], self.VW, self.u[j], self.inv_temperature, self.am[j], self.rep[j], self.lpa[j], self.lse[j],
-                self.mode, stream)
+                self.vm[j], self.VW, self.u[j], self.inv_temperature, self.top_k, self.top_p, self.am[j], self.rep[j],
+                self.lpa[j], self.lse[j], self.mode, stream)
         else:
             cz.cfgzip_masked_logsoftmax_argmax(
                 self.ctx, self.parts[0], self.row_part_arg, self.cm[j], self.KW, self.work[j], dt, self.V, self.B,
@@ -449,6 +451,66 @@ def _e2e(runner: StepRunner, torch, n_steps: int):
     return dt_s, h2d, d2h
 
 
+def _offline_grouping(cz, torch) -> dict:
+    """cfgzip_group_tokens on a Llama-size vocabulary of synthetic signatures (2048 classes, 8-word rows), with the oracle's
+    grouping of a sample beside it; the call allocates, synchronises and frees (an offline step), all inside the time."""
+    V, K, W = 128256, 2048, 8
+    part = synth.zipf_partition(V, K, 1.1, seed=3)
+    rows = (synth.rng.u64(synth.rng.stream_key(8), K * W) % np.uint64(7)).astype(np.int32).reshape(K, W)
+    rows[:, 1], rows[:, 2] = np.arange(K) // 7, np.arange(K) % 7
+    sig = torch.from_numpy(np.ascontiguousarray(rows[part.c])).cuda()
+    lens = torch.from_numpy((1 + synth.rng.u64(synth.rng.stream_key(9), V) % np.uint64(12)).astype(np.int32)).cuda()
+    c = torch.empty(V, dtype=torch.int32, device="cuda"); r = torch.empty_like(c); k = torch.empty(1, dtype=torch.int32, device="cuda")
+    off = torch.empty(V + 1, dtype=torch.int32, device="cuda"); tok = torch.empty_like(c)
+    best = None
+    for _ in range(5):
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        cz.cfgzip_group_tokens(sig, W, lens, V, c, r, k, off, tok, torch.cuda.current_stream())
+        dt_s = time.perf_counter() - t0
+        best = dt_s if best is None else min(best, dt_s)
+    ok = int(k.cpu()[0]) == K and bool((c.cpu().numpy() == _first_occurrence_ids(part.c)).all())
+    return {"V": V, "classes": K, "row_words": W, "ms": best * 1e3, "tokens_per_s": V / best, "matches_partition": ok,
+            "what": "grouping of equal signature rows into classes, representatives and class lists on the GPU, wall clock "
+                    "of the whole call (allocation, 7 launches, synchronisation)"}
+
+
+def _first_occurrence_ids(c: np.ndarray) -> np.ndarray:
+    """Relabel class ids in the order of their lowest token id (bookkeeping for the check above)."""
+    _, first, inverse = np.unique(c, return_index=True, return_inverse=True)
+    rank = np.empty(len(first), dtype=np.int64)
+    rank[np.argsort(first)] = np.arange(len(first))
+    return rank[inverse]
+
+
+def _multi_mask(cz, torch, device: int, B: int = 8, M: int = 16, steps: int = 200) -> dict:
+    """cfgzip_multi_mask_logsoftmax_argmax: M class masks against each of B Llama-size rows (logits read once)."""
+    w = synth.make_workload(2, B=B)
+    part = w.partitions[0]
+    ctx = cz.cfgzip_create(device)
+    pid = cz.cfgzip_load_partition(ctx, part.c, w.V, part.r, w.K)
+    z = torch.from_numpy(w.logits(0).view(np.int16)).cuda()
+    cms = torch.from_numpy(synth.class_mask_bernoulli(w.K, B * M, 0.1, synth.rng.stream_key(77)).view(np.int32)).cuda()
+    VW = (w.V + 31) // 32
+    vm = torch.empty((B * M, VW), dtype=torch.int32, device="cuda")
+    am = torch.empty(B * M, dtype=torch.int32, device="cuda"); rep = torch.empty_like(am)
+    lse = torch.empty(B * M, dtype=torch.float32, device="cuda"); lpa = torch.empty_like(lse)
+    st = torch.cuda.Stream()
+    def run(n):
+        with torch.cuda.stream(st):
+            for _ in range(n):
+                cz.cfgzip_multi_mask_logsoftmax_argmax(ctx, pid, cms, cms.shape[1], M, z, cz.BF16, w.V, B, vm, VW, am, rep, lpa, lse, st)
+    run(20)
+    st.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(st); run(steps); e1.record(st)
+    st.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / steps
+    cz.cfgzip_destroy(ctx)
+    return {"B": B, "masks_per_row": M, "us_per_step": us, "row_masks_per_s": B * M / us * 1e6,
+            "what": "V=128256 K=2048 bf16, one logits buffer (L2-resident: a latency figure, not an HBM one)"}
+
+
 def _cpu_baseline(runner, budget_s: float = 12.0) -> dict:
     """The CPU oracle timed on steps of the same workload: with one thread per host core (rows split over a thread
     pool) and with a single thread, each for about half of `budget_s`."""
@@ -494,7 +556,7 @@ def run_own(args):
 
     solo = rank == 0 and world == 1
     runner = StepRunner(cz, torch, local_rank, args.workload, B=args.batch, mode=args.mode, steps_hint=args.steps,
-                        tune=args.tune, inv_temperature=args.sample_inv_temperature)
+                        tune=args.tune, inv_temperature=args.sample_inv_temperature, top_k=args.top_k, top_p=args.top_p)
     props = torch.cuda.get_device_properties(local_rank)
     sampler = ClockSampler("GPU-" + str(props.uuid))
     seconds, timed_steps, launches = runner.timed(args.steps, args.warmup, barrier, sampler)
@@ -606,6 +668,17 @@ def run_own(args):
                          "frac_of_measured": r6.alg_bytes() / us6 / 1e3 / peak})
             r6.close()
         line["sampling_step_T0.2"] = samp
+        # the same sampling step restricted to the most probable tokens (top-k, top-p), at the paper's temperature
+        filt = []
+        for top_k, top_p in ((50, 1.0), (0, 0.9)):
+            r8 = StepRunner(cz, torch, local_rank, args.workload, B=args.batch, mode=args.mode, steps_hint=64, unique=2,
+                            tune=args.tune, inv_temperature=5.0, top_k=top_k, top_p=top_p)
+            us8, _, l8 = _measure(r8)
+            filt.append({"top_k": top_k, "top_p": top_p, "B": r8.B, "us_per_step": us8, "launches_per_step": l8})
+            r8.close()
+        line["filtered_sampling_step_T0.2"] = filt
+        line["offline_grouping"] = _offline_grouping(cz, torch)
+        line["multi_mask_step"] = _multi_mask(cz, torch, local_rank)
         # the same step on two buffers that stay in the 126 MB L2: NOT an HBM figure, only the latency floor
         r5 = StepRunner(cz, torch, local_rank, args.workload, B=args.batch, mode=args.mode, steps_hint=2, unique=2,
                         tune=args.tune, ring=2)
@@ -717,6 +790,8 @@ def main(argv=None):
                     help="library tuning knob (see cfgzip_set_tuning); may be repeated")
     ap.add_argument("--sample-inv-temperature", type=float, default=0.0, metavar="1/T",
                     help="time the sampling step (cfgzip_masked_sample) at this inverse temperature instead of the greedy one")
+    ap.add_argument("--top-k", type=int, default=0, help="with --sample-inv-temperature: keep the k most probable tokens")
+    ap.add_argument("--top-p", type=float, default=1.0, help="with --sample-inv-temperature: keep the top-p nucleus")
     ap.add_argument("--no-extras", action="store_true", help="skip the larger-batch sweep")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args(argv)

@@ -26,6 +26,7 @@ struct Part {
 };
 
 constexpr size_t kPartialSlots = size_t(1) << 18;  // 4 MB of (max, sum, pos) slots
+constexpr size_t kFiltSmem = size_t(kFiltList) * 12;  // candidate list of the filtered sampling kernel
 constexpr int kTwoOctetItemsPerWarp = 3;           // bf16: two octets per lane from this many work items per warp on
 constexpr int kDefaultRows = 16384;
 
@@ -660,8 +661,10 @@ int launch_sample(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, b
         const dim3 grid(unsigned(d.n_groups_ub) * unsigned(d.S)), block{unsigned(d.threads)};
         if ((rc = launch_pipe<DT>(ctx, a, d, grid, block, st)) != CFGZIP_OK) return rc;
         const unsigned rows_grid = unsigned(d.n_groups_ub) * kGroupRows;
-        if (filtered)
-            return launch(ctx, k_sample_filtered<DT>, dim3(rows_grid), dim3(kFiltThreads), 0, st, a, 1, top_k, top_p);
+        if (filtered) {
+            if ((rc = ensure_smem(k_sample_filtered<DT>, kFiltSmem)) != CFGZIP_OK) return rc;
+            return launch(ctx, k_sample_filtered<DT>, dim3(rows_grid), dim3(kFiltThreads), kFiltSmem, st, a, 1, top_k, top_p);
+        }
         const size_t pad = row_blocks_pad(ctx, rows_grid, a.B);
         if (pad && (rc = ensure_smem(k_sample_rows<DT>, pad)) != CFGZIP_OK) return rc;
         return launch(ctx, k_sample_rows<DT>, dim3(rows_grid), dim3(kSampleThreads), pad, st, a, 1);
@@ -676,9 +679,11 @@ int launch_sample(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, b
     a.tail_state = 0;
     a.p0 = ctx->parts[size_t(a.part0)].dev;
     if ((rc = launch(ctx, k_step_generic<DT, true>, dim3(unsigned(a.B)), dim3(256), 0, st, a)) != CFGZIP_OK) return rc;
-    if (filtered)
-        return launch(ctx, k_sample_filtered<DT>, dim3(unsigned(ceil_div(a.B, kGroupRows)) * kGroupRows), dim3(kFiltThreads), 0,
-                      st, a, aligned ? 1 : 0, top_k, top_p);
+    if (filtered) {
+        if ((rc = ensure_smem(k_sample_filtered<DT>, kFiltSmem)) != CFGZIP_OK) return rc;
+        return launch(ctx, k_sample_filtered<DT>, dim3(unsigned(ceil_div(a.B, kGroupRows)) * kGroupRows), dim3(kFiltThreads),
+                      kFiltSmem, st, a, aligned ? 1 : 0, top_k, top_p);
+    }
     return launch(ctx, k_sample_rows<DT>, dim3(unsigned(ceil_div(a.B, kGroupRows)) * kGroupRows), dim3(kSampleThreads), 0, st,
                   a, aligned ? 1 : 0);
 }

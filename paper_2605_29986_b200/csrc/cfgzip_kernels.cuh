@@ -1660,20 +1660,27 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample_rows(const __grid_con
 // The kept set is { key > tau } plus the first m tokens, in token order, with key == tau, where key is an
 // order-preserving integer image of the logit; tau is found by bisection on the key with counts and weights of
 // { key >= mid } as the test. Weights are 40-bit fixed-point integers (exp((z - M) / T) * 2^40), so every sum is
-// exact whatever the order of the addends: the result is deterministic. The tokens whose weight is at least 2^-24
-// are first collected in shared memory (up to kFiltList of them): when the searched threshold lies among them,
-// which is the rule at the temperatures used for constrained decoding, the bisection never goes back to the row.
+// exact whatever the order of the addends: the result is deterministic. The tokens whose weight is not zero in that
+// format are first collected in shared memory (up to kFiltList of them): when they all fit, which is the rule at the
+// temperatures used for constrained decoding, the bisection never goes back to the row (a token of weight zero can
+// change neither a cumulative weight nor the draw).
 // ---------------------------------------------------------------------------------------
-constexpr int kFiltThreads = 256;
-constexpr int kFiltList = 2048;
+constexpr int kFiltThreads = 1024;
+constexpr int kFiltList = 12288;  // entries of the candidate list (12 bytes each, dynamic shared memory)
 constexpr float kFixOne = 1099511627776.f;  // 2^40
 
+// Order-preserving integer image of a logit and its inverse. bf16 logits only use the upper half of the float's
+// bits, so their keys are 16 bits wide and a bisection over them takes half the steps.
+template <int DT>
 __device__ __forceinline__ uint32_t logit_key(float z) {
     z = z == 0.f ? 0.f : z;  // -0.0 and +0.0 are the same value
     const uint32_t b = __float_as_uint(z);
-    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+    const uint32_t k = (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+    return DT == kBF16 ? k >> 16 : k;
 }
+template <int DT>
 __device__ __forceinline__ float key_logit(uint32_t k) {
+    if (DT == kBF16) k = (k << 16) | ((k & 0x8000u) ? 0u : 0xFFFFu);  // the lower half of a negative value's key is all ones
     return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
 }
 __device__ __forceinline__ unsigned long long fixed_weight(float z, float M, float scale) {
@@ -1685,25 +1692,30 @@ struct CountMass {
     unsigned long long w;
 };
 
-// Sum of one (count, weight) pair per thread over the block; everybody gets the total. s_n / s_w: one entry per warp.
-__device__ __forceinline__ CountMass block_sum(CountMass v, unsigned int* s_n, unsigned long long* s_w) {
+// Sum of one (count, weight) pair per thread over the block; everybody gets the total. s_n / s_w: two sets of one
+// entry per warp, used in turn (`turn` flips with every call), so that one barrier per call is enough: a warp can only
+// write a set again after every warp has passed the barrier of the call in between, i.e. has read this one.
+__device__ __forceinline__ CountMass block_sum(CountMass v, unsigned int* s_n, unsigned long long* s_w, int& turn) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
     for (int d = 16; d >= 1; d >>= 1) {
         v.n += __shfl_xor_sync(0xFFFFFFFFu, v.n, d);
         v.w += __shfl_xor_sync(0xFFFFFFFFu, v.w, d);
     }
-    __syncthreads();  // the arrays may still be read from the call before
+    constexpr int kWarps = kFiltThreads / 32;
+    unsigned int* n = s_n + turn * kWarps;
+    unsigned long long* w = s_w + turn * kWarps;
+    turn ^= 1;
     if (lane == 0) {
-        s_n[warp] = v.n;
-        s_w[warp] = v.w;
+        n[warp] = v.n;
+        w[warp] = v.w;
     }
     __syncthreads();
     CountMass t{0u, 0ull};
 #pragma unroll
-    for (int w = 0; w < kFiltThreads / 32; ++w) {
-        t.n += s_n[w];
-        t.w += s_w[w];
+    for (int i = 0; i < kWarps; ++i) {
+        t.n += n[i];
+        t.w += w[i];
     }
     return t;
 }
@@ -1732,42 +1744,56 @@ __device__ __forceinline__ unsigned long long block_exclusive_scan_u64(unsigned 
     return before + inc - v;
 }
 
-// Visit every token of a row, the block's threads side by side (8 consecutive tokens per thread and round).
+// Eight consecutive logits of a row from token t0 on (-inf past `end`), as floats.
+template <int DT>
+__device__ __forceinline__ void load_eight(const char* rowp, int t0, int end, bool aligned, float (&e)[8]) {
+    if (aligned && t0 + 8 <= end) {
+        if (DT == kBF16) {
+            const uint4 v = __ldcg(reinterpret_cast<const uint4*>(rowp + size_t(t0) * 2));
+            e[0] = __uint_as_float(v.x << 16); e[1] = __uint_as_float(v.x & 0xFFFF0000u);
+            e[2] = __uint_as_float(v.y << 16); e[3] = __uint_as_float(v.y & 0xFFFF0000u);
+            e[4] = __uint_as_float(v.z << 16); e[5] = __uint_as_float(v.z & 0xFFFF0000u);
+            e[6] = __uint_as_float(v.w << 16); e[7] = __uint_as_float(v.w & 0xFFFF0000u);
+        } else {
+            const float4 v0 = __ldcg(reinterpret_cast<const float4*>(rowp + size_t(t0) * 4));
+            const float4 v1 = __ldcg(reinterpret_cast<const float4*>(rowp + size_t(t0) * 4 + 16));
+            e[0] = v0.x; e[1] = v0.y; e[2] = v0.z; e[3] = v0.w;
+            e[4] = v1.x; e[5] = v1.y; e[6] = v1.z; e[7] = v1.w;
+        }
+    } else {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) e[q] = t0 + q < end ? ldcg_elem<DT>(rowp, t0 + q) : -INFINITY;
+    }
+}
+
+// Visit every token of a row, the block's threads side by side (8 consecutive tokens per thread and round, four
+// rounds in flight together).
 template <int DT, typename F>
 __device__ __forceinline__ void row_visit(const char* rowp, int V, bool aligned, F&& f) {
-    for (int t0 = threadIdx.x * 8; t0 < V; t0 += kFiltThreads * 8) {
-        float e[8];
-        if (aligned && t0 + 8 <= V) {
-            if (DT == kBF16) {
-                const uint4 v = __ldcg(reinterpret_cast<const uint4*>(rowp + size_t(t0) * 2));
-                e[0] = __uint_as_float(v.x << 16); e[1] = __uint_as_float(v.x & 0xFFFF0000u);
-                e[2] = __uint_as_float(v.y << 16); e[3] = __uint_as_float(v.y & 0xFFFF0000u);
-                e[4] = __uint_as_float(v.z << 16); e[5] = __uint_as_float(v.z & 0xFFFF0000u);
-                e[6] = __uint_as_float(v.w << 16); e[7] = __uint_as_float(v.w & 0xFFFF0000u);
-            } else {
-                const float4 v0 = __ldcg(reinterpret_cast<const float4*>(rowp + size_t(t0) * 4));
-                const float4 v1 = __ldcg(reinterpret_cast<const float4*>(rowp + size_t(t0) * 4 + 16));
-                e[0] = v0.x; e[1] = v0.y; e[2] = v0.z; e[3] = v0.w;
-                e[4] = v1.x; e[5] = v1.y; e[6] = v1.z; e[7] = v1.w;
-            }
-        } else {
+    constexpr int kInFlight = 4;
+    for (int t0 = threadIdx.x * 8; t0 < V; t0 += kFiltThreads * 8 * kInFlight) {
+        float e[kInFlight][8];
 #pragma unroll
-            for (int q = 0; q < 8; ++q) e[q] = t0 + q < V ? ldcg_elem<DT>(rowp, t0 + q) : -INFINITY;
-        }
+        for (int r = 0; r < kInFlight; ++r) load_eight<DT>(rowp, t0 + r * kFiltThreads * 8, V, aligned, e[r]);
 #pragma unroll
-        for (int q = 0; q < 8; ++q)
-            if (e[q] > kRefFloor) f(t0 + q, e[q]);  // masked logits are -inf
+        for (int r = 0; r < kInFlight; ++r)
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                if (e[r][q] > kRefFloor) f(t0 + r * kFiltThreads * 8 + q, e[r][q]);  // masked logits are -inf
     }
 }
 
 template <int DT>
 __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_constant__ StepArgs a, int aligned, int top_k,
                                                                   float top_p) {
-    __shared__ uint32_t l_key[kFiltList];
-    __shared__ unsigned long long l_w[kFiltList];
-    __shared__ unsigned int s_n[kFiltThreads / 32];
-    __shared__ unsigned long long s_w[kFiltThreads / 32];
+    extern __shared__ __align__(16) unsigned long long filt_smem[];
+    unsigned long long* const l_w = filt_smem;                                  // kFiltList weights
+    uint32_t* const l_key = reinterpret_cast<uint32_t*>(filt_smem + kFiltList);  // kFiltList keys
+    __shared__ unsigned int s_n[2 * kFiltThreads / 32];
+    __shared__ unsigned long long s_w[2 * kFiltThreads / 32];
+    __shared__ unsigned long long s_scan[kFiltThreads / 32];
     __shared__ float s_max[kFiltThreads / 32];
+    int turn = 0;
     __shared__ unsigned int s_list_n;
     pdl_prologue();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -1816,15 +1842,16 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
     constexpr int ES = DT == kBF16 ? 2 : 4;
     const char* rowp = reinterpret_cast<const char*>(a.logits) + int64_t(row) * a.row_stride * ES;
     const float scale = a.scale;
-    const uint32_t key_max = logit_key(M);
-    // candidates of weight >= 2^-24 go to the list; counts and weights of the whole row on the way
-    const uint32_t key_list = logit_key(M - 24.f / scale);
+    const uint32_t key_max = logit_key<DT>(M);
+    // the tokens whose fixed-point weight is not zero (z >= M - 40 / scale) go to the list; counts and weights of the
+    // whole row on the way
+    const uint32_t key_list = logit_key<DT>(M - 40.f / scale);
     CountMass mine{0u, 0ull};
     row_visit<DT>(rowp, a.V, aligned != 0, [&](int, float z) {
         const unsigned long long w = fixed_weight(z, M, scale);
         mine.n += 1u;
         mine.w += w;
-        const uint32_t key = logit_key(z);
+        const uint32_t key = logit_key<DT>(z);
         if (key >= key_list) {
             const unsigned int at = atomicAdd(&s_list_n, 1u);
             if (at < kFiltList) {
@@ -1833,7 +1860,7 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
             }
         }
     });
-    const CountMass all = block_sum(mine, s_n, s_w);
+    const CountMass all = block_sum(mine, s_n, s_w, turn);
     const unsigned int n_list = s_list_n;
     const bool list_whole = n_list <= kFiltList;
 
@@ -1848,20 +1875,21 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
                 }
         } else {
             row_visit<DT>(rowp, a.V, aligned != 0, [&](int, float z) {
-                if (logit_key(z) >= lo) {
+                if (logit_key<DT>(z) >= lo) {
                     v.n += 1u;
                     v.w += fixed_weight(z, M, scale);
                 }
             });
         }
-        return block_sum(v, s_n, s_w);
+        return block_sum(v, s_n, s_w, turn);
     };
     // kept so far: { key > tau } and the first m tokens with key == tau; S their weight
     uint32_t tau = 0u;
     unsigned int m = 0xFFFFFFFFu;
     unsigned long long S = all.w;
-    if (top_k > 0 && unsigned(top_k) < all.n) {
-        const bool use_list = list_whole && n_list >= unsigned(top_k);
+    // (with the whole list in hand a top_k beyond it only adds tokens of weight zero: nothing to do)
+    if (top_k > 0 && unsigned(top_k) < all.n && !(list_whole && unsigned(top_k) >= n_list)) {
+        const bool use_list = list_whole;
         uint32_t lo = use_list ? key_list : 0u, hi = key_max;  // count(>= lo) >= top_k holds
         while (lo < hi) {
             const uint32_t mid = lo + (hi - lo + 1u) / 2u;
@@ -1870,15 +1898,14 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
         tau = lo;
         const CountMass gt = tau == key_max ? CountMass{0u, 0ull} : above(tau + 1u, use_list);
         m = unsigned(top_k) - gt.n;
-        S = gt.w + static_cast<unsigned long long>(m) * fixed_weight(key_logit(tau), M, scale);
+        S = gt.w + static_cast<unsigned long long>(m) * fixed_weight(key_logit<DT>(tau), M, scale);
     }
     if (top_p < 1.f) {
         // the target: top_p times the weight kept so far, rounded up; at least one unit so that one token is kept
         unsigned long long target = static_cast<unsigned long long>(ceil(static_cast<double>(S) * static_cast<double>(top_p)));
         target = target < 1ull ? 1ull : (target > S ? S : target);
-        // the list serves when it holds everything above tau, or when its weight alone reaches the target
-        bool use_list = list_whole && tau >= key_list;
-        if (!use_list && list_whole) use_list = above(key_list, true).w >= target;
+        // the whole list serves: whatever it leaves out has weight zero
+        const bool use_list = list_whole;
         const CountMass gt_tau = tau >= key_max ? CountMass{0u, 0ull} : above(tau + 1u, use_list);
         if (gt_tau.w >= target) {
             uint32_t lo = tau + 1u, hi = key_max;  // weight(>= lo) >= target holds
@@ -1888,7 +1915,7 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
             }
             const CountMass ge = above(lo, use_list);
             const CountMass gt = lo == key_max ? CountMass{0u, 0ull} : above(lo + 1u, use_list);
-            const unsigned long long w_tie = fixed_weight(key_logit(lo), M, scale);
+            const unsigned long long w_tie = fixed_weight(key_logit<DT>(lo), M, scale);
             unsigned int need = ge.n - gt.n;  // all the ties unless fewer reach the target
             if (w_tie > 0ull) {
                 const unsigned long long q = (target - gt.w + w_tie - 1ull) / w_tie;
@@ -1899,7 +1926,7 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
             S = gt.w + static_cast<unsigned long long>(m) * w_tie;
         } else {
             // the target is reached among the ties at tau itself
-            const unsigned long long w_tie = fixed_weight(key_logit(tau), M, scale);
+            const unsigned long long w_tie = fixed_weight(key_logit<DT>(tau), M, scale);
             if (w_tie > 0ull) {
                 const unsigned long long q = (target - gt_tau.w + w_tie - 1ull) / w_tie;
                 if (q < m) m = unsigned(q < 1ull ? 1ull : q);
@@ -1914,41 +1941,28 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
     const int seg = ((a.V + kFiltThreads - 1) / kFiltThreads + 7) & ~7;
     const int t_lo = min(tid * seg, a.V), t_hi = min(t_lo + seg, a.V);
     auto seg_visit = [&](auto&& f) {
-        for (int t0 = t_lo; t0 < t_hi; t0 += 8) {
-            float e[8];
-            if (aligned && t0 + 8 <= t_hi) {
-                if (DT == kBF16) {
-                    const uint4 v = __ldcg(reinterpret_cast<const uint4*>(rowp + size_t(t0) * 2));
-                    e[0] = __uint_as_float(v.x << 16); e[1] = __uint_as_float(v.x & 0xFFFF0000u);
-                    e[2] = __uint_as_float(v.y << 16); e[3] = __uint_as_float(v.y & 0xFFFF0000u);
-                    e[4] = __uint_as_float(v.z << 16); e[5] = __uint_as_float(v.z & 0xFFFF0000u);
-                    e[6] = __uint_as_float(v.w << 16); e[7] = __uint_as_float(v.w & 0xFFFF0000u);
-                } else {
-                    const float4 v0 = __ldcg(reinterpret_cast<const float4*>(rowp + size_t(t0) * 4));
-                    const float4 v1 = __ldcg(reinterpret_cast<const float4*>(rowp + size_t(t0) * 4 + 16));
-                    e[0] = v0.x; e[1] = v0.y; e[2] = v0.z; e[3] = v0.w;
-                    e[4] = v1.x; e[5] = v1.y; e[6] = v1.z; e[7] = v1.w;
-                }
-            } else {
+        for (int t0 = t_lo; t0 < t_hi; t0 += 32) {
+            float e[4][8];
 #pragma unroll
-                for (int q = 0; q < 8; ++q) e[q] = t0 + q < t_hi ? ldcg_elem<DT>(rowp, t0 + q) : -INFINITY;
-            }
+            for (int r = 0; r < 4; ++r) load_eight<DT>(rowp, t0 + 8 * r, t_hi, aligned != 0, e[r]);
 #pragma unroll
-            for (int q = 0; q < 8; ++q)
-                if (e[q] > kRefFloor) f(t0 + q, e[q]);
+            for (int r = 0; r < 4; ++r)
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    if (e[r][q] > kRefFloor) f(t0 + 8 * r + q, e[r][q]);
         }
     };
     unsigned long long my_ties = 0ull;
-    seg_visit([&](int, float z) { my_ties += logit_key(z) == tau ? 1ull : 0ull; });
+    seg_visit([&](int, float z) { my_ties += logit_key<DT>(z) == tau ? 1ull : 0ull; });
     unsigned long long total_ties;
-    const unsigned long long tie_base = block_exclusive_scan_u64(my_ties, s_w, total_ties);
+    const unsigned long long tie_base = block_exclusive_scan_u64(my_ties, s_scan, total_ties);
     unsigned long long my_w = 0ull, ties_seen = tie_base;
     seg_visit([&](int, float z) {
-        const uint32_t key = logit_key(z);
+        const uint32_t key = logit_key<DT>(z);
         if (key > tau || (key == tau && ties_seen++ < m)) my_w += fixed_weight(z, M, scale);
     });
     unsigned long long S_drawn;
-    const unsigned long long w_base = block_exclusive_scan_u64(my_w, s_w, S_drawn);
+    const unsigned long long w_base = block_exclusive_scan_u64(my_w, s_scan, S_drawn);
     // u * S rounded down: the first token whose cumulative weight exceeds it is drawn
     const float u = __ldg(a.u + row);
     unsigned long long thr = static_cast<unsigned long long>(static_cast<double>(u) * static_cast<double>(S_drawn));
@@ -1968,7 +1982,7 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
         float zt = 0.f;
         ties_seen = tie_base;
         seg_visit([&](int t, float z) {
-            const uint32_t key = logit_key(z);
+            const uint32_t key = logit_key<DT>(z);
             if (key > tau || (key == tau && ties_seen++ < m)) {
                 cum += fixed_weight(z, M, scale);
                 if (token < 0 && cum > thr) {
