@@ -26,7 +26,7 @@ struct Part {
 };
 
 constexpr size_t kPartialSlots = size_t(1) << 18;  // 4 MB of (max, sum, pos) slots
-constexpr size_t kFiltSmem = size_t(kFiltList) * 12;  // candidate list of the filtered sampling kernel
+constexpr size_t kFiltSmem = size_t(kFiltList) * 16;  // candidate list of the filtered sampling kernel
 constexpr int kTwoOctetItemsPerWarp = 3;           // bf16: two octets per lane from this many work items per warp on
 constexpr int kDefaultRows = 16384;
 

@@ -1663,10 +1663,10 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample_rows(const __grid_con
 // exact whatever the order of the addends: the result is deterministic. The tokens whose weight is not zero in that
 // format are first collected in shared memory (up to kFiltList of them): when they all fit, which is the rule at the
 // temperatures used for constrained decoding, the bisection never goes back to the row (a token of weight zero can
-// change neither a cumulative weight nor the draw).
+// change neither a cumulative weight nor the draw), and the draw itself is a bisection on the token id over the list.
 // ---------------------------------------------------------------------------------------
 constexpr int kFiltThreads = 1024;
-constexpr int kFiltList = 12288;  // entries of the candidate list (12 bytes each, dynamic shared memory)
+constexpr int kFiltList = 12288;  // entries of the candidate list (16 bytes each, dynamic shared memory)
 constexpr float kFixOne = 1099511627776.f;  // 2^40
 
 // Order-preserving integer image of a logit and its inverse. bf16 logits only use the upper half of the float's
@@ -1789,6 +1789,7 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
     extern __shared__ __align__(16) unsigned long long filt_smem[];
     unsigned long long* const l_w = filt_smem;                                  // kFiltList weights
     uint32_t* const l_key = reinterpret_cast<uint32_t*>(filt_smem + kFiltList);  // kFiltList keys
+    int* const l_id = reinterpret_cast<int*>(l_key + kFiltList);                 // kFiltList token ids
     __shared__ unsigned int s_n[2 * kFiltThreads / 32];
     __shared__ unsigned long long s_w[2 * kFiltThreads / 32];
     __shared__ unsigned long long s_scan[kFiltThreads / 32];
@@ -1847,7 +1848,7 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
     // whole row on the way
     const uint32_t key_list = logit_key<DT>(M - 40.f / scale);
     CountMass mine{0u, 0ull};
-    row_visit<DT>(rowp, a.V, aligned != 0, [&](int, float z) {
+    row_visit<DT>(rowp, a.V, aligned != 0, [&](int t, float z) {
         const unsigned long long w = fixed_weight(z, M, scale);
         mine.n += 1u;
         mine.w += w;
@@ -1857,6 +1858,7 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
             if (at < kFiltList) {
                 l_key[at] = key;
                 l_w[at] = w;
+                l_id[at] = t;
             }
         }
     });
@@ -1933,6 +1935,52 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
             }
             S = gt_tau.w + static_cast<unsigned long long>(m) * w_tie;
         }
+    }
+
+    if (list_whole) {
+        // Draw from the list (it holds every token that carries weight, in no particular order): the ties that are
+        // kept are those with the m lowest ids, i.e. the ids up to id_cut; the drawn token is the lowest id t with
+        // (kept weight at ids <= t) > floor(u * kept weight). Both are found by bisection on the token id with a sum
+        // over the list as the test.
+        auto list_sum = [&](auto&& pred) {
+            CountMass v{0u, 0ull};
+            for (unsigned int i = tid; i < n_list; i += kFiltThreads)
+                if (pred(l_key[i], l_id[i])) {
+                    v.n += 1u;
+                    v.w += l_w[i];
+                }
+            return block_sum(v, s_n, s_w, turn);
+        };
+        int id_cut = a.V;
+        const unsigned int n_ties = list_sum([&](uint32_t key, int) { return key == tau; }).n;
+        if (m < n_ties) {
+            int lo = 0, hi = a.V - 1;  // the smallest id with at least m ties at or below it
+            while (lo < hi) {
+                const int mid = lo + (hi - lo) / 2;
+                if (list_sum([&](uint32_t key, int id) { return key == tau && id <= mid; }).n >= m) hi = mid; else lo = mid + 1;
+            }
+            id_cut = lo;
+        }
+        auto kept = [&](uint32_t key, int id) { return key > tau || (key == tau && id <= id_cut); };
+        const unsigned long long S_kept = list_sum(kept).w;
+        const float u = __ldg(a.u + row);
+        unsigned long long thr = static_cast<unsigned long long>(static_cast<double>(u) * static_cast<double>(S_kept));
+        if (thr >= S_kept) thr = S_kept - 1ull;  // (S_kept > 0: the row maximum is always kept)
+        int lo = 0, hi = a.V - 1;
+        while (lo < hi) {
+            const int mid = lo + (hi - lo) / 2;
+            if (list_sum([&](uint32_t key, int id) { return id <= mid && kept(key, id); }).w > thr) hi = mid; else lo = mid + 1;
+        }
+        const float l = logf(static_cast<float>(S_kept) * (1.f / kFixOne));
+        for (unsigned int i = tid; i < n_list; i += kFiltThreads)
+            if (l_id[i] == lo) {  // the one thread that holds the drawn token writes the row's results
+                const float zt = key_logit<DT>(l_key[i]);
+                a.argmax[row] = lo;
+                if (a.rep) a.rep[row] = __ldg(P.trep + lo);
+                if (a.lse) a.lse[row] = fmaf(M, a.inv_t, l);
+                if (a.logp_argmax) a.logp_argmax[row] = (zt - M) * a.inv_t - l;
+            }
+        return;
     }
 
     // Draw in token order. Every thread owns one contiguous segment of the row: first the ties per segment (their

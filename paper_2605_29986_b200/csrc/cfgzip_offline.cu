@@ -289,18 +289,32 @@ __global__ void k_group_assign(const int32_t* slot_of, const int32_t* min_id, co
 }
 
 // Class lists in ascending token id: one warp walks the tokens in order, 32 at a time; lanes of the same class share
-// one cursor and take consecutive places in lane order.
-__global__ void __launch_bounds__(32) k_group_lists(const int32_t* c, int V, int32_t* cursor, int32_t* tok) {
+// one cursor and take consecutive places in lane order. The cursors (class offsets to start with) sit in shared
+// memory when there are few enough classes, which takes the round trip to L2 out of every step of the walk.
+constexpr int kListCursorsShared = 48 * 1024 / 4;
+
+__global__ void __launch_bounds__(32) k_group_lists(const int32_t* c, int V, const int32_t* n_classes, int32_t* cursor,
+                                                    int32_t* tok) {
+    __shared__ int32_t s_cursor[kListCursorsShared];
     const int lane = threadIdx.x;
+    const int K = *n_classes;
+    const bool shared = K <= kListCursorsShared;
+    int32_t* cur = shared ? s_cursor : cursor;
+    if (shared) {
+        for (int k = lane; k < K; k += 32) s_cursor[k] = cursor[k];
+        __syncwarp();
+    }
+    int k_next = lane < V ? c[lane] : 0;  // the class of this lane's next token is fetched one round ahead
     for (int base = 0; base < V; base += 32) {
         const int t = base + lane;
         const bool have = t < V;
-        const int k = have ? c[t] : -1 - lane;  // lanes without a token match nobody
+        const int k = have ? k_next : -1 - lane;  // lanes without a token match nobody
+        if (t + 32 < V) k_next = c[t + 32];
         const unsigned peers = __match_any_sync(0xFFFFFFFFu, k);
         const int rank = __popc(peers & ((1u << lane) - 1u));
         const int leader = __ffs(peers) - 1;
         int at = 0;
-        if (have && lane == leader) at = atomicAdd(cursor + k, __popc(peers));
+        if (have && lane == leader) at = atomicAdd(cur + k, __popc(peers));
         at = __shfl_sync(0xFFFFFFFFu, at, leader);
         if (have) tok[at + rank] = t;
         __syncwarp();
@@ -354,7 +368,7 @@ extern "C" int cfgzip_group_tokens(const int32_t* signatures, int32_t row_words,
             k_exclusive_scan<<<1, kScanThreads, 0, st>>>(count, V, nullptr);
             ok = cudaMemcpyAsync(class_off, count, size_t(V + 1) * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess &&
                  cudaMemcpyAsync(cursor, count, size_t(V) * 4, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
-            if (ok) k_group_lists<<<1, 32, 0, st>>>(token_to_class, V, cursor, class_tok);
+            if (ok) k_group_lists<<<1, 32, 0, st>>>(token_to_class, V, n_classes, cursor, class_tok);
         }
         ok = ok && cudaGetLastError() == cudaSuccess;
     }
