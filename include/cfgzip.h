@@ -153,14 +153,15 @@ int cfgzip_mask_logits(cfgzip_ctx* ctx, void* logits, int dtype, int64_t row_str
  *   vocab_mask  : nullable; as in cfgzip_expand_mask
  *   mode        : CFGZIP_DENSE streams every row through the gather; CFGZIP_SPARSE builds each row's vocab
  *                 mask from the class->token lists of its allowed classes and never reads a logit that
- *                 is not allowed; CFGZIP_AUTO decides on the GPU, for the 8 rows of a row batch at a
- *                 time (the rows the gather kernel streams together): the class-list kernel runs first,
- *                 adds up the sizes of the classes the batch's rows allow and finishes the batches that
- *                 allow under 4 % (f32) or 1 % (bf16) of their tokens, the measured break-even; the
- *                 gather kernel behind it streams the other batches. The extra launch costs about
- *                 10 us, so steps of less than 384 MB of logits are dense outright. Callers whose
- *                 class masks are still on the host can choose for free: see cfgzip_choose_mode. The
- *                 results do not depend on the mode.
+ *                 is not allowed. CFGZIP_AUTO: the class-list kernel pays off when under 4 % (f32) or 1 %
+ *                 (bf16) of the tokens are allowed, the measured break-even. Callers whose class masks are
+ *                 still in host memory, where the grammar engine leaves them, get that choice for free
+ *                 from cfgzip_choose_mode (cfgzip_decode_step_host with CFGZIP_AUTO uses it). On device
+ *                 masks the choice needs one more launch (the class-list kernel runs first, adds up the
+ *                 sizes of the classes the 8 rows of a row batch allow and finishes the batches below the
+ *                 break-even; the gather kernel behind it streams the others), which costs 6 to 16 % on a
+ *                 batch that turns out dense: so CFGZIP_AUTO means CFGZIP_DENSE here unless the caller
+ *                 opts in (tuning knob "auto_min_mbytes"). The results do not depend on the mode.
  * A row with no allowed token, or whose allowed logits are all -inf, gets lse =
  * logp_argmax = -inf (the latter still returns the lowest allowed id). +inf and NaN
  * logits are outside the contract for the reductions (the masking itself still copies
@@ -251,8 +252,8 @@ int cfgzip_map_tokens(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_
  * which is where the grammar engine leaves them (Section 3.1, "Inference": the engine produces the mask over the
  * classes; Section 4 runs it on the CPU). Adds up the sizes of the classes every row allows and returns
  * CFGZIP_SPARSE when under 4 % (f32) or 1 % (bf16) of the batch's tokens are allowed (the measured break-even of the
- * two kernels; tuning knob "auto_sparse_permille"), else CFGZIP_DENSE; a negative status on bad arguments. Touches
- * no GPU and launches nothing. row_part_host: NULL or host int32 [B].
+ * two kernels; tuning knob "auto_sparse_permille"), else CFGZIP_DENSE; a negative status on bad arguments. The count
+ * stops as soon as the batch is known to be dense. Touches no GPU and launches nothing. row_part_host: NULL or host int32 [B].
  */
 int cfgzip_choose_mode(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part_host,
                        const uint32_t* class_mask_host /*host [B, class_stride_words]*/, int64_t class_stride_words,
@@ -410,7 +411,8 @@ int cfgzip_launch_count(cfgzip_ctx* ctx, int64_t* out);
  *   "auto_sparse_permille"  CFGZIP_AUTO: a row batch stays with the class-list kernel when under this many
  *                  thousandths of its tokens are allowed (0..1000; 0 = always dense; -1 = by element type, the default: 40 for
  *                  f32, 10 for bf16)
- *   "auto_min_mbytes"  CFGZIP_AUTO: steps with fewer megabytes of logits are dense without looking (default 384)
+ *   "auto_min_mbytes"  CFGZIP_AUTO on device-resident masks: steps of at least this many megabytes of logits let the GPU
+ *                  choose per batch of 8 rows, at the price of one more launch (-1 = never, the default)
  *   "fold"         0 = every warp of the streaming kernel publishes its row states and a second launch (one block or
  *                  warp per row) folds them and writes the results (default: the fastest at every size measured);
  *                  1 = the streaming kernel's last block of every row group does that itself, one launch per step;

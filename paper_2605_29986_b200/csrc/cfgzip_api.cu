@@ -93,7 +93,8 @@ struct cfgzip_ctx {
     int32_t lane_octets = 0;  // bf16 pipelined kernel: octets per lane and row (0 = automatic, 1, 2)
     int32_t auto_permille = -1;  // automatic mode: groups that allow under this many thousandths of their tokens go to the
                                  // class lists; -1 = by element type (measured break-even: f32 40, bf16 10)
-    int64_t auto_min_bytes = int64_t(384) << 20;  // automatic mode: steps with fewer bytes of logits are dense outright
+    int64_t auto_min_bytes = -1;  // automatic mode on device-resident masks: steps of at least this many bytes of logits let the
+                                  // GPU choose (one more launch); -1 = never (dense): the choice from host masks costs nothing
     int32_t fold = 0;         // pipelined kernel: the last block of a row group writes the rows' results (one launch per step)
     int32_t expire_test = 0;  // test hook: the pipelined kernel reports its first completed wait as run out
 };
@@ -580,7 +581,8 @@ int launch_fused(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, in
             int sp_S = 0, sp_per = 0;
             const int permille = ctx->auto_permille >= 0 ? ctx->auto_permille : (DT == kBF16 ? 10 : 40);
             const bool choose = mode == CFGZIP_AUTO && d.depth > 0 && permille > 0 && ctx->d_row_mode != nullptr &&
-                                a.B <= ctx->reserved_rows && int64_t(a.B) * a.V * (DT == kBF16 ? 2 : 4) >= ctx->auto_min_bytes &&
+                                a.B <= ctx->reserved_rows && ctx->auto_min_bytes >= 0 &&
+                                int64_t(a.B) * a.V * (DT == kBF16 ? 2 : 4) >= ctx->auto_min_bytes &&
                                 plan_sparse(ctx, ps, a.B, true, &sp_S, &sp_per);
             if (choose) {
                 if (d.fold_off) d.smem -= size_t(kGroupRows) * (d.WT + 1) * sizeof(Partial);
@@ -1224,8 +1226,12 @@ int cfgzip_choose_mode(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row
     if (rc != CFGZIP_OK) return rc;
     if (B == 0) return CFGZIP_DENSE;
     if (!class_mask_host || class_stride_words < ps.maxKW) return CFGZIP_E_ARG;
-    unsigned long long allowed = 0, rows = 0;
-    for (int32_t b = 0; b < B; ++b) {
+    const int permille = ctx->auto_permille >= 0 ? ctx->auto_permille : (dtype == CFGZIP_BF16 ? 10 : 40);
+    // the gather kernel wins as soon as the allowed tokens reach permille / 1000 of the batch (rows with a bad partition
+    // id count as rows: they make the batch look sparser, never denser): stop counting there
+    const unsigned long long enough = (static_cast<unsigned long long>(permille) * unsigned(B) * unsigned(ps.V) + 999ull) / 1000ull;
+    unsigned long long allowed = 0;
+    for (int32_t b = 0; b < B && allowed < enough; ++b) {
         const int32_t id = row_part_host ? row_part_host[b] : part0;
         if (id < 0 || size_t(id) >= ctx->parts.size() || !ctx->parts[size_t(id)].live || ctx->parts[size_t(id)].V != ps.V) continue;
         const Part& p = ctx->parts[size_t(id)];
@@ -1238,10 +1244,8 @@ int cfgzip_choose_mode(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row
                 word &= word - 1u;
             }
         }
-        ++rows;
     }
-    const int permille = ctx->auto_permille >= 0 ? ctx->auto_permille : (dtype == CFGZIP_BF16 ? 10 : 40);
-    return allowed * 1000ull < static_cast<unsigned long long>(permille) * rows * unsigned(ps.V) ? CFGZIP_SPARSE : CFGZIP_DENSE;
+    return allowed * 1000ull < static_cast<unsigned long long>(permille) * unsigned(B) * unsigned(ps.V) ? CFGZIP_SPARSE : CFGZIP_DENSE;
 }
 
 int cfgzip_decode_step_host(cfgzip_ctx* ctx, cfgzip_part_id part0, const int32_t* row_part_host,
@@ -1415,8 +1419,8 @@ int cfgzip_set_tuning(cfgzip_ctx* ctx, const char* name, int32_t value) {
         if (value < -1 || value > 1000) return CFGZIP_E_ARG;
         ctx->auto_permille = value;
     } else if (!std::strcmp(name, "auto_min_mbytes")) {
-        if (value < 0) return CFGZIP_E_ARG;
-        ctx->auto_min_bytes = int64_t(value) << 20;
+        if (value < -1) return CFGZIP_E_ARG;
+        ctx->auto_min_bytes = value < 0 ? -1 : int64_t(value) << 20;
     } else if (!std::strcmp(name, "fold")) {
         if (value < 0 || value > 2) return CFGZIP_E_ARG;
         ctx->fold = value;
