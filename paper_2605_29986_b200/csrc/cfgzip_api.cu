@@ -78,6 +78,7 @@ struct cfgzip_ctx {
     int32_t row_warps = 0;
     int32_t pdl = 1;
     bool pdl_now = true;      // set per call: programmatic dependent launch only pays for short kernels
+    int cluster_now = 1;      // set around a launch: blocks per thread-block cluster
     // cuTensorMapEncodeTiled, looked up through the runtime (no link against the driver library)
     CUresult (*encode_tiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -121,11 +122,22 @@ int launch(cfgzip_ctx* ctx, void (*kernel)(KArgs...), dim3 grid, dim3 block, siz
     cfg.blockDim = block;
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    int n_attr = 0;
+    if (ctx->pdl == 2 || (ctx->pdl && ctx->pdl_now)) {
+        attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+        ++n_attr;
+    }
+    if (ctx->cluster_now > 1) {  // neighbouring blocks along x form a thread-block cluster
+        attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+        attr[n_attr].val.clusterDim.x = unsigned(ctx->cluster_now);
+        attr[n_attr].val.clusterDim.y = 1;
+        attr[n_attr].val.clusterDim.z = 1;
+        ++n_attr;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = (ctx->pdl == 2 || (ctx->pdl && ctx->pdl_now)) ? 1 : 0;
+    cfg.numAttrs = unsigned(n_attr);
     if (cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...) != cudaSuccess) {
         cudaGetLastError();
         return CFGZIP_E_CUDA;
@@ -637,6 +649,22 @@ int launch_fused(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, in
     return rc;
 }
 
+// The draw of a sampling step with top-k / top-p. One block per row leaves most of the device idle on a short batch,
+// so 4 or 2 blocks (a thread-block cluster) share a row while that many blocks still fit the device in one wave.
+template <int DT>
+int launch_filtered(cfgzip_ctx* ctx, const StepArgs& a, unsigned rows_grid, int aligned, int top_k, float top_p,
+                    cudaStream_t st) {
+    int rc;
+    if ((rc = ensure_smem(k_sample_filtered<DT>, kFiltSmem)) != CFGZIP_OK) return rc;
+    const unsigned sms = unsigned(std::max(ctx->sm_count, 1));
+    const unsigned per_row = rows_grid * 4 <= sms ? 4u : (rows_grid * 2 <= sms ? 2u : 1u);
+    ctx->cluster_now = int(per_row);
+    rc = launch(ctx, k_sample_filtered<DT>, dim3(rows_grid * per_row), dim3(kFiltThreads), kFiltSmem, st, a, aligned, top_k,
+                top_p);
+    ctx->cluster_now = 1;
+    return rc;
+}
+
 // A sampling step: the streaming kernel leaves the states of a row in token order, the sampling kernel
 // (one block per row) draws the token. Rows off the 16-byte grid, and shapes the pipelined kernel does not
 // take, go through the per-row kernel, whose single state per row stands for the whole row.
@@ -663,10 +691,7 @@ int launch_sample(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, b
         const dim3 grid(unsigned(d.n_groups_ub) * unsigned(d.S)), block{unsigned(d.threads)};
         if ((rc = launch_pipe<DT>(ctx, a, d, grid, block, st)) != CFGZIP_OK) return rc;
         const unsigned rows_grid = unsigned(d.n_groups_ub) * kGroupRows;
-        if (filtered) {
-            if ((rc = ensure_smem(k_sample_filtered<DT>, kFiltSmem)) != CFGZIP_OK) return rc;
-            return launch(ctx, k_sample_filtered<DT>, dim3(rows_grid), dim3(kFiltThreads), kFiltSmem, st, a, 1, top_k, top_p);
-        }
+        if (filtered) return launch_filtered<DT>(ctx, a, rows_grid, 1, top_k, top_p, st);
         const size_t pad = row_blocks_pad(ctx, rows_grid, a.B);
         if (pad && (rc = ensure_smem(k_sample_rows<DT>, pad)) != CFGZIP_OK) return rc;
         return launch(ctx, k_sample_rows<DT>, dim3(rows_grid), dim3(kSampleThreads), pad, st, a, 1);
@@ -681,11 +706,8 @@ int launch_sample(cfgzip_ctx* ctx, StepArgs& a, const PartSet& ps, bool mixed, b
     a.tail_state = 0;
     a.p0 = ctx->parts[size_t(a.part0)].dev;
     if ((rc = launch(ctx, k_step_generic<DT, true>, dim3(unsigned(a.B)), dim3(256), 0, st, a)) != CFGZIP_OK) return rc;
-    if (filtered) {
-        if ((rc = ensure_smem(k_sample_filtered<DT>, kFiltSmem)) != CFGZIP_OK) return rc;
-        return launch(ctx, k_sample_filtered<DT>, dim3(unsigned(ceil_div(a.B, kGroupRows)) * kGroupRows), dim3(kFiltThreads),
-                      kFiltSmem, st, a, aligned ? 1 : 0, top_k, top_p);
-    }
+    if (filtered)
+        return launch_filtered<DT>(ctx, a, unsigned(ceil_div(a.B, kGroupRows)) * kGroupRows, aligned ? 1 : 0, top_k, top_p, st);
     return launch(ctx, k_sample_rows<DT>, dim3(unsigned(ceil_div(a.B, kGroupRows)) * kGroupRows), dim3(kSampleThreads), 0, st,
                   a, aligned ? 1 : 0);
 }

@@ -5,6 +5,7 @@
 #pragma once
 
 #include <cuda.h>
+#include <type_traits>
 
 #include "cfgzip_device.cuh"
 
@@ -1658,12 +1659,13 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample_rows(const __grid_con
 // shortest beginning whose weight reaches top_p times the weight of what top_k kept (>= 1: all), then draws among
 // the kept tokens by inverse CDF in token order with the row's uniform number.
 // The kept set is { key > tau } plus the first m tokens, in token order, with key == tau, where key is an
-// order-preserving integer image of the logit; tau is found by bisection on the key with counts and weights of
-// { key >= mid } as the test. Weights are 40-bit fixed-point integers (exp((z - M) / T) * 2^40), so every sum is
+// order-preserving integer image of the logit; tau is the largest key with enough tokens (top-k) or enough weight
+// (top-p) at or above it. Weights are 40-bit fixed-point integers (exp((z - M) / T) * 2^40), so every sum is
 // exact whatever the order of the addends: the result is deterministic. The tokens whose weight is not zero in that
-// format are first collected in shared memory (up to kFiltList of them): when they all fit, which is the rule at the
-// temperatures used for constrained decoding, the bisection never goes back to the row (a token of weight zero can
-// change neither a cumulative weight nor the draw), and the draw itself is a bisection on the token id over the list.
+// format are first collected in shared memory (up to kFiltList of them). When they all fit, which is the rule at the
+// temperatures used for constrained decoding, nothing goes back to the row (a token of weight zero can change neither
+// a cumulative weight nor the draw): tau, the last tie that is kept and the drawn token each come out of a radix
+// search over the list, ten bits per round (list_select). Otherwise tau is found by bisection with passes over the row.
 // ---------------------------------------------------------------------------------------
 constexpr int kFiltThreads = 1024;
 constexpr int kFiltList = 12288;  // entries of the candidate list (16 bytes each, dynamic shared memory)
@@ -1783,6 +1785,180 @@ __device__ __forceinline__ void row_visit(const char* rowp, int V, bool aligned,
     }
 }
 
+// ---- thread-block cluster: rank, barrier, reads of a peer block's shared memory -----------------
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_blocks() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+    return r;
+}
+// every thread of every block of the cluster (a hardware barrier like the block's own: no flag is polled)
+__device__ __forceinline__ void cluster_barrier() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t peer_shared(const void* mine, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(mine)), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ uint32_t ld_peer_u32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ unsigned long long ld_peer_u64(uint32_t addr) {
+    unsigned long long v;
+    asm volatile("ld.shared::cluster.u64 %0, [%1];" : "=l"(v) : "r"(addr) : "memory");
+    return v;
+}
+
+// ---- the searches over the candidate list run on the first kSelThreads threads of the block (a list of a few
+// thousand entries does not feed more, and barriers and sums across 8 warps cost a fraction of those across 32)
+constexpr int kSelThreads = 256;
+constexpr int kSelBuckets = 1024;  // ten bits of the value per round; kSelBuckets / kSelThreads buckets per thread
+__device__ __forceinline__ void sel_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kSelThreads) : "memory"); }
+
+// Exclusive prefix of one (count, weight) pair per thread in thread order over those threads; total to everybody.
+// s_n / s_w: two sets of one entry per warp, used in turn as in block_sum.
+__device__ __forceinline__ CountMass sel_exclusive_scan(CountMass v, unsigned int* s_n, unsigned long long* s_w, int& turn,
+                                                        CountMass& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    CountMass inc = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const unsigned int un = __shfl_up_sync(0xFFFFFFFFu, inc.n, d);
+        const unsigned long long uw = __shfl_up_sync(0xFFFFFFFFu, inc.w, d);
+        if (lane >= d) {
+            inc.n += un;
+            inc.w += uw;
+        }
+    }
+    constexpr int kWarps = kSelThreads / 32;
+    unsigned int* n = s_n + turn * kWarps;
+    unsigned long long* w = s_w + turn * kWarps;
+    turn ^= 1;
+    if (lane == 31) {
+        n[warp] = inc.n;
+        w[warp] = inc.w;
+    }
+    sel_sync();
+    CountMass before{0u, 0ull}, all{0u, 0ull};
+#pragma unroll
+    for (int i = 0; i < kWarps; ++i) {
+        const unsigned int tn = n[i];
+        const unsigned long long tw = w[i];
+        if (i < warp) {
+            before.n += tn;
+            before.w += tw;
+        }
+        all.n += tn;
+        all.w += tw;
+    }
+    total = all;
+    return CountMass{before.n + inc.n - v.n, before.w + inc.w - v.w};
+}
+
+// Result of a search: the value found, (count, weight) of the entries below it and of the entries at it.
+struct Picked {
+    uint32_t x;
+    CountMass before, at;
+};
+
+// Smallest value x such that the entries of the list with value <= x together count (BY_WEIGHT: weigh) more than thr.
+// xg(i, x, gn, gw) gives entry i's value (below 2^bits), count and weight (both 0: the entry takes no part); the
+// caller guarantees that all entries together exceed thr. Ten bits of the value per round, highest first: a histogram
+// of the round's digit over the entries that agree with the digits found so far, a prefix sum over the buckets, and
+// the one bucket in which the running sum passes thr is the next digit. Weights are added as two 32-bit halves (the
+// carry out of the lower half is seen in the value the atomic returns), which keeps every atomic a native one.
+template <bool BY_WEIGHT, typename F>
+__device__ __forceinline__ Picked list_select(unsigned int n_list, int bits, unsigned long long thr, F&& xg, unsigned int* h_n,
+                                              unsigned int* h_lo, unsigned int* h_hi, unsigned long long* s_pick,
+                                              unsigned int* s_n, unsigned long long* s_w, int& turn) {
+    const int tid = threadIdx.x;
+    const int rounds = bits <= 10 ? 1 : (bits + 9) / 10;
+    constexpr int kPer = kSelBuckets / kSelThreads;
+    static_assert(kPer == 4, "a thread reads its buckets as one 16-byte vector per array");
+    unsigned long long prefix = 0ull;
+    CountMass carry{0u, 0ull}, at{0u, 0ull};  // carry: the entries below the digits found so far
+    for (int rd = rounds - 1; rd >= 0; --rd) {
+        const int shift = rd * 10;
+        unsigned long long* pick = s_pick + 8 * (rd & 1);
+        reinterpret_cast<uint4*>(h_n)[tid] = make_uint4(0u, 0u, 0u, 0u);
+        reinterpret_cast<uint4*>(h_lo)[tid] = make_uint4(0u, 0u, 0u, 0u);
+        reinterpret_cast<uint4*>(h_hi)[tid] = make_uint4(0u, 0u, 0u, 0u);
+        sel_sync();
+        if (tid == 0) {  // (what stands if no bucket qualifies: cannot happen under the caller's guarantee)
+            pick[0] = 0ull;
+            pick[1] = carry.n;
+            pick[2] = carry.w;
+            pick[3] = 0ull;
+            pick[4] = 0ull;
+        }
+        for (unsigned int i = tid; i < n_list; i += kSelThreads) {
+            uint32_t x;
+            unsigned int gn;
+            unsigned long long gw;
+            xg(i, x, gn, gw);
+            if ((gn != 0u || gw != 0ull) && (static_cast<unsigned long long>(x) >> (shift + 10)) == prefix) {
+                const uint32_t b = (x >> shift) & (kSelBuckets - 1);
+                if (gn) atomicAdd(&h_n[b], gn);
+                if (gw) {
+                    const uint32_t lo = static_cast<uint32_t>(gw);
+                    uint32_t hi = static_cast<uint32_t>(gw >> 32);
+                    if (lo) {
+                        const uint32_t old = atomicAdd(&h_lo[b], lo);
+                        hi += (old + lo) < old ? 1u : 0u;
+                    }
+                    if (hi) atomicAdd(&h_hi[b], hi);
+                }
+            }
+        }
+        sel_sync();
+        const uint4 vn = reinterpret_cast<const uint4*>(h_n)[tid];
+        const uint4 vl = reinterpret_cast<const uint4*>(h_lo)[tid];
+        const uint4 vh = reinterpret_cast<const uint4*>(h_hi)[tid];
+        const CountMass h[kPer] = {{vn.x, (static_cast<unsigned long long>(vh.x) << 32) | vl.x},
+                                   {vn.y, (static_cast<unsigned long long>(vh.y) << 32) | vl.y},
+                                   {vn.z, (static_cast<unsigned long long>(vh.z) << 32) | vl.z},
+                                   {vn.w, (static_cast<unsigned long long>(vh.w) << 32) | vl.w}};
+        CountMass mine{0u, 0ull}, total;
+#pragma unroll
+        for (int b = 0; b < kPer; ++b) {
+            mine.n += h[b].n;
+            mine.w += h[b].w;
+        }
+        CountMass run = sel_exclusive_scan(mine, s_n, s_w, turn, total);
+        run.n += carry.n;
+        run.w += carry.w;
+#pragma unroll
+        for (int b = 0; b < kPer; ++b) {
+            const unsigned long long below = BY_WEIGHT ? run.w : static_cast<unsigned long long>(run.n);
+            const unsigned long long here = BY_WEIGHT ? h[b].w : static_cast<unsigned long long>(h[b].n);
+            if (below <= thr && thr < below + here) {
+                pick[0] = static_cast<unsigned long long>(tid * kPer + b);
+                pick[1] = run.n;
+                pick[2] = run.w;
+                pick[3] = h[b].n;
+                pick[4] = h[b].w;
+            }
+            run.n += h[b].n;
+            run.w += h[b].w;
+        }
+        sel_sync();
+        prefix = (prefix << 10) | pick[0];
+        carry = CountMass{static_cast<unsigned int>(pick[1]), pick[2]};
+        at = CountMass{static_cast<unsigned int>(pick[3]), pick[4]};
+    }
+    return Picked{static_cast<uint32_t>(prefix), carry, at};
+}
+
+// One row per cluster of blocks (1, 2 or 4 of them: a short batch has fewer rows than the device has
+// multiprocessors). Every block collects the candidates of its share of the row; the first block of the cluster
+// then gathers the lists through the cluster's shared memory and carries on alone.
 template <int DT>
 __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_constant__ StepArgs a, int aligned, int top_k,
                                                                   float top_p) {
@@ -1793,12 +1969,21 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
     __shared__ unsigned int s_n[2 * kFiltThreads / 32];
     __shared__ unsigned long long s_w[2 * kFiltThreads / 32];
     __shared__ unsigned long long s_scan[kFiltThreads / 32];
+    __shared__ __align__(16) unsigned int s_hn[kSelBuckets], s_hlo[kSelBuckets], s_hhi[kSelBuckets];
+    __shared__ unsigned long long s_pick[16];
+    __shared__ unsigned long long s_top_w[kSelThreads];  // the entries with key >= tau when there are few of them
+    __shared__ uint32_t s_top_key[kSelThreads];
+    __shared__ int s_top_id[kSelThreads];
+    __shared__ unsigned int s_top_n;
     __shared__ float s_max[kFiltThreads / 32];
     int turn = 0;
     __shared__ unsigned int s_list_n;
     pdl_prologue();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int g = blockIdx.x / kGroupRows, j = blockIdx.x - g * kGroupRows;
+    const uint32_t n_peers = cluster_blocks(), crank = cluster_rank();
+    const int slot = blockIdx.x / n_peers;  // the blocks of a cluster are neighbours along x
+    const int g = slot / kGroupRows, j = slot - g * kGroupRows;
+    // (every way out before the cluster's barriers depends on the row alone, so the blocks of a cluster take it together)
     if (a.n_groups && g >= __ldg(a.n_groups)) return;
     int row;
     if (a.group_rows) {
@@ -1829,7 +2014,7 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
     for (int w = 0; w < kFiltThreads / 32; ++w) M = fmaxf(M, s_max[w]);
     if (!(M > kRefFloor)) {
         // nothing allowed, or only -inf allowed: the lowest allowed token (if any) and -inf logs
-        if (warp == 0) {
+        if (warp == 0 && crank == 0) {
             unsigned long long cand = first_allowed_share(a, P, row, lane, 32);
 #pragma unroll
             for (int d = 16; d >= 1; d >>= 1) {
@@ -1844,143 +2029,284 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
     const char* rowp = reinterpret_cast<const char*>(a.logits) + int64_t(row) * a.row_stride * ES;
     const float scale = a.scale;
     const uint32_t key_max = logit_key<DT>(M);
-    // the tokens whose fixed-point weight is not zero (z >= M - 40 / scale) go to the list; counts and weights of the
-    // whole row on the way
-    const uint32_t key_list = logit_key<DT>(M - 40.f / scale);
-    CountMass mine{0u, 0ull};
-    row_visit<DT>(rowp, a.V, aligned != 0, [&](int t, float z) {
-        const unsigned long long w = fixed_weight(z, M, scale);
-        mine.n += 1u;
-        mine.w += w;
-        const uint32_t key = logit_key<DT>(z);
-        if (key >= key_list) {
-            const unsigned int at = atomicAdd(&s_list_n, 1u);
-            if (at < kFiltList) {
-                l_key[at] = key;
-                l_w[at] = w;
-                l_id[at] = t;
+    // The tokens at or above M - 41 / scale are the candidates (below M - 40 / scale the fixed-point weight is zero;
+    // the extra unit covers the rounding of the threshold itself): this block lists those of its share of the row. z_cut is the lowest logit whose key reaches key_list, so one comparison of floats
+    // decides, and a round of eight logits is skipped as soon as its maximum falls short.
+    const uint32_t key_list = logit_key<DT>(M - 41.f / scale);
+    const float z_cut = key_logit<DT>(key_list);
+    {
+        const int share = ((a.V + int(n_peers) - 1) / int(n_peers) + 7) & ~7;
+        const int t_begin = min(int(crank) * share, a.V), t_end = min(t_begin + share, a.V);
+        constexpr int kInFlight = 4;
+        // (the loop bound is the same for the lanes of a warp: they reserve their places in the list together)
+        for (int tw = t_begin + warp * 256; tw < t_end; tw += kFiltThreads * 8 * kInFlight) {
+            const int t0 = tw + lane * 8;
+            float e[kInFlight][8];
+#pragma unroll
+            for (int r = 0; r < kInFlight; ++r) load_eight<DT>(rowp, t0 + r * kFiltThreads * 8, t_end, aligned != 0, e[r]);
+            uint32_t cand = 0u;  // bit 8 r + q: logit q of round r is a candidate
+#pragma unroll
+            for (int r = 0; r < kInFlight; ++r) {
+                const float top = fmax3(fmax3(e[r][0], e[r][1], e[r][2]), fmax3(e[r][3], e[r][4], e[r][5]), fmaxf(e[r][6], e[r][7]));
+                if (top >= z_cut) {
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) cand |= e[r][q] >= z_cut ? 1u << (8 * r + q) : 0u;
+                }
+            }
+            const int cnt = __popc(cand);
+            int inc = cnt;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int up = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+                if (lane >= d) inc += up;
+            }
+            const int warp_cnt = __shfl_sync(0xFFFFFFFFu, inc, 31);
+            if (warp_cnt == 0) continue;
+            unsigned int base = 0u;
+            if (lane == 31) base = atomicAdd(&s_list_n, unsigned(warp_cnt));
+            base = __shfl_sync(0xFFFFFFFFu, base, 31);
+            unsigned int at = base + unsigned(inc - cnt);
+#pragma unroll
+            for (int r = 0; r < kInFlight; ++r)
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    if ((cand >> (8 * r + q)) & 1u) {
+                        if (at < kFiltList) {  // (key and weight follow below, for the listed logits only)
+                            l_key[at] = __float_as_uint(e[r][q]);
+                            l_id[at] = t0 + r * kFiltThreads * 8 + q;
+                        }
+                        ++at;
+                    }
+        }
+    }
+    __syncthreads();
+    unsigned int n_list = s_list_n;
+    for (unsigned int i = tid; i < min(n_list, unsigned(kFiltList)); i += kFiltThreads) {
+        const float z = __uint_as_float(l_key[i]);
+        l_key[i] = logit_key<DT>(z);
+        l_w[i] = fixed_weight(z, M, scale);
+    }
+    if (n_peers == 1u) __syncthreads();
+    if (n_peers > 1u) {
+        cluster_barrier();  // the peers' lists are complete
+        if (crank == 0u) {
+            for (uint32_t p = 1; p < n_peers; ++p) {
+                const unsigned int n_p = ld_peer_u32(peer_shared(&s_list_n, p));
+                if (n_list <= kFiltList && n_p <= kFiltList && n_list + n_p <= kFiltList) {
+                    const uint32_t pw = peer_shared(l_w, p), pk = peer_shared(l_key, p), pi = peer_shared(l_id, p);
+                    for (unsigned int i = tid; i < n_p; i += kFiltThreads) {
+                        l_w[n_list + i] = ld_peer_u64(pw + i * 8u);
+                        l_key[n_list + i] = ld_peer_u32(pk + i * 4u);
+                        l_id[n_list + i] = int(ld_peer_u32(pi + i * 4u));
+                    }
+                    n_list += n_p;
+                } else {
+                    n_list = kFiltList + 1u;  // too many for the list
+                }
             }
         }
-    });
-    const CountMass all = block_sum(mine, s_n, s_w, turn);
-    const unsigned int n_list = s_list_n;
+        cluster_barrier();  // the peers' shared memory has been read: they may leave
+        if (crank != 0u) return;
+    }
     const bool list_whole = n_list <= kFiltList;
 
-    // (count, weight) of the tokens with key >= lo: from the list when it is known to hold them all, else from the row
-    auto above = [&](uint32_t lo, bool from_list) {
-        CountMass v{0u, 0ull};
-        if (from_list) {
-            for (unsigned int i = tid; i < n_list; i += kFiltThreads)
-                if (l_key[i] >= lo) {
-                    v.n += 1u;
-                    v.w += l_w[i];
-                }
-        } else {
-            row_visit<DT>(rowp, a.V, aligned != 0, [&](int, float z) {
-                if (logit_key<DT>(z) >= lo) {
-                    v.n += 1u;
-                    v.w += fixed_weight(z, M, scale);
-                }
-            });
-        }
-        return block_sum(v, s_n, s_w, turn);
-    };
-    // kept so far: { key > tau } and the first m tokens with key == tau; S their weight
+    // kept: { key > tau } and the first m tokens, in token order, with key == tau; S their weight
     uint32_t tau = 0u;
     unsigned int m = 0xFFFFFFFFu;
+
+    if (list_whole) {
+        // ---- everything from the list (it holds every token that carries weight, in no particular order)
+        if (tid >= kSelThreads) return;
+        auto select = [&](auto kind, int bits, unsigned long long thr, auto&& xg) {
+            return list_select<decltype(kind)::value>(n_list, bits, thr, xg, s_hn, s_hlo, s_hhi, s_pick, s_n, s_w, turn);
+        };
+        const std::integral_constant<bool, false> by_count;
+        const std::integral_constant<bool, true> by_weight;
+        // keys from the top: x = key_max - key, below 2^key_bits
+        const int key_bits = 32 - __clz(key_max - key_list);
+        auto from_top = [&](unsigned int i, uint32_t& x, unsigned int& gn, unsigned long long& gw) {
+            x = key_max - l_key[i];
+            gn = 1u;
+            gw = l_w[i];
+        };
+        unsigned long long S;  // weight of what is kept so far
+        {
+            CountMass mine{0u, 0ull}, all;
+            for (unsigned int i = tid; i < n_list; i += kSelThreads) mine.w += l_w[i];
+            sel_exclusive_scan(mine, s_n, s_w, turn, all);
+            S = all.w;
+        }
+        unsigned long long w_above = S;  // weight of the tokens with key > tau
+        unsigned int n_above = 0u;       // their number
+        unsigned int n_ties = 0u;        // tokens with key == tau
+        unsigned long long w_tie = 0ull; // weight of each of them
+        bool cut = false;
+        // (a top_k beyond the list only adds tokens of weight zero: nothing to do)
+        if (top_k > 0 && unsigned(top_k) < n_list) {
+            // the largest key with at least top_k entries at or above it
+            const Picked pk = select(by_count, key_bits, static_cast<unsigned long long>(top_k) - 1ull, from_top);
+            tau = key_max - pk.x;
+            m = unsigned(top_k) - pk.before.n;
+            n_ties = pk.at.n;
+            w_tie = fixed_weight(key_logit<DT>(tau), M, scale);
+            w_above = pk.before.w;
+            n_above = pk.before.n;
+            S = w_above + static_cast<unsigned long long>(m) * w_tie;
+            cut = true;
+        }
+        if (top_p < 1.f) {
+            // the target: top_p times the weight kept so far, rounded up; at least one unit so that one token is kept
+            unsigned long long target = static_cast<unsigned long long>(ceil(static_cast<double>(S) * static_cast<double>(top_p)));
+            target = target < 1ull ? 1ull : (target > S ? S : target);
+            if (w_above >= target) {
+                // the largest key whose entries, with those above it, reach the target
+                const Picked pk = select(by_weight, key_bits, target - 1ull, from_top);
+                tau = key_max - pk.x;
+                w_tie = fixed_weight(key_logit<DT>(tau), M, scale);
+                w_above = pk.before.w;
+                n_above = pk.before.n;
+                n_ties = pk.at.n;
+                unsigned int need = n_ties;  // all the ties unless fewer reach the target
+                if (w_tie > 0ull) {
+                    const unsigned long long q = (target - w_above + w_tie - 1ull) / w_tie;
+                    if (q < need) need = unsigned(q);
+                }
+                m = need < 1u ? 1u : need;
+                cut = true;
+            } else if (w_tie > 0ull) {
+                // the target is reached among the ties at tau itself
+                const unsigned long long q = (target - w_above + w_tie - 1ull) / w_tie;
+                if (q < m) m = unsigned(q < 1ull ? 1ull : q);
+            }
+        }
+        // The ties that are kept are those with the m lowest ids; the drawn token is the lowest id t with
+        // (kept weight at ids <= t) > floor(u * kept weight). All ties weigh the same, so the kept weight needs no pass.
+        const unsigned long long S_kept = cut ? w_above + static_cast<unsigned long long>(min(m, n_ties)) * w_tie : S;
+        const float u = __ldg(a.u + row);
+        unsigned long long thr = static_cast<unsigned long long>(static_cast<double>(u) * static_cast<double>(S_kept));
+        if (thr >= S_kept) thr = S_kept - 1ull;  // (S_kept > 0: the row maximum is always kept)
+        const float l = logf(static_cast<float>(S_kept) * (1.f / kFixOne));
+        if (cut && n_above + n_ties <= unsigned(kSelThreads)) {
+            // Few tokens at or above tau (the rule with top-k, and with top-p on a peaked distribution): one per thread,
+            // and every thread sums over all of them: the ties below its id for its rank, the kept weight up to its id
+            // for its place in the cumulative distribution.
+            const unsigned int n_top = n_above + n_ties;
+            if (tid == 0) s_top_n = 0u;
+            sel_sync();
+            for (unsigned int i = tid; i < n_list; i += kSelThreads)
+                if (l_key[i] >= tau) {
+                    const unsigned int at = atomicAdd(&s_top_n, 1u);
+                    s_top_key[at] = l_key[i];
+                    s_top_id[at] = l_id[i];
+                    s_top_w[at] = l_w[i];
+                }
+            sel_sync();
+            const bool have = unsigned(tid) < n_top;
+            const int my_id = have ? s_top_id[tid] : a.V;
+            const uint32_t my_key = have ? s_top_key[tid] : 0u;
+            unsigned long long my_w = have ? s_top_w[tid] : 0ull;
+            if (m < n_ties) {
+                unsigned int rank = 0u;
+                for (unsigned int k = 0; k < n_top; ++k) rank += (s_top_key[k] == tau && s_top_id[k] < my_id) ? 1u : 0u;
+                if (have && my_key == tau && rank >= m) {
+                    my_w = 0ull;
+                    s_top_w[tid] = 0ull;  // (read by the others only after the barrier below)
+                }
+            }
+            sel_sync();
+            unsigned long long cum = 0ull;
+            for (unsigned int k = 0; k < n_top; ++k) cum += s_top_id[k] <= my_id ? s_top_w[k] : 0ull;
+            if (my_w > 0ull && cum - my_w <= thr && thr < cum) {  // the one thread that holds the drawn token
+                const float zt = key_logit<DT>(my_key);
+                a.argmax[row] = my_id;
+                if (a.rep) a.rep[row] = __ldg(P.trep + my_id);
+                if (a.lse) a.lse[row] = fmaf(M, a.inv_t, l);
+                if (a.logp_argmax) a.logp_argmax[row] = (zt - M) * a.inv_t - l;
+            }
+            return;
+        }
+        const int id_bits = 32 - __clz(max(a.V - 1, 1));
+        int id_cut = a.V;  // the kept ties are those with ids up to id_cut
+        if (cut && m < n_ties)
+            id_cut = int(select(by_count, id_bits, static_cast<unsigned long long>(m) - 1ull,
+                                [&](unsigned int i, uint32_t& x, unsigned int& gn, unsigned long long& gw) {
+                                    x = uint32_t(l_id[i]);
+                                    gn = l_key[i] == tau ? 1u : 0u;
+                                    gw = 0ull;
+                                })
+                             .x);
+        const int token = int(select(by_weight, id_bits, thr,
+                                     [&](unsigned int i, uint32_t& x, unsigned int& gn, unsigned long long& gw) {
+                                         const uint32_t key = l_key[i];
+                                         const int id = l_id[i];
+                                         x = uint32_t(id);
+                                         gn = 0u;
+                                         gw = (!cut || key > tau || (key == tau && id <= id_cut)) ? l_w[i] : 0ull;
+                                     })
+                              .x);
+        for (unsigned int i = tid; i < n_list; i += kSelThreads)
+            if (l_id[i] == token) {  // the one thread that holds the drawn token writes the row's results
+                const float zt = key_logit<DT>(l_key[i]);
+                a.argmax[row] = token;
+                if (a.rep) a.rep[row] = __ldg(P.trep + token);
+                if (a.lse) a.lse[row] = fmaf(M, a.inv_t, l);
+                if (a.logp_argmax) a.logp_argmax[row] = (zt - M) * a.inv_t - l;
+            }
+        return;
+    }
+
+    // ---- more candidates than the list holds (a flat distribution): counts and weights come from passes over the
+    // row, tau by bisection on the key
+    auto above = [&](uint32_t lo) {  // (count, weight) of the tokens with key >= lo
+        CountMass v{0u, 0ull};
+        row_visit<DT>(rowp, a.V, aligned != 0, [&](int, float z) {
+            if (logit_key<DT>(z) >= lo) {
+                v.n += 1u;
+                v.w += fixed_weight(z, M, scale);
+            }
+        });
+        return block_sum(v, s_n, s_w, turn);
+    };
+    const CountMass all = above(0u);
     unsigned long long S = all.w;
-    // (with the whole list in hand a top_k beyond it only adds tokens of weight zero: nothing to do)
-    if (top_k > 0 && unsigned(top_k) < all.n && !(list_whole && unsigned(top_k) >= n_list)) {
-        const bool use_list = list_whole;
-        uint32_t lo = use_list ? key_list : 0u, hi = key_max;  // count(>= lo) >= top_k holds
+    if (top_k > 0 && unsigned(top_k) < all.n) {
+        uint32_t lo = 0u, hi = key_max;  // count(>= lo) >= top_k holds
         while (lo < hi) {
             const uint32_t mid = lo + (hi - lo + 1u) / 2u;
-            if (above(mid, use_list).n >= unsigned(top_k)) lo = mid; else hi = mid - 1u;
+            if (above(mid).n >= unsigned(top_k)) lo = mid; else hi = mid - 1u;
         }
         tau = lo;
-        const CountMass gt = tau == key_max ? CountMass{0u, 0ull} : above(tau + 1u, use_list);
+        const CountMass gt = tau == key_max ? CountMass{0u, 0ull} : above(tau + 1u);
         m = unsigned(top_k) - gt.n;
         S = gt.w + static_cast<unsigned long long>(m) * fixed_weight(key_logit<DT>(tau), M, scale);
     }
     if (top_p < 1.f) {
-        // the target: top_p times the weight kept so far, rounded up; at least one unit so that one token is kept
         unsigned long long target = static_cast<unsigned long long>(ceil(static_cast<double>(S) * static_cast<double>(top_p)));
         target = target < 1ull ? 1ull : (target > S ? S : target);
-        // the whole list serves: whatever it leaves out has weight zero
-        const bool use_list = list_whole;
-        const CountMass gt_tau = tau >= key_max ? CountMass{0u, 0ull} : above(tau + 1u, use_list);
+        const CountMass gt_tau = tau >= key_max ? CountMass{0u, 0ull} : above(tau + 1u);
         if (gt_tau.w >= target) {
             uint32_t lo = tau + 1u, hi = key_max;  // weight(>= lo) >= target holds
             while (lo < hi) {
                 const uint32_t mid = lo + (hi - lo + 1u) / 2u;
-                if (above(mid, use_list).w >= target) lo = mid; else hi = mid - 1u;
+                if (above(mid).w >= target) lo = mid; else hi = mid - 1u;
             }
-            const CountMass ge = above(lo, use_list);
-            const CountMass gt = lo == key_max ? CountMass{0u, 0ull} : above(lo + 1u, use_list);
+            const CountMass ge = above(lo);
+            const CountMass gt = lo == key_max ? CountMass{0u, 0ull} : above(lo + 1u);
             const unsigned long long w_tie = fixed_weight(key_logit<DT>(lo), M, scale);
-            unsigned int need = ge.n - gt.n;  // all the ties unless fewer reach the target
+            unsigned int need = ge.n - gt.n;
             if (w_tie > 0ull) {
                 const unsigned long long q = (target - gt.w + w_tie - 1ull) / w_tie;
                 if (q < need) need = unsigned(q);
             }
             tau = lo;
             m = need < 1u ? 1u : need;
-            S = gt.w + static_cast<unsigned long long>(m) * w_tie;
         } else {
-            // the target is reached among the ties at tau itself
             const unsigned long long w_tie = fixed_weight(key_logit<DT>(tau), M, scale);
             if (w_tie > 0ull) {
                 const unsigned long long q = (target - gt_tau.w + w_tie - 1ull) / w_tie;
                 if (q < m) m = unsigned(q < 1ull ? 1ull : q);
             }
-            S = gt_tau.w + static_cast<unsigned long long>(m) * w_tie;
         }
-    }
-
-    if (list_whole) {
-        // Draw from the list (it holds every token that carries weight, in no particular order): the ties that are
-        // kept are those with the m lowest ids, i.e. the ids up to id_cut; the drawn token is the lowest id t with
-        // (kept weight at ids <= t) > floor(u * kept weight). Both are found by bisection on the token id with a sum
-        // over the list as the test.
-        auto list_sum = [&](auto&& pred) {
-            CountMass v{0u, 0ull};
-            for (unsigned int i = tid; i < n_list; i += kFiltThreads)
-                if (pred(l_key[i], l_id[i])) {
-                    v.n += 1u;
-                    v.w += l_w[i];
-                }
-            return block_sum(v, s_n, s_w, turn);
-        };
-        int id_cut = a.V;
-        const unsigned int n_ties = list_sum([&](uint32_t key, int) { return key == tau; }).n;
-        if (m < n_ties) {
-            int lo = 0, hi = a.V - 1;  // the smallest id with at least m ties at or below it
-            while (lo < hi) {
-                const int mid = lo + (hi - lo) / 2;
-                if (list_sum([&](uint32_t key, int id) { return key == tau && id <= mid; }).n >= m) hi = mid; else lo = mid + 1;
-            }
-            id_cut = lo;
-        }
-        auto kept = [&](uint32_t key, int id) { return key > tau || (key == tau && id <= id_cut); };
-        const unsigned long long S_kept = list_sum(kept).w;
-        const float u = __ldg(a.u + row);
-        unsigned long long thr = static_cast<unsigned long long>(static_cast<double>(u) * static_cast<double>(S_kept));
-        if (thr >= S_kept) thr = S_kept - 1ull;  // (S_kept > 0: the row maximum is always kept)
-        int lo = 0, hi = a.V - 1;
-        while (lo < hi) {
-            const int mid = lo + (hi - lo) / 2;
-            if (list_sum([&](uint32_t key, int id) { return id <= mid && kept(key, id); }).w > thr) hi = mid; else lo = mid + 1;
-        }
-        const float l = logf(static_cast<float>(S_kept) * (1.f / kFixOne));
-        for (unsigned int i = tid; i < n_list; i += kFiltThreads)
-            if (l_id[i] == lo) {  // the one thread that holds the drawn token writes the row's results
-                const float zt = key_logit<DT>(l_key[i]);
-                a.argmax[row] = lo;
-                if (a.rep) a.rep[row] = __ldg(P.trep + lo);
-                if (a.lse) a.lse[row] = fmaf(M, a.inv_t, l);
-                if (a.logp_argmax) a.logp_argmax[row] = (zt - M) * a.inv_t - l;
-            }
-        return;
     }
 
     // Draw in token order. Every thread owns one contiguous segment of the row: first the ties per segment (their

@@ -151,6 +151,22 @@ def test_filtered_llama_size_rows_peaked_and_flat():
             assert np.array_equal(a[key].view(np.uint8), b[key].view(np.uint8)), key
 
 
+@pytest.mark.parametrize("B", [40, 150])
+def test_filtered_one_and_two_blocks_per_row(B):
+    # rows share thread-block clusters of 4 blocks up to 32 rows, of 2 up to 64, and have a block each beyond
+    V, K = 9001, 200
+    part = synth.zipf_partition(V, K, 1.1, seed=81)
+    cm = synth.class_mask_bernoulli(K, B, 0.3, rng.stream_key(82, B))
+    cm[:, 0] |= 1
+    z = synth.logits_normal(B, V, 2.0, "f32", (83, B))
+    u = rng.uniform(rng.stream_key(84, B), B).astype(np.float32)
+    with Ctx([part]) as ctx:
+        for inv_t, top_k, top_p in ((5.0, 20, 1.0), (5.0, 0, 0.9), (2.0, 300, 0.7)):
+            got = run_filtered(ctx, None, cm, z, V, u, inv_t, top_k, top_p)
+            close, near = check_filtered(got, [part], None, cm, z, V, u, inv_t, top_k, top_p, "B=%d k=%d p=%g" % (B, top_k, top_p))
+            assert close <= 2 and near <= 2
+
+
 def test_no_filter_is_the_plain_sampling_step_and_bad_filters_are_refused():
     w = synth.make_workload(2, B=16, V=20000, K=300)
     cm, z, u = w.class_masks(1), w.logits(1), w.uniforms(1)
