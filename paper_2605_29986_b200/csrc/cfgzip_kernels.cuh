@@ -1805,19 +1805,18 @@ __device__ __forceinline__ uint32_t peer_shared(const void* mine, uint32_t rank)
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(mine)), "r"(rank));
     return r;
 }
-__device__ __forceinline__ uint32_t ld_peer_u32(uint32_t addr) {
-    uint32_t v;
-    asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
-    return v;
+__device__ __forceinline__ unsigned int add_peer_u32(uint32_t addr, unsigned int v) {
+    unsigned int old;
+    asm volatile("atom.shared::cluster.add.u32 %0, [%1], %2;" : "=r"(old) : "r"(addr), "r"(v) : "memory");
+    return old;
 }
-__device__ __forceinline__ unsigned long long ld_peer_u64(uint32_t addr) {
-    unsigned long long v;
-    asm volatile("ld.shared::cluster.u64 %0, [%1];" : "=l"(v) : "r"(addr) : "memory");
-    return v;
+__device__ __forceinline__ void st_peer_u32(uint32_t addr, uint32_t v) {
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
 
-// ---- the searches over the candidate list run on the first kSelThreads threads of the block (a list of a few
-// thousand entries does not feed more, and barriers and sums across 8 warps cost a fraction of those across 32)
+// ---- searches over the candidate list: every thread of the block walks the list (a walk is a chain of dependent
+// shared-memory accesses per entry, so more threads shorten it), the first kSelThreads threads sum over the buckets
+// (barriers and sums across 8 warps cost a fraction of those across 32)
 constexpr int kSelThreads = 256;
 constexpr int kSelBuckets = 1024;  // ten bits of the value per round; kSelBuckets / kSelThreads buckets per thread
 __device__ __forceinline__ void sel_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kSelThreads) : "memory"); }
@@ -1862,35 +1861,39 @@ __device__ __forceinline__ CountMass sel_exclusive_scan(CountMass v, unsigned in
     return CountMass{before.n + inc.n - v.n, before.w + inc.w - v.w};
 }
 
-// Result of a search: the value found, (count, weight) of the entries below it and of the entries at it.
+// Result of a search: the value found, (count, weight) of the entries below it and of the entries at it, the
+// threshold that was used and (count, weight) of all entries that took part.
 struct Picked {
     uint32_t x;
-    CountMass before, at;
+    CountMass before, at, all;
+    unsigned long long thr;
 };
 
-// Smallest value x such that the entries of the list with value <= x together count (BY_WEIGHT: weigh) more than thr.
-// xg(i, x, gn, gw) gives entry i's value (below 2^bits), count and weight (both 0: the entry takes no part); the
-// caller guarantees that all entries together exceed thr. Ten bits of the value per round, highest first: a histogram
-// of the round's digit over the entries that agree with the digits found so far, a prefix sum over the buckets, and
-// the one bucket in which the running sum passes thr is the next digit. Weights are added as two 32-bit halves (the
-// carry out of the lower half is seen in the value the atomic returns), which keeps every atomic a native one.
-template <bool BY_WEIGHT, typename F>
-__device__ __forceinline__ Picked list_select(unsigned int n_list, int bits, unsigned long long thr, F&& xg, unsigned int* h_n,
+// Smallest value x such that the entries of the list with value <= x together count (BY_WEIGHT: weigh) more than thr,
+// where thr = thr_of(count and weight of all entries) is fixed once the first histogram is summed (so a threshold
+// that depends on the total weight costs no pass of its own). xg(i, x, gn, gw) gives entry i's value (below 2^bits),
+// count and weight (both 0: the entry takes no part); the caller guarantees that all entries together exceed thr.
+// Ten bits of the value per round, highest first: a histogram of the round's digit over the entries that agree with
+// the digits found so far, a prefix sum over the buckets, and the one bucket in which the running sum passes thr is
+// the next digit. Weights are added as two 32-bit halves (the carry out of the lower half is seen in the value the
+// atomic returns), which keeps every atomic a native one. Called by all threads of the block.
+template <bool BY_WEIGHT, typename T, typename F>
+__device__ __forceinline__ Picked list_select(unsigned int n_list, int bits, T&& thr_of, F&& xg, unsigned int* h_n,
                                               unsigned int* h_lo, unsigned int* h_hi, unsigned long long* s_pick,
                                               unsigned int* s_n, unsigned long long* s_w, int& turn) {
     const int tid = threadIdx.x;
     const int rounds = bits <= 10 ? 1 : (bits + 9) / 10;
     constexpr int kPer = kSelBuckets / kSelThreads;
-    static_assert(kPer == 4, "a thread reads its buckets as one 16-byte vector per array");
-    unsigned long long prefix = 0ull;
+    static_assert(kPer == 4 && kSelBuckets == kFiltThreads, "one bucket per thread to clear, four per summing thread");
+    unsigned long long prefix = 0ull, thr = 0ull;
     CountMass carry{0u, 0ull}, at{0u, 0ull};  // carry: the entries below the digits found so far
     for (int rd = rounds - 1; rd >= 0; --rd) {
         const int shift = rd * 10;
-        unsigned long long* pick = s_pick + 8 * (rd & 1);
-        reinterpret_cast<uint4*>(h_n)[tid] = make_uint4(0u, 0u, 0u, 0u);
-        reinterpret_cast<uint4*>(h_lo)[tid] = make_uint4(0u, 0u, 0u, 0u);
-        reinterpret_cast<uint4*>(h_hi)[tid] = make_uint4(0u, 0u, 0u, 0u);
-        sel_sync();
+        unsigned long long* pick = s_pick + 5 * (rd & 1);
+        h_n[tid] = 0u;
+        h_lo[tid] = 0u;
+        h_hi[tid] = 0u;
+        __syncthreads();
         if (tid == 0) {  // (what stands if no bucket qualifies: cannot happen under the caller's guarantee)
             pick[0] = 0ull;
             pick[1] = carry.n;
@@ -1898,7 +1901,7 @@ __device__ __forceinline__ Picked list_select(unsigned int n_list, int bits, uns
             pick[3] = 0ull;
             pick[4] = 0ull;
         }
-        for (unsigned int i = tid; i < n_list; i += kSelThreads) {
+        for (unsigned int i = tid; i < n_list; i += kFiltThreads) {
             uint32_t x;
             unsigned int gn;
             unsigned long long gw;
@@ -1917,48 +1920,58 @@ __device__ __forceinline__ Picked list_select(unsigned int n_list, int bits, uns
                 }
             }
         }
-        sel_sync();
-        const uint4 vn = reinterpret_cast<const uint4*>(h_n)[tid];
-        const uint4 vl = reinterpret_cast<const uint4*>(h_lo)[tid];
-        const uint4 vh = reinterpret_cast<const uint4*>(h_hi)[tid];
-        const CountMass h[kPer] = {{vn.x, (static_cast<unsigned long long>(vh.x) << 32) | vl.x},
-                                   {vn.y, (static_cast<unsigned long long>(vh.y) << 32) | vl.y},
-                                   {vn.z, (static_cast<unsigned long long>(vh.z) << 32) | vl.z},
-                                   {vn.w, (static_cast<unsigned long long>(vh.w) << 32) | vl.w}};
-        CountMass mine{0u, 0ull}, total;
+        __syncthreads();
+        if (tid < kSelThreads) {
+            const uint4 vn = reinterpret_cast<const uint4*>(h_n)[tid];
+            const uint4 vl = reinterpret_cast<const uint4*>(h_lo)[tid];
+            const uint4 vh = reinterpret_cast<const uint4*>(h_hi)[tid];
+            const CountMass h[kPer] = {{vn.x, (static_cast<unsigned long long>(vh.x) << 32) | vl.x},
+                                       {vn.y, (static_cast<unsigned long long>(vh.y) << 32) | vl.y},
+                                       {vn.z, (static_cast<unsigned long long>(vh.z) << 32) | vl.z},
+                                       {vn.w, (static_cast<unsigned long long>(vh.w) << 32) | vl.w}};
+            CountMass mine{0u, 0ull}, total;
 #pragma unroll
-        for (int b = 0; b < kPer; ++b) {
-            mine.n += h[b].n;
-            mine.w += h[b].w;
-        }
-        CountMass run = sel_exclusive_scan(mine, s_n, s_w, turn, total);
-        run.n += carry.n;
-        run.w += carry.w;
-#pragma unroll
-        for (int b = 0; b < kPer; ++b) {
-            const unsigned long long below = BY_WEIGHT ? run.w : static_cast<unsigned long long>(run.n);
-            const unsigned long long here = BY_WEIGHT ? h[b].w : static_cast<unsigned long long>(h[b].n);
-            if (below <= thr && thr < below + here) {
-                pick[0] = static_cast<unsigned long long>(tid * kPer + b);
-                pick[1] = run.n;
-                pick[2] = run.w;
-                pick[3] = h[b].n;
-                pick[4] = h[b].w;
+            for (int b = 0; b < kPer; ++b) {
+                mine.n += h[b].n;
+                mine.w += h[b].w;
             }
-            run.n += h[b].n;
-            run.w += h[b].w;
+            CountMass run = sel_exclusive_scan(mine, s_n, s_w, turn, total);
+            if (rd == rounds - 1) {  // the first round sees every entry
+                thr = thr_of(total);
+                if (tid == 0) {
+                    s_pick[10] = thr;
+                    s_pick[11] = total.n;
+                    s_pick[12] = total.w;
+                }
+            }
+            run.n += carry.n;
+            run.w += carry.w;
+#pragma unroll
+            for (int b = 0; b < kPer; ++b) {
+                const unsigned long long below = BY_WEIGHT ? run.w : static_cast<unsigned long long>(run.n);
+                const unsigned long long here = BY_WEIGHT ? h[b].w : static_cast<unsigned long long>(h[b].n);
+                if (below <= thr && thr < below + here) {
+                    pick[0] = static_cast<unsigned long long>(tid * kPer + b);
+                    pick[1] = run.n;
+                    pick[2] = run.w;
+                    pick[3] = h[b].n;
+                    pick[4] = h[b].w;
+                }
+                run.n += h[b].n;
+                run.w += h[b].w;
+            }
         }
-        sel_sync();
+        __syncthreads();
         prefix = (prefix << 10) | pick[0];
         carry = CountMass{static_cast<unsigned int>(pick[1]), pick[2]};
         at = CountMass{static_cast<unsigned int>(pick[3]), pick[4]};
     }
-    return Picked{static_cast<uint32_t>(prefix), carry, at};
+    return Picked{static_cast<uint32_t>(prefix), carry, at, CountMass{static_cast<unsigned int>(s_pick[11]), s_pick[12]}, s_pick[10]};
 }
 
 // One row per cluster of blocks (1, 2 or 4 of them: a short batch has fewer rows than the device has
-// multiprocessors). Every block collects the candidates of its share of the row; the first block of the cluster
-// then gathers the lists through the cluster's shared memory and carries on alone.
+// multiprocessors). Every block looks for the candidates in its share of the row and writes them, through the
+// cluster's shared memory, into the list of the cluster's first block, which carries on alone.
 template <int DT>
 __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_constant__ StepArgs a, int aligned, int top_k,
                                                                   float top_p) {
@@ -2034,7 +2047,11 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
     // decides, and a round of eight logits is skipped as soon as its maximum falls short.
     const uint32_t key_list = logit_key<DT>(M - 41.f / scale);
     const float z_cut = key_logit<DT>(key_list);
+    // The candidates of every block go straight into the list of the cluster's first block (places are reserved in its
+    // counter, a warp at a time): no lists to merge afterwards.
+    cluster_barrier();  // the first block's counter is cleared before anybody adds to it
     {
+        const uint32_t list_n0 = peer_shared(&s_list_n, 0u), list_key0 = peer_shared(l_key, 0u), list_id0 = peer_shared(l_id, 0u);
         const int share = ((a.V + int(n_peers) - 1) / int(n_peers) + 7) & ~7;
         const int t_begin = min(int(crank) * share, a.V), t_end = min(t_begin + share, a.V);
         constexpr int kInFlight = 4;
@@ -2063,7 +2080,7 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
             const int warp_cnt = __shfl_sync(0xFFFFFFFFu, inc, 31);
             if (warp_cnt == 0) continue;
             unsigned int base = 0u;
-            if (lane == 31) base = atomicAdd(&s_list_n, unsigned(warp_cnt));
+            if (lane == 31) base = add_peer_u32(list_n0, unsigned(warp_cnt));
             base = __shfl_sync(0xFFFFFFFFu, base, 31);
             unsigned int at = base + unsigned(inc - cnt);
 #pragma unroll
@@ -2072,42 +2089,22 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
                 for (int q = 0; q < 8; ++q)
                     if ((cand >> (8 * r + q)) & 1u) {
                         if (at < kFiltList) {  // (key and weight follow below, for the listed logits only)
-                            l_key[at] = __float_as_uint(e[r][q]);
-                            l_id[at] = t0 + r * kFiltThreads * 8 + q;
+                            st_peer_u32(list_key0 + at * 4u, __float_as_uint(e[r][q]));
+                            st_peer_u32(list_id0 + at * 4u, uint32_t(t0 + r * kFiltThreads * 8 + q));
                         }
                         ++at;
                     }
         }
     }
-    __syncthreads();
-    unsigned int n_list = s_list_n;
+    cluster_barrier();  // every block's candidates have arrived; the other blocks are done
+    if (crank != 0u) return;
+    const unsigned int n_list = s_list_n;
     for (unsigned int i = tid; i < min(n_list, unsigned(kFiltList)); i += kFiltThreads) {
         const float z = __uint_as_float(l_key[i]);
         l_key[i] = logit_key<DT>(z);
         l_w[i] = fixed_weight(z, M, scale);
     }
-    if (n_peers == 1u) __syncthreads();
-    if (n_peers > 1u) {
-        cluster_barrier();  // the peers' lists are complete
-        if (crank == 0u) {
-            for (uint32_t p = 1; p < n_peers; ++p) {
-                const unsigned int n_p = ld_peer_u32(peer_shared(&s_list_n, p));
-                if (n_list <= kFiltList && n_p <= kFiltList && n_list + n_p <= kFiltList) {
-                    const uint32_t pw = peer_shared(l_w, p), pk = peer_shared(l_key, p), pi = peer_shared(l_id, p);
-                    for (unsigned int i = tid; i < n_p; i += kFiltThreads) {
-                        l_w[n_list + i] = ld_peer_u64(pw + i * 8u);
-                        l_key[n_list + i] = ld_peer_u32(pk + i * 4u);
-                        l_id[n_list + i] = int(ld_peer_u32(pi + i * 4u));
-                    }
-                    n_list += n_p;
-                } else {
-                    n_list = kFiltList + 1u;  // too many for the list
-                }
-            }
-        }
-        cluster_barrier();  // the peers' shared memory has been read: they may leave
-        if (crank != 0u) return;
-    }
+    __syncthreads();
     const bool list_whole = n_list <= kFiltList;
 
     // kept: { key > tau } and the first m tokens, in token order, with key == tau; S their weight
@@ -2116,9 +2113,8 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
 
     if (list_whole) {
         // ---- everything from the list (it holds every token that carries weight, in no particular order)
-        if (tid >= kSelThreads) return;
-        auto select = [&](auto kind, int bits, unsigned long long thr, auto&& xg) {
-            return list_select<decltype(kind)::value>(n_list, bits, thr, xg, s_hn, s_hlo, s_hhi, s_pick, s_n, s_w, turn);
+        auto select = [&](auto kind, int bits, auto&& thr_of, auto&& xg) {
+            return list_select<decltype(kind)::value>(n_list, bits, thr_of, xg, s_hn, s_hlo, s_hhi, s_pick, s_n, s_w, turn);
         };
         const std::integral_constant<bool, false> by_count;
         const std::integral_constant<bool, true> by_weight;
@@ -2129,22 +2125,22 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
             gn = 1u;
             gw = l_w[i];
         };
-        unsigned long long S;  // weight of what is kept so far
-        {
-            CountMass mine{0u, 0ull}, all;
-            for (unsigned int i = tid; i < n_list; i += kSelThreads) mine.w += l_w[i];
-            sel_exclusive_scan(mine, s_n, s_w, turn, all);
-            S = all.w;
-        }
-        unsigned long long w_above = S;  // weight of the tokens with key > tau
-        unsigned int n_above = 0u;       // their number
-        unsigned int n_ties = 0u;        // tokens with key == tau
-        unsigned long long w_tie = 0ull; // weight of each of them
+        // the target of top-p: that share of the weight kept so far, rounded up; at least one unit so that one token is kept
+        auto target_of = [&](unsigned long long S) {
+            const unsigned long long t = static_cast<unsigned long long>(ceil(static_cast<double>(S) * static_cast<double>(top_p)));
+            return t < 1ull ? 1ull : (t > S ? S : t);
+        };
+        unsigned long long S = 0ull;        // weight of what is kept so far (once something has been cut)
+        unsigned long long w_above = 0ull;  // weight of the tokens with key > tau
+        unsigned int n_above = 0u;          // their number
+        unsigned int n_ties = 0u;           // tokens with key == tau
+        unsigned long long w_tie = 0ull;    // weight of each of them
         bool cut = false;
         // (a top_k beyond the list only adds tokens of weight zero: nothing to do)
         if (top_k > 0 && unsigned(top_k) < n_list) {
             // the largest key with at least top_k entries at or above it
-            const Picked pk = select(by_count, key_bits, static_cast<unsigned long long>(top_k) - 1ull, from_top);
+            const Picked pk = select(by_count, key_bits, [&](CountMass) { return static_cast<unsigned long long>(top_k) - 1ull; },
+                                     from_top);
             tau = key_max - pk.x;
             m = unsigned(top_k) - pk.before.n;
             n_ties = pk.at.n;
@@ -2155,12 +2151,13 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
             cut = true;
         }
         if (top_p < 1.f) {
-            // the target: top_p times the weight kept so far, rounded up; at least one unit so that one token is kept
-            unsigned long long target = static_cast<unsigned long long>(ceil(static_cast<double>(S) * static_cast<double>(top_p)));
-            target = target < 1ull ? 1ull : (target > S ? S : target);
-            if (w_above >= target) {
-                // the largest key whose entries, with those above it, reach the target
-                const Picked pk = select(by_weight, key_bits, target - 1ull, from_top);
+            const unsigned long long target = cut ? target_of(S) : 0ull;
+            if (!cut || w_above >= target) {
+                // the largest key whose entries, with those above it, reach the target (without a cut so far the target
+                // follows from the weight of the whole list, which the search sums on its way)
+                const Picked pk = select(by_weight, key_bits,
+                                         [&](CountMass all) { return (cut ? target : target_of(all.w)) - 1ull; }, from_top);
+                const unsigned long long tgt = pk.thr + 1ull;
                 tau = key_max - pk.x;
                 w_tie = fixed_weight(key_logit<DT>(tau), M, scale);
                 w_above = pk.before.w;
@@ -2168,7 +2165,7 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
                 n_ties = pk.at.n;
                 unsigned int need = n_ties;  // all the ties unless fewer reach the target
                 if (w_tie > 0ull) {
-                    const unsigned long long q = (target - w_above + w_tie - 1ull) / w_tie;
+                    const unsigned long long q = (tgt - w_above + w_tie - 1ull) / w_tie;
                     if (q < need) need = unsigned(q);
                 }
                 m = need < 1u ? 1u : need;
@@ -2181,26 +2178,29 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
         }
         // The ties that are kept are those with the m lowest ids; the drawn token is the lowest id t with
         // (kept weight at ids <= t) > floor(u * kept weight). All ties weigh the same, so the kept weight needs no pass.
-        const unsigned long long S_kept = cut ? w_above + static_cast<unsigned long long>(min(m, n_ties)) * w_tie : S;
         const float u = __ldg(a.u + row);
-        unsigned long long thr = static_cast<unsigned long long>(static_cast<double>(u) * static_cast<double>(S_kept));
-        if (thr >= S_kept) thr = S_kept - 1ull;  // (S_kept > 0: the row maximum is always kept)
-        const float l = logf(static_cast<float>(S_kept) * (1.f / kFixOne));
+        auto threshold_of = [&](unsigned long long S_kept) {  // (S_kept > 0: the row maximum is always kept)
+            const unsigned long long t = static_cast<unsigned long long>(static_cast<double>(u) * static_cast<double>(S_kept));
+            return t >= S_kept ? S_kept - 1ull : t;
+        };
         if (cut && n_above + n_ties <= unsigned(kSelThreads)) {
             // Few tokens at or above tau (the rule with top-k, and with top-p on a peaked distribution): one per thread,
             // and every thread sums over all of them: the ties below its id for its rank, the kept weight up to its id
             // for its place in the cumulative distribution.
+            const unsigned long long S_kept = w_above + static_cast<unsigned long long>(min(m, n_ties)) * w_tie;
+            const unsigned long long thr = threshold_of(S_kept);
             const unsigned int n_top = n_above + n_ties;
             if (tid == 0) s_top_n = 0u;
-            sel_sync();
-            for (unsigned int i = tid; i < n_list; i += kSelThreads)
+            __syncthreads();
+            for (unsigned int i = tid; i < n_list; i += kFiltThreads)
                 if (l_key[i] >= tau) {
                     const unsigned int at = atomicAdd(&s_top_n, 1u);
                     s_top_key[at] = l_key[i];
                     s_top_id[at] = l_id[i];
                     s_top_w[at] = l_w[i];
                 }
-            sel_sync();
+            __syncthreads();
+            if (tid >= kSelThreads) return;
             const bool have = unsigned(tid) < n_top;
             const int my_id = have ? s_top_id[tid] : a.V;
             const uint32_t my_key = have ? s_top_key[tid] : 0u;
@@ -2217,6 +2217,7 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
             unsigned long long cum = 0ull;
             for (unsigned int k = 0; k < n_top; ++k) cum += s_top_id[k] <= my_id ? s_top_w[k] : 0ull;
             if (my_w > 0ull && cum - my_w <= thr && thr < cum) {  // the one thread that holds the drawn token
+                const float l = logf(static_cast<float>(S_kept) * (1.f / kFixOne));
                 const float zt = key_logit<DT>(my_key);
                 a.argmax[row] = my_id;
                 if (a.rep) a.rep[row] = __ldg(P.trep + my_id);
@@ -2228,23 +2229,25 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
         const int id_bits = 32 - __clz(max(a.V - 1, 1));
         int id_cut = a.V;  // the kept ties are those with ids up to id_cut
         if (cut && m < n_ties)
-            id_cut = int(select(by_count, id_bits, static_cast<unsigned long long>(m) - 1ull,
+            id_cut = int(select(by_count, id_bits, [&](CountMass) { return static_cast<unsigned long long>(m) - 1ull; },
                                 [&](unsigned int i, uint32_t& x, unsigned int& gn, unsigned long long& gw) {
                                     x = uint32_t(l_id[i]);
                                     gn = l_key[i] == tau ? 1u : 0u;
                                     gw = 0ull;
                                 })
                              .x);
-        const int token = int(select(by_weight, id_bits, thr,
-                                     [&](unsigned int i, uint32_t& x, unsigned int& gn, unsigned long long& gw) {
-                                         const uint32_t key = l_key[i];
-                                         const int id = l_id[i];
-                                         x = uint32_t(id);
-                                         gn = 0u;
-                                         gw = (!cut || key > tau || (key == tau && id <= id_cut)) ? l_w[i] : 0ull;
-                                     })
-                              .x);
-        for (unsigned int i = tid; i < n_list; i += kSelThreads)
+        // (the kept weight is the weight of everything that takes part in the search for the token)
+        const Picked drawn = select(by_weight, id_bits, [&](CountMass all) { return threshold_of(all.w); },
+                                    [&](unsigned int i, uint32_t& x, unsigned int& gn, unsigned long long& gw) {
+                                        const uint32_t key = l_key[i];
+                                        const int id = l_id[i];
+                                        x = uint32_t(id);
+                                        gn = 0u;
+                                        gw = (!cut || key > tau || (key == tau && id <= id_cut)) ? l_w[i] : 0ull;
+                                    });
+        const int token = int(drawn.x);
+        const float l = logf(static_cast<float>(drawn.all.w) * (1.f / kFixOne));
+        for (unsigned int i = tid; i < n_list; i += kFiltThreads)
             if (l_id[i] == token) {  // the one thread that holds the drawn token writes the row's results
                 const float zt = key_logit<DT>(l_key[i]);
                 a.argmax[row] = token;
