@@ -1669,6 +1669,8 @@ __global__ void __launch_bounds__(kSampleThreads) k_sample_rows(const __grid_con
 // ---------------------------------------------------------------------------------------
 constexpr int kFiltThreads = 1024;
 constexpr int kFiltList = 12288;  // entries of the candidate list (16 bytes each, dynamic shared memory)
+constexpr int kFiltAttempts = 5;  // passes over the row with the bar for the list raised each time it overflows
+constexpr int kFiltPeers = 4;     // most blocks that share a row
 constexpr float kFixOne = 1099511627776.f;  // 2^40
 
 // Order-preserving integer image of a logit and its inverse. bf16 logits only use the upper half of the float's
@@ -1809,6 +1811,14 @@ __device__ __forceinline__ unsigned int add_peer_u32(uint32_t addr, unsigned int
     unsigned int old;
     asm volatile("atom.shared::cluster.add.u32 %0, [%1], %2;" : "=r"(old) : "r"(addr), "r"(v) : "memory");
     return old;
+}
+__device__ __forceinline__ uint32_t ld_peer_u32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_peer_u64(uint32_t addr, unsigned long long v) {
+    asm volatile("st.shared::cluster.u64 [%0], %1;" ::"r"(addr), "l"(v) : "memory");
 }
 __device__ __forceinline__ void st_peer_u32(uint32_t addr, uint32_t v) {
     asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
@@ -1990,7 +2000,9 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
     __shared__ unsigned int s_top_n;
     __shared__ float s_max[kFiltThreads / 32];
     int turn = 0;
-    __shared__ unsigned int s_list_n;
+    __shared__ unsigned int s_list_n[kFiltAttempts];  // candidates counted in each pass over the row
+    __shared__ unsigned int s_low_n[kFiltPeers];      // per block of the cluster: the tokens with weight that stayed
+    __shared__ unsigned long long s_low_w[kFiltPeers];  // below the bar of the last pass, and their weight
     pdl_prologue();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t n_peers = cluster_blocks(), crank = cluster_rank();
@@ -2021,7 +2033,7 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
 #pragma unroll
     for (int d = 16; d >= 1; d >>= 1) M = fmaxf(M, __shfl_xor_sync(0xFFFFFFFFu, M, d));
     if (lane == 0) s_max[warp] = M;
-    if (tid == 0) s_list_n = 0u;
+    if (tid < kFiltAttempts) s_list_n[tid] = 0u;
     __syncthreads();
 #pragma unroll
     for (int w = 0; w < kFiltThreads / 32; ++w) M = fmaxf(M, s_max[w]);
@@ -2042,63 +2054,90 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
     const char* rowp = reinterpret_cast<const char*>(a.logits) + int64_t(row) * a.row_stride * ES;
     const float scale = a.scale;
     const uint32_t key_max = logit_key<DT>(M);
-    // The tokens at or above M - 41 / scale are the candidates (below M - 40 / scale the fixed-point weight is zero;
-    // the extra unit covers the rounding of the threshold itself): this block lists those of its share of the row. z_cut is the lowest logit whose key reaches key_list, so one comparison of floats
-    // decides, and a round of eight logits is skipped as soon as its maximum falls short.
-    const uint32_t key_list = logit_key<DT>(M - 41.f / scale);
-    const float z_cut = key_logit<DT>(key_list);
-    // The candidates of every block go straight into the list of the cluster's first block (places are reserved in its
-    // counter, a warp at a time): no lists to merge afterwards.
-    cluster_barrier();  // the first block's counter is cleared before anybody adds to it
+    // The candidates are the tokens at or above M - 41 / scale (below M - 40 / scale the fixed-point weight is zero;
+    // the extra unit covers the rounding of the threshold itself). The candidates of every block go straight into the
+    // list of the cluster's first block (places are reserved in its counter, a warp at a time). A comparison of
+    // floats decides (z_cut is the lowest logit whose key reaches key_list), and a round of eight logits is skipped as
+    // soon as its maximum falls short. When the list overflows (a flat row, or a mask that allows most of the
+    // vocabulary) the row is gone over again with the bar half as far below M; what carries weight below the bar is
+    // then only counted and summed (low): enough as long as top-k and top-p end inside the list.
+    const float z_zero = key_logit<DT>(logit_key<DT>(M - 41.f / scale));
+    uint32_t key_list = 0u;
+    unsigned int n_list = 0u;
+    int attempt = 0;
     {
-        const uint32_t list_n0 = peer_shared(&s_list_n, 0u), list_key0 = peer_shared(l_key, 0u), list_id0 = peer_shared(l_id, 0u);
+        const uint32_t list_key0 = peer_shared(l_key, 0u), list_id0 = peer_shared(l_id, 0u);
         const int share = ((a.V + int(n_peers) - 1) / int(n_peers) + 7) & ~7;
         const int t_begin = min(int(crank) * share, a.V), t_end = min(t_begin + share, a.V);
         constexpr int kInFlight = 4;
-        // (the loop bound is the same for the lanes of a warp: they reserve their places in the list together)
-        for (int tw = t_begin + warp * 256; tw < t_end; tw += kFiltThreads * 8 * kInFlight) {
-            const int t0 = tw + lane * 8;
-            float e[kInFlight][8];
+        float units = 41.f;
+        cluster_barrier();  // the first block's counters are cleared before anybody adds to them
+        for (;; ++attempt, units *= 0.5f) {
+            key_list = logit_key<DT>(M - units / scale);
+            const float z_cut = key_logit<DT>(key_list);
+            const uint32_t list_n0 = peer_shared(&s_list_n[attempt], 0u);
+            CountMass low{0u, 0ull};
+            // (the loop bound is the same for the lanes of a warp: they reserve their places in the list together)
+            for (int tw = t_begin + warp * 256; tw < t_end; tw += kFiltThreads * 8 * kInFlight) {
+                const int t0 = tw + lane * 8;
+                float e[kInFlight][8];
 #pragma unroll
-            for (int r = 0; r < kInFlight; ++r) load_eight<DT>(rowp, t0 + r * kFiltThreads * 8, t_end, aligned != 0, e[r]);
-            uint32_t cand = 0u;  // bit 8 r + q: logit q of round r is a candidate
+                for (int r = 0; r < kInFlight; ++r) load_eight<DT>(rowp, t0 + r * kFiltThreads * 8, t_end, aligned != 0, e[r]);
+                uint32_t cand = 0u;  // bit 8 r + q: logit q of round r is a candidate
 #pragma unroll
-            for (int r = 0; r < kInFlight; ++r) {
-                const float top = fmax3(fmax3(e[r][0], e[r][1], e[r][2]), fmax3(e[r][3], e[r][4], e[r][5]), fmaxf(e[r][6], e[r][7]));
-                if (top >= z_cut) {
+                for (int r = 0; r < kInFlight; ++r) {
+                    const float top = fmax3(fmax3(e[r][0], e[r][1], e[r][2]), fmax3(e[r][3], e[r][4], e[r][5]), fmaxf(e[r][6], e[r][7]));
+                    if (top >= z_cut) {
 #pragma unroll
-                    for (int q = 0; q < 8; ++q) cand |= e[r][q] >= z_cut ? 1u << (8 * r + q) : 0u;
+                        for (int q = 0; q < 8; ++q) cand |= e[r][q] >= z_cut ? 1u << (8 * r + q) : 0u;
+                    }
+                    if (attempt > 0 && top >= z_zero) {
+#pragma unroll
+                        for (int q = 0; q < 8; ++q)
+                            if (e[r][q] >= z_zero && e[r][q] < z_cut) {
+                                low.n += 1u;
+                                low.w += fixed_weight(e[r][q], M, scale);
+                            }
+                    }
+                }
+                const int cnt = __popc(cand);
+                int inc = cnt;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const int up = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+                    if (lane >= d) inc += up;
+                }
+                const int warp_cnt = __shfl_sync(0xFFFFFFFFu, inc, 31);
+                if (warp_cnt == 0) continue;
+                unsigned int base = 0u;
+                if (lane == 31) base = add_peer_u32(list_n0, unsigned(warp_cnt));
+                base = __shfl_sync(0xFFFFFFFFu, base, 31);
+                unsigned int at = base + unsigned(inc - cnt);
+#pragma unroll
+                for (int r = 0; r < kInFlight; ++r)
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        if ((cand >> (8 * r + q)) & 1u) {
+                            if (at < kFiltList) {  // (key and weight follow below, for the listed logits only)
+                                st_peer_u32(list_key0 + at * 4u, __float_as_uint(e[r][q]));
+                                st_peer_u32(list_id0 + at * 4u, uint32_t(t0 + r * kFiltThreads * 8 + q));
+                            }
+                            ++at;
+                        }
+            }
+            if (attempt > 0) {
+                const CountMass mine = block_sum(low, s_n, s_w, turn);
+                if (tid == 0) {
+                    st_peer_u32(peer_shared(&s_low_n[crank], 0u), mine.n);
+                    st_peer_u64(peer_shared(&s_low_w[crank], 0u), mine.w);
                 }
             }
-            const int cnt = __popc(cand);
-            int inc = cnt;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const int up = __shfl_up_sync(0xFFFFFFFFu, inc, d);
-                if (lane >= d) inc += up;
-            }
-            const int warp_cnt = __shfl_sync(0xFFFFFFFFu, inc, 31);
-            if (warp_cnt == 0) continue;
-            unsigned int base = 0u;
-            if (lane == 31) base = add_peer_u32(list_n0, unsigned(warp_cnt));
-            base = __shfl_sync(0xFFFFFFFFu, base, 31);
-            unsigned int at = base + unsigned(inc - cnt);
-#pragma unroll
-            for (int r = 0; r < kInFlight; ++r)
-#pragma unroll
-                for (int q = 0; q < 8; ++q)
-                    if ((cand >> (8 * r + q)) & 1u) {
-                        if (at < kFiltList) {  // (key and weight follow below, for the listed logits only)
-                            st_peer_u32(list_key0 + at * 4u, __float_as_uint(e[r][q]));
-                            st_peer_u32(list_id0 + at * 4u, uint32_t(t0 + r * kFiltThreads * 8 + q));
-                        }
-                        ++at;
-                    }
+            cluster_barrier();  // every block's candidates have arrived
+            n_list = ld_peer_u32(list_n0);
+            if (n_list <= kFiltList || attempt == kFiltAttempts - 1) break;  // (the same in every block of the cluster)
         }
     }
-    cluster_barrier();  // every block's candidates have arrived; the other blocks are done
-    if (crank != 0u) return;
-    const unsigned int n_list = s_list_n;
+    if (crank != 0u) return;  // (the first block touches no other block's memory from here on)
     for (unsigned int i = tid; i < min(n_list, unsigned(kFiltList)); i += kFiltThreads) {
         const float z = __uint_as_float(l_key[i]);
         l_key[i] = logit_key<DT>(z);
@@ -2106,13 +2145,20 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
     }
     __syncthreads();
     const bool list_whole = n_list <= kFiltList;
+    CountMass low{0u, 0ull};  // what carries weight and is not in the list
+    if (attempt > 0)
+        for (uint32_t p = 0; p < n_peers; ++p) {
+            low.n += s_low_n[p];
+            low.w += s_low_w[p];
+        }
 
     // kept: { key > tau } and the first m tokens, in token order, with key == tau; S their weight
     uint32_t tau = 0u;
     unsigned int m = 0xFFFFFFFFu;
 
-    if (list_whole) {
-        // ---- everything from the list (it holds every token that carries weight, in no particular order)
+    if (list_whole) do {
+        // ---- everything from the list (it holds the tokens that carry weight, or the heaviest of them, in no
+        // particular order); leaves for the passes over the row below when top-k or top-p reach past the list
         auto select = [&](auto kind, int bits, auto&& thr_of, auto&& xg) {
             return list_select<decltype(kind)::value>(n_list, bits, thr_of, xg, s_hn, s_hlo, s_hhi, s_pick, s_n, s_w, turn);
         };
@@ -2136,7 +2182,8 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
         unsigned int n_ties = 0u;           // tokens with key == tau
         unsigned long long w_tie = 0ull;    // weight of each of them
         bool cut = false;
-        // (a top_k beyond the list only adds tokens of weight zero: nothing to do)
+        // (a top_k beyond everything that carries weight only adds tokens of weight zero: nothing to do)
+        if (top_k > 0 && unsigned(top_k) >= n_list && unsigned(top_k) - n_list < low.n) break;  // ends below the list
         if (top_k > 0 && unsigned(top_k) < n_list) {
             // the largest key with at least top_k entries at or above it
             const Picked pk = select(by_count, key_bits, [&](CountMass) { return static_cast<unsigned long long>(top_k) - 1ull; },
@@ -2156,8 +2203,9 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
                 // the largest key whose entries, with those above it, reach the target (without a cut so far the target
                 // follows from the weight of the whole list, which the search sums on its way)
                 const Picked pk = select(by_weight, key_bits,
-                                         [&](CountMass all) { return (cut ? target : target_of(all.w)) - 1ull; }, from_top);
+                                         [&](CountMass all) { return (cut ? target : target_of(all.w + low.w)) - 1ull; }, from_top);
                 const unsigned long long tgt = pk.thr + 1ull;
+                if (pk.all.w < tgt) break;  // the list does not hold the target (only possible with tokens left below it)
                 tau = key_max - pk.x;
                 w_tie = fixed_weight(key_logit<DT>(tau), M, scale);
                 w_above = pk.before.w;
@@ -2178,6 +2226,7 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
         }
         // The ties that are kept are those with the m lowest ids; the drawn token is the lowest id t with
         // (kept weight at ids <= t) > floor(u * kept weight). All ties weigh the same, so the kept weight needs no pass.
+        if (!cut && low.n > 0u) break;  // nothing is cut away: the draw is over the whole row
         const float u = __ldg(a.u + row);
         auto threshold_of = [&](unsigned long long S_kept) {  // (S_kept > 0: the row maximum is always kept)
             const unsigned long long t = static_cast<unsigned long long>(static_cast<double>(u) * static_cast<double>(S_kept));
@@ -2256,10 +2305,12 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
                 if (a.logp_argmax) a.logp_argmax[row] = (zt - M) * a.inv_t - l;
             }
         return;
-    }
+    } while (false);
 
-    // ---- more candidates than the list holds (a flat distribution): counts and weights come from passes over the
-    // row, tau by bisection on the key
+    // ---- the list does not reach (a flat distribution): counts and weights come from passes over the row, tau by
+    // bisection on the key
+    tau = 0u;
+    m = 0xFFFFFFFFu;
     auto above = [&](uint32_t lo) {  // (count, weight) of the tokens with key >= lo
         CountMass v{0u, 0ull};
         row_visit<DT>(rowp, a.V, aligned != 0, [&](int, float z) {

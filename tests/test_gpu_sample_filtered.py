@@ -151,6 +151,23 @@ def test_filtered_llama_size_rows_peaked_and_flat():
             assert np.array_equal(a[key].view(np.uint8), b[key].view(np.uint8)), key
 
 
+def test_filtered_masks_that_allow_most_of_the_vocabulary():
+    # nearly every class allowed: at T = 0.2 far more tokens carry weight than the candidate list holds, so the row is
+    # gone over again with a higher bar for the list and the rest is only summed; top-k / top-p that end inside the
+    # list are served from it, the others (k = 5000; k beyond every token with weight and no top-p) from the row
+    w = synth.make_workload(2, B=8)
+    cm = np.full_like(w.class_masks(0), 0xFFFFFFFF)
+    cm[3, 0] &= ~np.uint32(1)
+    z, u = w.logits(0), w.uniforms(0)
+    with Ctx(w.partitions) as ctx:
+        for inv_t, top_k, top_p in ((5.0, 50, 1.0), (5.0, 0, 0.9), (5.0, 0, 0.99), (5.0, 5000, 1.0), (5.0, 100000, 1.0),
+                                    (5.0, 200, 0.5), (2.0, 20, 1.0)):
+            got = run_filtered(ctx, None, cm, z, w.V, u, inv_t, top_k, top_p)
+            close, near = check_filtered(got, w.partitions, None, cm, z, w.V, u, inv_t, top_k, top_p,
+                                         "1/T=%g k=%d p=%g" % (inv_t, top_k, top_p))
+            assert close <= 1 and near <= 1
+
+
 @pytest.mark.parametrize("B", [40, 150])
 def test_filtered_one_and_two_blocks_per_row(B):
     # rows share thread-block clusters of 4 blocks up to 32 rows, of 2 up to 64, and have a block each beyond
