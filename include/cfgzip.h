@@ -420,6 +420,9 @@ int cfgzip_launch_count(cfgzip_ctx* ctx, int64_t* out);
  *   "lane_octets"  bf16 streaming kernel: octets (8 tokens) a lane handles per row of a work item: 1 = 16 bytes,
  *                  2 = 32 bytes (chunks of 512 tokens, at most 12 warps per block), 0 = automatic (default; currently
  *                  always 1: two octets measured 2 % faster at 256 rows with 8 warps x 3 stages and slower elsewhere)
+ *   "rotate"       1 (default) = the round-robin deal of a row batch's chunks to the warps of the streaming kernel
+ *                  starts at another warp for every row batch, so that the warps that get one chunk more differ from
+ *                  row batch to row batch; 0 = always at the first warp
  *   "test_expire_waits"  test hook, default 0: 1 makes every warp of the streaming kernel report its first wait
  *                  for an asynchronous copy as run out AFTER the wait has completed, so that the error path
  *                  (flag, bounded drain of the copies in flight, cfgzip_poll_status -> CFGZIP_E_CUDA) can be

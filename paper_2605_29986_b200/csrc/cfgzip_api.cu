@@ -79,6 +79,7 @@ struct cfgzip_ctx {
     int32_t pdl = 1;
     bool pdl_now = true;      // set per call: programmatic dependent launch only pays for short kernels
     int cluster_now = 1;      // set around a launch: blocks per thread-block cluster
+    int rotate = 1;           // the chunk deal of the pipelined kernel starts at another warp slot for every row batch
     // cuTensorMapEncodeTiled, looked up through the runtime (no link against the driver library)
     CUresult (*encode_tiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
@@ -483,6 +484,7 @@ void fill_groups(cfgzip_ctx* ctx, StepArgs& a, const DensePlan& d) {
     a.fold = d.fold;
     a.fold_off = d.fold_off;
     a.chunk_tokens = 256 * d.opl;
+    a.rot_chunks = ctx->rotate ? std::max(1, d.S * d.WT / ceil_div(std::min<int>(a.B, kGroupRows), kBatchRows)) : 0;
     a.expire_test = ctx->expire_test;
     a.p0 = ctx->parts[size_t(a.part0)].dev;
 }
@@ -1443,6 +1445,8 @@ int cfgzip_set_tuning(cfgzip_ctx* ctx, const char* name, int32_t value) {
     } else if (!std::strcmp(name, "auto_min_mbytes")) {
         if (value < -1) return CFGZIP_E_ARG;
         ctx->auto_min_bytes = value < 0 ? -1 : int64_t(value) << 20;
+    } else if (!std::strcmp(name, "rotate")) {
+        ctx->rotate = value != 0;
     } else if (!std::strcmp(name, "fold")) {
         if (value < 0 || value > 2) return CFGZIP_E_ARG;
         ctx->fold = value;

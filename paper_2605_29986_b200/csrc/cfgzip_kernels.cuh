@@ -46,6 +46,8 @@ struct StepArgs {
     int32_t run_chunks;         // sampling step: every warp slot of the pipelined kernel takes one contiguous run of this
                                 // many chunks, so that the published states of a row follow the token order
     int32_t chunk_tokens;       // tokens of one chunk of the pipelined kernel (256 or 512): sampling kernel's run length unit
+    int32_t rot_chunks;         // pipelined kernel, greedy step: the round-robin deal of a row batch's chunks starts this many
+                                // warp slots further on for every next row batch of the group
     int32_t expire_test;        // test hook: the pipelined kernel reports its first completed wait as run out
     int32_t fold;               // pipelined kernel: the last block of a row group folds the group's states and writes the
                                 // rows' results itself (no second kernel); tickets[g] counts the group's finished blocks
@@ -825,10 +827,18 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
     // range per block, and as fast as handing chunks out through global counters.
     // In a sampling step (TEMPERED) the states of a row must follow the token order: every warp slot then
     // takes one contiguous run of run_chunks chunks instead.
+    // The number of chunks is rarely a multiple of the number of warp slots, so some slots get one chunk more than
+    // the others; the deal starts at a different slot for every row batch (rot_chunks further on), which spreads the
+    // extra chunks evenly over the warps and the blocks instead of giving the first ones one more in every row batch.
     const int n_chunks = (n_full + G::kChunkOctets - 1) / G::kChunkOctets;
-    const int first_chunk = TEMPERED ? (split * a.WT + wt) * a.run_chunks : split * a.WT + wt;  // this warp's first chunk
     const int stride_chunks = TEMPERED ? 1 : a.S * a.WT;  // round-robin: warps that share a row batch of the group
-    const int chunk_end = TEMPERED ? min(first_chunk + a.run_chunks, n_chunks) : n_chunks;
+    auto first_chunk_of = [&](int rb) {  // this warp's first chunk of row batch rb
+        if (TEMPERED) return (split * a.WT + wt) * a.run_chunks;
+        int c = split * a.WT + wt - rb * a.rot_chunks;
+        c %= stride_chunks;
+        return c < 0 ? c + stride_chunks : c;
+    };
+    const int chunk_end = TEMPERED ? min(first_chunk_of(0) + a.run_chunks, n_chunks) : n_chunks;
     int* const slot_info = ring_info + warp * depth; // (rb << 24) | chunk of the item in each slot, -1 = no more items
 
     // automatic mode: bit r = row slot r was finished by the class-list kernel (set after the wait below)
@@ -850,7 +860,7 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
                 continue;
             }
             if (p_first) {
-                chunk = first_chunk;
+                chunk = first_chunk_of(p_rb);
                 p_first = false;
             } else {
                 chunk = p_chunk + stride_chunks;
