@@ -2002,6 +2002,9 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
     __shared__ unsigned int s_n[2 * kFiltThreads / 32];
     __shared__ unsigned long long s_w[2 * kFiltThreads / 32];
     __shared__ unsigned long long s_scan[kFiltThreads / 32];
+    __shared__ unsigned int s_sel_n[2 * kSelThreads / 32];  // the searches' own sets (only some threads sum there, so
+    __shared__ unsigned long long s_sel_w[2 * kSelThreads / 32];  // their turn must not be that of the block's sums)
+    int turn_sel = 0;
     __shared__ __align__(16) unsigned int s_hn[kSelBuckets], s_hlo[kSelBuckets], s_hhi[kSelBuckets];
     __shared__ unsigned long long s_pick[16];
     __shared__ unsigned long long s_top_w[kSelThreads];  // the entries with key >= tau when there are few of them
@@ -2170,7 +2173,7 @@ __global__ void __launch_bounds__(kFiltThreads) k_sample_filtered(const __grid_c
         // ---- everything from the list (it holds the tokens that carry weight, or the heaviest of them, in no
         // particular order); leaves for the passes over the row below when top-k or top-p reach past the list
         auto select = [&](auto kind, int bits, auto&& thr_of, auto&& xg) {
-            return list_select<decltype(kind)::value>(n_list, bits, thr_of, xg, s_hn, s_hlo, s_hhi, s_pick, s_n, s_w, turn);
+            return list_select<decltype(kind)::value>(n_list, bits, thr_of, xg, s_hn, s_hlo, s_hhi, s_pick, s_sel_n, s_sel_w, turn_sel);
         };
         const std::integral_constant<bool, false> by_count;
         const std::integral_constant<bool, true> by_weight;

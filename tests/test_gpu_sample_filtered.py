@@ -154,18 +154,39 @@ def test_filtered_llama_size_rows_peaked_and_flat():
 def test_filtered_masks_that_allow_most_of_the_vocabulary():
     # nearly every class allowed: at T = 0.2 far more tokens carry weight than the candidate list holds, so the row is
     # gone over again with a higher bar for the list and the rest is only summed; top-k / top-p that end inside the
-    # list are served from it, the others (k = 5000; k beyond every token with weight and no top-p) from the row
+    # list are served from it, the others (k = 5000; k beyond every token with weight and no top-p; at T = 1 a nucleus
+    # of 99 %, found too large only after the search over the list) from the row
     w = synth.make_workload(2, B=8)
     cm = np.full_like(w.class_masks(0), 0xFFFFFFFF)
     cm[3, 0] &= ~np.uint32(1)
     z, u = w.logits(0), w.uniforms(0)
     with Ctx(w.partitions) as ctx:
         for inv_t, top_k, top_p in ((5.0, 50, 1.0), (5.0, 0, 0.9), (5.0, 0, 0.99), (5.0, 5000, 1.0), (5.0, 100000, 1.0),
-                                    (5.0, 200, 0.5), (2.0, 20, 1.0)):
+                                    (5.0, 200, 0.5), (2.0, 20, 1.0), (1.0, 0, 0.99), (1.0, 0, 0.3)):
             got = run_filtered(ctx, None, cm, z, w.V, u, inv_t, top_k, top_p)
             close, near = check_filtered(got, w.partitions, None, cm, z, w.V, u, inv_t, top_k, top_p,
                                          "1/T=%g k=%d p=%g" % (inv_t, top_k, top_p))
-            assert close <= 1 and near <= 1
+            # (at T = 1 a nucleus ends among tokens of about 1e-7 of the weight each: every cut there is too close to
+            # call between fixed point and fp64, and only the validity of the draw is checked)
+            assert near <= 1 and (close <= 1 or inv_t < 2.0)
+
+
+def test_filtered_nucleus_larger_than_the_list_found_after_the_search():
+    # f32, T = 1, 18 thousand allowed tokens: the list overflows, is rebuilt with a higher bar, the search for the
+    # top-p cut runs over it and finds that the list does not hold 99 % of the weight: the passes over the row take over
+    V, K, B = 183926, 1426, 36
+    part = synth.zipf_partition(V, K, 1.1, seed=54)
+    cm = synth.class_mask_bernoulli(K, B, 0.1, rng.stream_key(91))
+    cm[:, 0] |= 1
+    z = synth.logits_normal(B, V + 2, 2.0, "f32", (92,))
+    u = rng.uniform(rng.stream_key(93), B).astype(np.float32)
+    with Ctx([part]) as ctx:
+        for top_k, top_p in ((0, 0.99), (0, 0.9), (15000, 0.95)):
+            got = run_filtered(ctx, None, cm, z, V, u, 1.0, top_k, top_p, stride=V + 2)
+            close, near = check_filtered(got, [part], None, cm, z, V, u, 1.0, top_k, top_p, "k=%d p=%g" % (top_k, top_p))
+            # (most cuts among so many light tokens are too close to call between fixed point and fp64; the rows
+            # that can be called must match, and there must be some)
+            assert near <= 1 and close <= B - 3, (top_k, top_p, close, near)
 
 
 @pytest.mark.parametrize("B", [40, 150])
