@@ -205,6 +205,38 @@ def test_filtered_one_and_two_blocks_per_row(B):
             assert close <= 2 and near <= 2
 
 
+@pytest.mark.parametrize("case", range(32))
+def test_filtered_random_shapes(case):
+    # shape, element type, padding, temperature, mask density, spread of the logits and both filters drawn per case
+    u = rng.u64(rng.stream_key(7101, case), 12)
+    V = int(u[0] % np.uint64([3000, 40000, 200000][int(u[9] % np.uint64(3))])) + 1
+    K = int(u[1] % np.uint64(min(V, 5000))) + 1
+    B = [1, 7, 32, 33, 64, 65, 150][int(u[2] % np.uint64(7))]
+    dtype = "bf16" if u[3] & np.uint64(1) else "f32"
+    pad = (-V) % 8 if (u[4] % np.uint64(4)) else 3
+    inv_t = [0.5, 1.0, 5.0, 20.0][int(u[5] % np.uint64(4))]
+    density = [0.01, 0.1, 0.5, 1.0][int(u[6] % np.uint64(4))]
+    top_k = [0, 1, 5, 50, 300, 3000, 100000000][int(u[7] % np.uint64(7))]
+    top_p = [1.0, 0.5, 0.9, 0.99, 0.1][int(u[8] % np.uint64(5))]
+    if top_k == 0 and top_p == 1.0:
+        top_k = 20
+    sigma = [0.5, 2.0, 6.0][int(u[10] % np.uint64(3))]
+    part = synth.zipf_partition(V, K, 1.1, seed=case)
+    cm = synth.class_mask_bernoulli(K, B, density, rng.stream_key(7102, case))
+    cm[:, 0] |= 1
+    if density == 1.0:
+        cm[:] = 0xFFFFFFFF
+    unique = min(B, 16)
+    z = np.tile(synth.logits_normal(unique, V + pad, sigma, dtype, (7103, case)), (-(-B // unique), 1))[:B]
+    uu = rng.uniform(rng.stream_key(7104, case), B).astype(np.float32)
+    sel = np.unique(np.linspace(0, B - 1, min(B, 12)).astype(np.int64))  # rows checked against the oracle
+    what = "V=%d K=%d B=%d %s pad=%d 1/T=%g density=%g k=%d p=%g sigma=%g" % (V, K, B, dtype, pad, inv_t, density, top_k, top_p, sigma)
+    with Ctx([part]) as ctx:
+        got = run_filtered(ctx, None, cm, z, V, uu, inv_t, top_k, top_p, stride=V + pad)
+    sub = {k: v[sel] for k, v in got.items()}
+    check_filtered(sub, [part], None, cm[sel], z[sel], V, uu[sel], inv_t, top_k, top_p, what)
+
+
 def test_no_filter_is_the_plain_sampling_step_and_bad_filters_are_refused():
     w = synth.make_workload(2, B=16, V=20000, K=300)
     cm, z, u = w.class_masks(1), w.logits(1), w.uniforms(1)
