@@ -145,10 +145,11 @@ def test_filtered_llama_size_rows_peaked_and_flat():
             assert near <= 2
         assert total_close <= 3
         # twice the same call: the same bits (integer sums do not depend on the order of the addends)
-        a = run_filtered(ctx, None, cm, z, w.V, u, 1.0, 0, 0.5)
-        b = run_filtered(ctx, None, cm, z, w.V, u, 1.0, 0, 0.5)
-        for key in ("token", "lse", "logp_token"):
-            assert np.array_equal(a[key].view(np.uint8), b[key].view(np.uint8)), key
+        for inv_t, top_k, top_p in ((1.0, 0, 0.5), (5.0, 50, 0.9), (5.0, 2000, 1.0)):  # over the row; list, few kept; list, many kept
+            a = run_filtered(ctx, None, cm, z, w.V, u, inv_t, top_k, top_p)
+            b = run_filtered(ctx, None, cm, z, w.V, u, inv_t, top_k, top_p)
+            for key in ("token", "lse", "logp_token"):
+                assert np.array_equal(a[key].view(np.uint8), b[key].view(np.uint8)), (key, inv_t, top_k, top_p)
 
 
 def test_filtered_masks_that_allow_most_of_the_vocabulary():
