@@ -664,6 +664,8 @@ int launch_filtered(cfgzip_ctx* ctx, const StepArgs& a, unsigned rows_grid, int 
     rc = launch(ctx, k_sample_filtered<DT>, dim3(rows_grid * per_row), dim3(kFiltThreads), kFiltSmem, st, a, aligned, top_k,
                 top_p);
     ctx->cluster_now = 1;
+    if (rc != CFGZIP_OK && per_row > 1)  // a device that cannot place such a cluster: one block per row
+        rc = launch(ctx, k_sample_filtered<DT>, dim3(rows_grid), dim3(kFiltThreads), kFiltSmem, st, a, aligned, top_k, top_p);
     return rc;
 }
 
