@@ -224,7 +224,7 @@ class StepRunner:
 
     def __init__(self, cz, torch, device: int, config: int, B: int = None, mode: str = "dense", steps_hint: int = 1000,
                  unique: int = 8, tune=(), kind: str = "fused", ring: int = 0, inv_temperature: float = 0.0, top_k: int = 0,
-                 top_p: float = 1.0):
+                 top_p: float = 1.0, allow_all: bool = False):
         self.cz, self.torch = cz, torch
         # kind: "fused" the whole step; "unfused" separate expand + mask calls (no reductions); "floor" the in-place
         # read-modify-write kernel over the same buffers (what a pass over these bytes costs at least)
@@ -262,6 +262,8 @@ class StepRunner:
             self.host_logits.append(z)
             self.pristine.append(torch.from_numpy(z.view(np.int16) if self.dtype == "bf16" else z).cuda())
         self.host_cm = np.stack([self.w.class_masks(j) for j in range(self.R)])
+        if allow_all:  # every class allowed (an unconstrained position of the grammar): the masks allow the whole vocabulary
+            self.host_cm[:] = 0xFFFFFFFF
         self.cm = torch.from_numpy(self.host_cm.view(np.int32)).cuda()
         self.row_part_host = None if self.w.row_part is None else np.ascontiguousarray(self.w.row_part, dtype=np.int32)
         self.row_part = None if self.row_part_host is None else torch.from_numpy(self.row_part_host).cuda()
@@ -692,6 +694,14 @@ def run_own(args):
             us8, _, l8 = _measure(r8)
             filt.append({"top_k": top_k, "top_p": top_p, "B": r8.B, "us_per_step": us8, "launches_per_step": l8})
             r8.close()
+        # the same with masks that allow every class: far more tokens carry weight than the candidate list holds, and
+        # the row is gone over a second time with a higher bar for the list
+        r9 = StepRunner(cz, torch, local_rank, args.workload, B=args.batch, mode=args.mode, steps_hint=64, unique=2,
+                        tune=args.tune, inv_temperature=5.0, top_k=50, top_p=0.9, allow_all=True)
+        us9, _, l9 = _measure(r9)
+        filt.append({"top_k": 50, "top_p": 0.9, "B": r9.B, "us_per_step": us9, "launches_per_step": l9,
+                     "masks": "every class allowed"})
+        r9.close()
         line["filtered_sampling_step_T0.2"] = filt
         line["offline_grouping"] = _offline_grouping(cz, torch)
         line["multi_mask_step"] = _multi_mask(cz, torch, local_rank)
