@@ -420,6 +420,10 @@ int cfgzip_launch_count(cfgzip_ctx* ctx, int64_t* out);
  *   "lane_octets"  bf16 streaming kernel: octets (8 tokens) a lane handles per row of a work item: 1 = 16 bytes,
  *                  2 = 32 bytes (chunks of 512 tokens, at most 12 warps per block), 0 = automatic (default; currently
  *                  always 1: two octets measured 2 % faster at 256 rows with 8 warps x 3 stages and slower elsewhere)
+ *   "prefetch_items"  work items per warp of the streaming kernel whose logits are asked into the L2 (a hint, nothing is
+ *                  read) while the kernel in front is still finishing, on programmatic launches of steps of at least
+ *                  "prefetch_min_mbytes" megabytes of logits (0..64, default 4; 0 = none)
+ *   "prefetch_min_mbytes"  see above (default 48: shorter steps were measured slower with the hint)
  *   "rotate"       1 (default) = the round-robin deal of a row batch's chunks to the warps of the streaming kernel
  *                  starts at another warp for every row batch, so that the warps that get one chunk more differ from
  *                  row batch to row batch; 0 = always at the first warp

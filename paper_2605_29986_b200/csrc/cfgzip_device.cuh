@@ -378,6 +378,14 @@ __device__ __forceinline__ void tma_g2s_2d(void* dst_smem, const void* tensor_ma
         "l"(tensor_map), "r"(x), "r"(y), "r"(smem_u32(bar))
         : "memory");
 }
+// The same box into the L2 only (a hint: nothing is delivered, no barrier involved).
+__device__ __forceinline__ void tma_prefetch_2d(const void* tensor_map, int x, int y) {
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(tensor_map), "r"(x), "r"(y) : "memory");
+}
+// size and address multiples of 16 bytes; into the L2 only
+__device__ __forceinline__ void bulk_prefetch(const void* src_gmem, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src_gmem), "r"(bytes) : "memory");
+}
 // size and both addresses are multiples of 16 bytes
 __device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(

@@ -46,6 +46,8 @@ struct StepArgs {
     int32_t run_chunks;         // sampling step: every warp slot of the pipelined kernel takes one contiguous run of this
                                 // many chunks, so that the published states of a row follow the token order
     int32_t chunk_tokens;       // tokens of one chunk of the pipelined kernel (256 or 512): sampling kernel's run length unit
+    int32_t prefetch_items;     // pipelined kernel without a row plan: work items per warp whose logits are asked into the L2
+                                // before the wait for the kernel in front (a hint; nothing is read until after the wait)
     int32_t rot_chunks;         // pipelined kernel, greedy step: the round-robin deal of a row batch's chunks starts this many
                                 // warp slots further on for every next row batch of the group
     int32_t expire_test;        // test hook: the pipelined kernel reports its first completed wait as run out
@@ -908,6 +910,29 @@ __global__ void __launch_bounds__(LBT, MINB) k_step_dense_pipe(const __grid_cons
         for (int d = 0; d < depth; ++d) mbar_init(bar + d, 1);
         if (warp == 0 && !early_cm) mbar_init(&cm_bar, 1);
         mbar_init_fence();
+    }
+    if (implicit && a.prefetch_items > 0 && lane == 0 && !p_done) {
+        // While the kernel in front is finishing, DRAM has little to do: ask this warp's first work items (and the
+        // group's class masks) into the L2. These are hints only: they deliver nothing, and whatever the kernel in
+        // front may still write reaches the same L2, so nothing stale can be read after the wait.
+        const int row0 = g * kGroupRows + wr * kBatchRows;
+        const int live0 = min(kBatchRows, nrow - wr * kBatchRows);
+        int chunk = first_chunk_of(wr);
+        for (int d = 0; d < a.prefetch_items && chunk < chunk_end; ++d, chunk += TEMPERED ? 1 : stride_chunks) {
+            const int o0 = chunk * G::kChunkOctets;
+            const uint32_t nvec = uint32_t(min(n_full - o0, G::kChunkOctets));
+            if (TMAP) {
+                tma_prefetch_2d(&tmap, o0 * 8, row0);
+                if (OPL == 2 && nvec > 32u) tma_prefetch_2d(&tmap, o0 * 8 + 256, row0);
+            } else {
+                for (int i = 0; i < live0; ++i)
+                    bulk_prefetch(reinterpret_cast<const char*>(a.logits) + (int64_t(row0 + i) * a.row_stride * ES + int64_t(o0) * 8 * ES),
+                                  nvec * G::kOctetBytes);
+            }
+        }
+        if (warp == 0 && a.cm_bulk)
+            for (int r = 0; r < nrow; ++r)
+                bulk_prefetch(a.class_mask + int64_t(g * kGroupRows + r) * a.cm_stride, uint32_t(a.p0.KW) * 4u);
     }
     if (implicit) pdl_wait();
     // automatic mode: row batches that allow few tokens were finished by the class-list kernel in front and get no
