@@ -52,13 +52,13 @@ LOG_TOL = 1e-4                # absolute, fp32-accumulated log quantities agains
 # DRAM traffic of the dominant (streaming) kernel per launch = per step (dram__bytes_read.sum +
 # dram__bytes_write.sum from one ncu capture, see profiles/), keyed by workload; valid only for the kernel
 # sources whose digest is recorded with it. A workload without a capture of the current sources reports null.
-_CAPTURED = "0970c426c414458b"
+_CAPTURED = "02183c84a4d7b29e"
 NCU_TRAFFIC = {
-    "cfg2_B32_dense": {"digest": _CAPTURED, "bytes_per_launch": 14788352},      # 8.24 MB read + 6.55 MB written (L2 still filling)
-    "cfg2_B1024_dense": {"digest": _CAPTURED, "bytes_per_launch": 541683797},   # 263.2 MB read + 278.5 MB written
-    "cfg4_B256_dense": {"digest": _CAPTURED, "bytes_per_launch": 269616555},    # 132.5 MB read + 137.1 MB written
-    "cfg5_B1024_dense": {"digest": _CAPTURED, "bytes_per_launch": 1066656512},  # 526.3 MB read + 540.3 MB written
-    "cfg5_B1024_sparse": {"digest": _CAPTURED, "bytes_per_launch": 611926613},  # 65.2 MB read + 546.8 MB written
+    "cfg2_B32_dense": {"digest": _CAPTURED, "bytes_per_launch": 14954837},      # 8.24 MB read + 6.71 MB written (L2 still filling)
+    "cfg2_B1024_dense": {"digest": _CAPTURED, "bytes_per_launch": 541736960},   # 263.2 MB read + 278.5 MB written
+    "cfg4_B256_dense": {"digest": _CAPTURED, "bytes_per_launch": 269750784},    # 132.4 MB read + 137.4 MB written
+    "cfg5_B1024_dense": {"digest": _CAPTURED, "bytes_per_launch": 1067131051},  # 526.5 MB read + 540.6 MB written
+    "cfg5_B1024_sparse": {"digest": _CAPTURED, "bytes_per_launch": 611983872},  # 65.1 MB read + 546.9 MB written
 }
 
 
